@@ -1,0 +1,112 @@
+"""fp64 CPU oracle for shared-prefix batched causal attention (ctypes wrapper).
+
+TEST INFRASTRUCTURE ONLY: tests, the smoke check and the CPU-baseline leg of
+the benchmark may import this package; the product path never does, and this
+package imports nothing from the CUDA package.
+
+``attn_fwd`` / ``attn_bwd`` take numpy arrays of any float dtype, widen them
+to fp64 and call the plain-C program in ``pskv_oracle.c`` (paper Eq. 2 over
+the per-candidate duplicated prefix cache of Eq. 3).  Inputs that are meant
+to be bf16 must already hold bf16-representable values; the oracle does not
+round anything.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pskv_oracle.c")
+_LIB = os.path.join(_HERE, "libpskv_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile pskv_oracle.c with gcc (OpenMP) into libpskv_oracle.so."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + ".tmp.%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        dp = ctypes.POINTER(ctypes.c_double)
+        ints = [ctypes.c_int] * 6
+        lib.pskv_oracle_attn_fwd.argtypes = [dp] * 5 + [ctypes.c_double] + [dp] * 2 + ints
+        lib.pskv_oracle_attn_fwd.restype = ctypes.c_int
+        lib.pskv_oracle_attn_bwd.argtypes = [dp] * 6 + [ctypes.c_double] + [dp] * 3 + ints
+        lib.pskv_oracle_attn_bwd.restype = ctypes.c_int
+        lib.pskv_oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the C program uses (OpenMP max threads)."""
+    return int(_load().pskv_oracle_num_threads())
+
+
+def _f64(a, shape):
+    a = np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+    if a.shape != tuple(shape):
+        raise ValueError("expected shape %s, got %s" % (tuple(shape), a.shape))
+    return a
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _dims(q, prefix_k, suffix_k):
+    q = np.asarray(q)
+    B, Hq, S, d = q.shape
+    Hkv, P = np.asarray(prefix_k).shape[:2]
+    return B, Hq, Hkv, S, P, d
+
+
+def attn_fwd(q, prefix_k, prefix_v, suffix_k, suffix_v, scale):
+    """out [B,Hq,S,d] and lse [B,Hq,S] (fp64) per Eq. 2 with the duplicated cache of Eq. 3."""
+    B, Hq, Hkv, S, P, d = _dims(q, prefix_k, suffix_k)
+    q = _f64(q, (B, Hq, S, d))
+    pk = _f64(prefix_k, (Hkv, P, d))
+    pv = _f64(prefix_v, (Hkv, P, d))
+    sk = _f64(suffix_k, (B, Hkv, S, d))
+    sv = _f64(suffix_v, (B, Hkv, S, d))
+    out = np.empty((B, Hq, S, d), dtype=np.float64)
+    lse = np.empty((B, Hq, S), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_fwd(_ptr(q), _ptr(pk), _ptr(pv), _ptr(sk), _ptr(sv),
+                                      float(scale), _ptr(out), _ptr(lse), B, Hq, Hkv, S, P, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_fwd failed with code %d" % rc)
+    return out, lse
+
+
+def attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, scale):
+    """dq, dk_suffix, dv_suffix (fp64) of L = sum(out * dout); prefix K/V frozen."""
+    B, Hq, Hkv, S, P, d = _dims(q, prefix_k, suffix_k)
+    do = _f64(dout, (B, Hq, S, d))
+    q = _f64(q, (B, Hq, S, d))
+    pk = _f64(prefix_k, (Hkv, P, d))
+    pv = _f64(prefix_v, (Hkv, P, d))
+    sk = _f64(suffix_k, (B, Hkv, S, d))
+    sv = _f64(suffix_v, (B, Hkv, S, d))
+    dq = np.empty((B, Hq, S, d), dtype=np.float64)
+    dk = np.empty((B, Hkv, S, d), dtype=np.float64)
+    dv = np.empty((B, Hkv, S, d), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_bwd(_ptr(do), _ptr(q), _ptr(pk), _ptr(pv), _ptr(sk), _ptr(sv),
+                                      float(scale), _ptr(dq), _ptr(dk), _ptr(dv),
+                                      B, Hq, Hkv, S, P, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_bwd failed with code %d" % rc)
+    return dq, dk, dv

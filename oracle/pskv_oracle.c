@@ -1,0 +1,200 @@
+/*
+ * fp64 CPU oracle for shared-prefix batched causal attention.
+ *
+ * TEST INFRASTRUCTURE ONLY.  Nothing on the product path may call, link or
+ * import this file; it exists so that the CUDA kernels can be compared with
+ * an independent, slow, obviously-correct program.  It shares no code with
+ * the CUDA path.
+ *
+ * What it computes (paper Sec. 3, Eq. 2 with the cache of Eq. 3):
+ *   every candidate b gets its OWN physical copy of the prefix keys/values
+ *   (the "Repeat(K, V, times = N)" of Eq. 3, i.e. the standard-KV-cache
+ *   formulation), the candidate's suffix keys/values are appended
+ *   (Sec. 4.2: the prefix cache is concatenated with the suffix-side K/V
+ *   of the current layer), and ordinary causal scaled-dot-product attention
+ *   (Eq. 2) is run for the S suffix-side query rows: row i sees the P
+ *   prefix keys and suffix keys 0..i.
+ *
+ *   Grouped-query attention (Appendix E: several query heads share one KV
+ *   head): query head h reads KV head g = h / (Hq / Hkv).
+ *
+ * Layouts (dense, row-major, last index fastest), all fp64:
+ *   q, out, dout, dq     [B][Hq][S][d]
+ *   prefix_k, prefix_v   [Hkv][P][d]
+ *   suffix_k, suffix_v   [B][Hkv][S][d]      (also dk_suffix, dv_suffix)
+ *   lse                  [B][Hq][S]          natural log of sum_j exp(s_j)
+ *
+ * Parity pins (tests/test_oracle_pins.py): full-sequence no-cache attention
+ * through a library routine, closed forms (zero queries, constant values,
+ * key shift, the P=1,S=1 logistic form), prefix/suffix split invariance,
+ * candidate permutation, GQA-vs-repeated-MHA, the log-sum-exp merge
+ * identity, and central finite differences for the backward pass.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int pskv_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* K_full[b,g] = prefix_k[g] (+) suffix_k[b,g]  -- the per-candidate physical
+ * duplicate of Eq. 3, followed by the concatenation of Sec. 4.2. */
+static void build_full_kv(const double *prefix, const double *suffix, double *full,
+                          int b, int g, int Hkv, int S, int P, int d)
+{
+    memcpy(full, prefix + (size_t)g * P * d, sizeof(double) * (size_t)P * d);
+    memcpy(full + (size_t)P * d, suffix + ((size_t)b * Hkv + g) * S * d,
+           sizeof(double) * (size_t)S * d);
+}
+
+/* Eq. 2 for one query row against its n_vis visible keys.
+ * s[j] = scale * <q, K[j]>, returns lse = m + ln sum exp(s - m) and leaves
+ * the normalised probabilities in p[0..n_vis). */
+static double softmax_row(const double *qrow, const double *K, int n_vis, int d,
+                          double scale, double *p)
+{
+    double m = -INFINITY;
+    for (int j = 0; j < n_vis; ++j) {
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c) acc += qrow[c] * K[(size_t)j * d + c];
+        p[j] = scale * acc;
+        if (p[j] > m) m = p[j];
+    }
+    double l = 0.0;
+    for (int j = 0; j < n_vis; ++j) {
+        p[j] = exp(p[j] - m);
+        l += p[j];
+    }
+    for (int j = 0; j < n_vis; ++j) p[j] /= l;
+    return m + log(l);
+}
+
+int pskv_oracle_attn_fwd(const double *q, const double *prefix_k, const double *prefix_v,
+                         const double *suffix_k, const double *suffix_v, double scale,
+                         double *out, double *lse,
+                         int B, int Hq, int Hkv, int S, int P, int d)
+{
+    if (B < 1 || Hq < 1 || Hkv < 1 || S < 1 || P < 0 || d < 1 || Hq % Hkv != 0) return 1;
+    const int n_rep = Hq / Hkv;
+    const int T = P + S;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        if (!Kf || !Vf || !p) {
+            failed = 1;
+        } else {
+            for (int g = 0; g < Hkv; ++g) {
+                build_full_kv(prefix_k, suffix_k, Kf, b, g, Hkv, S, P, d);
+                build_full_kv(prefix_v, suffix_v, Vf, b, g, Hkv, S, P, d);
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < S; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * S + i;
+                        const int n_vis = P + i + 1;
+                        lse[row] = softmax_row(q + row * d, Kf, n_vis, d, scale, p);
+                        double *o = out + row * d;
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+    }
+    return failed ? 2 : 0;
+}
+
+/*
+ * Closed-form backward of L = sum(out * dout) (no autodiff).  From the
+ * softmax Jacobian d o / d s_j = p_j (v_j - o):
+ *   D    = <dout_row, out_row>
+ *   dp_j = <dout_row, V[j]>
+ *   ds_j = p_j (dp_j - D)
+ *   dq_row        = scale * sum_j ds_j K[j]
+ *   dK[j]        += scale * ds_j q_row          (kept only for suffix keys j >= P)
+ *   dV[j]        += p_j dout_row                (kept only for suffix keys j >= P)
+ * Suffix-key gradients are summed over the query rows that see the key and
+ * over the Hq/Hkv query heads that share the KV head.  The prefix cache is
+ * computed once and frozen (Sec. 4.2: only gradients with respect to the
+ * suffix side are needed), so contributions to prefix keys are discarded.
+ * The forward quantities (p, out) are recomputed here in fp64.
+ */
+int pskv_oracle_attn_bwd(const double *dout, const double *q,
+                         const double *prefix_k, const double *prefix_v,
+                         const double *suffix_k, const double *suffix_v, double scale,
+                         double *dq, double *dk_suffix, double *dv_suffix,
+                         int B, int Hq, int Hkv, int S, int P, int d)
+{
+    if (B < 1 || Hq < 1 || Hkv < 1 || S < 1 || P < 0 || d < 1 || Hq % Hkv != 0) return 1;
+    const int n_rep = Hq / Hkv;
+    const int T = P + S;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        double *o = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!Kf || !Vf || !p || !o) {
+            failed = 1;
+        } else {
+            for (int g = 0; g < Hkv; ++g) {
+                build_full_kv(prefix_k, suffix_k, Kf, b, g, Hkv, S, P, d);
+                build_full_kv(prefix_v, suffix_v, Vf, b, g, Hkv, S, P, d);
+                double *dKs = dk_suffix + ((size_t)b * Hkv + g) * S * d;
+                double *dVs = dv_suffix + ((size_t)b * Hkv + g) * S * d;
+                for (size_t e = 0; e < (size_t)S * d; ++e) { dKs[e] = 0.0; dVs[e] = 0.0; }
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < S; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * S + i;
+                        const int n_vis = P + i + 1;
+                        const double *qr = q + row * d;
+                        const double *go = dout + row * d;
+                        softmax_row(qr, Kf, n_vis, d, scale, p);
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                        double D = 0.0;
+                        for (int c = 0; c < d; ++c) D += go[c] * o[c];
+                        double *dqr = dq + row * d;
+                        for (int c = 0; c < d; ++c) dqr[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j) {
+                            double dp = 0.0;
+                            for (int c = 0; c < d; ++c) dp += go[c] * Vf[(size_t)j * d + c];
+                            const double ds = p[j] * (dp - D);
+                            for (int c = 0; c < d; ++c) dqr[c] += scale * ds * Kf[(size_t)j * d + c];
+                            if (j >= P) {
+                                const int t = j - P;
+                                for (int c = 0; c < d; ++c) {
+                                    dKs[(size_t)t * d + c] += scale * ds * qr[c];
+                                    dVs[(size_t)t * d + c] += p[j] * go[c];
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+        free(o);
+    }
+    return failed ? 2 : 0;
+}
