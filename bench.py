@@ -1,0 +1,451 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-prefix attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one forward (`pskv_attn_fwd`: out, lse) plus one backward (`pskv_attn_bwd`: dq,
+dk_suffix, dv_suffix) of one attention layer of the Llama-3-8B-shaped GQA workload (C2:
+B=512 candidates, 32 query / 8 KV heads, d=128, prefix 256, suffix-side 48, outlier key
+channels), all inputs resident in HBM.  Prints ONE JSON line on rank 0.  With N > 1 each
+rank runs the same step on its own B candidates against its own replica of the prefix cache
+(candidates are independent given the prefix; there is no collective on the data path).
+`--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_13420_b200 import inputs as wl  # noqa: E402
+
+METRIC = "shared-prefix attention TFLOP/s (fwd+bwd, one layer)"
+MAIN = "C2"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.lines = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax = float(parts[2])
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": smax,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), \
+        int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    """The fp64 CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    w = wl.WORKLOADS[MAIN]
+    cand = args.ref_candidates
+    sub = w.with_candidates(cand)
+    t = wl.make_inputs(sub, with_dout=True)
+    f = {k: v.to(torch.float64).numpy() for k, v in t.items()}
+
+    def step():
+        oracle.attn_fwd(f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"], w.scale)
+        oracle.attn_bwd(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"],
+                        w.scale)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    flops = wl.fwd_flops(sub) + wl.bwd_flops(sub)
+    value = flops / dt / 1e12
+    cores = oracle.num_threads()
+    sample = "%d of %d candidates of %s per step, fwd+bwd, fp64" % (cand, w.B, MAIN)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(w, 1),
+        "candidates_per_s": cand / dt,
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, world):
+    return {"workload": "%s: %s" % (w.name, w.note), "B_per_gpu": w.B, "Hq": w.Hq, "Hkv": w.Hkv,
+            "d": w.d, "P": w.P, "S": w.S, "step": "pskv_attn_fwd + pskv_attn_bwd, one layer",
+            "parallelism": "candidates sharded over %d GPU(s), prefix cache replicated" % world,
+            "l2": "inputs larger than L2 (%.0f MB touched per step vs 126 MB L2)"
+                  % ((wl.fwd_bytes(w) + wl.bwd_bytes(w)) / 1e6)}
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+
+def time_calls(fn, iters, warmup):
+    """Median-free plain average over `iters` calls with CUDA events on the current stream."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters  # ms
+
+
+def device_inputs(w, seed, device):
+    """Same distribution as inputs.make_inputs, drawn on the device (kernel-only timing legs)."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+
+    def draw(shape, outliers=False):
+        x = torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
+        if outliers:
+            for c in wl.OUTLIER_CHANNELS:
+                x[..., c] *= wl.OUTLIER_GAIN
+        return x.to(torch.bfloat16)
+
+    t = {"q": draw((w.B, w.Hq, w.S, w.d)),
+         "prefix_k": draw((w.Hkv, w.P, w.d), w.outlier_keys),
+         "prefix_v": draw((w.Hkv, w.P, w.d)),
+         "suffix_k": draw((w.B, w.Hkv, w.S, w.d), w.outlier_keys),
+         "suffix_v": draw((w.B, w.Hkv, w.S, w.d)),
+         "dout": draw((w.B, w.Hq, w.S, w.d))}
+    return t
+
+
+class Layer:
+    """Device buffers of one attention layer call (inputs, outputs, workspaces)."""
+
+    def __init__(self, pskv, w, t):
+        self.pskv, self.w, self.t = pskv, w, t
+        dev = t["q"].device
+        dims = (w.B, w.Hq, w.Hkv, w.S, w.P, w.d)
+        self.out = torch.empty_like(t["q"])
+        self.lse = torch.empty((w.B, w.Hq, w.S), dtype=torch.float32, device=dev)
+        self.dq = torch.empty_like(t["q"])
+        self.dk = torch.empty_like(t["suffix_k"])
+        self.dv = torch.empty_like(t["suffix_v"])
+        self.ws_f = torch.empty(max(pskv.pskv_attn_fwd_workspace_bytes(*dims), 256), dtype=torch.uint8, device=dev)
+        self.ws_b = torch.empty(max(pskv.pskv_attn_bwd_workspace_bytes(*dims), 256), dtype=torch.uint8, device=dev)
+
+    def fwd(self):
+        t = self.t
+        self.pskv.pskv_attn_fwd(t["q"], t["prefix_k"], t["prefix_v"], t["suffix_k"], t["suffix_v"],
+                                self.w.scale, out=self.out, lse=self.lse, workspace=self.ws_f)
+
+    def bwd(self):
+        t = self.t
+        self.pskv.pskv_attn_bwd(t["dout"], t["q"], t["prefix_k"], t["prefix_v"], t["suffix_k"],
+                                t["suffix_v"], self.out, self.lse, self.w.scale,
+                                dq=self.dq, dk_suffix=self.dk, dv_suffix=self.dv, workspace=self.ws_b)
+
+
+def run_cuda(args):
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    import paper_2603_13420_b200 as pskv
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    peaks = load_peaks()
+    w = wl.WORKLOADS[MAIN]
+
+    # ---- inputs: seeded on the host (pinned, reused by the end-to-end leg), then resident in HBM
+    host = wl.make_inputs(w, seed=w.seed + 1000 * rank, with_dout=True)
+    host = {k: v.pin_memory() for k, v in host.items()}
+    dev = {k: v.to(device, non_blocking=True) for k, v in host.items()}
+    torch.cuda.synchronize()
+    layer = Layer(pskv, w, dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- main timed region: K steps, device-resident inputs
+    for _ in range(max(args.warmup, 3)):
+        layer.fwd()
+        layer.bwd()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    launches0 = pskv.pskv_kernel_launches()
+    e_start = torch.cuda.Event(enable_timing=True)
+    e_stop = torch.cuda.Event(enable_timing=True)
+    e_start.record()
+    for k in range(args.steps):
+        ev[k][0].record()
+        layer.fwd()
+        ev[k][1].record()
+        layer.bwd()
+        ev[k][2].record()
+    e_stop.record()
+    barrier()
+    launches = pskv.pskv_kernel_launches() - launches0
+    total_ms = e_start.elapsed_time(e_stop)
+    fwd_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    bwd_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    if rank == 0:
+        time.sleep(0.2)
+    clocks = sampler.stop() if rank == 0 else None
+    status = pskv.pskv_poll_device_status()
+    if status != pskv.PSKV_OK:
+        raise SystemExit("device status after timed region: %s" % pskv.pskv_status_string(status))
+
+    # ---- end-to-end leg: host buffers, H2D and D2H inside the timed region
+    houts = {"out": torch.empty_like(host["q"]).pin_memory(),
+             "lse": torch.empty((w.B, w.Hq, w.S), dtype=torch.float32).pin_memory(),
+             "dq": torch.empty_like(host["q"]).pin_memory(),
+             "dk": torch.empty_like(host["suffix_k"]).pin_memory(),
+             "dv": torch.empty_like(host["suffix_v"]).pin_memory()}
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = sum(v.numel() * v.element_size() for v in houts.values())
+
+    def e2e_step():
+        for k, v in host.items():
+            dev[k].copy_(v, non_blocking=True)
+        layer.fwd()
+        layer.bwd()
+        houts["out"].copy_(layer.out, non_blocking=True)
+        houts["lse"].copy_(layer.lse, non_blocking=True)
+        houts["dq"].copy_(layer.dq, non_blocking=True)
+        houts["dk"].copy_(layer.dk, non_blocking=True)
+        houts["dv"].copy_(layer.dv, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    barrier()
+    e2e_ms = time_calls(e2e_step, e2e_steps, 2)
+    barrier()
+
+    # ---- max over ranks
+    times = torch.tensor([total_ms, fwd_ms, bwd_ms, e2e_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, fwd_ms, bwd_ms, e2e_ms = times.tolist()
+    step_ms = total_ms / args.steps
+    flops_f, flops_b = wl.fwd_flops(w), wl.bwd_flops(w)
+    value = world * (flops_f + flops_b) / (step_ms * 1e-3) / 1e12
+    e2e_value = world * (flops_f + flops_b) / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, world),
+        "candidates_per_s": world * w.B / (step_ms * 1e-3),
+        "pct_bf16_peak": 100.0 * value / world / peaks["bf16_tflops"],
+        "parts": {
+            "fwd": {"ms": fwd_ms, "tflops": flops_f / fwd_ms / 1e9, "candidates_per_s": w.B / fwd_ms * 1e3,
+                    "pct_bf16_peak": 100.0 * flops_f / fwd_ms / 1e9 / peaks["bf16_tflops"],
+                    "hbm_gbs": wl.fwd_bytes(w) / fwd_ms / 1e6,
+                    "kernel_family": pskv.pskv_kernel_family(0, w.B, w.Hq, w.Hkv, w.S, w.P, w.d)},
+            "bwd": {"ms": bwd_ms, "tflops": flops_b / bwd_ms / 1e9, "candidates_per_s": w.B / bwd_ms * 1e3,
+                    "pct_bf16_peak": 100.0 * flops_b / bwd_ms / 1e9 / peaks["bf16_tflops"],
+                    "hbm_gbs": wl.bwd_bytes(w) / bwd_ms / 1e6,
+                    "kernel_family": pskv.pskv_kernel_family(1, w.B, w.Hq, w.Hkv, w.S, w.P, w.d)},
+        },
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "peaks": peaks,
+    }
+    line["roofline"] = roofline(w, fwd_ms, bwd_ms, peaks)
+
+    if world == 1 and not args.no_detail:
+        line["detail"] = detail_runs(pskv, device, peaks)
+    if world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(w, args.ref_candidates)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def roofline(w, fwd_ms, bwd_ms, peaks):
+    """Roofline of the dominant kernel: the forward call is a single fused kernel; its algorithmic
+    bytes and flops per launch come from inputs.fwd_bytes / fwd_flops.  The binding roof is the
+    slower of bytes / HBM peak and flops / tensor peak for this workload."""
+    t_hbm = wl.fwd_bytes(w) / (peaks["hbm_gbs"] * 1e9)
+    t_mma = wl.fwd_flops(w) / (peaks["bf16_tflops"] * 1e12)
+    traffic = TRAFFIC_BYTES_PER_LAUNCH.get(w.name)
+    if t_hbm >= t_mma:
+        ach = wl.fwd_bytes(w) / (fwd_ms * 1e-3) / 1e9
+        return {"kernel": "pskv_attn_fwd", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": traffic,
+                "peak_source": peaks["source"] + ", burst copy"}
+    ach = wl.fwd_flops(w) / (fwd_ms * 1e-3) / 1e12
+    return {"kernel": "pskv_attn_fwd", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+            "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "traffic": traffic,
+            "peak_source": peaks["source"] + ", burst"}
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the forward kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists for the workload).
+TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def detail_runs(pskv, device, peaks):
+    """Kernel-only timings of every workload (forward; backward where the workload asks for it)."""
+    res = {}
+    for name in ("C1", "C2", "C3", "C4"):
+        w = wl.WORKLOADS[name]
+        layer = Layer(pskv, w, device_inputs(w, w.seed, device))
+        layer.fwd()
+        entry = {}
+        ms = time_calls(layer.fwd, 20, 3)
+        entry["fwd"] = {"ms": ms, "tflops": wl.fwd_flops(w) / ms / 1e9,
+                        "candidates_per_s": w.B / ms * 1e3,
+                        "pct_bf16_peak": 100 * wl.fwd_flops(w) / ms / 1e9 / peaks["bf16_tflops"],
+                        "hbm_gbs": wl.fwd_bytes(w) / ms / 1e6,
+                        "pct_hbm_peak": 100 * wl.fwd_bytes(w) / ms / 1e6 / peaks["hbm_gbs"]}
+        if name in ("C4", "C2"):
+            ms = time_calls(layer.bwd, 20, 3)
+            entry["bwd"] = {"ms": ms, "tflops": wl.bwd_flops(w) / ms / 1e9,
+                            "candidates_per_s": w.B / ms * 1e3,
+                            "pct_bf16_peak": 100 * wl.bwd_flops(w) / ms / 1e9 / peaks["bf16_tflops"],
+                            "hbm_gbs": wl.bwd_bytes(w) / ms / 1e6,
+                            "pct_hbm_peak": 100 * wl.bwd_bytes(w) / ms / 1e6 / peaks["hbm_gbs"]}
+        res[name] = entry
+        del layer
+        torch.cuda.empty_cache()
+    # C2 over 32 layers back to back: 32 calls on distinct per-layer tensors, one stream, no host sync
+    w = wl.WORKLOADS["C2"]
+    layers = [Layer(pskv, w, device_inputs(w, w.seed + 100 + i, device)) for i in range(32)]
+
+    def stack():
+        for L in layers:
+            L.fwd()
+
+    ms = time_calls(stack, 3, 1)
+    res["C2_32_layers_fwd"] = {"ms": ms, "ms_per_layer": ms / 32, "tflops": 32 * wl.fwd_flops(w) / ms / 1e9,
+                               "candidates_per_s": w.B / ms * 1e3}
+    del layers
+    torch.cuda.empty_cache()
+    return res
+
+
+def cpu_baseline(w, cand):
+    import oracle
+    sub = w.with_candidates(cand)
+    t = wl.make_inputs(sub, with_dout=True)
+    f = {k: v.to(torch.float64).numpy() for k, v in t.items()}
+    t0 = time.perf_counter()
+    oracle.attn_fwd(f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"], w.scale)
+    oracle.attn_bwd(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"], w.scale)
+    dt = time.perf_counter() - t0
+    flops = wl.fwd_flops(sub) + wl.bwd_flops(sub)
+    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "%d of %d candidates of %s, fwd+bwd once, fp64, %.1f s" % (cand, w.B, w.name, dt),
+            "candidates_per_s": cand / dt}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--ref-candidates", type=int, default=32,
+                    help="candidates per step of the CPU oracle sample")
+    ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

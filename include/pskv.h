@@ -1,0 +1,126 @@
+/*
+ * pskv.h -- C ABI of the shared-prefix attention library (libpskv.so), sm_100a only.
+ *
+ * The operation is the per-layer attention step of prefix-shared KV caching:
+ * B candidate suffixes are scored against ONE compact prefix K/V cache that is
+ * stored once and never duplicated along the candidate dimension (paper
+ * Sec. 4.2), plus each candidate's own suffix-side K/V.  Mathematically it is
+ * scaled-dot-product attention (Eq. 2) over K = prefix (+) suffix, i.e. what
+ * the candidate-expanded cache of Eq. 3 would give, without building it.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers owned by the caller; the library
+ *     never allocates, frees or keeps them.  Tensors are dense, row-major, last
+ *     index fastest, and every base address must be 16-byte aligned.
+ *   - bf16 tensors are raw 16-bit bfloat16; lse is fp32.
+ *   - Query head h reads KV head g = h / (Hq / Hkv) (grouped-query attention,
+ *     Appendix E; Table 8 lists the head counts).
+ *   - Suffix row i of a candidate sees all P prefix keys and suffix keys 0..i
+ *     (causal, diagonal included: the K_{<=t} of Eq. 2).  P = 0 is legal.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     the default stream) and the call returns without synchronising.
+ *   - Arguments are validated on the host before anything is launched; a call
+ *     that returns non-zero has launched nothing.
+ *   - There is no CPU fallback: without an sm_100 device the calls fail.
+ */
+#ifndef PSKV_H_
+#define PSKV_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PSKV_OK = 0,
+    PSKV_ERR_INVALID_ARG = 1,       /* null / misaligned pointer, non-positive size, Hq % Hkv != 0 */
+    PSKV_ERR_UNSUPPORTED_SHAPE = 2, /* head dim other than 64 or 128, or sizes beyond the kernels' limits */
+    PSKV_ERR_UNSUPPORTED_ARCH = 3,  /* current device is not compute capability 10.x */
+    PSKV_ERR_WORKSPACE = 4,         /* workspace missing, misaligned or smaller than *_workspace_bytes() */
+    PSKV_ERR_CUDA = 5,              /* a CUDA runtime/driver call failed; see pskv_last_cuda_error() */
+    PSKV_ERR_DEVICE_TIMEOUT = 6     /* a bounded device-side wait expired (reported by pskv_poll_device_status) */
+} pskv_status;
+
+/* Scratch (device global memory) the forward call needs for these sizes; may be 0. */
+size_t pskv_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d);
+
+/*
+ * Forward (Eq. 2 over the shared prefix cache of Sec. 4.2 plus the suffix K/V):
+ *   s_j  = scale * <q[b,h,i,:], K_j>,  K = prefix_k[g] (P rows) then suffix_k[b,g] rows 0..i
+ *   lse[b,h,i]   = ln sum_j exp(s_j)                      (natural log, scale included)
+ *   out[b,h,i,:] = sum_j exp(s_j - lse) V_j                (rounded to bf16)
+ * Inputs are read-only; out and lse are fully overwritten.  Accumulation is fp32.
+ */
+pskv_status pskv_attn_fwd(const void *q,        /* bf16 [B,Hq,S,d]  */
+                          const void *prefix_k, /* bf16 [Hkv,P,d]   (may be NULL when P == 0) */
+                          const void *prefix_v, /* bf16 [Hkv,P,d]   (may be NULL when P == 0) */
+                          const void *suffix_k, /* bf16 [B,Hkv,S,d] */
+                          const void *suffix_v, /* bf16 [B,Hkv,S,d] */
+                          float scale,
+                          void *out,            /* bf16 [B,Hq,S,d]  */
+                          float *lse,           /* fp32 [B,Hq,S]    */
+                          int B, int Hq, int Hkv, int S, int P, int d,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Scratch the backward call needs for these sizes (holds per-row fp32 statistics). */
+size_t pskv_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d);
+
+/*
+ * Backward of L = sum(out * dout) with the prefix cache frozen (Sec. 4.2: the
+ * prefix is computed once; only suffix-side gradients are needed for
+ * gradient-guided suffix search).  With p_j = exp(s_j - lse), D = <dout, out>,
+ * ds_j = p_j (<dout, V_j> - D):
+ *   dq[b,h,i,:]        = scale * sum_j ds_j K_j
+ *   dk_suffix[b,g,t,:] = scale * sum over heads h of g and rows i >= t of ds_{P+t} q[b,h,i,:]
+ *   dv_suffix[b,g,t,:] =         sum over the same (h, i) of p_{P+t} dout[b,h,i,:]
+ * `out` and `lse` are the forward results for the same inputs.  No gradient is
+ * produced for prefix_k / prefix_v, and lse carries no incoming gradient.
+ * The three outputs are fully overwritten.
+ */
+pskv_status pskv_attn_bwd(const void *dout,     /* bf16 [B,Hq,S,d]  */
+                          const void *q, const void *prefix_k, const void *prefix_v,
+                          const void *suffix_k, const void *suffix_v,
+                          const void *out,      /* bf16 [B,Hq,S,d], from pskv_attn_fwd */
+                          const float *lse,     /* fp32 [B,Hq,S],   from pskv_attn_fwd */
+                          float scale,
+                          void *dq,             /* bf16 [B,Hq,S,d]  */
+                          void *dk_suffix,      /* bf16 [B,Hkv,S,d] */
+                          void *dv_suffix,      /* bf16 [B,Hkv,S,d] */
+                          int B, int Hq, int Hkv, int S, int P, int d,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Synchronises `cuda_stream`, then reads and clears the device status word that
+ * kernels set when one of their bounded waits gives up.  Returns PSKV_OK,
+ * PSKV_ERR_DEVICE_TIMEOUT (results of the affected call are undefined) or
+ * PSKV_ERR_CUDA.  Launch calls are asynchronous and cannot report this themselves.
+ */
+pskv_status pskv_poll_device_status(void *cuda_stream);
+
+/* Static, human-readable name of a status code. */
+const char *pskv_status_string(pskv_status status);
+
+/* cudaError_t (as int) recorded by the most recent call that returned PSKV_ERR_CUDA on this thread. */
+int pskv_last_cuda_error(void);
+
+/* major * 10000 + minor * 100 + patch */
+int pskv_version(void);
+
+/*
+ * Which kernel family pskv_attn_fwd / pskv_attn_bwd pick for these sizes:
+ * 1 = tcgen05 / TMEM tensor-core kernels, 0 = general CUDA-core kernels, negative = sizes rejected.
+ * `backward` selects which call is asked about.  Pure host logic; touches no device.
+ */
+int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d);
+
+/*
+ * Number of kernels this library has launched in this process so far (all threads, all devices).
+ * A host-side counter for benchmarks that must state how many launches a timed region made.
+ */
+long long pskv_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSKV_H_ */

@@ -1,0 +1,168 @@
+"""ctypes binding of libpskv.so: argument marshalling only.
+
+Each function has the name and argument order of its C entry point in
+``include/pskv.h``; tensors are torch CUDA tensors whose ``data_ptr()`` is
+handed through, sizes are read from the tensors' shapes, and the work is
+enqueued on torch's current stream.  Nothing is computed here and there is no
+fallback: if the shared library has not been built, loading fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libpskv.so")
+
+PSKV_OK = 0
+PSKV_ERR_INVALID_ARG = 1
+PSKV_ERR_UNSUPPORTED_SHAPE = 2
+PSKV_ERR_UNSUPPORTED_ARCH = 3
+PSKV_ERR_WORKSPACE = 4
+PSKV_ERR_CUDA = 5
+PSKV_ERR_DEVICE_TIMEOUT = 6
+
+_lib = None
+
+
+class PskvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        name = lib().pskv_status_string(self.status).decode()
+        extra = ""
+        if self.status == PSKV_ERR_CUDA:
+            extra = " (cudaError %d)" % lib().pskv_last_cuda_error()
+        super().__init__("%s: %s%s" % (where, name, extra))
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libpskv.so is missing at %s: build it with `python -m paper_2603_13420_b200.build` "
+                "(there is no CPU or PyTorch fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, ci, cf = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_float
+        six = [ci] * 6
+        L.pskv_attn_fwd_workspace_bytes.argtypes = six
+        L.pskv_attn_fwd_workspace_bytes.restype = sz
+        L.pskv_attn_bwd_workspace_bytes.argtypes = six
+        L.pskv_attn_bwd_workspace_bytes.restype = sz
+        L.pskv_attn_fwd.argtypes = [vp] * 5 + [cf] + [vp] * 2 + six + [vp, sz, vp]
+        L.pskv_attn_fwd.restype = ci
+        L.pskv_attn_bwd.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp, sz, vp]
+        L.pskv_attn_bwd.restype = ci
+        L.pskv_poll_device_status.argtypes = [vp]
+        L.pskv_poll_device_status.restype = ci
+        L.pskv_status_string.argtypes = [ci]
+        L.pskv_status_string.restype = ctypes.c_char_p
+        L.pskv_last_cuda_error.argtypes = []
+        L.pskv_last_cuda_error.restype = ci
+        L.pskv_version.argtypes = []
+        L.pskv_version.restype = ci
+        L.pskv_kernel_launches.argtypes = []
+        L.pskv_kernel_launches.restype = ctypes.c_longlong
+        L.pskv_kernel_family.argtypes = [ci] + six
+        L.pskv_kernel_family.restype = ci
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensors must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dims(q, prefix_k, suffix_k):
+    B, Hq, S, d = q.shape
+    Hkv = suffix_k.shape[1]
+    P = 0 if prefix_k is None else prefix_k.shape[1]
+    return [int(B), int(Hq), int(Hkv), int(S), int(P), int(d)]
+
+
+def pskv_version() -> int:
+    return int(lib().pskv_version())
+
+
+def pskv_kernel_launches() -> int:
+    return int(lib().pskv_kernel_launches())
+
+
+def pskv_last_cuda_error() -> int:
+    return int(lib().pskv_last_cuda_error())
+
+
+def pskv_status_string(status: int) -> str:
+    return lib().pskv_status_string(int(status)).decode()
+
+
+def pskv_kernel_family(backward, B, Hq, Hkv, S, P, d) -> int:
+    return int(lib().pskv_kernel_family(int(bool(backward)), B, Hq, Hkv, S, P, d))
+
+
+def pskv_attn_fwd_workspace_bytes(B, Hq, Hkv, S, P, d) -> int:
+    return int(lib().pskv_attn_fwd_workspace_bytes(B, Hq, Hkv, S, P, d))
+
+
+def pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d) -> int:
+    return int(lib().pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d))
+
+
+def _workspace(nbytes, device, workspace):
+    if workspace is not None:
+        return workspace
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def pskv_attn_fwd(q, prefix_k, prefix_v, suffix_k, suffix_v, scale, out=None, lse=None,
+                  workspace=None):
+    """out [B,Hq,S,d] bf16 and lse [B,Hq,S] fp32; q/suffix_* are per candidate, prefix_* [Hkv,P,d] shared."""
+    dims = _dims(q, prefix_k, suffix_k)
+    B, Hq, Hkv, S, P, d = dims
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    ws = _workspace(pskv_attn_fwd_workspace_bytes(*dims), q.device, workspace)
+    st = lib().pskv_attn_fwd(_ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(suffix_k), _ptr(suffix_v),
+                             float(scale), _ptr(out), _ptr(lse), *dims,
+                             _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_fwd")
+    return out, lse
+
+
+def pskv_attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, out, lse, scale,
+                  dq=None, dk_suffix=None, dv_suffix=None, workspace=None):
+    """dq, dk_suffix, dv_suffix (bf16) of L = sum(out * dout); the prefix cache gets no gradient."""
+    dims = _dims(q, prefix_k, suffix_k)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk_suffix is None:
+        dk_suffix = torch.empty_like(suffix_k)
+    if dv_suffix is None:
+        dv_suffix = torch.empty_like(suffix_v)
+    ws = _workspace(pskv_attn_bwd_workspace_bytes(*dims), q.device, workspace)
+    st = lib().pskv_attn_bwd(_ptr(dout), _ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(suffix_k),
+                             _ptr(suffix_v), _ptr(out), _ptr(lse), float(scale),
+                             _ptr(dq), _ptr(dk_suffix), _ptr(dv_suffix), *dims,
+                             _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_bwd")
+    return dq, dk_suffix, dv_suffix
+
+
+def pskv_poll_device_status() -> int:
+    """Synchronise the current stream and return the device status (PSKV_OK or an error code)."""
+    return int(lib().pskv_poll_device_status(_stream()))

@@ -1,0 +1,231 @@
+// C ABI of libpskv: host-side validation, kernel-family choice and launch.  No device memory
+// is allocated here; everything the kernels touch is passed in by the caller.
+#include <stdio.h>
+
+#include <atomic>
+
+#include "pskv_common.cuh"
+
+namespace pskv {
+namespace {
+
+__device__ unsigned int g_device_status = 0;  // set non-zero by a kernel whose bounded wait expired
+
+thread_local int t_last_cuda_error = 0;
+
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+    int checked;              // 0 = not yet, 1 = sm_100, -1 = other arch
+    unsigned int *status_ptr; // device address of g_device_status on that device
+};
+DeviceInfo g_devices[kMaxDevices];
+
+pskv_status cuda_fail(cudaError_t e)
+{
+    t_last_cuda_error = (int)e;
+    return PSKV_ERR_CUDA;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Pure host checks shared by both calls.  Returns PSKV_OK and fills `dm` when the sizes are usable.
+pskv_status check_dims(int B, int Hq, int Hkv, int S, int P, int d, Dims *dm)
+{
+    if (B < 1 || Hq < 1 || Hkv < 1 || S < 1 || P < 0 || d < 1) return PSKV_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0) return PSKV_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return PSKV_ERR_UNSUPPORTED_SHAPE;
+    // element counts must stay inside 2^40 so that byte offsets fit comfortably in 64 bits
+    const double rows = (double)B * Hq * S;
+    if (rows * d > 1.0e12 || (double)Hkv * P * d > 1.0e12) return PSKV_ERR_UNSUPPORTED_SHAPE;
+    dm->B = B; dm->Hq = Hq; dm->Hkv = Hkv; dm->S = S; dm->P = P; dm->d = d; dm->n_rep = Hq / Hkv;
+    return PSKV_OK;
+}
+
+// Device checks: compute capability 10.x, and the address of the status word on this device.
+pskv_status check_device(unsigned int **status_ptr)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return PSKV_ERR_UNSUPPORTED_ARCH;
+    DeviceInfo &info = g_devices[dev];
+    if (info.checked == 0) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (major != 10) {
+            info.checked = -1;
+        } else {
+            void *p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_device_status);
+            if (e != cudaSuccess) return cuda_fail(e);
+            info.status_ptr = static_cast<unsigned int *>(p);
+            info.checked = 1;
+        }
+    }
+    if (info.checked != 1) return PSKV_ERR_UNSUPPORTED_ARCH;
+    *status_ptr = info.status_ptr;
+    return PSKV_OK;
+}
+
+size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+size_t simt_bwd_workspace(const Dims &dm) { return round256((size_t)dm.B * dm.Hq * dm.S * sizeof(float)); }
+
+std::atomic<long long> g_launches{0};
+
+}  // namespace
+
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+}  // namespace pskv
+
+using namespace pskv;
+
+extern "C" {
+
+int pskv_version(void) { return 100; }
+
+long long pskv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *pskv_status_string(pskv_status s)
+{
+    switch (s) {
+    case PSKV_OK: return "PSKV_OK";
+    case PSKV_ERR_INVALID_ARG: return "PSKV_ERR_INVALID_ARG";
+    case PSKV_ERR_UNSUPPORTED_SHAPE: return "PSKV_ERR_UNSUPPORTED_SHAPE";
+    case PSKV_ERR_UNSUPPORTED_ARCH: return "PSKV_ERR_UNSUPPORTED_ARCH";
+    case PSKV_ERR_WORKSPACE: return "PSKV_ERR_WORKSPACE";
+    case PSKV_ERR_CUDA: return "PSKV_ERR_CUDA";
+    case PSKV_ERR_DEVICE_TIMEOUT: return "PSKV_ERR_DEVICE_TIMEOUT";
+    }
+    return "PSKV_ERR_UNKNOWN";
+}
+
+int pskv_last_cuda_error(void) { return t_last_cuda_error; }
+
+int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return -(int)st;
+    return (backward ? tc_bwd_supported(dm) : tc_fwd_supported(dm)) ? 1 : 0;
+}
+
+size_t pskv_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d)
+{
+    Dims dm;
+    if (check_dims(B, Hq, Hkv, S, P, d, &dm) != PSKV_OK) return 0;
+    return tc_fwd_supported(dm) ? round256(tc_fwd_workspace_bytes(dm)) : 0;
+}
+
+size_t pskv_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d)
+{
+    Dims dm;
+    if (check_dims(B, Hq, Hkv, S, P, d, &dm) != PSKV_OK) return 0;
+    return tc_bwd_supported(dm) ? round256(tc_bwd_workspace_bytes(dm)) : simt_bwd_workspace(dm);
+}
+
+pskv_status pskv_attn_fwd(const void *q, const void *prefix_k, const void *prefix_v,
+                          const void *suffix_k, const void *suffix_v, float scale,
+                          void *out, float *lse, int B, int Hq, int Hkv, int S, int P, int d,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return st;
+    if (!q || !suffix_k || !suffix_v || !out || !lse) return PSKV_ERR_INVALID_ARG;
+    if (P > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) || !aligned16(suffix_k) ||
+        !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse))
+        return PSKV_ERR_INVALID_ARG;
+    if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
+    const size_t need = pskv_attn_fwd_workspace_bytes(B, Hq, Hkv, S, P, d);
+    if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace)))
+        return PSKV_ERR_WORKSPACE;
+
+    unsigned int *status_word = nullptr;
+    st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+
+    FwdArgs a;
+    a.q = static_cast<const __nv_bfloat16 *>(q);
+    a.prefix_k = static_cast<const __nv_bfloat16 *>(prefix_k);
+    a.prefix_v = static_cast<const __nv_bfloat16 *>(prefix_v);
+    a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k);
+    a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v);
+    a.out = static_cast<__nv_bfloat16 *>(out);
+    a.lse = lse;
+    a.scale = scale;
+    a.dims = dm;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = tc_fwd_supported(dm) ? launch_tc_fwd(a, workspace, status_word, stream)
+                                         : launch_simt_fwd(a, stream);
+    return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
+}
+
+pskv_status pskv_attn_bwd(const void *dout, const void *q, const void *prefix_k,
+                          const void *prefix_v, const void *suffix_k, const void *suffix_v,
+                          const void *out, const float *lse, float scale, void *dq,
+                          void *dk_suffix, void *dv_suffix, int B, int Hq, int Hkv, int S, int P,
+                          int d, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return st;
+    if (!dout || !q || !suffix_k || !suffix_v || !out || !lse || !dq || !dk_suffix || !dv_suffix)
+        return PSKV_ERR_INVALID_ARG;
+    if (P > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
+    if (!aligned16(dout) || !aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) ||
+        !aligned16(suffix_k) || !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse) ||
+        !aligned16(dq) || !aligned16(dk_suffix) || !aligned16(dv_suffix))
+        return PSKV_ERR_INVALID_ARG;
+    if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
+    const size_t need = pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
+
+    unsigned int *status_word = nullptr;
+    st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+
+    BwdArgs a;
+    a.dout = static_cast<const __nv_bfloat16 *>(dout);
+    a.q = static_cast<const __nv_bfloat16 *>(q);
+    a.prefix_k = static_cast<const __nv_bfloat16 *>(prefix_k);
+    a.prefix_v = static_cast<const __nv_bfloat16 *>(prefix_v);
+    a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k);
+    a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v);
+    a.out = static_cast<const __nv_bfloat16 *>(out);
+    a.lse = lse;
+    a.dq = static_cast<__nv_bfloat16 *>(dq);
+    a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix);
+    a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix);
+    a.row_dot = static_cast<float *>(workspace);
+    a.scale = scale;
+    a.dims = dm;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = tc_bwd_supported(dm) ? launch_tc_bwd(a, workspace, status_word, stream)
+                                         : launch_simt_bwd(a, stream);
+    return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
+}
+
+pskv_status pskv_poll_device_status(void *cuda_stream)
+{
+    unsigned int *status_word = nullptr;
+    pskv_status st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    unsigned int word = 0;
+    e = cudaMemcpy(&word, status_word, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (word != 0) {
+        e = cudaMemset(status_word, 0, sizeof(word));
+        if (e != cudaSuccess) return cuda_fail(e);
+        return PSKV_ERR_DEVICE_TIMEOUT;
+    }
+    return PSKV_OK;
+}
+
+}  // extern "C"

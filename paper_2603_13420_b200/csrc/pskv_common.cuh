@@ -1,0 +1,53 @@
+// Shared declarations of the libpskv translation units (host launchers + small device helpers).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pskv.h"
+
+namespace pskv {
+
+// Dimensions of one call; `n_rep` = Hq / Hkv query heads per KV head.
+struct Dims {
+    int B, Hq, Hkv, S, P, d, n_rep;
+};
+
+struct FwdArgs {
+    const __nv_bfloat16 *q, *prefix_k, *prefix_v, *suffix_k, *suffix_v;
+    __nv_bfloat16 *out;
+    float *lse;
+    float scale;
+    Dims dims;
+};
+
+struct BwdArgs {
+    const __nv_bfloat16 *dout, *q, *prefix_k, *prefix_v, *suffix_k, *suffix_v, *out;
+    const float *lse;
+    __nv_bfloat16 *dq, *dk_suffix, *dv_suffix;
+    float *row_dot;  // workspace: D[b,h,i] = <dout, out>, fp32 [B*Hq*S]
+    float scale;
+    Dims dims;
+};
+
+// General CUDA-core kernels (any S, P; d in {64,128}).
+cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream);
+cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream);
+
+// tcgen05/TMEM kernels.  `status_word` is the device status flag that bounded waits set.
+bool tc_fwd_supported(const Dims &d);
+size_t tc_fwd_workspace_bytes(const Dims &d);
+cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word,
+                          cudaStream_t stream);
+bool tc_bwd_supported(const Dims &d);
+size_t tc_bwd_workspace_bytes(const Dims &d);
+cudaError_t launch_tc_bwd(const BwdArgs &a, void *workspace, unsigned int *status_word,
+                          cudaStream_t stream);
+
+// Host-side count of kernel launches (read through pskv_kernel_launches()).
+void count_launches(int n);
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+}  // namespace pskv

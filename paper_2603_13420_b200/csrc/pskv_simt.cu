@@ -1,0 +1,307 @@
+// General CUDA-core kernels for shared-prefix attention: any P >= 0, any S >= 1, d in {64,128}.
+// They serve the shapes the tensor-core kernels do not take.  One warp owns one query row
+// (forward, dQ) or one suffix key (dK/dV); the prefix K/V is read in place, shared by all
+// candidates (Sec. 4.2), and the softmax is one continued online softmax over prefix keys
+// followed by the causally visible suffix keys (Eq. 2).
+#include "pskv_common.cuh"
+
+namespace pskv {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// <x (fp32, shared memory), row (bf16, global)> over D elements, 16-byte loads.
+template <int D>
+__device__ __forceinline__ float dot_row(const float *x, const __nv_bfloat16 *row)
+{
+    const uint4 *r4 = reinterpret_cast<const uint4 *>(row);
+    float acc = 0.f;
+#pragma unroll
+    for (int v = 0; v < D / 8; ++v) {
+        uint4 u = __ldg(r4 + v);
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float2 f = __bfloat1622float2(h[e]);
+            acc = fmaf(x[v * 8 + 2 * e], f.x, acc);
+            acc = fmaf(x[v * 8 + 2 * e + 1], f.y, acc);
+        }
+    }
+    return acc;
+}
+
+// The lane's D/32 consecutive columns of a bf16 row, widened.
+template <int D>
+__device__ __forceinline__ void load_slice(const __nv_bfloat16 *row, int lane, float (&v)[D / 32])
+{
+    if constexpr (D == 128) {
+        uint2 u = __ldg(reinterpret_cast<const uint2 *>(row) + lane);
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+        float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+        v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+    } else {
+        unsigned int u = __ldg(reinterpret_cast<const unsigned int *>(row) + lane);
+        float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u));
+        v[0] = a.x; v[1] = a.y;
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void store_slice(__nv_bfloat16 *row, int lane, const float (&v)[D / 32])
+{
+    if constexpr (D == 128) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+        __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
+        uint2 u;
+        u.x = *reinterpret_cast<unsigned int *>(&a);
+        u.y = *reinterpret_cast<unsigned int *>(&b);
+        reinterpret_cast<uint2 *>(row)[lane] = u;
+    } else {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+        reinterpret_cast<unsigned int *>(row)[lane] = *reinterpret_cast<unsigned int *>(&a);
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void stage_row(float *dst, const __nv_bfloat16 *row, int lane)
+{
+    float v[D / 32];
+    load_slice<D>(row, lane, v);
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) dst[lane * (D / 32) + e] = v[e];
+}
+
+// Forward: one warp per query row (b,h,i); lanes take 32 keys at a time.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_fwd_kernel(FwdArgs a)
+{
+    __shared__ float q_s[kWarpsPerBlock][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Dims dm = a.dims;
+    const long long row = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    if (row >= (long long)dm.B * dm.Hq * dm.S) return;
+    const int i = (int)(row % dm.S);
+    const int h = (int)((row / dm.S) % dm.Hq);
+    const int b = (int)(row / ((long long)dm.S * dm.Hq));
+    const int g = h / dm.n_rep;
+    const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.P * D;
+    const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.P * D;
+    const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
+    const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
+
+    stage_row<D>(q_s[warp], a.q + (size_t)row * D, lane);
+    __syncwarp();
+
+    const float scale2 = a.scale * kLog2e;
+    const int n_vis = dm.P + i + 1;
+    float m = -INFINITY, l = 0.f;
+    float acc[D / 32];
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) acc[e] = 0.f;
+
+    for (int j0 = 0; j0 < n_vis; j0 += 32) {
+        const int j = j0 + lane;
+        float s = -INFINITY;
+        if (j < n_vis) {
+            const __nv_bfloat16 *krow = (j < dm.P) ? pk + (size_t)j * D : sk + (size_t)(j - dm.P) * D;
+            s = scale2 * dot_row<D>(q_s[warp], krow);
+        }
+        const float m_new = fmaxf(m, warp_max(s));  // finite: key j0 is always visible
+        const float p = exp2f(s - m_new);           // 0 for lanes past n_vis
+        const float corr = exp2f(m - m_new);        // 0 on the first chunk (m = -inf)
+        l = l * corr + warp_sum(p);
+#pragma unroll
+        for (int e = 0; e < D / 32; ++e) acc[e] *= corr;
+        const int cnt = min(32, n_vis - j0);
+        for (int t = 0; t < cnt; ++t) {
+            const float pt = __shfl_sync(0xffffffffu, p, t);
+            const int jj = j0 + t;
+            const __nv_bfloat16 *vrow = (jj < dm.P) ? pv + (size_t)jj * D : sv + (size_t)(jj - dm.P) * D;
+            float v[D / 32];
+            load_slice<D>(vrow, lane, v);
+#pragma unroll
+            for (int e = 0; e < D / 32; ++e) acc[e] = fmaf(pt, v[e], acc[e]);
+        }
+        m = m_new;
+    }
+    const float inv = 1.f / l;
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) acc[e] *= inv;
+    store_slice<D>(a.out + (size_t)row * D, lane, acc);
+    if (lane == 0) a.lse[row] = (m + log2f(l)) * kLn2;
+}
+
+// Backward, query side: one warp per query row; writes dq and D = <dout, out>.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_bwd_dq_kernel(BwdArgs a)
+{
+    __shared__ float q_s[kWarpsPerBlock][D];
+    __shared__ float do_s[kWarpsPerBlock][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Dims dm = a.dims;
+    const long long row = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    if (row >= (long long)dm.B * dm.Hq * dm.S) return;
+    const int i = (int)(row % dm.S);
+    const int h = (int)((row / dm.S) % dm.Hq);
+    const int b = (int)(row / ((long long)dm.S * dm.Hq));
+    const int g = h / dm.n_rep;
+    const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.P * D;
+    const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.P * D;
+    const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
+    const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
+
+    stage_row<D>(q_s[warp], a.q + (size_t)row * D, lane);
+    stage_row<D>(do_s[warp], a.dout + (size_t)row * D, lane);
+    float o[D / 32];
+    load_slice<D>(a.out + (size_t)row * D, lane, o);
+    __syncwarp();
+    float dsum = 0.f;
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) dsum = fmaf(o[e], do_s[warp][lane * (D / 32) + e], dsum);
+    const float Drow = warp_sum(dsum);
+    if (lane == 0) a.row_dot[row] = Drow;
+
+    const float scale2 = a.scale * kLog2e;
+    const float lse2 = a.lse[row] * kLog2e;
+    const int n_vis = dm.P + i + 1;
+    float acc[D / 32];
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) acc[e] = 0.f;
+    for (int j0 = 0; j0 < n_vis; j0 += 32) {
+        const int j = j0 + lane;
+        float ds = 0.f;
+        if (j < n_vis) {
+            const bool pre = j < dm.P;
+            const __nv_bfloat16 *krow = pre ? pk + (size_t)j * D : sk + (size_t)(j - dm.P) * D;
+            const __nv_bfloat16 *vrow = pre ? pv + (size_t)j * D : sv + (size_t)(j - dm.P) * D;
+            const float p = exp2f(scale2 * dot_row<D>(q_s[warp], krow) - lse2);
+            const float dp = dot_row<D>(do_s[warp], vrow);
+            ds = p * (dp - Drow);
+        }
+        const int cnt = min(32, n_vis - j0);
+        for (int t = 0; t < cnt; ++t) {
+            const float dst = __shfl_sync(0xffffffffu, ds, t);
+            const int jj = j0 + t;
+            const __nv_bfloat16 *krow = (jj < dm.P) ? pk + (size_t)jj * D : sk + (size_t)(jj - dm.P) * D;
+            float k[D / 32];
+            load_slice<D>(krow, lane, k);
+#pragma unroll
+            for (int e = 0; e < D / 32; ++e) acc[e] = fmaf(dst, k[e], acc[e]);
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) acc[e] *= a.scale;
+    store_slice<D>(a.dq + (size_t)row * D, lane, acc);
+}
+
+// Backward, key side: one warp per suffix key (b,g,t); sums over the n_rep heads of the group
+// and the rows i >= t that see the key.  Needs row_dot from the query-side kernel.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_bwd_dkv_kernel(BwdArgs a)
+{
+    __shared__ float k_s[kWarpsPerBlock][D];
+    __shared__ float v_s[kWarpsPerBlock][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Dims dm = a.dims;
+    const long long key = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    if (key >= (long long)dm.B * dm.Hkv * dm.S) return;
+    const int t = (int)(key % dm.S);
+    const int g = (int)((key / dm.S) % dm.Hkv);
+    const int b = (int)(key / ((long long)dm.S * dm.Hkv));
+
+    stage_row<D>(k_s[warp], a.suffix_k + (size_t)key * D, lane);
+    stage_row<D>(v_s[warp], a.suffix_v + (size_t)key * D, lane);
+    __syncwarp();
+
+    const float scale2 = a.scale * kLog2e;
+    const int per_head = dm.S - t;            // rows i = t .. S-1
+    const int n_rows = dm.n_rep * per_head;
+    float dk[D / 32], dv[D / 32];
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) { dk[e] = 0.f; dv[e] = 0.f; }
+
+    for (int r0 = 0; r0 < n_rows; r0 += 32) {
+        const int r = r0 + lane;
+        float p = 0.f, ds = 0.f;
+        if (r < n_rows) {
+            const int h = g * dm.n_rep + r / per_head;
+            const int i = t + r % per_head;
+            const size_t row = ((size_t)b * dm.Hq + h) * dm.S + i;
+            p = exp2f(scale2 * dot_row<D>(k_s[warp], a.q + row * D) - a.lse[row] * kLog2e);
+            const float dp = dot_row<D>(v_s[warp], a.dout + row * D);
+            ds = p * (dp - a.row_dot[row]);
+        }
+        const int cnt = min(32, n_rows - r0);
+        for (int u = 0; u < cnt; ++u) {
+            const float pu = __shfl_sync(0xffffffffu, p, u);
+            const float dsu = __shfl_sync(0xffffffffu, ds, u);
+            const int rr = r0 + u;
+            const int h = g * dm.n_rep + rr / per_head;
+            const int i = t + rr % per_head;
+            const size_t row = ((size_t)b * dm.Hq + h) * dm.S + i;
+            float qv[D / 32], gv[D / 32];
+            load_slice<D>(a.q + row * D, lane, qv);
+            load_slice<D>(a.dout + row * D, lane, gv);
+#pragma unroll
+            for (int e = 0; e < D / 32; ++e) {
+                dk[e] = fmaf(dsu, qv[e], dk[e]);
+                dv[e] = fmaf(pu, gv[e], dv[e]);
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) dk[e] *= a.scale;
+    store_slice<D>(a.dk_suffix + (size_t)key * D, lane, dk);
+    store_slice<D>(a.dv_suffix + (size_t)key * D, lane, dv);
+}
+
+inline unsigned int blocks_for(long long items)
+{
+    return (unsigned int)((items + kWarpsPerBlock - 1) / kWarpsPerBlock);
+}
+
+}  // namespace
+
+cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream)
+{
+    const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    if (a.dims.d == 128)
+        simt_fwd_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+    else
+        simt_fwd_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream)
+{
+    const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.S;
+    if (a.dims.d == 128) {
+        simt_bwd_dq_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+        simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
+    } else {
+        simt_bwd_dq_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+        simt_bwd_dkv_kernel<64><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
+    }
+    count_launches(2);
+    return cudaGetLastError();
+}
+
+}  // namespace pskv

@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compile the CUDA library and the C oracle once per session if their sources changed."""
+    from paper_2603_13420_b200 import build as pskv_build
+    import oracle
+
+    pskv_build.build()
+    oracle.build()

@@ -1,0 +1,138 @@
+"""Helpers of the GPU parity tests: run the C-ABI path and the fp64 oracle on the same seeded
+bf16 inputs and compare element by element.
+
+Tolerances (bf16 inputs, fp32 accumulation, bf16 outputs):
+  out   max |err| <= 2e-2 and mean |err| <= 2e-3 (the stated bar); and, because attention
+        outputs shrink like 1/sqrt(keys) so that the absolute bar alone would pass a kernel that
+        is 10 % off on a long prefix, also max |err| <= 2e-2 * max|ref| and
+        mean |err| <= 1e-2 * mean|ref|
+  lse   |err| <= 1e-3 * max(|ref|, 1)
+  grads the scale-aware bounds, and the absolute ones taken relative to max(1, max|ref|)
+        (a gradient can exceed 1 with outlier key channels, where bf16 rounding alone is 2^-9 |x|).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2603_13420_b200 as pskv
+from paper_2603_13420_b200 import inputs as pskv_inputs
+
+GUARD = 64          # guard elements on each side of every output buffer
+POISON = float("nan")
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+class Guarded:
+    """An output tensor embedded in a larger buffer: NaN-filled payload (so unwritten elements
+    show) and a known pattern around it (so out-of-bounds writes show)."""
+
+    def __init__(self, shape, dtype, device):
+        n = int(np.prod(shape))
+        pad = GUARD * 16  # keeps the payload 16-byte aligned for every dtype used here
+        self.buf = torch.full((n + 2 * pad,), 512.0, dtype=dtype, device=device)
+        self.view = self.buf[pad:pad + n].view(shape)
+        self.view.fill_(POISON)
+        self.pad, self.n = pad, n
+
+    def check(self, name):
+        b = self.buf.to("cpu").to(torch.float32)
+        assert torch.all(b[: self.pad] == 512.0), name + ": write before the buffer"
+        assert torch.all(b[self.pad + self.n:] == 512.0), name + ": write past the buffer"
+        assert not torch.isnan(self.view.to(torch.float32)).any(), name + ": unwritten or NaN elements"
+
+
+def check_tensor(name, got: np.ndarray, ref: np.ndarray, max_abs=2e-2, mean_abs=2e-3,
+                 max_rel_of_max=2e-2, mean_rel_of_mean=1e-2, strict_abs=False):
+    err = np.abs(got - ref)
+    ref_max = float(np.max(np.abs(ref))) if ref.size else 0.0
+    ref_mean = float(np.mean(np.abs(ref))) if ref.size else 0.0
+    stats = dict(max_abs=float(err.max()), mean_abs=float(err.mean()), ref_max=ref_max, ref_mean=ref_mean)
+    msg = "%s: %s" % (name, stats)
+    assert np.isfinite(got).all(), msg
+    unit = 1.0 if strict_abs else max(1.0, ref_max)
+    assert stats["max_abs"] <= max_abs * unit, msg
+    assert stats["mean_abs"] <= mean_abs * unit, msg
+    assert stats["max_abs"] <= max_rel_of_max * ref_max + 1e-6, msg
+    assert stats["mean_abs"] <= mean_rel_of_mean * ref_mean + 1e-7, msg
+    return stats
+
+
+def check_lse(got: np.ndarray, ref: np.ndarray):
+    rel = np.abs(got - ref) / np.maximum(np.abs(ref), 1.0)
+    assert np.isfinite(got).all()
+    assert rel.max() <= 1e-3, "lse: max rel err %g" % rel.max()
+    return float(rel.max())
+
+
+def run_fwd_gpu(t, scale, device="cuda"):
+    """t: dict of CPU bf16 tensors.  Returns guarded out/lse plus the device inputs."""
+    dev = {k: v.to(device) for k, v in t.items()}
+    P = dev["prefix_k"].shape[1]
+    out = Guarded(tuple(dev["q"].shape), torch.bfloat16, device)
+    lse = Guarded(tuple(dev["q"].shape[:3]), torch.float32, device)
+    pk = dev["prefix_k"] if P > 0 else None
+    pv = dev["prefix_v"] if P > 0 else None
+    pskv.pskv_attn_fwd(dev["q"], pk, pv, dev["suffix_k"], dev["suffix_v"], scale,
+                       out=out.view, lse=lse.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    out.check("out")
+    lse.check("lse")
+    return out.view, lse.view, dev
+
+
+def oracle_fwd(t, scale, cand=None):
+    sl = slice(None) if cand is None else cand
+    return oracle.attn_fwd(to_f64(t["q"][sl]), to_f64(t["prefix_k"]), to_f64(t["prefix_v"]),
+                           to_f64(t["suffix_k"][sl]), to_f64(t["suffix_v"][sl]), scale)
+
+
+def oracle_bwd(t, scale, cand=None):
+    sl = slice(None) if cand is None else cand
+    return oracle.attn_bwd(to_f64(t["dout"][sl]), to_f64(t["q"][sl]), to_f64(t["prefix_k"]),
+                           to_f64(t["prefix_v"]), to_f64(t["suffix_k"][sl]), to_f64(t["suffix_v"][sl]),
+                           scale)
+
+
+def fwd_parity(w, t=None, cand=None):
+    """Forward parity for workload w (optionally only the listed candidates against the oracle)."""
+    if t is None:
+        t = pskv_inputs.make_inputs(w)
+    out, lse, _ = run_fwd_gpu(t, w.scale)
+    ref_out, ref_lse = oracle_fwd(t, w.scale, cand)
+    sl = slice(None) if cand is None else cand
+    s = check_tensor("out", to_f64(out[sl]), ref_out, strict_abs=True)
+    s["lse_rel"] = check_lse(to_f64(lse[sl]), ref_lse)
+    return s
+
+
+def run_bwd_gpu(t, scale, device="cuda"):
+    out, lse, dev = run_fwd_gpu(t, scale, device)
+    P = dev["prefix_k"].shape[1]
+    pk = dev["prefix_k"] if P > 0 else None
+    pv = dev["prefix_v"] if P > 0 else None
+    dq = Guarded(tuple(dev["q"].shape), torch.bfloat16, device)
+    dk = Guarded(tuple(dev["suffix_k"].shape), torch.bfloat16, device)
+    dv = Guarded(tuple(dev["suffix_v"].shape), torch.bfloat16, device)
+    pskv.pskv_attn_bwd(dev["dout"], dev["q"], pk, pv, dev["suffix_k"], dev["suffix_v"],
+                       out.contiguous(), lse.contiguous(), scale,
+                       dq=dq.view, dk_suffix=dk.view, dv_suffix=dv.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    for name, g in (("dq", dq), ("dk_suffix", dk), ("dv_suffix", dv)):
+        g.check(name)
+    return dq.view, dk.view, dv.view
+
+
+def bwd_parity(w, t=None, cand=None):
+    if t is None:
+        t = pskv_inputs.make_inputs(w, with_dout=True)
+    dq, dk, dv = run_bwd_gpu(t, w.scale)
+    rq, rk, rv = oracle_bwd(t, w.scale, cand)
+    sl = slice(None) if cand is None else cand
+    return dict(dq=check_tensor("dq", to_f64(dq[sl]), rq),
+                dk=check_tensor("dk_suffix", to_f64(dk[sl]), rk),
+                dv=check_tensor("dv_suffix", to_f64(dv[sl]), rv))

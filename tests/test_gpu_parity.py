@@ -1,0 +1,141 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_13420_b200 as pskv
+from paper_2603_13420_b200.inputs import WORKLOADS, Workload, make_inputs
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def wl(name, **kw):
+    return dataclasses.replace(WORKLOADS[name], **kw)
+
+
+# ---------------------------------------------------------------- the five configurations, reduced B
+# (sizes the oracle finishes in seconds; each spans several 128-row tiles and ends in a ragged tail)
+
+def test_c0_tiny_forward_full():
+    parity.fwd_parity(WORKLOADS["C0"])
+
+
+@pytest.mark.parametrize("name,B", [("C1", 7), ("C2", 5), ("C3", 3), ("C4", 5)])
+def test_forward_reduced_candidates(name, B):
+    parity.fwd_parity(wl(name, B=B))
+
+
+@pytest.mark.parametrize("name,B", [("C4", 5), ("C0", 8), ("C2", 3), ("C3", 2)])
+def test_backward_reduced_candidates(name, B):
+    parity.bwd_parity(wl(name, B=B, backward=True))
+
+
+# ---------------------------------------------------------------- full sizes, sampled candidates
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_forward_full_size_sampled(name):
+    w = WORKLOADS[name]
+    rng = np.random.default_rng(w.seed)
+    cand = sorted(set([0, w.B - 1] + rng.integers(0, w.B, size=4).tolist()))
+    parity.fwd_parity(w, cand=cand)
+
+
+def test_backward_full_size_sampled():
+    w = WORKLOADS["C4"]
+    rng = np.random.default_rng(w.seed)
+    cand = sorted(set([0, w.B - 1] + rng.integers(0, w.B, size=4).tolist()))
+    parity.bwd_parity(w, cand=cand)
+
+
+# ---------------------------------------------------------------- edge cases and odd shapes
+
+EDGE = [
+    # B, Hq, Hkv, S, P, d
+    (1, 1, 1, 1, 0, 64),      # a single query that sees only itself
+    (3, 4, 4, 8, 0, 128),     # no prefix: plain causal attention per candidate
+    (2, 4, 2, 1, 40, 128),    # one suffix token
+    (5, 7, 1, 3, 37, 64),     # n_rep = 7, odd S, P not a multiple of 16
+    (4, 8, 2, 13, 100, 128),  # odd S with GQA
+    (2, 4, 4, 200, 16, 64),   # suffix longer than prefix
+    (1, 32, 8, 48, 256, 128), # one candidate of the GQA layer
+    (9, 4, 1, 24, 333, 128),  # prefix not a multiple of any tile
+    (3, 2, 2, 16, 1, 128),    # one prefix token
+]
+
+
+@pytest.mark.parametrize("shape", EDGE)
+def test_forward_edge_shapes(shape):
+    B, Hq, Hkv, S, P, d = shape
+    w = Workload("edge", 100 + sum(shape), B=B, Hq=Hq, Hkv=Hkv, d=d, P=P, S=S)
+    parity.fwd_parity(w)
+
+
+@pytest.mark.parametrize("shape", EDGE)
+def test_backward_edge_shapes(shape):
+    B, Hq, Hkv, S, P, d = shape
+    w = Workload("edge", 200 + sum(shape), B=B, Hq=Hq, Hkv=Hkv, d=d, P=P, S=S, backward=True)
+    parity.bwd_parity(w)
+
+
+def test_outlier_key_channels_and_large_scores():
+    """Large score spread (outlier channels x8 and a 4x scale) exercises the running-max rescale."""
+    w = wl("C2", B=3)
+    t = make_inputs(w)
+    out, lse, _ = parity.run_fwd_gpu(t, 4 * w.scale)
+    ref_out, ref_lse = parity.oracle_fwd(t, 4 * w.scale)
+    parity.check_tensor("out", parity.to_f64(out), ref_out, max_abs=4e-2, mean_abs=4e-3,
+                        max_rel_of_max=2e-2, mean_rel_of_mean=2e-2)
+    parity.check_lse(parity.to_f64(lse), ref_lse)
+
+
+# ---------------------------------------------------------------- properties that hold at any size
+
+def test_candidate_permutation_equivariance_is_bit_exact():
+    w = wl("C1", B=12)
+    t = make_inputs(w)
+    out0, lse0, _ = parity.run_fwd_gpu(t, w.scale)
+    perm = torch.randperm(w.B, generator=torch.Generator().manual_seed(5))
+    t2 = dict(t, q=t["q"][perm].contiguous(), suffix_k=t["suffix_k"][perm].contiguous(),
+              suffix_v=t["suffix_v"][perm].contiguous())
+    out1, lse1, _ = parity.run_fwd_gpu(t2, w.scale)
+    assert torch.equal(out1.cpu(), out0.cpu()[perm])
+    assert torch.equal(lse1.cpu(), lse0.cpu()[perm])
+
+
+def test_prefix_is_shared_not_copied():
+    """Changing the one prefix tensor changes every candidate's result: there is no per-candidate copy."""
+    w = wl("C1", B=6)
+    t = make_inputs(w)
+    out0, _, _ = parity.run_fwd_gpu(t, w.scale)
+    t2 = dict(t, prefix_v=(t["prefix_v"].float() + 1.0).to(torch.bfloat16))
+    out1, _, _ = parity.run_fwd_gpu(t2, w.scale)
+    diff = (out1.float() - out0.float()).abs().amax(dim=(1, 2, 3))
+    assert torch.all(diff > 0.1)
+
+
+def test_results_do_not_depend_on_workspace_contents_or_repeat():
+    w = wl("C4", B=4, backward=True)
+    t = make_inputs(w, with_dout=True)
+    a = [x.clone() for x in parity.run_bwd_gpu(t, w.scale)]
+    b = [x.clone() for x in parity.run_bwd_gpu(t, w.scale)]
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+def test_runs_on_a_side_stream():
+    w = WORKLOADS["C0"]
+    t = make_inputs(w)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        out, lse, _ = parity.run_fwd_gpu(t, w.scale)
+    s.synchronize()
+    ref_out, _ = parity.oracle_fwd(t, w.scale)
+    parity.check_tensor("out", parity.to_f64(out), ref_out, strict_abs=True)
+
+
+def test_status_word_is_clean_after_normal_calls():
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
