@@ -64,6 +64,14 @@ EDGE = [
     (1, 32, 8, 48, 256, 128), # one candidate of the GQA layer
     (9, 4, 1, 24, 333, 128),  # prefix not a multiple of any tile
     (3, 2, 2, 16, 1, 128),    # one prefix token
+    # shapes the tensor-core kernels take (S a multiple of 8)
+    (3, 8, 2, 16, 300, 128),  # prefix blocks streamed through the 2-stage ring (d = 128)
+    (2, 4, 4, 24, 600, 64),   # prefix blocks streamed through the 4-stage ring (d = 64)
+    (5, 7, 1, 8, 37, 64),     # n_rep = 7, partial prefix block
+    (6, 4, 2, 128, 20, 64),   # S = 128: a tile is half of one candidate's group
+    (3, 2, 2, 72, 50, 128),   # rows per candidate (72) force 72-row tiles
+    (40, 4, 4, 8, 16, 128),   # sixteen candidates share one tile
+    (37, 2, 1, 40, 129, 128), # ragged last tile, prefix one key past a block
 ]
 
 
@@ -94,7 +102,10 @@ def test_outlier_key_channels_and_large_scores():
 
 # ---------------------------------------------------------------- properties that hold at any size
 
-def test_candidate_permutation_equivariance_is_bit_exact():
+def test_candidate_permutation_equivariance():
+    """Permuting the candidates permutes the results.  A candidate's position decides which rows
+    share its tile and where its suffix keys sit inside the key block, i.e. the fp32 summation
+    order, so equality holds up to one rounding of the bf16 result, not bit for bit."""
     w = wl("C1", B=12)
     t = make_inputs(w)
     out0, lse0, _ = parity.run_fwd_gpu(t, w.scale)
@@ -102,8 +113,9 @@ def test_candidate_permutation_equivariance_is_bit_exact():
     t2 = dict(t, q=t["q"][perm].contiguous(), suffix_k=t["suffix_k"][perm].contiguous(),
               suffix_v=t["suffix_v"][perm].contiguous())
     out1, lse1, _ = parity.run_fwd_gpu(t2, w.scale)
-    assert torch.equal(out1.cpu(), out0.cpu()[perm])
-    assert torch.equal(lse1.cpu(), lse0.cpu()[perm])
+    a, b = out1.cpu().float(), out0.cpu()[perm].float()
+    assert torch.all((a - b).abs() <= 2.0 ** -7 * torch.maximum(a.abs(), b.abs()) + 1e-6)
+    assert torch.all((lse1.cpu() - lse0.cpu()[perm]).abs() <= 1e-5)
 
 
 def test_prefix_is_shared_not_copied():
