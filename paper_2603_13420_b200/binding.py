@@ -14,7 +14,8 @@ import os
 import torch
 
 _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG_DIR, "libpskv.so")
+# PSKV_LIBRARY_PATH selects another build of the same library (e.g. one compiled with tracing).
+LIB_PATH = os.environ.get("PSKV_LIBRARY_PATH") or os.path.join(_PKG_DIR, "libpskv.so")
 
 PSKV_OK = 0
 PSKV_ERR_INVALID_ARG = 1

@@ -71,6 +71,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     const long long start = clock64();
     for (unsigned int spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
+#ifdef PSKV_WAIT_SLEEP_NS
+        __nanosleep(PSKV_WAIT_SLEEP_NS);
+#endif
         if ((spin & 63u) == 0u) {
             if (*abort_flag != 0) return false;
             if (clock64() - start > kWaitBudgetCycles) {

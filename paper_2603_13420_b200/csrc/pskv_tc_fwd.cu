@@ -33,6 +33,24 @@ constexpr int kThreads = 352;
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 constexpr float kRescaleGap = 8.0f;      // log2 units the running max may lag before O is rescaled
 
+// Optional event trace of CTA 0 (lane 0 of each warp): compiled in only with -DPSKV_TRACE.
+#ifdef PSKV_TRACE
+__device__ long long g_trace[2 * 32768];
+__device__ unsigned int g_trace_n;
+#define PSKV_TRACE_EVENT(tag, val)                                                        \
+    do {                                                                                  \
+        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0 && (threadIdx.x & 31) == 0) { \
+            const unsigned int ti_ = atomicAdd(&g_trace_n, 1u);                           \
+            if (ti_ < 32768u) {                                                           \
+                g_trace[2 * ti_] = clock64();                                             \
+                g_trace[2 * ti_ + 1] = ((long long)(tag) << 32) | (unsigned int)(val);    \
+            }                                                                             \
+        }                                                                                 \
+    } while (0)
+#else
+#define PSKV_TRACE_EVENT(tag, val) do { } while (0)
+#endif
+
 enum : unsigned int {
     kErrProducerK = 0x101, kErrProducerV = 0x102, kErrMma = 0x103, kErrSoftmax = 0x104,
     kErrEpilogue = 0x105, kErrAlign = 0x106
@@ -182,6 +200,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 // MMA of the previous tile has completed
                 ok = mbar_wait(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
                 if (!ok) break;
+                PSKV_TRACE_EVENT(1, tl);
                 const int nseg = t.rows / p.seg_rows;  // one box per run of seg_rows rows
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
@@ -272,105 +291,123 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (lane == 0) {
             const int total_items = n_tiles * nitems;
             int i_qk = 0, i_pv = 0;
-            uint32_t kuse = 0, vuse = 0;  // streaming mode: prefix blocks consumed
+            int tl_qk = 0, k_qk = 0, tl_pv = 0, k_pv = 0;  // (tile, block) of the next score / value item
+            uint32_t kuse = 0, vuse = 0;                    // streaming mode: prefix blocks consumed
+            TileInfo tq = tile_info(p, t_begin, t_begin), tv = tq;
+            // descriptors are built once; per MMA only the 16-byte-granular start address moves
+            const uint64_t q_desc = make_smem_desc(sbase + C::kOffQ, 0, 1024);
+            const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
             bool ok = true;
             while (ok && i_pv < total_items) {
                 if (i_qk < total_items && i_qk < i_pv + kSlots) {
                     // ---- scores of item i_qk:  S[128 x N] = Q[128 x D] * K_blk[N x D]^T
-                    const int tl = i_qk / nitems, k = i_qk - tl * nitems;
-                    const TileInfo t = tile_info(p, t_begin + tl, t_begin);
                     const int slot = i_qk % kSlots;
-                    if (k == 0) {
-                        ok = mbar_wait(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMma);
+                    if (k_qk == 0) {
+                        ok = mbar_wait(bar(kBarQFull), tl_qk & 1, abort_flag, p.status, kErrMma);
                         if (!ok) break;
                     }
                     uint32_t kaddr;
                     int n;
-                    if (k < p.nblk_p) {
-                        n = prefix_block_cols(p, k);
+                    if (k_qk < p.nblk_p) {
+                        n = prefix_block_cols(p, k_qk);
                         if (p.resident) {
-                            if (t.first_of_g)
-                                ok = mbar_wait(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMma);
-                            kaddr = sbase + C::kOffPK + k * C::kTileBytes;
+                            if (tq.first_of_g)
+                                ok = mbar_wait(bar(kBarKFull + k_qk), (tq.g - g_first) & 1, abort_flag, p.status, kErrMma);
+                            kaddr = sbase + C::kOffPK + k_qk * C::kTileBytes;
                         } else {
                             const uint32_t ks = kuse % C::kStages;
                             ok = mbar_wait(bar(kBarKFull + ks), (kuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
                             kaddr = sbase + C::kOffPK + ks * C::kTileBytes;
                         }
                     } else {
-                        n = t.n_sfx;
-                        ok = mbar_wait(bar(kBarSKFull), tl & 1, abort_flag, p.status, kErrMma);
+                        n = tq.n_sfx;
+                        ok = mbar_wait(bar(kBarSKFull), tl_qk & 1, abort_flag, p.status, kErrMma);
                         kaddr = sbase + C::kOffSK;
                     }
                     if (!ok) break;
+                    PSKV_TRACE_EVENT(10, i_qk);
                     tc_fence_after();
                     const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
                     const uint32_t d_tmem = tmem + slot * kBlockN;
+                    const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
 #pragma unroll
                     for (int ks16 = 0; ks16 < D / 16; ++ks16) {
-                        const uint32_t off = (ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32;
-                        mma_ss(d_tmem, make_smem_desc(sbase + C::kOffQ + off, 0, 1024),
-                               make_smem_desc(kaddr + off, 0, 1024), idesc, ks16 > 0 ? 1u : 0u);
+                        const uint64_t off = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
+                        mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks16 > 0 ? 1u : 0u);
                     }
                     tc_commit(bar(kBarSFull + slot));
-                    if (k < p.nblk_p) {
+                    if (k_qk < p.nblk_p) {
                         if (!p.resident) { tc_commit(bar(kBarKFree + (kuse % C::kStages))); ++kuse; }
                     } else {
                         tc_commit(bar(kBarQkFree));  // the suffix block is the tile's last score block
                     }
                     ++i_qk;
+                    if (++k_qk == nitems) {
+                        k_qk = 0;
+                        if (++tl_qk < n_tiles) tq = tile_info(p, t_begin + tl_qk, t_begin);
+                    }
                 } else {
                     // ---- values of item i_pv:  O[128 x D] (+)= P[128 x N] * V_blk[N x D]
-                    const int tl = i_pv / nitems, k = i_pv - tl * nitems;
-                    const TileInfo t = tile_info(p, t_begin + tl, t_begin);
                     const int slot = i_pv % kSlots;
                     ok = mbar_wait(bar(kBarPReady + slot), (i_pv / kSlots) & 1, abort_flag, p.status, kErrMma);
                     if (!ok) break;
-                    if (k == 0 && tl > 0) {
+                    if (k_pv == 0 && tl_pv > 0) {
                         // O of the previous tile must have been read out by the epilogue warps
-                        ok = mbar_wait(bar(kBarOFree), (tl - 1) & 1, abort_flag, p.status, kErrMma);
+                        ok = mbar_wait(bar(kBarOFree), (tl_pv - 1) & 1, abort_flag, p.status, kErrMma);
                         if (!ok) break;
                     }
                     uint32_t vaddr;
                     int n;
-                    if (k < p.nblk_p) {
-                        n = prefix_block_cols(p, k);
+                    if (k_pv < p.nblk_p) {
+                        n = prefix_block_cols(p, k_pv);
                         if (p.resident) {
-                            if (t.first_of_g)
-                                ok = mbar_wait(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMma);
-                            vaddr = sbase + C::kOffPV + k * C::kTileBytes;
+                            if (tv.first_of_g)
+                                ok = mbar_wait(bar(kBarVFull + k_pv), (tv.g - g_first) & 1, abort_flag, p.status, kErrMma);
+                            vaddr = sbase + C::kOffPV + k_pv * C::kTileBytes;
                         } else {
                             const uint32_t vs = vuse % C::kStages;
                             ok = mbar_wait(bar(kBarVFull + vs), (vuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
                             vaddr = sbase + C::kOffPV + vs * C::kTileBytes;
                         }
                     } else {
-                        n = t.n_sfx;
-                        ok = mbar_wait(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMma);
+                        n = tv.n_sfx;
+                        ok = mbar_wait(bar(kBarSVFull), tl_pv & 1, abort_flag, p.status, kErrMma);
                         vaddr = sbase + C::kOffSV;
                     }
                     if (!ok) break;
+                    PSKV_TRACE_EVENT(11, i_pv);
                     tc_fence_after();
-                    const uint32_t idesc = make_idesc_bf16(kTileM, D, 1);
                     const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
-                    for (int ks16 = 0; ks16 < n / 16; ++ks16)
-                        mma_ts(tmem + kOCol, p_tmem + ks16 * 8,
-                               make_smem_desc(vaddr + ks16 * 2048, C::kSlabBytes, 1024), idesc,
-                               (k > 0 || ks16 > 0) ? 1u : 0u);
+                    const uint64_t v_desc = make_smem_desc(vaddr, C::kSlabBytes, 1024);
+                    const int nk = n >> 4;
+#pragma unroll
+                    for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
+                        if (ks16 < nk)
+                            mma_ts(tmem + kOCol, p_tmem + ks16 * 8, v_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_pv,
+                                   (k_pv > 0 || ks16 > 0) ? 1u : 0u);
+                    }
                     tc_commit(bar(kBarPvDone + slot));
-                    if (k < p.nblk_p) {
+                    if (k_pv < p.nblk_p) {
                         if (!p.resident) { tc_commit(bar(kBarVFree + (vuse % C::kStages))); ++vuse; }
                     } else {
                         tc_commit(bar(kBarSVFree));
                         tc_commit(bar(kBarOFull));
                     }
                     ++i_pv;
+                    if (++k_pv == nitems) {
+                        k_pv = 0;
+                        if (++tl_pv < n_tiles) tv = tile_info(p, t_begin + tl_pv, t_begin);
+                    }
                 }
             }
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ softmax warps
-        const int row = 32 * (warp & 3) + lane;                  // tensor-memory lane of this thread
+        // Each thread owns one query row (tensor-memory lane).  Per item: pass 1 reads the score
+        // block 32 columns at a time and takes the row max; pass 2 reads it again, exponentiates
+        // and writes bf16 probabilities over the first half of the same slot (a probability chunk
+        // only ever overwrites score columns that pass 2 has already consumed).
+        const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
         int item = 0;
         bool ok = true;
@@ -379,12 +416,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const bool valid = row < t.rows;
             const int R = t.R0 + (valid ? row : 0);
             const int b = R / p.Rg, r = R - b * p.Rg;
-            const int sfx_lo = (b - t.b_first) * p.S;            // first suffix column of this row's candidate
-            const int sfx_hi = sfx_lo + (r % p.S);               // causal: suffix keys 0..i
+            const int sfx_lo = (b - t.b_first) * p.S;   // first suffix column of this row's candidate
+            const int sfx_hi = sfx_lo + (r % p.S);      // causal: suffix keys 0..i
             float m_ref = 0.f, l = 0.f;
             for (int k = 0; k < nitems && ok; ++k, ++item) {
                 const int slot = item % kSlots;
-                int n, lo, hi;                                     // valid columns of this row: [lo, hi]
+                int n, lo, hi;                            // valid columns of this row: [lo, hi]
                 if (k < p.nblk_p) {
                     n = prefix_block_cols(p, k);
                     lo = 0;
@@ -395,33 +432,46 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     hi = valid ? sfx_hi : 0;
                 }
                 const int nch = (n + 31) >> 5;
+                // chunks [ch_b, ch_e] hold at least one valid column of some row of this warp
+                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1) && ((n & 31) == 0);
+                int ch_b = 0, ch_e = nch - 1;
+                if (!full) {
+                    const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
+                    const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
+                    ch_b = wlo >> 5;
+                    ch_e = min(nch - 1, whi >> 5);
+                }
+                const unsigned span = (unsigned)(hi - lo);  // hi < lo wraps to a huge span only if hi-lo < 0
+                const bool any_col = hi >= lo;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag,
                                                        p.status, kErrSoftmax));
                 if (!ok) break;
+                if (warp == 2) PSKV_TRACE_EVENT(20, item);
                 tc_fence_after();
                 const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
-                uint32_t sr[kBlockN];
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch)
-                    if (ch < nch) tmem_ld32(s_tmem + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
-                tmem_wait_ld();
-                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1 && (n & 31) == 0);
+
+                // ---- pass 1: row max of the block
                 float mb = -INFINITY;
+                {
+                    float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    for (int ch = ch_b; ch <= ch_e; ++ch) {
+                        uint32_t rr[32];
+                        tmem_ld32(s_tmem + ch * 32, rr);
+                        tmem_wait_ld();
+                        if (full) {
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    if (ch < nch) {
+                            for (int c = 0; c < 32; ++c) m4[c & 3] = fmaxf(m4[c & 3], __uint_as_float(rr[c]));
+                        } else {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            float v = __uint_as_float(sr[ch * 32 + c]);
-                            if (!full) {
-                                const int col = ch * 32 + c;
-                                v = (col >= lo && col <= hi) ? v : -INFINITY;
-                                sr[ch * 32 + c] = __float_as_uint(v);
+                            for (int c = 0; c < 32; ++c) {
+                                const bool in = any_col && (unsigned)(ch * 32 + c - lo) <= span;
+                                m4[c & 3] = fmaxf(m4[c & 3], in ? __uint_as_float(rr[c]) : -INFINITY);
                             }
-                            mb = fmaxf(mb, v);
                         }
                     }
+                    mb = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                 }
+                if (warp == 2) PSKV_TRACE_EVENT(22, item);
                 const float mx = mb * p.sl2;
                 if (k == 0) {
                     m_ref = (mb == -INFINITY) ? 0.f : mx;
@@ -449,24 +499,46 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         tmem_wait_st();
                     }
                 }
+
+                // ---- pass 2: p = 2^(s * sl2 - m_ref), row sum, bf16 pairs back to tensor memory
                 const float neg_m = -m_ref;
-                float lsum = 0.f;
+                float ls0 = 0.f, ls1 = 0.f;
+                for (int ch = 0; ch < nch; ++ch) {
+                    uint32_t pk[16];
+                    if (ch >= ch_b && ch <= ch_e) {
+                        uint32_t rr[32];
+                        tmem_ld32(s_tmem + ch * 32, rr);
+                        tmem_wait_ld();
+                        if (full) {
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    if (ch < nch) {
-                        uint32_t pk[16];
+                            for (int c = 0; c < 16; ++c) {
+                                const float p0 = exp2f(fmaf(__uint_as_float(rr[2 * c]), p.sl2, neg_m));
+                                const float p1 = exp2f(fmaf(__uint_as_float(rr[2 * c + 1]), p.sl2, neg_m));
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[c] = pack_bf16x2(p0, p1);
+                            }
+                        } else {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const float p0 = exp2f(fmaf(__uint_as_float(sr[ch * 32 + 2 * c]), p.sl2, neg_m));
-                            const float p1 = exp2f(fmaf(__uint_as_float(sr[ch * 32 + 2 * c + 1]), p.sl2, neg_m));
-                            lsum += p0 + p1;
-                            pk[c] = pack_bf16x2(p0, p1);
+                            for (int c = 0; c < 16; ++c) {
+                                const bool in0 = any_col && (unsigned)(ch * 32 + 2 * c - lo) <= span;
+                                const bool in1 = any_col && (unsigned)(ch * 32 + 2 * c + 1 - lo) <= span;
+                                const float p0 = in0 ? exp2f(fmaf(__uint_as_float(rr[2 * c]), p.sl2, neg_m)) : 0.f;
+                                const float p1 = in1 ? exp2f(fmaf(__uint_as_float(rr[2 * c + 1]), p.sl2, neg_m)) : 0.f;
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[c] = pack_bf16x2(p0, p1);
+                            }
                         }
-                        tmem_st16(s_tmem + ch * 16, pk);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
                     }
+                    tmem_st16(s_tmem + ch * 16, pk);
                 }
-                l += lsum;
+                l += ls0 + ls1;
                 if (k == nitems - 1) ml[(tl & 1) * kTileM + row] = make_float2(l, m_ref + log2f(l));
+                if (warp == 2) PSKV_TRACE_EVENT(23, item);
                 tmem_wait_st();
                 tc_fence_before();
                 __threadfence_block();
@@ -482,13 +554,20 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             if (!__all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), tl & 1, abort_flag, p.status, kErrEpilogue)))
                 break;
+            if (warp == 6) PSKV_TRACE_EVENT(30, tl);
             tc_fence_after();
             const float2 lm = ml[(tl & 1) * kTileM + row];
-            uint32_t o[D];
+            const float inv = 1.f / lm.x;
+            uint32_t ob[D / 2];  // normalised row as bf16 pairs
 #pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch)
-                tmem_ld32(tmem + lane_addr + kOCol + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&o[ch * 32]));
-            tmem_wait_ld();
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_addr + kOCol + ch * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                    ob[ch * 16 + c] = pack_bf16x2(__uint_as_float(o[2 * c]) * inv, __uint_as_float(o[2 * c + 1]) * inv);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarOFree));
@@ -496,19 +575,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int R = t.R0 + row;
                 const int b = R / p.Rg, r = R - b * p.Rg;
                 const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
-                const float inv = 1.f / lm.x;
                 uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D);
 #pragma unroll
-                for (int v = 0; v < D / 8; ++v) {
-                    uint4 u;
-                    u.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-                    u.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-                    u.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-                    u.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                    dst[v] = u;
-                }
+                for (int v = 0; v < D / 8; ++v) dst[v] = make_uint4(ob[4 * v], ob[4 * v + 1], ob[4 * v + 2], ob[4 * v + 3]);
                 p.lse[grow] = lm.y * kLn2;
             }
+            if (warp == 6) PSKV_TRACE_EVENT(31, tl);
         }
     }
 
@@ -661,6 +733,22 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_
 }
 
 }  // namespace
+
+#ifdef PSKV_TRACE
+// Debug builds only: copies the event trace of CTA 0 to the host and resets it.
+extern "C" int pskv_debug_read_trace(long long *host, int max_events)
+{
+    unsigned int n = 0;
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n));
+    if (n > 32768u) n = 32768u;
+    if ((int)n > max_events) n = (unsigned int)max_events;
+    cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 2 * n);
+    unsigned int zero = 0;
+    cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero));
+    return (int)n;
+}
+#endif
 
 bool tc_fwd_supported(const Dims &dm)
 {
