@@ -85,6 +85,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// All 32 lanes wait (the warp's control flow stays uniform); true only if every lane saw the phase.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                               unsigned int *status_word, unsigned int code)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status_word, code));
+}
+
+// One lane of a fully converged warp gets a non-zero result.
+__device__ __forceinline__ uint32_t elect_one_sync()
+{
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred P1;\n\t"
+        "elect.sync _|P1, %1;\n\t"
+        "@P1 mov.s32 %0, 1;\n\t"
+        "}"
+        : "+r"(pred)
+        : "r"(0xffffffffu));
+    return pred;
+}
+
 // ---------------------------------------------------------------------------------------------
 // TMA tile loads (global -> shared, completion on an mbarrier)
 

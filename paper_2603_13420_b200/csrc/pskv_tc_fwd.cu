@@ -33,21 +33,30 @@ constexpr int kThreads = 352;
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 constexpr float kRescaleGap = 8.0f;      // log2 units the running max may lag before O is rescaled
 
-// Optional event trace of CTA 0 (lane 0 of each warp): compiled in only with -DPSKV_TRACE.
+// Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
+// costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
 #ifdef PSKV_TRACE
-__device__ long long g_trace[2 * 32768];
-__device__ unsigned int g_trace_n;
-#define PSKV_TRACE_EVENT(tag, val)                                                        \
-    do {                                                                                  \
-        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0 && (threadIdx.x & 31) == 0) { \
-            const unsigned int ti_ = atomicAdd(&g_trace_n, 1u);                           \
-            if (ti_ < 32768u) {                                                           \
-                g_trace[2 * ti_] = clock64();                                             \
-                g_trace[2 * ti_ + 1] = ((long long)(tag) << 32) | (unsigned int)(val);    \
-            }                                                                             \
-        }                                                                                 \
+constexpr int kTraceWarps = 11, kTraceCap = 4096;
+__device__ long long g_trace[kTraceWarps * kTraceCap * 2];
+__device__ unsigned int g_trace_n[kTraceWarps];
+#define PSKV_TRACE_DECL unsigned int trace_i_ = 0
+#define PSKV_TRACE_EVENT(tag, val)                                                                     \
+    do {                                                                                               \
+        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0 && (threadIdx.x & 31) == 0 &&        \
+            trace_i_ < (unsigned int)kTraceCap) {                                                      \
+            long long *e_ = g_trace + ((size_t)(threadIdx.x >> 5) * kTraceCap + trace_i_) * 2;         \
+            e_[0] = clock64();                                                                         \
+            e_[1] = ((long long)(tag) << 32) | (unsigned int)(val);                                    \
+            ++trace_i_;                                                                                \
+        }                                                                                              \
+    } while (0)
+#define PSKV_TRACE_FLUSH                                                                               \
+    do {                                                                                               \
+        if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
     } while (0)
 #else
+#define PSKV_TRACE_DECL do { } while (0)
+#define PSKV_TRACE_FLUSH do { } while (0)
 #define PSKV_TRACE_EVENT(tag, val) do { } while (0)
 #endif
 
@@ -143,7 +152,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
+    PSKV_TRACE_DECL;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + C::kOffBar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -186,22 +197,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int nitems = p.nblk_p + 1;  // prefix blocks + the suffix block
     const int g_first = t_begin / p.tiles_per_group;
 
+    // The producer and MMA warps run their loops with all 32 lanes (warp-uniform control flow and
+    // addresses, so descriptors can live in uniform registers); one elected lane issues the
+    // asynchronous instructions.
     if (warp == 0) {
         // ------------------------------------------------------------------ producer, score side
         if (lane == 0) {
             prefetch_tensormap(&tm_q);
             prefetch_tensormap(&tm_sk);
             if (p.P > 0) prefetch_tensormap(&tm_pk);
-            uint32_t kload = 0;  // streaming mode: prefix K blocks loaded so far
-            bool ok = true;
-            for (int tl = 0; tl < n_tiles && ok; ++tl) {
-                const TileInfo t = tile_info(p, t_begin + tl, t_begin);
-                // Q, suffix K and (resident mode) the prefix K blocks are free once every score
-                // MMA of the previous tile has completed
-                ok = mbar_wait(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
-                if (!ok) break;
-                PSKV_TRACE_EVENT(1, tl);
-                const int nseg = t.rows / p.seg_rows;  // one box per run of seg_rows rows
+        }
+        uint32_t kload = 0;  // streaming mode: prefix K blocks loaded so far
+        bool ok = true;
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            // Q, suffix K and (resident mode) the prefix K blocks are free once every score MMA of
+            // the previous tile has completed
+            ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
+            if (!ok) break;
+            PSKV_TRACE_EVENT(1, tl);
+            const int nseg = t.rows / p.seg_rows;  // one box per run of seg_rows rows
+            if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
                     const int R = t.R0 + s * p.seg_rows;
@@ -210,194 +226,219 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         tma_load_4d(sbase + C::kOffQ + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
                                     bar(kBarQFull), sl * 64, r, t.g, b);
                 }
-                if (p.resident) {
-                    if (t.first_of_g) {
-                        for (int k = 0; k < p.nblk_p; ++k) {
-                            mbar_arrive_expect_tx(bar(kBarKFull + k), C::kTileBytes);
-                            for (int sl = 0; sl < C::kSlabs; ++sl)
-                                tma_load_3d(sbase + C::kOffPK + k * C::kTileBytes + sl * C::kSlabBytes, &tm_pk,
-                                            bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
-                        }
-                    }
-                } else {
+            }
+            __syncwarp();
+            if (p.resident) {
+                if (t.first_of_g && elect_one_sync()) {
                     for (int k = 0; k < p.nblk_p; ++k) {
-                        const uint32_t ks = kload % C::kStages;
-                        ok = mbar_wait(bar(kBarKFree + ks), ((kload / C::kStages) & 1) ^ 1, abort_flag, p.status,
-                                       kErrProducerK);
-                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(kBarKFull + k), C::kTileBytes);
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_3d(sbase + C::kOffPK + k * C::kTileBytes + sl * C::kSlabBytes, &tm_pk,
+                                        bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
+                    }
+                }
+                __syncwarp();
+            } else {
+                for (int k = 0; k < p.nblk_p; ++k) {
+                    const uint32_t ks = kload % C::kStages;
+                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / C::kStages) & 1) ^ 1, abort_flag, p.status,
+                                        kErrProducerK);
+                    if (!ok) break;
+                    if (elect_one_sync()) {
                         mbar_arrive_expect_tx(bar(kBarKFull + ks), C::kTileBytes);
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + C::kOffPK + ks * C::kTileBytes + sl * C::kSlabBytes, &tm_pk,
                                         bar(kBarKFull + ks), sl * 64, k * kBlockN, t.g);
-                        ++kload;
                     }
-                    if (!ok) break;
+                    __syncwarp();
+                    ++kload;
                 }
-                // suffix K of the candidates this tile touches: one box per candidate
+                if (!ok) break;
+            }
+            // suffix K of the candidates this tile touches: one box per candidate
+            if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarSKFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
                 for (int c = 0; c < t.nc; ++c)
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + C::kOffSK + sl * C::kSlabBytes + c * p.S * 128, &tm_sk,
                                     bar(kBarSKFull), sl * 64, 0, t.g, t.b_first + c);
             }
+            __syncwarp();
         }
     } else if (warp == 10) {
         // ------------------------------------------------------------------ producer, value side
         if (lane == 0) {
             prefetch_tensormap(&tm_sv);
             if (p.P > 0) prefetch_tensormap(&tm_pv);
-            uint32_t vload = 0;
-            bool ok = true;
-            for (int tl = 0; tl < n_tiles && ok; ++tl) {
-                const TileInfo t = tile_info(p, t_begin + tl, t_begin);
-                if (p.resident) {
-                    // suffix V and the resident prefix V blocks are free once every value MMA of
-                    // the previous tile has completed
-                    ok = mbar_wait(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
-                    if (!ok) break;
-                    if (t.first_of_g) {
-                        for (int k = 0; k < p.nblk_p; ++k) {
-                            mbar_arrive_expect_tx(bar(kBarVFull + k), C::kTileBytes);
-                            for (int sl = 0; sl < C::kSlabs; ++sl)
-                                tma_load_3d(sbase + C::kOffPV + k * C::kTileBytes + sl * C::kSlabBytes, &tm_pv,
-                                            bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
-                        }
-                    }
-                } else {
+        }
+        uint32_t vload = 0;
+        bool ok = true;
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            if (p.resident) {
+                // suffix V and the resident prefix V blocks are free once every value MMA of the
+                // previous tile has completed
+                ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
+                if (!ok) break;
+                if (t.first_of_g && elect_one_sync()) {
                     for (int k = 0; k < p.nblk_p; ++k) {
-                        const uint32_t vs = vload % C::kStages;
-                        ok = mbar_wait(bar(kBarVFree + vs), ((vload / C::kStages) & 1) ^ 1, abort_flag, p.status,
-                                       kErrProducerV);
-                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(kBarVFull + k), C::kTileBytes);
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_3d(sbase + C::kOffPV + k * C::kTileBytes + sl * C::kSlabBytes, &tm_pv,
+                                        bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
+                    }
+                }
+                __syncwarp();
+            } else {
+                for (int k = 0; k < p.nblk_p; ++k) {
+                    const uint32_t vs = vload % C::kStages;
+                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / C::kStages) & 1) ^ 1, abort_flag, p.status,
+                                        kErrProducerV);
+                    if (!ok) break;
+                    if (elect_one_sync()) {
                         mbar_arrive_expect_tx(bar(kBarVFull + vs), C::kTileBytes);
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + C::kOffPV + vs * C::kTileBytes + sl * C::kSlabBytes, &tm_pv,
                                         bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
-                        ++vload;
                     }
-                    if (!ok) break;
-                    ok = mbar_wait(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
-                    if (!ok) break;
+                    __syncwarp();
+                    ++vload;
                 }
+                if (!ok) break;
+                ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
+                if (!ok) break;
+            }
+            if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
                 for (int c = 0; c < t.nc; ++c)
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + C::kOffSV + sl * C::kSlabBytes + c * p.S * 128, &tm_sv,
                                     bar(kBarSVFull), sl * 64, 0, t.g, t.b_first + c);
             }
+            __syncwarp();
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const int total_items = n_tiles * nitems;
-            int i_qk = 0, i_pv = 0;
-            int tl_qk = 0, k_qk = 0, tl_pv = 0, k_pv = 0;  // (tile, block) of the next score / value item
-            uint32_t kuse = 0, vuse = 0;                    // streaming mode: prefix blocks consumed
-            TileInfo tq = tile_info(p, t_begin, t_begin), tv = tq;
-            // descriptors are built once; per MMA only the 16-byte-granular start address moves
-            const uint64_t q_desc = make_smem_desc(sbase + C::kOffQ, 0, 1024);
-            const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
-            bool ok = true;
-            while (ok && i_pv < total_items) {
-                if (i_qk < total_items && i_qk < i_pv + kSlots) {
-                    // ---- scores of item i_qk:  S[128 x N] = Q[128 x D] * K_blk[N x D]^T
-                    const int slot = i_qk % kSlots;
-                    if (k_qk == 0) {
-                        ok = mbar_wait(bar(kBarQFull), tl_qk & 1, abort_flag, p.status, kErrMma);
-                        if (!ok) break;
-                    }
-                    uint32_t kaddr;
-                    int n;
-                    if (k_qk < p.nblk_p) {
-                        n = prefix_block_cols(p, k_qk);
-                        if (p.resident) {
-                            if (tq.first_of_g)
-                                ok = mbar_wait(bar(kBarKFull + k_qk), (tq.g - g_first) & 1, abort_flag, p.status, kErrMma);
-                            kaddr = sbase + C::kOffPK + k_qk * C::kTileBytes;
-                        } else {
-                            const uint32_t ks = kuse % C::kStages;
-                            ok = mbar_wait(bar(kBarKFull + ks), (kuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
-                            kaddr = sbase + C::kOffPK + ks * C::kTileBytes;
-                        }
-                    } else {
-                        n = tq.n_sfx;
-                        ok = mbar_wait(bar(kBarSKFull), tl_qk & 1, abort_flag, p.status, kErrMma);
-                        kaddr = sbase + C::kOffSK;
-                    }
+        const int total_items = n_tiles * nitems;
+        int i_qk = 0, i_pv = 0;
+        int tl_qk = 0, k_qk = 0, tl_pv = 0, k_pv = 0;  // (tile, block) of the next score / value item
+        uint32_t kuse = 0, vuse = 0;                    // streaming mode: prefix blocks consumed
+        TileInfo tq = tile_info(p, t_begin, t_begin), tv = tq;
+        // descriptors are built once; per MMA only the 16-byte-granular start address moves
+        const uint64_t q_desc = make_smem_desc(sbase + C::kOffQ, 0, 1024);
+        const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
+        bool ok = true;
+        while (ok && i_pv < total_items) {
+            PSKV_TRACE_EVENT(16, i_pv);
+            if (i_qk < total_items && i_qk < i_pv + kSlots) {
+                // ---- scores of item i_qk:  S[128 x N] = Q[128 x D] * K_blk[N x D]^T
+                const int slot = i_qk % kSlots;
+                if (k_qk == 0) {
+                    ok = mbar_wait_warp(bar(kBarQFull), tl_qk & 1, abort_flag, p.status, kErrMma);
                     if (!ok) break;
-                    PSKV_TRACE_EVENT(10, i_qk);
-                    tc_fence_after();
-                    const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
-                    const uint32_t d_tmem = tmem + slot * kBlockN;
-                    const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
+                }
+                uint32_t kaddr;
+                int n;
+                if (k_qk < p.nblk_p) {
+                    n = prefix_block_cols(p, k_qk);
+                    if (p.resident) {
+                        if (tq.first_of_g)
+                            ok = mbar_wait_warp(bar(kBarKFull + k_qk), (tq.g - g_first) & 1, abort_flag, p.status, kErrMma);
+                        kaddr = sbase + C::kOffPK + k_qk * C::kTileBytes;
+                    } else {
+                        const uint32_t ks = kuse % C::kStages;
+                        ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
+                        kaddr = sbase + C::kOffPK + ks * C::kTileBytes;
+                    }
+                } else {
+                    n = tq.n_sfx;
+                    ok = mbar_wait_warp(bar(kBarSKFull), tl_qk & 1, abort_flag, p.status, kErrMma);
+                    kaddr = sbase + C::kOffSK;
+                }
+                if (!ok) break;
+                PSKV_TRACE_EVENT(10, i_qk);
+                tc_fence_after();
+                const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
+                const uint32_t d_tmem = tmem + slot * kBlockN;
+                const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
+                const bool last_of_tile = k_qk == nitems - 1;
+                const bool free_stage = k_qk < p.nblk_p && !p.resident;
+                if (elect_one_sync()) {
 #pragma unroll
                     for (int ks16 = 0; ks16 < D / 16; ++ks16) {
                         const uint64_t off = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
                         mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks16 > 0 ? 1u : 0u);
                     }
                     tc_commit(bar(kBarSFull + slot));
-                    if (k_qk < p.nblk_p) {
-                        if (!p.resident) { tc_commit(bar(kBarKFree + (kuse % C::kStages))); ++kuse; }
+                    if (free_stage) tc_commit(bar(kBarKFree + (kuse % C::kStages)));
+                    if (last_of_tile) tc_commit(bar(kBarQkFree));  // the suffix block ends the tile's scores
+                }
+                __syncwarp();
+                PSKV_TRACE_EVENT(12, i_qk);
+                if (free_stage) ++kuse;
+                ++i_qk;
+                if (++k_qk == nitems) {
+                    k_qk = 0;
+                    if (++tl_qk < n_tiles) tq = tile_info(p, t_begin + tl_qk, t_begin);
+                }
+            } else {
+                // ---- values of item i_pv:  O[128 x D] (+)= P[128 x N] * V_blk[N x D]
+                const int slot = i_pv % kSlots;
+                ok = mbar_wait_warp(bar(kBarPReady + slot), (i_pv / kSlots) & 1, abort_flag, p.status, kErrMma);
+                if (!ok) break;
+                if (k_pv == 0 && tl_pv > 0) {
+                    // O of the previous tile must have been read out by the epilogue warps
+                    ok = mbar_wait_warp(bar(kBarOFree), (tl_pv - 1) & 1, abort_flag, p.status, kErrMma);
+                    if (!ok) break;
+                }
+                uint32_t vaddr;
+                int n;
+                if (k_pv < p.nblk_p) {
+                    n = prefix_block_cols(p, k_pv);
+                    if (p.resident) {
+                        if (tv.first_of_g)
+                            ok = mbar_wait_warp(bar(kBarVFull + k_pv), (tv.g - g_first) & 1, abort_flag, p.status, kErrMma);
+                        vaddr = sbase + C::kOffPV + k_pv * C::kTileBytes;
                     } else {
-                        tc_commit(bar(kBarQkFree));  // the suffix block is the tile's last score block
-                    }
-                    ++i_qk;
-                    if (++k_qk == nitems) {
-                        k_qk = 0;
-                        if (++tl_qk < n_tiles) tq = tile_info(p, t_begin + tl_qk, t_begin);
+                        const uint32_t vs = vuse % C::kStages;
+                        ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
+                        vaddr = sbase + C::kOffPV + vs * C::kTileBytes;
                     }
                 } else {
-                    // ---- values of item i_pv:  O[128 x D] (+)= P[128 x N] * V_blk[N x D]
-                    const int slot = i_pv % kSlots;
-                    ok = mbar_wait(bar(kBarPReady + slot), (i_pv / kSlots) & 1, abort_flag, p.status, kErrMma);
-                    if (!ok) break;
-                    if (k_pv == 0 && tl_pv > 0) {
-                        // O of the previous tile must have been read out by the epilogue warps
-                        ok = mbar_wait(bar(kBarOFree), (tl_pv - 1) & 1, abort_flag, p.status, kErrMma);
-                        if (!ok) break;
-                    }
-                    uint32_t vaddr;
-                    int n;
-                    if (k_pv < p.nblk_p) {
-                        n = prefix_block_cols(p, k_pv);
-                        if (p.resident) {
-                            if (tv.first_of_g)
-                                ok = mbar_wait(bar(kBarVFull + k_pv), (tv.g - g_first) & 1, abort_flag, p.status, kErrMma);
-                            vaddr = sbase + C::kOffPV + k_pv * C::kTileBytes;
-                        } else {
-                            const uint32_t vs = vuse % C::kStages;
-                            ok = mbar_wait(bar(kBarVFull + vs), (vuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
-                            vaddr = sbase + C::kOffPV + vs * C::kTileBytes;
-                        }
-                    } else {
-                        n = tv.n_sfx;
-                        ok = mbar_wait(bar(kBarSVFull), tl_pv & 1, abort_flag, p.status, kErrMma);
-                        vaddr = sbase + C::kOffSV;
-                    }
-                    if (!ok) break;
-                    PSKV_TRACE_EVENT(11, i_pv);
-                    tc_fence_after();
-                    const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
-                    const uint64_t v_desc = make_smem_desc(vaddr, C::kSlabBytes, 1024);
-                    const int nk = n >> 4;
+                    n = tv.n_sfx;
+                    ok = mbar_wait_warp(bar(kBarSVFull), tl_pv & 1, abort_flag, p.status, kErrMma);
+                    vaddr = sbase + C::kOffSV;
+                }
+                if (!ok) break;
+                PSKV_TRACE_EVENT(11, i_pv);
+                tc_fence_after();
+                const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
+                const uint64_t v_desc = make_smem_desc(vaddr, C::kSlabBytes, 1024);
+                const int nk = n >> 4;
+                const bool last_of_tile = k_pv == nitems - 1;
+                const bool free_stage = k_pv < p.nblk_p && !p.resident;
+                const uint32_t acc0 = k_pv > 0 ? 1u : 0u;
+                if (elect_one_sync()) {
 #pragma unroll
                     for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
                         if (ks16 < nk)
                             mma_ts(tmem + kOCol, p_tmem + ks16 * 8, v_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_pv,
-                                   (k_pv > 0 || ks16 > 0) ? 1u : 0u);
+                                   ks16 > 0 ? 1u : acc0);
                     }
                     tc_commit(bar(kBarPvDone + slot));
-                    if (k_pv < p.nblk_p) {
-                        if (!p.resident) { tc_commit(bar(kBarVFree + (vuse % C::kStages))); ++vuse; }
-                    } else {
+                    if (free_stage) tc_commit(bar(kBarVFree + (vuse % C::kStages)));
+                    if (last_of_tile) {
                         tc_commit(bar(kBarSVFree));
                         tc_commit(bar(kBarOFull));
                     }
-                    ++i_pv;
-                    if (++k_pv == nitems) {
-                        k_pv = 0;
-                        if (++tl_pv < n_tiles) tv = tile_info(p, t_begin + tl_pv, t_begin);
-                    }
+                }
+                __syncwarp();
+                PSKV_TRACE_EVENT(13, i_pv);
+                if (free_stage) ++vuse;
+                ++i_pv;
+                if (++k_pv == nitems) {
+                    k_pv = 0;
+                    if (++tl_pv < n_tiles) tv = tile_info(p, t_begin + tl_pv, t_begin);
                 }
             }
         }
@@ -523,8 +564,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                             for (int c = 0; c < 16; ++c) {
                                 const bool in0 = any_col && (unsigned)(ch * 32 + 2 * c - lo) <= span;
                                 const bool in1 = any_col && (unsigned)(ch * 32 + 2 * c + 1 - lo) <= span;
-                                const float p0 = in0 ? exp2f(fmaf(__uint_as_float(rr[2 * c]), p.sl2, neg_m)) : 0.f;
-                                const float p1 = in1 ? exp2f(fmaf(__uint_as_float(rr[2 * c + 1]), p.sl2, neg_m)) : 0.f;
+                                const float p0 = exp2f(in0 ? fmaf(__uint_as_float(rr[2 * c]), p.sl2, neg_m) : -INFINITY);
+                                const float p1 = exp2f(in1 ? fmaf(__uint_as_float(rr[2 * c + 1]), p.sl2, neg_m) : -INFINITY);
                                 ls0 += p0;
                                 ls1 += p1;
                                 pk[c] = pack_bf16x2(p0, p1);
@@ -585,6 +626,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
 
     // ---------------------------------------------------------------------- teardown
+    PSKV_TRACE_FLUSH;
     if (*abort_flag != 0) __nanosleep(20000);  // let copies and MMAs still in flight drain
     tc_fence_before();
     __syncthreads();
@@ -735,18 +777,21 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_
 }  // namespace
 
 #ifdef PSKV_TRACE
-// Debug builds only: copies the event trace of CTA 0 to the host and resets it.
+// Debug builds only: copies the event trace of CTA 0 to the host (all warps' events concatenated).
 extern "C" int pskv_debug_read_trace(long long *host, int max_events)
 {
-    unsigned int n = 0;
+    static long long buf[kTraceWarps * kTraceCap * 2];
+    unsigned int cnt[kTraceWarps];
     cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n));
-    if (n > 32768u) n = 32768u;
-    if ((int)n > max_events) n = (unsigned int)max_events;
-    cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 2 * n);
-    unsigned int zero = 0;
-    cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero));
-    return (int)n;
+    cudaMemcpyFromSymbol(cnt, g_trace_n, sizeof(cnt));
+    cudaMemcpyFromSymbol(buf, g_trace, sizeof(buf));
+    int n = 0;
+    for (int w = 0; w < kTraceWarps; ++w)
+        for (unsigned int i = 0; i < cnt[w] && i < (unsigned int)kTraceCap && n < max_events; ++i, ++n) {
+            host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
+            host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1];
+        }
+    return n;
 }
 #endif
 
