@@ -39,6 +39,8 @@ constexpr float kRescaleGap = 8.0f;      // log2 units the running max may lag b
 constexpr int kTraceWarps = 11, kTraceCap = 4096;
 __device__ long long g_trace[kTraceWarps * kTraceCap * 2];
 __device__ unsigned int g_trace_n[kTraceWarps];
+__device__ long long g_trace2[kTraceWarps * kTraceCap * 2];
+__device__ unsigned int g_trace_n2[kTraceWarps];
 #define PSKV_TRACE_DECL unsigned int trace_i_ = 0
 #define PSKV_TRACE_EVENT(tag, val)                                                                     \
     do {                                                                                               \
@@ -50,12 +52,25 @@ __device__ unsigned int g_trace_n[kTraceWarps];
             ++trace_i_;                                                                                \
         }                                                                                              \
     } while (0)
+#define PSKV_TRACE_EVENT_ONE(tag, val)                                                                 \
+    do {                                                                                               \
+        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0) {                                   \
+            unsigned int *n_ = &g_trace_n2[threadIdx.x >> 5];                                          \
+            if (*n_ < (unsigned int)kTraceCap) {                                                       \
+                long long *e_ = g_trace2 + ((size_t)(threadIdx.x >> 5) * kTraceCap + *n_) * 2;         \
+                e_[0] = clock64();                                                                     \
+                e_[1] = ((long long)(tag) << 32) | (unsigned int)(val);                                \
+                *n_ += 1;                                                                              \
+            }                                                                                          \
+        }                                                                                              \
+    } while (0)
 #define PSKV_TRACE_FLUSH                                                                               \
     do {                                                                                               \
         if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
     } while (0)
 #else
 #define PSKV_TRACE_DECL do { } while (0)
+#define PSKV_TRACE_EVENT_ONE(tag, val) do { } while (0)
 #define PSKV_TRACE_FLUSH do { } while (0)
 #define PSKV_TRACE_EVENT(tag, val) do { } while (0)
 #endif
@@ -358,7 +373,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (!ok) break;
                 PSKV_TRACE_EVENT(10, i_qk);
                 tc_fence_after();
+#ifdef PSKV_X_QKN
+                const uint32_t idesc = make_idesc_bf16(kTileM, PSKV_X_QKN, 0);
+#else
                 const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
+#endif
                 const uint32_t d_tmem = tmem + slot * kBlockN;
                 const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
                 const bool last_of_tile = k_qk == nitems - 1;
@@ -368,6 +387,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     for (int ks16 = 0; ks16 < D / 16; ++ks16) {
                         const uint64_t off = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
                         mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks16 > 0 ? 1u : 0u);
+                        PSKV_TRACE_EVENT_ONE(17, i_qk * 8 + ks16);
                     }
                     tc_commit(bar(kBarSFull + slot));
                     if (free_stage) tc_commit(bar(kBarKFree + (kuse % C::kStages)));
@@ -618,6 +638,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
                 uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D);
 #pragma unroll
+#ifdef PSKV_X_NOSTORE
+                if (ob[0] == 0x12345678u)
+#endif
                 for (int v = 0; v < D / 8; ++v) dst[v] = make_uint4(ob[4 * v], ob[4 * v + 1], ob[4 * v + 2], ob[4 * v + 3]);
                 p.lse[grow] = lm.y * kLn2;
             }
@@ -791,6 +814,15 @@ extern "C" int pskv_debug_read_trace(long long *host, int max_events)
             host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
             host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1];
         }
+    cudaMemcpyFromSymbol(cnt, g_trace_n2, sizeof(cnt));
+    cudaMemcpyFromSymbol(buf, g_trace2, sizeof(buf));
+    for (int w = 0; w < kTraceWarps; ++w)
+        for (unsigned int i = 0; i < cnt[w] && i < (unsigned int)kTraceCap && n < max_events; ++i, ++n) {
+            host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
+            host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1];
+        }
+    unsigned int zeros[kTraceWarps] = {0};
+    cudaMemcpyToSymbol(g_trace_n2, zeros, sizeof(zeros));
     return n;
 }
 #endif
