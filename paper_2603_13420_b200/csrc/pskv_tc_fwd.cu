@@ -9,15 +9,18 @@
 // partial results by their log-sum-exp), probabilities go back to tensor memory as bf16 and are
 // the A operand of the P*V contraction; `out` and `lse` are written once.
 //
-// Persistent CTA, one per SM, 11 warps:
+// Persistent CTA, one per SM, 12 warps:
 //   warp 0      TMA producer, score side (Q tile, prefix K blocks, suffix K of the tile)
-//   warp 1      tcgen05.mma issuer; score blocks run up to three items ahead of P*V
-//   warps 2-5   softmax: thread <-> query row (tensor-memory lane)
-//   warps 6-9   epilogue: O from tensor memory, normalise, bf16, store; writes lse
-//   warp 10     TMA producer, value side (prefix V blocks, suffix V of the tile)
+//   warp 1      tcgen05.mma issuer for the score blocks  S = Q K^T
+//   warp 2      tcgen05.mma issuer for the value blocks  O += P V   (owns the TMEM allocation)
+//   warp 3      TMA producer, value side (prefix V blocks, suffix V of the tile)
+//   warps 4-7   softmax: thread <-> query row (tensor-memory lane)
+//   warps 8-11  epilogue: O from tensor memory, normalise, bf16, shared-memory staging, TMA store
 // An "item" is one (tile, key block) pair; score blocks rotate through three 128-column slots of
-// tensor memory, O has its own 128 columns.  The two producers wait only on completions of
-// score-side resp. value-side MMAs of earlier items, so no wait cycle can form.
+// tensor memory, O has its own 128 columns.  Every wait is on an event produced by an earlier
+// item of a role that never waits on the waiter, so no wait cycle can form; every wait is bounded.
+#include <string.h>
+
 #include "pskv_common.cuh"
 #include "pskv_sm100.cuh"
 
@@ -29,18 +32,19 @@ using namespace sm100;
 constexpr int kTileM = 128;    // rows of one MMA tile (tensor-memory lanes)
 constexpr int kBlockN = 128;   // keys per block
 constexpr int kSlots = 3;      // score slots in tensor memory
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 constexpr float kRescaleGap = 8.0f;      // log2 units the running max may lag before O is rescaled
+constexpr int kMaxStages = 4;
+constexpr int kStagingBytes = kTileM * 128;  // one 64-column slab of the output tile
+constexpr int kMaxSmem = 232448;
 
 // Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
 // costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
 #ifdef PSKV_TRACE
-constexpr int kTraceWarps = 11, kTraceCap = 4096;
+constexpr int kTraceWarps = 12, kTraceCap = 4096;
 __device__ long long g_trace[kTraceWarps * kTraceCap * 2];
 __device__ unsigned int g_trace_n[kTraceWarps];
-__device__ long long g_trace2[kTraceWarps * kTraceCap * 2];
-__device__ unsigned int g_trace_n2[kTraceWarps];
 #define PSKV_TRACE_DECL unsigned int trace_i_ = 0
 #define PSKV_TRACE_EVENT(tag, val)                                                                     \
     do {                                                                                               \
@@ -52,65 +56,45 @@ __device__ unsigned int g_trace_n2[kTraceWarps];
             ++trace_i_;                                                                                \
         }                                                                                              \
     } while (0)
-#define PSKV_TRACE_EVENT_ONE(tag, val)                                                                 \
-    do {                                                                                               \
-        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0) {                                   \
-            unsigned int *n_ = &g_trace_n2[threadIdx.x >> 5];                                          \
-            if (*n_ < (unsigned int)kTraceCap) {                                                       \
-                long long *e_ = g_trace2 + ((size_t)(threadIdx.x >> 5) * kTraceCap + *n_) * 2;         \
-                e_[0] = clock64();                                                                     \
-                e_[1] = ((long long)(tag) << 32) | (unsigned int)(val);                                \
-                *n_ += 1;                                                                              \
-            }                                                                                          \
-        }                                                                                              \
-    } while (0)
 #define PSKV_TRACE_FLUSH                                                                               \
     do {                                                                                               \
         if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
     } while (0)
 #else
 #define PSKV_TRACE_DECL do { } while (0)
-#define PSKV_TRACE_EVENT_ONE(tag, val) do { } while (0)
 #define PSKV_TRACE_FLUSH do { } while (0)
 #define PSKV_TRACE_EVENT(tag, val) do { } while (0)
 #endif
 
 enum : unsigned int {
-    kErrProducerK = 0x101, kErrProducerV = 0x102, kErrMma = 0x103, kErrSoftmax = 0x104,
-    kErrEpilogue = 0x105, kErrAlign = 0x106
+    kErrProducerK = 0x101, kErrProducerV = 0x102, kErrMmaQk = 0x103, kErrMmaPv = 0x104,
+    kErrSoftmax = 0x105, kErrEpilogue = 0x106, kErrAlign = 0x107
 };
 
 struct TcFwdParams {
-    __nv_bfloat16 *out;
     float *lse;
     unsigned int *status;
     float sl2;            // scale * log2(e)
     int B, Hq, Hkv, S, P, n_rep;
     int Rg;               // rows per candidate in one KV-head group: n_rep * S
     int tile_rows;        // rows of the flat row list per tile (<= 128, multiple of seg_rows)
-    int seg_rows;         // rows per Q TMA box: gcd(Rg, tile_rows)
+    int seg_rows;         // rows per Q / out TMA box: gcd(Rg, tile_rows)
     int tiles_per_group;
     int total_tiles;
     int nblk_p;           // prefix key blocks: ceil(P / 128)
+    int tail_rows;        // rows held by the last prefix block (multiple of 16, <= 128)
     int resident;         // 1 when all prefix blocks of a KV head stay in shared memory
+    int stages;           // streaming mode: stages of the prefix K and V rings
+    int sfx_rows;         // rows of the suffix K / V buffers (multiple of 16, <= 128)
+    // shared-memory carve-up (byte offsets from the 1024-byte aligned base)
+    int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml;
 };
 
 template <int D>
 struct Cfg {
-    static constexpr int kSlabs = D / 64;                 // 64-column (128-byte) swizzle slabs per row
-    static constexpr int kSlabBytes = kTileM * 128;       // 128 rows x 128 bytes
+    static constexpr int kSlabs = D / 64;              // 64-column (128-byte) swizzle slabs per row
+    static constexpr int kSlabBytes = kTileM * 128;    // a full slab: 128 rows x 128 bytes
     static constexpr int kTileBytes = kSlabs * kSlabBytes;
-    static constexpr int kStages = (D == 128) ? 2 : 4;    // prefix K/V block stages
-    static constexpr int kOffPK = 0;
-    static constexpr int kOffPV = kStages * kTileBytes;
-    static constexpr int kOffQ = 2 * kStages * kTileBytes;
-    static constexpr int kOffSK = kOffQ + kTileBytes;
-    static constexpr int kOffSV = kOffSK + kTileBytes;
-    static constexpr int kDataBytes = kOffSV + kTileBytes;
-    static constexpr int kOffBar = kDataBytes;            // mbarriers, 8 bytes each
-    static constexpr int kOffMisc = kOffBar + 512;        // tmem base, abort flag
-    static constexpr int kOffMl = kOffMisc + 64;          // float2 (l, lse2) [2][128]
-    static constexpr int kSmemBytes = kOffMl + 2 * kTileM * 8;
 };
 
 // barrier indices
@@ -122,16 +106,19 @@ enum {
     kBarSVFree,      // all value MMAs of a tile completed: suffix-V buffer is free
     kBarOFull,       // O of a tile is complete in tensor memory
     kBarOFree,       // epilogue has read O out (4 arrivals)
+    kBarStageFull,   // the epilogue warps have written a slab of the output tile (4 arrivals)
+    kBarStageFree,   // the TMA stores of that slab have read it
     kBarSFull,                        // [kSlots] scores of an item are in tensor memory
     kBarPReady = kBarSFull + kSlots,  // [kSlots] probabilities written (4 arrivals)
     kBarPvDone = kBarPReady + kSlots, // [kSlots] value MMAs of an item completed
     kBarKFull = kBarPvDone + kSlots,  // [stages]
-    kBarVFull = kBarKFull + 4,
-    kBarKFree = kBarVFull + 4,
-    kBarVFree = kBarKFree + 4,
-    kNumBars = kBarVFree + 4
+    kBarVFull = kBarKFull + kMaxStages,
+    kBarKFree = kBarVFull + kMaxStages,
+    kBarVFree = kBarKFree + kMaxStages,
+    kNumBars = kBarVFree + kMaxStages
 };
-static_assert(kNumBars * 8 <= 512, "barrier area");
+constexpr int kBarBytes = 512;
+static_assert(kNumBars * 8 <= kBarBytes, "barrier area");
 
 struct TileInfo {
     int g, R0, rows, b_first, nc, n_sfx;  // n_sfx: suffix columns rounded up to 16
@@ -154,16 +141,64 @@ __device__ __forceinline__ TileInfo tile_info(const TcFwdParams &p, int tile, in
     return t;
 }
 
-__device__ __forceinline__ int prefix_block_cols(const TcFwdParams &p, int k)
+// rows held (and MMA N used) by prefix block k
+__device__ __forceinline__ int prefix_block_rows(const TcFwdParams &p, int k)
 {
-    return min(kBlockN, (p.P - k * kBlockN + 15) & ~15);
+    return k == p.nblk_p - 1 ? p.tail_rows : kBlockN;
+}
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(map),
+                 "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// ---- softmax building blocks (one thread = one row; `rr` = 32 score columns of that row) -------
+
+// max over the valid columns [lo, lo + span] of chunk `ch`
+template <bool kMasked>
+__device__ __forceinline__ void chunk_max(const uint32_t (&rr)[32], float (&m4)[4], int ch, int lo, unsigned span,
+                                          bool any_col)
+{
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+        float v = __uint_as_float(rr[c]);
+        if (kMasked) v = (any_col && (unsigned)(ch * 32 + c - lo) <= span) ? v : -INFINITY;
+        m4[c & 3] = fmaxf(m4[c & 3], v);
+    }
+}
+
+// p = 2^(s * sl2 - m_ref) for chunk `ch`, packed to bf16 pairs; adds to the two partial row sums
+template <bool kMasked>
+__device__ __forceinline__ void chunk_exp(const uint32_t (&rr)[32], uint32_t (&pk)[16], float &ls0, float &ls1,
+                                          float sl2, float neg_m, int ch, int lo, unsigned span, bool any_col)
+{
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        float x0 = fmaf(__uint_as_float(rr[2 * c]), sl2, neg_m);
+        float x1 = fmaf(__uint_as_float(rr[2 * c + 1]), sl2, neg_m);
+        if (kMasked) {
+            x0 = (any_col && (unsigned)(ch * 32 + 2 * c - lo) <= span) ? x0 : -INFINITY;
+            x1 = (any_col && (unsigned)(ch * 32 + 2 * c + 1 - lo) <= span) ? x1 : -INFINITY;
+        }
+        const float p0 = exp2f(x0), p1 = exp2f(x1);
+        ls0 += p0;
+        ls1 += p1;
+        pk[c] = pack_bf16x2(p0, p1);
+    }
 }
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_pk,
-              const __grid_constant__ CUtensorMap tm_pv, const __grid_constant__ CUtensorMap tm_sk,
-              const __grid_constant__ CUtensorMap tm_sv, const TcFwdParams p)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_out,
+              const __grid_constant__ CUtensorMap tm_pk, const __grid_constant__ CUtensorMap tm_pv,
+              const __grid_constant__ CUtensorMap tm_pk_tail, const __grid_constant__ CUtensorMap tm_pv_tail,
+              const __grid_constant__ CUtensorMap tm_sk, const __grid_constant__ CUtensorMap tm_sv,
+              const TcFwdParams p)
 {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -171,11 +206,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
     PSKV_TRACE_DECL;
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar0 = sbase + C::kOffBar;
+    const uint32_t bar0 = sbase + p.off_bar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::kOffMisc + 4);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kOffMisc);
-    float2 *ml = reinterpret_cast<float2 *>(smem + C::kOffMl);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + p.off_misc + 4);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + p.off_misc);
+    float2 *ml = reinterpret_cast<float2 *>(smem + p.off_ml);  // (row sum, reference max) [2][128]
 
     if ((sbase & 1023u) != 0u) {  // the swizzled layouts need a 1024-byte aligned base
         if (tid == 0) atomicCAS(p.status, 0u, (unsigned int)kErrAlign);
@@ -184,11 +219,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 
     // Zero the data area: rows that no TMA box ever writes (tile padding) must hold finite values,
     // because a zero probability times a NaN value row would still poison the accumulator.
-    for (int i = tid; i < C::kDataBytes / 16; i += kThreads)
-        reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
-            const bool four = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree;
+            const bool four = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
             mbar_init(bar(i), four ? 4u : 1u);
         }
         *abort_flag = 0;
@@ -196,7 +230,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     fence_proxy_async();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 2) {
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
     }
@@ -211,6 +245,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int n_tiles = t_end - t_begin;
     const int nitems = p.nblk_p + 1;  // prefix blocks + the suffix block
     const int g_first = t_begin / p.tiles_per_group;
+    const int sfx_slab = p.sfx_rows * 128;
+    const int tail_slab = p.tail_rows * 128;
 
     // The producer and MMA warps run their loops with all 32 lanes (warp-uniform control flow and
     // addresses, so descriptors can live in uniform registers); one elected lane issues the
@@ -220,7 +256,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (lane == 0) {
             prefetch_tensormap(&tm_q);
             prefetch_tensormap(&tm_sk);
-            if (p.P > 0) prefetch_tensormap(&tm_pk);
+            if (p.P > 0) { prefetch_tensormap(&tm_pk); prefetch_tensormap(&tm_pk_tail); }
         }
         uint32_t kload = 0;  // streaming mode: prefix K blocks loaded so far
         bool ok = true;
@@ -238,7 +274,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const int R = t.R0 + s * p.seg_rows;
                     const int b = R / p.Rg, r = R - b * p.Rg;
                     for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + C::kOffQ + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
+                        tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
                                     bar(kBarQFull), sl * 64, r, t.g, b);
                 }
             }
@@ -246,23 +282,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (p.resident) {
                 if (t.first_of_g && elect_one_sync()) {
                     for (int k = 0; k < p.nblk_p; ++k) {
-                        mbar_arrive_expect_tx(bar(kBarKFull + k), C::kTileBytes);
+                        const bool tail = k == p.nblk_p - 1;
+                        const int slab = tail ? tail_slab : C::kSlabBytes;
+                        mbar_arrive_expect_tx(bar(kBarKFull + k), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + C::kOffPK + k * C::kTileBytes + sl * C::kSlabBytes, &tm_pk,
+                            tma_load_3d(sbase + p.off_pk + k * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
                                         bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
                     }
                 }
                 __syncwarp();
             } else {
                 for (int k = 0; k < p.nblk_p; ++k) {
-                    const uint32_t ks = kload % C::kStages;
-                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / C::kStages) & 1) ^ 1, abort_flag, p.status,
-                                        kErrProducerK);
+                    const uint32_t ks = kload % (uint32_t)p.stages;
+                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
+                                        p.status, kErrProducerK);
                     if (!ok) break;
+                    const bool tail = k == p.nblk_p - 1;
+                    const int slab = tail ? tail_slab : C::kSlabBytes;
                     if (elect_one_sync()) {
-                        mbar_arrive_expect_tx(bar(kBarKFull + ks), C::kTileBytes);
+                        mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + C::kOffPK + ks * C::kTileBytes + sl * C::kSlabBytes, &tm_pk,
+                            tma_load_3d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
                                         bar(kBarKFull + ks), sl * 64, k * kBlockN, t.g);
                     }
                     __syncwarp();
@@ -275,16 +315,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 mbar_arrive_expect_tx(bar(kBarSKFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
                 for (int c = 0; c < t.nc; ++c)
                     for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + C::kOffSK + sl * C::kSlabBytes + c * p.S * 128, &tm_sk,
-                                    bar(kBarSKFull), sl * 64, 0, t.g, t.b_first + c);
+                        tma_load_4d(sbase + p.off_sk + sl * sfx_slab + c * p.S * 128, &tm_sk, bar(kBarSKFull),
+                                    sl * 64, 0, t.g, t.b_first + c);
             }
             __syncwarp();
         }
-    } else if (warp == 10) {
+    } else if (warp == 3) {
         // ------------------------------------------------------------------ producer, value side
         if (lane == 0) {
             prefetch_tensormap(&tm_sv);
-            if (p.P > 0) prefetch_tensormap(&tm_pv);
+            if (p.P > 0) { prefetch_tensormap(&tm_pv); prefetch_tensormap(&tm_pv_tail); }
         }
         uint32_t vload = 0;
         bool ok = true;
@@ -297,23 +337,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (!ok) break;
                 if (t.first_of_g && elect_one_sync()) {
                     for (int k = 0; k < p.nblk_p; ++k) {
-                        mbar_arrive_expect_tx(bar(kBarVFull + k), C::kTileBytes);
+                        const bool tail = k == p.nblk_p - 1;
+                        const int slab = tail ? tail_slab : C::kSlabBytes;
+                        mbar_arrive_expect_tx(bar(kBarVFull + k), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + C::kOffPV + k * C::kTileBytes + sl * C::kSlabBytes, &tm_pv,
+                            tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
                                         bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
                     }
                 }
                 __syncwarp();
             } else {
                 for (int k = 0; k < p.nblk_p; ++k) {
-                    const uint32_t vs = vload % C::kStages;
-                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / C::kStages) & 1) ^ 1, abort_flag, p.status,
-                                        kErrProducerV);
+                    const uint32_t vs = vload % (uint32_t)p.stages;
+                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
+                                        p.status, kErrProducerV);
                     if (!ok) break;
+                    const bool tail = k == p.nblk_p - 1;
+                    const int slab = tail ? tail_slab : C::kSlabBytes;
                     if (elect_one_sync()) {
-                        mbar_arrive_expect_tx(bar(kBarVFull + vs), C::kTileBytes);
+                        mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + C::kOffPV + vs * C::kTileBytes + sl * C::kSlabBytes, &tm_pv,
+                            tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
                                         bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
                     }
                     __syncwarp();
@@ -327,151 +371,161 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
                 for (int c = 0; c < t.nc; ++c)
                     for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + C::kOffSV + sl * C::kSlabBytes + c * p.S * 128, &tm_sv,
-                                    bar(kBarSVFull), sl * 64, 0, t.g, t.b_first + c);
+                        tma_load_4d(sbase + p.off_sv + sl * sfx_slab + c * p.S * 128, &tm_sv, bar(kBarSVFull),
+                                    sl * 64, 0, t.g, t.b_first + c);
             }
             __syncwarp();
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ score MMAs: S = Q K^T
         const int total_items = n_tiles * nitems;
-        int i_qk = 0, i_pv = 0;
-        int tl_qk = 0, k_qk = 0, tl_pv = 0, k_pv = 0;  // (tile, block) of the next score / value item
-        uint32_t kuse = 0, vuse = 0;                    // streaming mode: prefix blocks consumed
-        TileInfo tq = tile_info(p, t_begin, t_begin), tv = tq;
-        // descriptors are built once; per MMA only the 16-byte-granular start address moves
-        const uint64_t q_desc = make_smem_desc(sbase + C::kOffQ, 0, 1024);
-        const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
+        int tl = 0, k = 0;
+        uint32_t kuse = 0;  // streaming mode: prefix K blocks consumed
+        TileInfo t = tile_info(p, t_begin, t_begin);
+        const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
         bool ok = true;
-        while (ok && i_pv < total_items) {
-            PSKV_TRACE_EVENT(16, i_pv);
-            if (i_qk < total_items && i_qk < i_pv + kSlots) {
-                // ---- scores of item i_qk:  S[128 x N] = Q[128 x D] * K_blk[N x D]^T
-                const int slot = i_qk % kSlots;
-                if (k_qk == 0) {
-                    ok = mbar_wait_warp(bar(kBarQFull), tl_qk & 1, abort_flag, p.status, kErrMma);
-                    if (!ok) break;
-                }
-                uint32_t kaddr;
-                int n;
-                if (k_qk < p.nblk_p) {
-                    n = prefix_block_cols(p, k_qk);
-                    if (p.resident) {
-                        if (tq.first_of_g)
-                            ok = mbar_wait_warp(bar(kBarKFull + k_qk), (tq.g - g_first) & 1, abort_flag, p.status, kErrMma);
-                        kaddr = sbase + C::kOffPK + k_qk * C::kTileBytes;
-                    } else {
-                        const uint32_t ks = kuse % C::kStages;
-                        ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
-                        kaddr = sbase + C::kOffPK + ks * C::kTileBytes;
-                    }
-                } else {
-                    n = tq.n_sfx;
-                    ok = mbar_wait_warp(bar(kBarSKFull), tl_qk & 1, abort_flag, p.status, kErrMma);
-                    kaddr = sbase + C::kOffSK;
-                }
+        for (int i = 0; i < total_items && ok; ++i) {
+            const int slot = i % kSlots;
+            // the slot is free once the value MMAs of item i-3 (which read P from it) have completed
+            ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
+            if (!ok) break;
+            if (k == 0) {
+                ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaQk);
                 if (!ok) break;
-                PSKV_TRACE_EVENT(10, i_qk);
-                tc_fence_after();
-#ifdef PSKV_X_QKN
-                const uint32_t idesc = make_idesc_bf16(kTileM, PSKV_X_QKN, 0);
-#else
-                const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
-#endif
-                const uint32_t d_tmem = tmem + slot * kBlockN;
-                const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
-                const bool last_of_tile = k_qk == nitems - 1;
-                const bool free_stage = k_qk < p.nblk_p && !p.resident;
-                if (elect_one_sync()) {
-#pragma unroll
-                    for (int ks16 = 0; ks16 < D / 16; ++ks16) {
-                        const uint64_t off = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
-                        mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks16 > 0 ? 1u : 0u);
-                        PSKV_TRACE_EVENT_ONE(17, i_qk * 8 + ks16);
-                    }
-                    tc_commit(bar(kBarSFull + slot));
-                    if (free_stage) tc_commit(bar(kBarKFree + (kuse % C::kStages)));
-                    if (last_of_tile) tc_commit(bar(kBarQkFree));  // the suffix block ends the tile's scores
-                }
-                __syncwarp();
-                PSKV_TRACE_EVENT(12, i_qk);
-                if (free_stage) ++kuse;
-                ++i_qk;
-                if (++k_qk == nitems) {
-                    k_qk = 0;
-                    if (++tl_qk < n_tiles) tq = tile_info(p, t_begin + tl_qk, t_begin);
+            }
+            uint32_t kaddr;
+            int n, slab;
+            if (k < p.nblk_p) {
+                n = prefix_block_rows(p, k);
+                slab = n * 128;
+                if (p.resident) {
+                    if (t.first_of_g)
+                        ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaQk);
+                    kaddr = sbase + p.off_pk + k * C::kTileBytes;
+                } else {
+                    const uint32_t ks = kuse % (uint32_t)p.stages;
+                    ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / (uint32_t)p.stages) & 1, abort_flag, p.status,
+                                        kErrMmaQk);
+                    kaddr = sbase + p.off_pk + ks * C::kTileBytes;
                 }
             } else {
-                // ---- values of item i_pv:  O[128 x D] (+)= P[128 x N] * V_blk[N x D]
-                const int slot = i_pv % kSlots;
-                ok = mbar_wait_warp(bar(kBarPReady + slot), (i_pv / kSlots) & 1, abort_flag, p.status, kErrMma);
-                if (!ok) break;
-                if (k_pv == 0 && tl_pv > 0) {
-                    // O of the previous tile must have been read out by the epilogue warps
-                    ok = mbar_wait_warp(bar(kBarOFree), (tl_pv - 1) & 1, abort_flag, p.status, kErrMma);
-                    if (!ok) break;
-                }
-                uint32_t vaddr;
-                int n;
-                if (k_pv < p.nblk_p) {
-                    n = prefix_block_cols(p, k_pv);
-                    if (p.resident) {
-                        if (tv.first_of_g)
-                            ok = mbar_wait_warp(bar(kBarVFull + k_pv), (tv.g - g_first) & 1, abort_flag, p.status, kErrMma);
-                        vaddr = sbase + C::kOffPV + k_pv * C::kTileBytes;
-                    } else {
-                        const uint32_t vs = vuse % C::kStages;
-                        ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / C::kStages) & 1, abort_flag, p.status, kErrMma);
-                        vaddr = sbase + C::kOffPV + vs * C::kTileBytes;
-                    }
-                } else {
-                    n = tv.n_sfx;
-                    ok = mbar_wait_warp(bar(kBarSVFull), tl_pv & 1, abort_flag, p.status, kErrMma);
-                    vaddr = sbase + C::kOffSV;
-                }
-                if (!ok) break;
-                PSKV_TRACE_EVENT(11, i_pv);
-                tc_fence_after();
-                const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
-                const uint64_t v_desc = make_smem_desc(vaddr, C::kSlabBytes, 1024);
-                const int nk = n >> 4;
-                const bool last_of_tile = k_pv == nitems - 1;
-                const bool free_stage = k_pv < p.nblk_p && !p.resident;
-                const uint32_t acc0 = k_pv > 0 ? 1u : 0u;
-                if (elect_one_sync()) {
+                n = t.n_sfx;
+                slab = sfx_slab;
+                ok = mbar_wait_warp(bar(kBarSKFull), tl & 1, abort_flag, p.status, kErrMmaQk);
+                kaddr = sbase + p.off_sk;
+            }
+            if (!ok) break;
+            PSKV_TRACE_EVENT(10, i);
+            tc_fence_after();
+            const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
+            const uint32_t d_tmem = tmem + slot * kBlockN;
+            const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
+            const uint64_t k_slab = (uint64_t)(slab >> 4);
+            const bool last_of_tile = k == nitems - 1;
+            const bool free_stage = k < p.nblk_p && !p.resident;
+            if (elect_one_sync()) {
 #pragma unroll
-                    for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
-                        if (ks16 < nk)
-                            mma_ts(tmem + kOCol, p_tmem + ks16 * 8, v_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_pv,
-                                   ks16 > 0 ? 1u : acc0);
-                    }
-                    tc_commit(bar(kBarPvDone + slot));
-                    if (free_stage) tc_commit(bar(kBarVFree + (vuse % C::kStages)));
-                    if (last_of_tile) {
-                        tc_commit(bar(kBarSVFree));
-                        tc_commit(bar(kBarOFull));
-                    }
+                for (int ks16 = 0; ks16 < D / 16; ++ks16) {
+                    const uint64_t qoff = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
+                    const uint64_t koff = (uint64_t)(ks16 >> 2) * k_slab + (uint64_t)(((ks16 & 3) * 32) >> 4);
+                    mma_ss(d_tmem, q_desc + qoff, k_desc + koff, idesc, ks16 > 0 ? 1u : 0u);
                 }
-                __syncwarp();
-                PSKV_TRACE_EVENT(13, i_pv);
-                if (free_stage) ++vuse;
-                ++i_pv;
-                if (++k_pv == nitems) {
-                    k_pv = 0;
-                    if (++tl_pv < n_tiles) tv = tile_info(p, t_begin + tl_pv, t_begin);
-                }
+                tc_commit(bar(kBarSFull + slot));
+                if (free_stage) tc_commit(bar(kBarKFree + (kuse % (uint32_t)p.stages)));
+                if (last_of_tile) tc_commit(bar(kBarQkFree));  // the suffix block ends the tile's scores
+            }
+            __syncwarp();
+            PSKV_TRACE_EVENT(12, i);
+            if (free_stage) ++kuse;
+            if (++k == nitems) {
+                k = 0;
+                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
-    } else if (warp < 6) {
-        // ------------------------------------------------------------------ softmax warps
-        // Each thread owns one query row (tensor-memory lane).  Per item: pass 1 reads the score
-        // block 32 columns at a time and takes the row max; pass 2 reads it again, exponentiates
-        // and writes bf16 probabilities over the first half of the same slot (a probability chunk
-        // only ever overwrites score columns that pass 2 has already consumed).
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ value MMAs: O += P V
+        const int total_items = n_tiles * nitems;
+        int tl = 0, k = 0;
+        uint32_t vuse = 0;
+        TileInfo t = tile_info(p, t_begin, t_begin);
+        const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
+        bool ok = true;
+        for (int i = 0; i < total_items && ok; ++i) {
+            const int slot = i % kSlots;
+            ok = mbar_wait_warp(bar(kBarPReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaPv);
+            if (!ok) break;
+            if (k == 0 && tl > 0) {
+                // O of the previous tile must have been read out by the epilogue warps
+                ok = mbar_wait_warp(bar(kBarOFree), (tl - 1) & 1, abort_flag, p.status, kErrMmaPv);
+                if (!ok) break;
+            }
+            uint32_t vaddr;
+            int n, slab;
+            if (k < p.nblk_p) {
+                n = prefix_block_rows(p, k);
+                slab = n * 128;
+                if (p.resident) {
+                    if (t.first_of_g)
+                        ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaPv);
+                    vaddr = sbase + p.off_pv + k * C::kTileBytes;
+                } else {
+                    const uint32_t vs = vuse % (uint32_t)p.stages;
+                    ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / (uint32_t)p.stages) & 1, abort_flag, p.status,
+                                        kErrMmaPv);
+                    vaddr = sbase + p.off_pv + vs * C::kTileBytes;
+                }
+            } else {
+                n = t.n_sfx;
+                slab = sfx_slab;
+                ok = mbar_wait_warp(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMmaPv);
+                vaddr = sbase + p.off_sv;
+            }
+            if (!ok) break;
+            PSKV_TRACE_EVENT(11, i);
+            tc_fence_after();
+            const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
+            const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
+            const int nk = n >> 4;
+            const bool last_of_tile = k == nitems - 1;
+            const bool free_stage = k < p.nblk_p && !p.resident;
+            const uint32_t acc0 = k > 0 ? 1u : 0u;
+            if (elect_one_sync()) {
+#pragma unroll
+                for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
+                    if (ks16 < nk)
+                        mma_ts(tmem + kOCol, p_tmem + ks16 * 8, v_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_pv,
+                               ks16 > 0 ? 1u : acc0);
+                }
+                tc_commit(bar(kBarPvDone + slot));
+                if (free_stage) tc_commit(bar(kBarVFree + (vuse % (uint32_t)p.stages)));
+                if (last_of_tile) {
+                    tc_commit(bar(kBarSVFree));
+                    tc_commit(bar(kBarOFull));
+                }
+            }
+            __syncwarp();
+            PSKV_TRACE_EVENT(13, i);
+            if (free_stage) ++vuse;
+            if (++k == nitems) {
+                k = 0;
+                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+            }
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------------ softmax warps (4..7)
+        // Each thread owns one query row (tensor-memory lane).  Per item the score block is read 32
+        // columns at a time, twice: once for the row max, once to exponentiate.  The max pass of
+        // the next item (when it is an unmasked prefix block whose scores are already there) is
+        // folded into the exponentiation pass of the current one, where the exponential unit is
+        // the bound and the other pipes are idle.  bf16 probabilities overwrite the first half of
+        // the item's own score slot, chunk by chunk, behind the reads.
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+        const int total_items = n_tiles * nitems;
         int item = 0;
         bool ok = true;
+        bool have_mb = false;  // the block max of `item` was already taken during the previous item
+        float mb_next = -INFINITY;
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             const bool valid = row < t.rows;
@@ -482,57 +536,50 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             float m_ref = 0.f, l = 0.f;
             for (int k = 0; k < nitems && ok; ++k, ++item) {
                 const int slot = item % kSlots;
-                int n, lo, hi;                            // valid columns of this row: [lo, hi]
+                // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
+                // blocks like real rows (their scores are finite and never stored) and see no suffix key.
+                int n, lo, hi;
                 if (k < p.nblk_p) {
-                    n = prefix_block_cols(p, k);
+                    n = prefix_block_rows(p, k);
                     lo = 0;
-                    hi = valid ? min(kBlockN, p.P - k * kBlockN) - 1 : -1;
+                    hi = min(kBlockN, p.P - k * kBlockN) - 1;
                 } else {
                     n = t.n_sfx;
                     lo = valid ? sfx_lo : 1;
                     hi = valid ? sfx_hi : 0;
                 }
                 const int nch = (n + 31) >> 5;
-                // chunks [ch_b, ch_e] hold at least one valid column of some row of this warp
                 const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1) && ((n & 31) == 0);
-                int ch_b = 0, ch_e = nch - 1;
+                int ch_b = 0, ch_e = nch - 1;  // chunks that hold a valid column of some row of this warp
                 if (!full) {
                     const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
                     const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
                     ch_b = wlo >> 5;
                     ch_e = min(nch - 1, whi >> 5);
                 }
-                const unsigned span = (unsigned)(hi - lo);  // hi < lo wraps to a huge span only if hi-lo < 0
+                const unsigned span = (unsigned)(hi - lo);
                 const bool any_col = hi >= lo;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag,
-                                                       p.status, kErrSoftmax));
-                if (!ok) break;
-                if (warp == 2) PSKV_TRACE_EVENT(20, item);
-                tc_fence_after();
                 const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
 
-                // ---- pass 1: row max of the block
-                float mb = -INFINITY;
-                {
+                // ---- block max (unless it was taken while the previous item was exponentiated)
+                float mb;
+                if (have_mb) {
+                    mb = mb_next;
+                } else {
+                    ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
+                    if (!ok) break;
+                    tc_fence_after();
                     float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                     for (int ch = ch_b; ch <= ch_e; ++ch) {
                         uint32_t rr[32];
                         tmem_ld32(s_tmem + ch * 32, rr);
                         tmem_wait_ld();
-                        if (full) {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) m4[c & 3] = fmaxf(m4[c & 3], __uint_as_float(rr[c]));
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) {
-                                const bool in = any_col && (unsigned)(ch * 32 + c - lo) <= span;
-                                m4[c & 3] = fmaxf(m4[c & 3], in ? __uint_as_float(rr[c]) : -INFINITY);
-                            }
-                        }
+                        if (full) chunk_max<false>(rr, m4, ch, lo, span, any_col);
+                        else chunk_max<true>(rr, m4, ch, lo, span, any_col);
                     }
                     mb = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                 }
-                if (warp == 2) PSKV_TRACE_EVENT(22, item);
+                PSKV_TRACE_EVENT(22, item);
                 const float mx = mb * p.sl2;
                 if (k == 0) {
                     m_ref = (mb == -INFINITY) ? 0.f : mx;
@@ -542,8 +589,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         // Rare: the running max jumped.  Rescale this row's O in tensor memory after the
                         // previous item's P*V has completed, and before this item's P is handed over.
                         const int prev = item - 1;
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPvDone + prev % kSlots), (prev / kSlots) & 1,
-                                                               abort_flag, p.status, kErrSoftmax));
+                        ok = mbar_wait_warp(bar(kBarPvDone + prev % kSlots), (prev / kSlots) & 1, abort_flag,
+                                            p.status, kErrSoftmax);
                         if (!ok) break;
                         tc_fence_after();
                         const float f = need ? exp2f(m_ref - mx) : 1.f;
@@ -561,45 +608,50 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     }
                 }
 
-                // ---- pass 2: p = 2^(s * sl2 - m_ref), row sum, bf16 pairs back to tensor memory
+                // ---- is the next item an unmasked prefix block whose scores have already arrived?
+                have_mb = false;
+                int nch_next = 0;
+                uint32_t s_tmem_next = 0;
+                if (item + 1 < total_items) {
+                    const int kn = (k + 1 == nitems) ? 0 : k + 1;
+                    if (kn < p.nblk_p && (prefix_block_rows(p, kn) & 31) == 0 &&
+                        min(kBlockN, p.P - kn * kBlockN) == prefix_block_rows(p, kn)) {
+                        const int slot_n = (item + 1) % kSlots;
+                        if (__all_sync(0xffffffffu, mbar_try_wait(bar(kBarSFull + slot_n), ((item + 1) / kSlots) & 1))) {
+                            tc_fence_after();
+                            have_mb = true;
+                            nch_next = prefix_block_rows(p, kn) >> 5;
+                            s_tmem_next = tmem + lane_addr + slot_n * kBlockN;
+                        }
+                    }
+                }
+
+                // ---- p = 2^(s * sl2 - m_ref), row sum, bf16 pairs back to tensor memory
                 const float neg_m = -m_ref;
                 float ls0 = 0.f, ls1 = 0.f;
-                for (int ch = 0; ch < nch; ++ch) {
-                    uint32_t pk[16];
-                    if (ch >= ch_b && ch <= ch_e) {
-                        uint32_t rr[32];
-                        tmem_ld32(s_tmem + ch * 32, rr);
-                        tmem_wait_ld();
-                        if (full) {
-#pragma unroll
-                            for (int c = 0; c < 16; ++c) {
-                                const float p0 = exp2f(fmaf(__uint_as_float(rr[2 * c]), p.sl2, neg_m));
-                                const float p1 = exp2f(fmaf(__uint_as_float(rr[2 * c + 1]), p.sl2, neg_m));
-                                ls0 += p0;
-                                ls1 += p1;
-                                pk[c] = pack_bf16x2(p0, p1);
-                            }
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 16; ++c) {
-                                const bool in0 = any_col && (unsigned)(ch * 32 + 2 * c - lo) <= span;
-                                const bool in1 = any_col && (unsigned)(ch * 32 + 2 * c + 1 - lo) <= span;
-                                const float p0 = exp2f(in0 ? fmaf(__uint_as_float(rr[2 * c]), p.sl2, neg_m) : -INFINITY);
-                                const float p1 = exp2f(in1 ? fmaf(__uint_as_float(rr[2 * c + 1]), p.sl2, neg_m) : -INFINITY);
-                                ls0 += p0;
-                                ls1 += p1;
-                                pk[c] = pack_bf16x2(p0, p1);
-                            }
-                        }
+                float n4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                const int nloop = max(nch, nch_next);
+                for (int ch = 0; ch < nloop; ++ch) {
+                    uint32_t rr[32], rn[32], pk[16];
+                    const bool act = ch >= ch_b && ch <= ch_e && ch < nch;
+                    const bool nxt = ch < nch_next;
+                    if (act) tmem_ld32(s_tmem + ch * 32, rr);
+                    if (nxt) tmem_ld32(s_tmem_next + ch * 32, rn);
+                    if (act || nxt) tmem_wait_ld();
+                    if (act) {
+                        if (full) chunk_exp<false>(rr, pk, ls0, ls1, p.sl2, neg_m, ch, lo, span, any_col);
+                        else chunk_exp<true>(rr, pk, ls0, ls1, p.sl2, neg_m, ch, lo, span, any_col);
                     } else {
 #pragma unroll
                         for (int c = 0; c < 16; ++c) pk[c] = 0u;
                     }
-                    tmem_st16(s_tmem + ch * 16, pk);
+                    if (nxt) chunk_max<false>(rn, n4, ch, 0, 0u, true);
+                    if (ch < nch) tmem_st16(s_tmem + ch * 16, pk);
                 }
+                mb_next = fmaxf(fmaxf(n4[0], n4[1]), fmaxf(n4[2], n4[3]));
                 l += ls0 + ls1;
-                if (k == nitems - 1) ml[(tl & 1) * kTileM + row] = make_float2(l, m_ref + log2f(l));
-                if (warp == 2) PSKV_TRACE_EVENT(23, item);
+                if (k == nitems - 1) ml[(tl & 1) * kTileM + row] = make_float2(l, m_ref);
+                PSKV_TRACE_EVENT(23, item);
                 tmem_wait_st();
                 tc_fence_before();
                 __threadfence_block();
@@ -608,18 +660,23 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue warps (6..9)
-        const int row = 32 * (warp & 3) + lane;
-        const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-        for (int tl = 0; tl < n_tiles; ++tl) {
+        // ------------------------------------------------------------------ epilogue warps (8..11)
+        const int ew = warp & 3;
+        const int row = 32 * ew + lane;
+        const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
+        const uint32_t stage = sbase + p.off_stage;
+        const bool issuer = warp == 8;  // this warp's elected lane issues the TMA stores
+        if (issuer && lane == 0) prefetch_tensormap(&tm_out);
+        bool ok = true;
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), tl & 1, abort_flag, p.status, kErrEpilogue)))
-                break;
-            if (warp == 6) PSKV_TRACE_EVENT(30, tl);
+            ok = mbar_wait_warp(bar(kBarOFull), tl & 1, abort_flag, p.status, kErrEpilogue);
+            if (!ok) break;
+            PSKV_TRACE_EVENT(30, tl);
             tc_fence_after();
             const float2 lm = ml[(tl & 1) * kTileM + row];
             const float inv = 1.f / lm.x;
-            uint32_t ob[D / 2];  // normalised row as bf16 pairs
+            uint32_t ob[D / 2];  // the normalised row as bf16 pairs
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
                 uint32_t o[32];
@@ -636,16 +693,43 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int R = t.R0 + row;
                 const int b = R / p.Rg, r = R - b * p.Rg;
                 const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
-                uint4 *dst = reinterpret_cast<uint4 *>(p.out + grow * D);
-#pragma unroll
-#ifdef PSKV_X_NOSTORE
-                if (ob[0] == 0x12345678u)
-#endif
-                for (int v = 0; v < D / 8; ++v) dst[v] = make_uint4(ob[4 * v], ob[4 * v + 1], ob[4 * v + 2], ob[4 * v + 3]);
-                p.lse[grow] = lm.y * kLn2;
+                p.lse[grow] = (lm.y + log2f(lm.x)) * kLn2;
             }
-            if (warp == 6) PSKV_TRACE_EVENT(31, tl);
+            // out: one 64-column slab at a time through the swizzled staging buffer, then TMA stores
+            const int nseg = t.rows / p.seg_rows;
+#pragma unroll
+            for (int sl = 0; sl < C::kSlabs; ++sl) {
+                const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
+                ok = mbar_wait_warp(bar(kBarStageFree), (round & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
+                if (!ok) break;
+                uint8_t *srow = smem + p.off_stage + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(ob[sl * 32 + 4 * c], ob[sl * 32 + 4 * c + 1], ob[sl * 32 + 4 * c + 2],
+                                   ob[sl * 32 + 4 * c + 3]);
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarStageFull));
+                if (issuer) {
+                    ok = mbar_wait_warp(bar(kBarStageFull), round & 1, abort_flag, p.status, kErrEpilogue);
+                    if (!ok) break;
+                    if (elect_one_sync()) {
+                        for (int s = 0; s < nseg; ++s) {
+                            const int R = t.R0 + s * p.seg_rows;
+                            const int b = R / p.Rg, r = R - b * p.Rg;
+                            tma_store_4d(&tm_out, stage + s * p.seg_rows * 128, sl * 64, r, t.g, b);
+                        }
+                        tma_store_commit();
+                        tma_store_wait_read();  // the staging buffer may be overwritten after this
+                        mbar_arrive(bar(kBarStageFree));
+                    }
+                    __syncwarp();
+                }
+            }
+            PSKV_TRACE_EVENT(31, tl);
         }
+        if (issuer && elect_one_sync()) tma_store_wait_all();
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -653,27 +737,34 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     if (*abort_flag != 0) __nanosleep(20000);  // let copies and MMAs still in flight drain
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 512);
+    if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------ host side
 
 struct TilePlan {
     bool ok;
-    int tile_rows, seg_rows, tiles_per_group;
+    int tile_rows, seg_rows, tiles_per_group, sfx_rows;
+    int nblk_p, tail_rows, resident, stages;
+    int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml, smem_bytes;
 };
 
 int gcd_int(int a, int b) { return b == 0 ? a : gcd_int(b, a % b); }
+int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-// Picks the rows per tile: the largest multiple of 8 up to 128 such that the suffix keys of all
-// candidates a tile can touch fit one 128-key block (candidates x S <= 128).
+// Picks the rows per tile -- the largest multiple of 8 up to 128 such that the suffix keys of all
+// candidates a tile can touch fit one 128-key block (candidates x S <= 128) -- and lays out shared
+// memory: all prefix blocks of a KV head if they fit beside the other buffers (resident mode), else
+// rings of 2..4 block stages.
 TilePlan plan_tiles(const Dims &dm)
 {
-    TilePlan best{false, 0, 0, 0};
-    if (dm.S % 8 != 0 || dm.S > kBlockN) return best;
+    TilePlan pl;
+    memset(&pl, 0, sizeof(pl));
+    if (dm.S % 8 != 0 || dm.S > kBlockN) return pl;
     const int Rg = dm.n_rep * dm.S;
     const long long total = (long long)dm.B * Rg;
-    for (int m = kTileM; m >= 8; m -= 8) {
+    int nc_best = 0;
+    for (int m = kTileM; m >= 8 && !pl.tile_rows; m -= 8) {
         const int seg = gcd_int(Rg, m);
         if (seg % 8 != 0) continue;
         // worst number of candidates a window [t*m, t*m + m) overlaps; the pattern repeats every Rg/seg tiles
@@ -689,13 +780,47 @@ TilePlan plan_tiles(const Dims &dm)
             if (nc > nc_max) nc_max = nc;
         }
         if (nc_max * dm.S > kBlockN) continue;
-        best.ok = true;
-        best.tile_rows = m;
-        best.seg_rows = seg;
-        best.tiles_per_group = (int)ntiles;
-        return best;
+        pl.tile_rows = m;
+        pl.seg_rows = seg;
+        pl.tiles_per_group = (int)ntiles;
+        nc_best = nc_max;
     }
-    return best;
+    if (!pl.tile_rows) return pl;
+    pl.sfx_rows = round_up(nc_best * dm.S, 16);
+    pl.nblk_p = (dm.P + kBlockN - 1) / kBlockN;
+    pl.tail_rows = pl.nblk_p ? round_up(dm.P - (pl.nblk_p - 1) * kBlockN, 16) : 0;
+
+    const int slabs = dm.d / 64;
+    const int tile_bytes = slabs * kTileM * 128;
+    const int sfx_bytes = round_up(slabs * pl.sfx_rows * 128, 1024);
+    const int tail_bytes = round_up(slabs * pl.tail_rows * 128, 1024);
+    const int tail_area = 2 * kTileM * 8 /*ml*/ + 64 /*misc*/ + kBarBytes;
+    const int fixed = tile_bytes /*Q*/ + 2 * sfx_bytes + kStagingBytes + tail_area;
+    const int resident_bytes = pl.nblk_p ? (pl.nblk_p - 1) * tile_bytes + tail_bytes : 0;
+    int kv_bytes = 0;  // bytes of the prefix K area (the V area has the same size)
+    if (pl.nblk_p <= kMaxStages && fixed + 2 * resident_bytes <= kMaxSmem) {
+        pl.resident = 1;
+        pl.stages = pl.nblk_p;
+        kv_bytes = resident_bytes;
+    } else {
+        int st = (kMaxSmem - fixed) / (2 * tile_bytes);
+        if (st > kMaxStages) st = kMaxStages;
+        if (st < 2) return pl;  // does not fit: the general kernels take the shape
+        pl.stages = st;
+        kv_bytes = st * tile_bytes;
+    }
+    pl.off_pk = 0;
+    pl.off_pv = pl.off_pk + kv_bytes;
+    pl.off_q = pl.off_pv + kv_bytes;
+    pl.off_sk = pl.off_q + tile_bytes;
+    pl.off_sv = pl.off_sk + sfx_bytes;
+    pl.off_stage = pl.off_sv + sfx_bytes;
+    pl.off_bar = pl.off_stage + kStagingBytes;
+    pl.off_misc = pl.off_bar + kBarBytes;
+    pl.off_ml = pl.off_misc + 64;
+    pl.smem_bytes = pl.off_ml + 2 * kTileM * 8;
+    pl.ok = pl.smem_bytes <= kMaxSmem;
+    return pl;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -743,18 +868,20 @@ int sm_count()
 template <int D>
 cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_word, cudaStream_t stream)
 {
-    using C = Cfg<D>;
     const Dims &dm = a.dims;
     const int Rg = dm.n_rep * dm.S;
-    CUtensorMap tm_q, tm_pk, tm_pv, tm_sk, tm_sv;
+    CUtensorMap tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail, tm_sk, tm_sv;
     memset(&tm_pk, 0, sizeof(tm_pk));
     memset(&tm_pv, 0, sizeof(tm_pv));
+    memset(&tm_pk_tail, 0, sizeof(tm_pk_tail));
+    memset(&tm_pv_tail, 0, sizeof(tm_pv_tail));
     {
-        // q viewed as [B][Hkv][Rg][D]: the n_rep heads of a KV head are contiguous rows
+        // q / out viewed as [B][Hkv][Rg][D]: the n_rep heads of a KV head are contiguous rows
         cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Rg, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
         cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)Rg * D * 2, (cuuint64_t)dm.Hkv * Rg * D * 2};
         cuuint32_t box[4] = {64, (cuuint32_t)plan.seg_rows, 1, 1};
         if (!encode_map(&tm_q, a.q, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_out, a.out, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
     {
         cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)dm.S, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
@@ -767,11 +894,13 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_
         cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
         cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.P * D * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
+        cuuint32_t box_tail[3] = {64, (cuuint32_t)plan.tail_rows, 1};
         if (!encode_map(&tm_pk, a.prefix_k, 3, dims, str, box)) return cudaErrorInvalidValue;
         if (!encode_map(&tm_pv, a.prefix_v, 3, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_pk_tail, a.prefix_k, 3, dims, str, box_tail)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_pv_tail, a.prefix_v, 3, dims, str, box_tail)) return cudaErrorInvalidValue;
     }
     TcFwdParams p;
-    p.out = a.out;
     p.lse = a.lse;
     p.status = status_word;
     p.sl2 = a.scale * kLog2e;
@@ -781,18 +910,24 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_
     p.seg_rows = plan.seg_rows;
     p.tiles_per_group = plan.tiles_per_group;
     p.total_tiles = plan.tiles_per_group * dm.Hkv;
-    p.nblk_p = (dm.P + kBlockN - 1) / kBlockN;
-    p.resident = p.nblk_p <= C::kStages ? 1 : 0;
+    p.nblk_p = plan.nblk_p;
+    p.tail_rows = plan.tail_rows;
+    p.resident = plan.resident;
+    p.stages = plan.stages > 0 ? plan.stages : 1;
+    p.sfx_rows = plan.sfx_rows;
+    p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_sk = plan.off_sk;
+    p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
+    p.off_ml = plan.off_ml;
 
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
-    tc_fwd_kernel<D><<<grid, kThreads, C::kSmemBytes, stream>>>(tm_q, tm_pk, tm_pv, tm_sk, tm_sv, p);
+    tc_fwd_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail,
+                                                                  tm_sk, tm_sv, p);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -814,15 +949,6 @@ extern "C" int pskv_debug_read_trace(long long *host, int max_events)
             host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
             host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1];
         }
-    cudaMemcpyFromSymbol(cnt, g_trace_n2, sizeof(cnt));
-    cudaMemcpyFromSymbol(buf, g_trace2, sizeof(buf));
-    for (int w = 0; w < kTraceWarps; ++w)
-        for (unsigned int i = 0; i < cnt[w] && i < (unsigned int)kTraceCap && n < max_events; ++i, ++n) {
-            host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
-            host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1];
-        }
-    unsigned int zeros[kTraceWarps] = {0};
-    cudaMemcpyToSymbol(g_trace_n2, zeros, sizeof(zeros));
     return n;
 }
 #endif
