@@ -16,8 +16,8 @@
 //   warp 3      TMA producer, value side (prefix V blocks, suffix V of the tile)
 //   warps 4-7   softmax: thread <-> query row (tensor-memory lane)
 //   warps 8-11  epilogue: O from tensor memory, normalise, bf16, shared-memory staging, TMA store
-// An "item" is one (tile, key block) pair; score blocks rotate through three 128-column slots of
-// tensor memory, O has its own 128 columns.  Every wait is on an event produced by an earlier
+// An "item" is one (tile, key block) pair; tensor memory holds two 128-column score slots, two
+// 64-column probability slots and the 128 columns of O.  Every wait is on an event produced by an earlier
 // item of a role that never waits on the waiter, so no wait cycle can form; every wait is bounded.
 #include <string.h>
 
@@ -31,10 +31,14 @@ using namespace sm100;
 
 constexpr int kTileM = 128;    // rows of one MMA tile (tensor-memory lanes)
 constexpr int kBlockN = 128;   // keys per block
-constexpr int kSlots = 3;      // score slots in tensor memory
+constexpr int kSlots = 2;      // score slots (128 columns each) and probability slots (64 columns each)
 constexpr int kThreads = 384;
-constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
-constexpr float kRescaleGap = 8.0f;      // log2 units the running max may lag before O is rescaled
+constexpr int kPCol = kSlots * kBlockN;              // first tensor-memory column of the probability slots
+constexpr int kOCol = kPCol + kSlots * kBlockN / 2;  // first tensor-memory column of O
+// Probabilities are 2^(score - reference) with a per-row reference taken from the first keys the
+// row sees; bf16 and fp32 share their exponent range, so any reference within this many powers of
+// two of the true row max is exact, and only a larger lag triggers the (rare) rescale path.
+constexpr float kRescaleGap = 64.0f;
 constexpr int kMaxStages = 4;
 constexpr int kStagingBytes = kTileM * 128;  // one 64-column slab of the output tile
 constexpr int kMaxSmem = 232448;
@@ -109,7 +113,8 @@ enum {
     kBarStageFull,   // the epilogue warps have written a slab of the output tile (4 arrivals)
     kBarStageFree,   // the TMA stores of that slab have read it
     kBarSFull,                        // [kSlots] scores of an item are in tensor memory
-    kBarPReady = kBarSFull + kSlots,  // [kSlots] probabilities written (4 arrivals)
+    kBarSFree = kBarSFull + kSlots,   // [kSlots] the softmax warps are done with a score slot (4 arrivals)
+    kBarPReady = kBarSFree + kSlots,  // [kSlots] probabilities written (4 arrivals)
     kBarPvDone = kBarPReady + kSlots, // [kSlots] value MMAs of an item completed
     kBarKFull = kBarPvDone + kSlots,  // [stages]
     kBarVFull = kBarKFull + kMaxStages,
@@ -222,7 +227,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
-            const bool four = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
+            const bool four = (i >= kBarSFree && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
             mbar_init(bar(i), four ? 4u : 1u);
         }
         *abort_flag = 0;
@@ -386,8 +391,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
         for (int i = 0; i < total_items && ok; ++i) {
             const int slot = i % kSlots;
-            // the slot is free once the value MMAs of item i-3 (which read P from it) have completed
-            ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
+            // the score slot is free once the softmax warps have read item i-2 out of it
+            ok = mbar_wait_warp(bar(kBarSFree + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
             if (!ok) break;
             if (k == 0) {
                 ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaQk);
@@ -483,7 +488,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (!ok) break;
             PSKV_TRACE_EVENT(11, i);
             tc_fence_after();
-            const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
+            const uint32_t p_tmem = tmem + kPCol + slot * (kBlockN / 2);  // bf16 pairs: 8 columns per 16 keys
             const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
             const int nk = n >> 4;
             const bool last_of_tile = k == nitems - 1;
@@ -513,19 +518,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         }
     } else if (warp < 8) {
         // ------------------------------------------------------------------ softmax warps (4..7)
-        // Each thread owns one query row (tensor-memory lane).  Per item the score block is read 32
-        // columns at a time, twice: once for the row max, once to exponentiate.  The max pass of
-        // the next item (when it is an unmasked prefix block whose scores are already there) is
-        // folded into the exponentiation pass of the current one, where the exponential unit is
-        // the bound and the other pipes are idle.  bf16 probabilities overwrite the first half of
-        // the item's own score slot, chunk by chunk, behind the reads.
+        // Each thread owns one query row (tensor-memory lane) and makes ONE pass over a score block,
+        // 16 columns at a time with the next 16 in flight: running max (for the reference and the
+        // overflow check), p = 2^(s*sl2 - m_ref), row sum, bf16 pairs into the item's probability
+        // slot.  m_ref is fixed by the first columns in which the row sees a key; scores stay intact
+        // in their slot, so the rare item whose max runs more than kRescaleGap ahead of m_ref is
+        // simply redone with a new reference after O and the row sum have been rescaled.  The loops
+        // are kept small on purpose: one warp per scheduler runs this code, and straight-line code
+        // longer than the instruction cache close to the scheduler stalls on fetch.
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-        const int total_items = n_tiles * nitems;
         int item = 0;
         bool ok = true;
-        bool have_mb = false;  // the block max of `item` was already taken during the previous item
-        float mb_next = -INFINITY;
+#pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             const bool valid = row < t.rows;
@@ -534,6 +539,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const int sfx_lo = (b - t.b_first) * p.S;   // first suffix column of this row's candidate
             const int sfx_hi = sfx_lo + (r % p.S);      // causal: suffix keys 0..i
             float m_ref = 0.f, l = 0.f;
+            bool m_set = false;
+#pragma unroll 1
             for (int k = 0; k < nitems && ok; ++k, ++item) {
                 const int slot = item % kSlots;
                 // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
@@ -548,107 +555,109 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     lo = valid ? sfx_lo : 1;
                     hi = valid ? sfx_hi : 0;
                 }
-                const int nch = (n + 31) >> 5;
-                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1) && ((n & 31) == 0);
-                int ch_b = 0, ch_e = nch - 1;  // chunks that hold a valid column of some row of this warp
+                const int nh = n >> 4;  // 16-column pieces
+                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1);
+                int h_b = 0, h_e = nh - 1;  // pieces that hold a valid column of some row of this warp
                 if (!full) {
                     const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
                     const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
-                    ch_b = wlo >> 5;
-                    ch_e = min(nch - 1, whi >> 5);
+                    h_b = wlo >> 4;
+                    h_e = min(nh - 1, whi >> 4);
                 }
                 const unsigned span = (unsigned)(hi - lo);
                 const bool any_col = hi >= lo;
                 const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
+                const uint32_t p_tmem = tmem + lane_addr + kPCol + slot * (kBlockN / 2);
 
-                // ---- block max (unless it was taken while the previous item was exponentiated)
-                float mb;
-                if (have_mb) {
-                    mb = mb_next;
-                } else {
-                    ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
-                    if (!ok) break;
-                    tc_fence_after();
-                    float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                    for (int ch = ch_b; ch <= ch_e; ++ch) {
-                        uint32_t rr[32];
-                        tmem_ld32(s_tmem + ch * 32, rr);
-                        tmem_wait_ld();
-                        if (full) chunk_max<false>(rr, m4, ch, lo, span, any_col);
-                        else chunk_max<true>(rr, m4, ch, lo, span, any_col);
+                ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
+                if (!ok) break;
+                // the probability slot is free once the value MMAs of item-2 have completed
+                ok = mbar_wait_warp(bar(kBarPvDone + slot), ((item / kSlots) & 1) ^ 1, abort_flag, p.status, kErrSoftmax);
+                if (!ok) break;
+                tc_fence_after();
+                PSKV_TRACE_EVENT(20, item);
+
+                const float l_before = l;
+                float ls0 = 0.f, ls1 = 0.f, item_max = -INFINITY;
+                bool ovf = false;
+                // one 16-column piece: max, reference / overflow bookkeeping, exponentials, store
+                auto piece = [&](int h, const uint32_t (&rr)[16]) {
+                    uint32_t pk[8];
+                    if (h >= h_b && h <= h_e) {
+                        float v[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            v[c] = __uint_as_float(rr[c]);
+                            if (!full) v[c] = (any_col && (unsigned)(h * 16 + c - lo) <= span) ? v[c] : -INFINITY;
+                        }
+                        float m0 = fmaxf(v[0], v[1]), m1 = fmaxf(v[2], v[3]), m2 = fmaxf(v[4], v[5]), m3 = fmaxf(v[6], v[7]);
+                        m0 = fmaxf(m0, fmaxf(v[8], v[9]));
+                        m1 = fmaxf(m1, fmaxf(v[10], v[11]));
+                        m2 = fmaxf(m2, fmaxf(v[12], v[13]));
+                        m3 = fmaxf(m3, fmaxf(v[14], v[15]));
+                        const float cmax = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                        item_max = fmaxf(item_max, cmax);
+                        if (!m_set && cmax > -INFINITY) { m_ref = cmax * p.sl2; m_set = true; }
+                        ovf = ovf || (cmax * p.sl2 - m_ref > kRescaleGap);
+                        const float neg_m = -m_ref;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const float p0 = exp2f(fmaf(v[2 * c], p.sl2, neg_m));      // -inf stays -inf -> 0
+                            const float p1 = exp2f(fmaf(v[2 * c + 1], p.sl2, neg_m));
+                            ls0 += p0;
+                            ls1 += p1;
+                            pk[c] = pack_bf16x2(p0, p1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) pk[c] = 0u;
                     }
-                    mb = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-                }
-                PSKV_TRACE_EVENT(22, item);
-                const float mx = mb * p.sl2;
-                if (k == 0) {
-                    m_ref = (mb == -INFINITY) ? 0.f : mx;
-                } else {
-                    const bool need = mx > m_ref + kRescaleGap;
-                    if (__any_sync(0xffffffffu, need)) {
-                        // Rare: the running max jumped.  Rescale this row's O in tensor memory after the
-                        // previous item's P*V has completed, and before this item's P is handed over.
+                    tmem_st8(p_tmem + h * 8, pk);
+                };
+#pragma unroll 1
+                for (int pass = 0; pass < 2; ++pass) {
+                    uint32_t ra[16], rb[16];
+                    if (h_b <= h_e && h_b == 0) tmem_ld16(s_tmem, ra);
+#pragma unroll 1
+                    for (int h = 0; h < nh; h += 2) {
+                        tmem_wait_ld();
+                        if (h + 1 >= h_b && h + 1 <= h_e) tmem_ld16(s_tmem + (h + 1) * 16, rb);
+                        piece(h, ra);
+                        if (h + 1 < nh) {
+                            tmem_wait_ld();
+                            if (h + 2 >= h_b && h + 2 <= h_e) tmem_ld16(s_tmem + (h + 2) * 16, ra);
+                            piece(h + 1, rb);
+                        }
+                    }
+                    if (!__any_sync(0xffffffffu, ovf)) break;
+                    // Rare: this item's scores run far ahead of the reference.  Move the reference of the
+                    // affected rows to the item's max, rescale what has been accumulated so far (row sum
+                    // and, once the previous item's P*V has completed, O), and redo the item.
+                    const float m_new = ovf ? item_max * p.sl2 : m_ref;
+                    const float f = exp2f(m_ref - m_new);
+                    m_ref = m_new;
+                    l = l_before * f;
+                    ls0 = 0.f;
+                    ls1 = 0.f;
+                    ovf = false;
+                    if (k > 0) {
                         const int prev = item - 1;
                         ok = mbar_wait_warp(bar(kBarPvDone + prev % kSlots), (prev / kSlots) & 1, abort_flag,
                                             p.status, kErrSoftmax);
                         if (!ok) break;
                         tc_fence_after();
-                        const float f = need ? exp2f(m_ref - mx) : 1.f;
-                        if (need) { l *= f; m_ref = mx; }
 #pragma unroll 1
-                        for (int ch = 0; ch < D / 32; ++ch) {
-                            uint32_t o[32];
-                            tmem_ld32(tmem + lane_addr + kOCol + ch * 32, o);
+                        for (int ch = 0; ch < D / 16; ++ch) {
+                            uint32_t o[16];
+                            tmem_ld16(tmem + lane_addr + kOCol + ch * 16, o);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
-                            tmem_st32(tmem + lane_addr + kOCol + ch * 32, o);
-                        }
-                        tmem_wait_st();
-                    }
-                }
-
-                // ---- is the next item an unmasked prefix block whose scores have already arrived?
-                have_mb = false;
-                int nch_next = 0;
-                uint32_t s_tmem_next = 0;
-                if (item + 1 < total_items) {
-                    const int kn = (k + 1 == nitems) ? 0 : k + 1;
-                    if (kn < p.nblk_p && (prefix_block_rows(p, kn) & 31) == 0 &&
-                        min(kBlockN, p.P - kn * kBlockN) == prefix_block_rows(p, kn)) {
-                        const int slot_n = (item + 1) % kSlots;
-                        if (__all_sync(0xffffffffu, mbar_try_wait(bar(kBarSFull + slot_n), ((item + 1) / kSlots) & 1))) {
-                            tc_fence_after();
-                            have_mb = true;
-                            nch_next = prefix_block_rows(p, kn) >> 5;
-                            s_tmem_next = tmem + lane_addr + slot_n * kBlockN;
+                            for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                            tmem_st16(tmem + lane_addr + kOCol + ch * 16, o);
                         }
                     }
                 }
-
-                // ---- p = 2^(s * sl2 - m_ref), row sum, bf16 pairs back to tensor memory
-                const float neg_m = -m_ref;
-                float ls0 = 0.f, ls1 = 0.f;
-                float n4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                const int nloop = max(nch, nch_next);
-                for (int ch = 0; ch < nloop; ++ch) {
-                    uint32_t rr[32], rn[32], pk[16];
-                    const bool act = ch >= ch_b && ch <= ch_e && ch < nch;
-                    const bool nxt = ch < nch_next;
-                    if (act) tmem_ld32(s_tmem + ch * 32, rr);
-                    if (nxt) tmem_ld32(s_tmem_next + ch * 32, rn);
-                    if (act || nxt) tmem_wait_ld();
-                    if (act) {
-                        if (full) chunk_exp<false>(rr, pk, ls0, ls1, p.sl2, neg_m, ch, lo, span, any_col);
-                        else chunk_exp<true>(rr, pk, ls0, ls1, p.sl2, neg_m, ch, lo, span, any_col);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
-                    }
-                    if (nxt) chunk_max<false>(rn, n4, ch, 0, 0u, true);
-                    if (ch < nch) tmem_st16(s_tmem + ch * 16, pk);
-                }
-                mb_next = fmaxf(fmaxf(n4[0], n4[1]), fmaxf(n4[2], n4[3]));
+                if (!ok) break;
                 l += ls0 + ls1;
                 if (k == nitems - 1) ml[(tl & 1) * kTileM + row] = make_float2(l, m_ref);
                 PSKV_TRACE_EVENT(23, item);
@@ -656,7 +665,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 tc_fence_before();
                 __threadfence_block();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPReady + slot));
+                if (lane == 0) {
+                    mbar_arrive(bar(kBarSFree + slot));
+                    mbar_arrive(bar(kBarPReady + slot));
+                }
             }
         }
     } else {
