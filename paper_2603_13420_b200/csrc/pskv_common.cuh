@@ -33,6 +33,8 @@ struct BwdArgs {
 // General CUDA-core kernels (any S, P; d in {64,128}).
 cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream);
 cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream);
+// Recomputes the rows whose lse is NaN, if *redo_count != 0 (a device counter); `blocks` CTAs.
+cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream);
 
 // tcgen05/TMEM kernels.  `status_word` is the device status flag that bounded waits set.
 bool tc_fwd_supported(const Dims &d);

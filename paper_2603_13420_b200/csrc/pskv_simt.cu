@@ -84,16 +84,12 @@ __device__ __forceinline__ void stage_row(float *dst, const __nv_bfloat16 *row, 
     for (int e = 0; e < D / 32; ++e) dst[lane * (D / 32) + e] = v[e];
 }
 
-// Forward: one warp per query row (b,h,i); lanes take 32 keys at a time.
+// Forward for one query row (b,h,i) by one warp; lanes take 32 keys at a time.  `q_s` is this
+// warp's D floats of shared memory.
 template <int D>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-simt_fwd_kernel(FwdArgs a)
+__device__ __forceinline__ void fwd_row(const FwdArgs &a, long long row, float *q_s, int lane)
 {
-    __shared__ float q_s[kWarpsPerBlock][D];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Dims dm = a.dims;
-    const long long row = (long long)blockIdx.x * kWarpsPerBlock + warp;
-    if (row >= (long long)dm.B * dm.Hq * dm.S) return;
     const int i = (int)(row % dm.S);
     const int h = (int)((row / dm.S) % dm.Hq);
     const int b = (int)(row / ((long long)dm.S * dm.Hq));
@@ -103,7 +99,7 @@ simt_fwd_kernel(FwdArgs a)
     const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
     const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
 
-    stage_row<D>(q_s[warp], a.q + (size_t)row * D, lane);
+    stage_row<D>(q_s, a.q + (size_t)row * D, lane);
     __syncwarp();
 
     const float scale2 = a.scale * kLog2e;
@@ -118,7 +114,7 @@ simt_fwd_kernel(FwdArgs a)
         float s = -INFINITY;
         if (j < n_vis) {
             const __nv_bfloat16 *krow = (j < dm.P) ? pk + (size_t)j * D : sk + (size_t)(j - dm.P) * D;
-            s = scale2 * dot_row<D>(q_s[warp], krow);
+            s = scale2 * dot_row<D>(q_s, krow);
         }
         const float m_new = fmaxf(m, warp_max(s));  // finite: key j0 is always visible
         const float p = exp2f(s - m_new);           // 0 for lanes past n_vis
@@ -143,6 +139,36 @@ simt_fwd_kernel(FwdArgs a)
     for (int e = 0; e < D / 32; ++e) acc[e] *= inv;
     store_slice<D>(a.out + (size_t)row * D, lane, acc);
     if (lane == 0) a.lse[row] = (m + log2f(l)) * kLn2;
+    __syncwarp();
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_fwd_kernel(FwdArgs a)
+{
+    __shared__ float q_s[kWarpsPerBlock][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    if (row >= (long long)a.dims.B * a.dims.Hq * a.dims.S) return;
+    fwd_row<D>(a, row, q_s[warp], lane);
+}
+
+// Redo pass behind the tensor-core forward: that kernel subtracts no running max and marks the rare
+// rows whose exponents leave the safe range with a NaN lse; if any were marked, every row is
+// scanned and the marked ones are recomputed here.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_fwd_redo_kernel(FwdArgs a, const unsigned int *redo_count)
+{
+    __shared__ float q_s[kWarpsPerBlock][D];
+    if (*redo_count == 0u) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    for (long long row = (long long)blockIdx.x * kWarpsPerBlock + warp; row < rows;
+         row += (long long)gridDim.x * kWarpsPerBlock) {
+        const float v = a.lse[row];
+        if (v != v) fwd_row<D>(a, row, q_s[warp], lane);
+    }
 }
 
 // Backward, query side: one warp per query row; writes dq and D = <dout, out>.
@@ -285,6 +311,16 @@ cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream)
         simt_fwd_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
     else
         simt_fwd_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream)
+{
+    if (a.dims.d == 128)
+        simt_fwd_redo_kernel<128><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(a, redo_count);
+    else
+        simt_fwd_redo_kernel<64><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(a, redo_count);
     count_launches(1);
     return cudaGetLastError();
 }

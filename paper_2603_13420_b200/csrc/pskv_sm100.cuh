@@ -85,6 +85,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Bounded wait until a monotonically increasing shared-memory counter reaches `target`.
+__device__ __forceinline__ bool spin_wait_ge(volatile int *counter, int target, volatile int *abort_flag,
+                                             unsigned int *status_word, unsigned int code)
+{
+    if (*counter >= target) return true;
+    const long long start = clock64();
+    for (unsigned int spin = 1;; ++spin) {
+        if (*counter >= target) return true;
+        if ((spin & 63u) == 0u) {
+            if (*abort_flag != 0) return false;
+            if (clock64() - start > kWaitBudgetCycles) {
+                *abort_flag = 1;
+                atomicCAS(status_word, 0u, code);
+                return false;
+            }
+        }
+    }
+}
+
 // All 32 lanes wait (the warp's control flow stays uniform); true only if every lane saw the phase.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                                unsigned int *status_word, unsigned int code)

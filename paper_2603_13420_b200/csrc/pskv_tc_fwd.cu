@@ -9,15 +9,15 @@
 // partial results by their log-sum-exp), probabilities go back to tensor memory as bf16 and are
 // the A operand of the P*V contraction; `out` and `lse` are written once.
 //
-// Persistent CTA, one per SM, 12 warps:
+// Persistent CTA, one per SM, 16 warps:
 //   warp 0      TMA producer, score side (Q tile, prefix K blocks, suffix K of the tile)
 //   warp 1      tcgen05.mma issuer for the score blocks  S = Q K^T
 //   warp 2      tcgen05.mma issuer for the value blocks  O += P V   (owns the TMEM allocation)
 //   warp 3      TMA producer, value side (prefix V blocks, suffix V of the tile)
-//   warps 4-7   softmax: thread <-> query row (tensor-memory lane)
-//   warps 8-11  epilogue: O from tensor memory, normalise, bf16, shared-memory staging, TMA store
-// An "item" is one (tile, key block) pair; tensor memory holds two 128-column score slots, two
-// 64-column probability slots and the 128 columns of O.  Every wait is on an event produced by an earlier
+//   warps 4-11  softmax, two warpgroups on alternate items: thread <-> query row (TMEM lane)
+//   warps 12-15 epilogue: O from tensor memory, normalise, bf16, shared-memory staging, TMA store
+// An "item" is one (tile, key block) pair; tensor memory holds three 128-column score slots (the
+// bf16 probabilities of an item overwrite the first half of its own slot) and the 128 columns of O.  Every wait is on an event produced by an earlier
 // item of a role that never waits on the waiter, so no wait cycle can form; every wait is bounded.
 #include <string.h>
 
@@ -31,14 +31,13 @@ using namespace sm100;
 
 constexpr int kTileM = 128;    // rows of one MMA tile (tensor-memory lanes)
 constexpr int kBlockN = 128;   // keys per block
-constexpr int kSlots = 2;      // score slots (128 columns each) and probability slots (64 columns each)
-constexpr int kThreads = 384;
-constexpr int kPCol = kSlots * kBlockN;              // first tensor-memory column of the probability slots
-constexpr int kOCol = kPCol + kSlots * kBlockN / 2;  // first tensor-memory column of O
-// Probabilities are 2^(score - reference) with a per-row reference taken from the first keys the
-// row sees; bf16 and fp32 share their exponent range, so any reference within this many powers of
-// two of the true row max is exact, and only a larger lag triggers the (rare) rescale path.
-constexpr float kRescaleGap = 64.0f;
+constexpr int kSlots = 3;      // score slots of 128 columns; an item's probabilities overwrite its own scores
+constexpr int kThreads = 512;
+constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
+// Probabilities are 2^(s * sl2) with no max subtracted; rows whose largest exponent exceeds
+// kMaxLog2 or whose row sum falls below kMinRowSum are redone by the general kernel.
+constexpr float kMaxLog2 = 100.0f;
+constexpr float kMinRowSum = 7.8886090522101181e-31f;  // 2^-100
 constexpr int kMaxStages = 4;
 constexpr int kStagingBytes = kTileM * 128;  // one 64-column slab of the output tile
 constexpr int kMaxSmem = 232448;
@@ -46,7 +45,7 @@ constexpr int kMaxSmem = 232448;
 // Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
 // costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
 #ifdef PSKV_TRACE
-constexpr int kTraceWarps = 12, kTraceCap = 4096;
+constexpr int kTraceWarps = 16, kTraceCap = 4096;
 __device__ long long g_trace[kTraceWarps * kTraceCap * 2];
 __device__ unsigned int g_trace_n[kTraceWarps];
 #define PSKV_TRACE_DECL unsigned int trace_i_ = 0
@@ -78,6 +77,7 @@ enum : unsigned int {
 struct TcFwdParams {
     float *lse;
     unsigned int *status;
+    unsigned int *redo_count;  // rows marked for the general kernel (zeroed before the launch)
     float sl2;            // scale * log2(e)
     int B, Hq, Hkv, S, P, n_rep;
     int Rg;               // rows per candidate in one KV-head group: n_rep * S
@@ -113,8 +113,7 @@ enum {
     kBarStageFull,   // the epilogue warps have written a slab of the output tile (4 arrivals)
     kBarStageFree,   // the TMA stores of that slab have read it
     kBarSFull,                        // [kSlots] scores of an item are in tensor memory
-    kBarSFree = kBarSFull + kSlots,   // [kSlots] the softmax warps are done with a score slot (4 arrivals)
-    kBarPReady = kBarSFree + kSlots,  // [kSlots] probabilities written (4 arrivals)
+    kBarPReady = kBarSFull + kSlots,  // [kSlots] probabilities written (4 arrivals)
     kBarPvDone = kBarPReady + kSlots, // [kSlots] value MMAs of an item completed
     kBarKFull = kBarPvDone + kSlots,  // [stages]
     kBarVFull = kBarKFull + kMaxStages,
@@ -161,6 +160,15 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t sr
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+#ifndef PSKV_PIECE
+#define PSKV_PIECE 32
+#endif
+constexpr int kPiece = PSKV_PIECE;  // score columns a softmax thread handles per tensor-memory load
+__device__ __forceinline__ void tmem_ld_piece(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld16(taddr, r); }
+__device__ __forceinline__ void tmem_ld_piece(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld32(taddr, r); }
+__device__ __forceinline__ void tmem_st_piece(uint32_t taddr, const uint32_t (&r)[8]) { tmem_st8(taddr, r); }
+__device__ __forceinline__ void tmem_st_piece(uint32_t taddr, const uint32_t (&r)[16]) { tmem_st16(taddr, r); }
 
 // ---- softmax building blocks (one thread = one row; `rr` = 32 score columns of that row) -------
 
@@ -215,7 +223,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + p.off_misc + 4);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + p.off_misc);
-    float2 *ml = reinterpret_cast<float2 *>(smem + p.off_ml);  // (row sum, reference max) [2][128]
+    volatile int *ml_read = reinterpret_cast<volatile int *>(smem + p.off_misc + 16);  // [4] tiles read, per quadrant
+    float *ml = reinterpret_cast<float *>(smem + p.off_ml);  // partial row sums [tile parity][softmax group][128]
 
     if ((sbase & 1023u) != 0u) {  // the swizzled layouts need a 1024-byte aligned base
         if (tid == 0) atomicCAS(p.status, 0u, (unsigned int)kErrAlign);
@@ -227,10 +236,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
-            const bool four = (i >= kBarSFree && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
+            const bool four = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
             mbar_init(bar(i), four ? 4u : 1u);
         }
         *abort_flag = 0;
+        for (int i = 0; i < 4; ++i) ml_read[i] = 0;
         fence_barrier_init();
     }
     fence_proxy_async();
@@ -391,8 +401,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
         for (int i = 0; i < total_items && ok; ++i) {
             const int slot = i % kSlots;
-            // the score slot is free once the softmax warps have read item i-2 out of it
-            ok = mbar_wait_warp(bar(kBarSFree + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
+            // the slot is free once the value MMAs of item i-3 (which read P from it) have completed
+            ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
             if (!ok) break;
             if (k == 0) {
                 ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaQk);
@@ -488,7 +498,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (!ok) break;
             PSKV_TRACE_EVENT(11, i);
             tc_fence_after();
-            const uint32_t p_tmem = tmem + kPCol + slot * (kBlockN / 2);  // bf16 pairs: 8 columns per 16 keys
+            const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
             const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
             const int nk = n >> 4;
             const bool last_of_tile = k == nitems - 1;
@@ -516,33 +526,42 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
-    } else if (warp < 8) {
-        // ------------------------------------------------------------------ softmax warps (4..7)
-        // Each thread owns one query row (tensor-memory lane) and makes ONE pass over a score block,
-        // 16 columns at a time with the next 16 in flight: running max (for the reference and the
-        // overflow check), p = 2^(s*sl2 - m_ref), row sum, bf16 pairs into the item's probability
-        // slot.  m_ref is fixed by the first columns in which the row sees a key; scores stay intact
-        // in their slot, so the rare item whose max runs more than kRescaleGap ahead of m_ref is
-        // simply redone with a new reference after O and the row sum have been rescaled.  The loops
-        // are kept small on purpose: one warp per scheduler runs this code, and straight-line code
-        // longer than the instruction cache close to the scheduler stalls on fetch.
+    } else if (warp < 12) {
+        // ------------------------------------------------------------------ softmax warps (4..11)
+        // Two warpgroups take alternate items (group = item parity), so
+        // that one group's tensor-memory round trips hide behind the other's exponentials.  Each
+        // thread owns one query row (tensor-memory lane) and makes one pass over a score block, a
+        // piece of columns at a time with the next piece in flight: p = 2^(s * sl2), row sum, bf16
+        // pairs into the item's probability slot.  No running max is subtracted: bf16 and fp32
+        // share an 8-bit exponent, so the quotient O / l is exact to rounding for any row whose
+        // largest s * sl2 lies within +-kMaxLog2; a row outside that range (essentially never, it
+        // means logits beyond +-69 nats) is marked through a NaN row sum and redone afterwards by
+        // the general kernel with max subtraction.  The groups share no state; their partial row
+        // sums meet in the epilogue.
+        const int wg = (warp - 4) >> 2;
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-        int item = 0;
         bool ok = true;
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const int item0 = tl * nitems;
+            // my items of this tile: k with (item0 + k) parity == wg
+            const int k_first = ((item0 & 1) == wg) ? 0 : 1;
+            if (k_first >= nitems) continue;
+            const int k_last = k_first + ((nitems - 1 - k_first) & ~1);
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             const bool valid = row < t.rows;
             const int R = t.R0 + (valid ? row : 0);
             const int b = R / p.Rg, r = R - b * p.Rg;
             const int sfx_lo = (b - t.b_first) * p.S;   // first suffix column of this row's candidate
             const int sfx_hi = sfx_lo + (r % p.S);      // causal: suffix keys 0..i
-            float m_ref = 0.f, l = 0.f;
-            bool m_set = false;
+            float l = 0.f, smax = -INFINITY;
 #pragma unroll 1
-            for (int k = 0; k < nitems && ok; ++k, ++item) {
-                const int slot = item % kSlots;
+            for (int k = k_first; k < nitems && ok; k += 2) {
+                const int item = item0 + k, slot = item % kSlots;
+                // scores and (over their first half, piece by piece behind the reads) probabilities
+                const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
+                const uint32_t p_tmem = s_tmem;
                 // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
                 // blocks like real rows (their scores are finite and never stored) and see no suffix key.
                 int n, lo, hi;
@@ -555,139 +574,111 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     lo = valid ? sfx_lo : 1;
                     hi = valid ? sfx_hi : 0;
                 }
-                const int nh = n >> 4;  // 16-column pieces
-                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1);
+                const int nh = (n + kPiece - 1) / kPiece;
+                // `full`: no column of any piece needs masking (also none past n in the last piece)
+                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1) && (n % kPiece == 0);
                 int h_b = 0, h_e = nh - 1;  // pieces that hold a valid column of some row of this warp
                 if (!full) {
                     const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
                     const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
-                    h_b = wlo >> 4;
-                    h_e = min(nh - 1, whi >> 4);
+                    h_b = wlo / kPiece;
+                    h_e = min(nh - 1, whi / kPiece);
                 }
                 const unsigned span = (unsigned)(hi - lo);
                 const bool any_col = hi >= lo;
-                const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
-                const uint32_t p_tmem = tmem + lane_addr + kPCol + slot * (kBlockN / 2);
 
                 ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
-                if (!ok) break;
-                // the probability slot is free once the value MMAs of item-2 have completed
-                ok = mbar_wait_warp(bar(kBarPvDone + slot), ((item / kSlots) & 1) ^ 1, abort_flag, p.status, kErrSoftmax);
                 if (!ok) break;
                 tc_fence_after();
                 PSKV_TRACE_EVENT(20, item);
 
-                const float l_before = l;
-                float ls0 = 0.f, ls1 = 0.f, item_max = -INFINITY;
-                bool ovf = false;
-                // one 16-column piece: max, reference / overflow bookkeeping, exponentials, store
-                auto piece = [&](int h, const uint32_t (&rr)[16]) {
-                    uint32_t pk[8];
+                float ls0 = 0.f, ls1 = 0.f;
+                float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                auto piece = [&](int h, const uint32_t (&rr)[kPiece]) {
+                    uint32_t pk[kPiece / 2];
                     if (h >= h_b && h <= h_e) {
-                        float v[16];
+                        float v[kPiece];
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
+                        for (int c = 0; c < kPiece; ++c) {
                             v[c] = __uint_as_float(rr[c]);
-                            if (!full) v[c] = (any_col && (unsigned)(h * 16 + c - lo) <= span) ? v[c] : -INFINITY;
+                            if (!full) v[c] = (any_col && (unsigned)(h * kPiece + c - lo) <= span) ? v[c] : -INFINITY;
+                            m4[c & 3] = fmaxf(m4[c & 3], v[c]);
                         }
-                        float m0 = fmaxf(v[0], v[1]), m1 = fmaxf(v[2], v[3]), m2 = fmaxf(v[4], v[5]), m3 = fmaxf(v[6], v[7]);
-                        m0 = fmaxf(m0, fmaxf(v[8], v[9]));
-                        m1 = fmaxf(m1, fmaxf(v[10], v[11]));
-                        m2 = fmaxf(m2, fmaxf(v[12], v[13]));
-                        m3 = fmaxf(m3, fmaxf(v[14], v[15]));
-                        const float cmax = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-                        item_max = fmaxf(item_max, cmax);
-                        if (!m_set && cmax > -INFINITY) { m_ref = cmax * p.sl2; m_set = true; }
-                        ovf = ovf || (cmax * p.sl2 - m_ref > kRescaleGap);
-                        const float neg_m = -m_ref;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const float p0 = exp2f(fmaf(v[2 * c], p.sl2, neg_m));      // -inf stays -inf -> 0
-                            const float p1 = exp2f(fmaf(v[2 * c + 1], p.sl2, neg_m));
+                        for (int c = 0; c < kPiece / 2; ++c) {
+                            const float p0 = exp2f(v[2 * c] * p.sl2);  // -inf -> 0
+                            const float p1 = exp2f(v[2 * c + 1] * p.sl2);
                             ls0 += p0;
                             ls1 += p1;
                             pk[c] = pack_bf16x2(p0, p1);
                         }
                     } else {
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) pk[c] = 0u;
+                        for (int c = 0; c < kPiece / 2; ++c) pk[c] = 0u;
                     }
-                    tmem_st8(p_tmem + h * 8, pk);
+                    tmem_st_piece(p_tmem + h * (kPiece / 2), pk);
                 };
-#pragma unroll 1
-                for (int pass = 0; pass < 2; ++pass) {
-                    uint32_t ra[16], rb[16];
-                    if (h_b <= h_e && h_b == 0) tmem_ld16(s_tmem, ra);
+                {
+                    uint32_t ra[kPiece], rb[kPiece];
+                    if (h_b == 0 && h_e >= 0) tmem_ld_piece(s_tmem, ra);
 #pragma unroll 1
                     for (int h = 0; h < nh; h += 2) {
                         tmem_wait_ld();
-                        if (h + 1 >= h_b && h + 1 <= h_e) tmem_ld16(s_tmem + (h + 1) * 16, rb);
+                        if (h + 1 >= h_b && h + 1 <= h_e) tmem_ld_piece(s_tmem + (h + 1) * kPiece, rb);
                         piece(h, ra);
                         if (h + 1 < nh) {
                             tmem_wait_ld();
-                            if (h + 2 >= h_b && h + 2 <= h_e) tmem_ld16(s_tmem + (h + 2) * 16, ra);
+                            if (h + 2 >= h_b && h + 2 <= h_e) tmem_ld_piece(s_tmem + (h + 2) * kPiece, ra);
                             piece(h + 1, rb);
                         }
                     }
-                    if (!__any_sync(0xffffffffu, ovf)) break;
-                    // Rare: this item's scores run far ahead of the reference.  Move the reference of the
-                    // affected rows to the item's max, rescale what has been accumulated so far (row sum
-                    // and, once the previous item's P*V has completed, O), and redo the item.
-                    const float m_new = ovf ? item_max * p.sl2 : m_ref;
-                    const float f = exp2f(m_ref - m_new);
-                    m_ref = m_new;
-                    l = l_before * f;
-                    ls0 = 0.f;
-                    ls1 = 0.f;
-                    ovf = false;
-                    if (k > 0) {
-                        const int prev = item - 1;
-                        ok = mbar_wait_warp(bar(kBarPvDone + prev % kSlots), (prev / kSlots) & 1, abort_flag,
-                                            p.status, kErrSoftmax);
-                        if (!ok) break;
-                        tc_fence_after();
-#pragma unroll 1
-                        for (int ch = 0; ch < D / 16; ++ch) {
-                            uint32_t o[16];
-                            tmem_ld16(tmem + lane_addr + kOCol + ch * 16, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
-                            tmem_st16(tmem + lane_addr + kOCol + ch * 16, o);
-                        }
-                    }
                 }
-                if (!ok) break;
                 l += ls0 + ls1;
-                if (k == nitems - 1) ml[(tl & 1) * kTileM + row] = make_float2(l, m_ref);
+                smax = fmaxf(smax, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+                if (k == k_last) {
+                    // hand this group's partial row sum to the epilogue; the buffer of tile tl-2 must
+                    // have been read first
+                    if (tl >= 2) {
+                        ok = __all_sync(0xffffffffu, spin_wait_ge(ml_read + (warp & 3), tl - 1, abort_flag, p.status,
+                                                                  kErrSoftmax));
+                        if (!ok) break;
+                        __threadfence_block();
+                    }
+                    ml[((tl & 1) * 2 + wg) * kTileM + row] = (smax * p.sl2 > kMaxLog2) ? __int_as_float(0x7fc00000) : l;
+                }
                 PSKV_TRACE_EVENT(23, item);
                 tmem_wait_st();
                 tc_fence_before();
                 __threadfence_block();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(bar(kBarSFree + slot));
-                    mbar_arrive(bar(kBarPReady + slot));
-                }
+                if (lane == 0) mbar_arrive(bar(kBarPReady + slot));
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue warps (8..11)
+        // ------------------------------------------------------------------ epilogue warps (12..15)
         const int ew = warp & 3;
         const int row = 32 * ew + lane;
         const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
         const uint32_t stage = sbase + p.off_stage;
-        const bool issuer = warp == 8;  // this warp's elected lane issues the TMA stores
+        const bool issuer = warp == 12;  // this warp's elected lane issues the TMA stores
         if (issuer && lane == 0) prefetch_tensormap(&tm_out);
         bool ok = true;
+#pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             ok = mbar_wait_warp(bar(kBarOFull), tl & 1, abort_flag, p.status, kErrEpilogue);
             if (!ok) break;
             PSKV_TRACE_EVENT(30, tl);
             tc_fence_after();
-            const float2 lm = ml[(tl & 1) * kTileM + row];
-            const float inv = 1.f / lm.x;
+            // row sum = the partial sums of the softmax groups that had an item in this tile
+            const int par0 = (tl * nitems) & 1;
+            float lsum = ml[((tl & 1) * 2 + par0) * kTileM + row];
+            if (nitems > 1) lsum += ml[((tl & 1) * 2 + (par0 ^ 1)) * kTileM + row];
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) ml_read[ew] = tl + 1;  // this warp's rows of the tile's partial sums have been read
+            const bool row_ok = lsum >= kMinRowSum;  // false for NaN (marked row) and for underflow
+            const float inv = 1.f / lsum;
             uint32_t ob[D / 2];  // the normalised row as bf16 pairs
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
@@ -701,12 +692,15 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarOFree));
-            if (row < t.rows) {
+            const bool stored = row < t.rows;
+            if (stored) {
                 const int R = t.R0 + row;
                 const int b = R / p.Rg, r = R - b * p.Rg;
                 const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
-                p.lse[grow] = (lm.y + log2f(lm.x)) * kLn2;
+                p.lse[grow] = row_ok ? log2f(lsum) * kLn2 : __int_as_float(0x7fc00000);
             }
+            const unsigned bad = __ballot_sync(0xffffffffu, stored && !row_ok);
+            if (bad != 0u && lane == 0) atomicAdd(p.redo_count, (unsigned int)__popc(bad));
             // out: one 64-column slab at a time through the swizzled staging buffer, then TMA stores
             const int nseg = t.rows / p.seg_rows;
 #pragma unroll
@@ -878,7 +872,8 @@ int sm_count()
 }
 
 template <int D>
-cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_word, cudaStream_t stream)
+cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsigned int *status_word,
+                   cudaStream_t stream)
 {
     const Dims &dm = a.dims;
     const int Rg = dm.n_rep * dm.S;
@@ -915,6 +910,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_
     TcFwdParams p;
     p.lse = a.lse;
     p.status = status_word;
+    p.redo_count = static_cast<unsigned int *>(workspace);
     p.sl2 = a.scale * kLog2e;
     p.B = dm.B; p.Hq = dm.Hq; p.Hkv = dm.Hkv; p.S = dm.S; p.P = dm.P; p.n_rep = dm.n_rep;
     p.Rg = Rg;
@@ -937,11 +933,16 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, unsigned int *status_
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    cudaError_t e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), stream);
+    if (e != cudaSuccess) return e;
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
     tc_fwd_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail,
                                                                   tm_sk, tm_sv, p);
     count_launches(1);
-    return cudaGetLastError();
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    // rows the tensor-core kernel marked (NaN lse) are recomputed with max subtraction
+    return launch_simt_fwd_redo(a, p.redo_count, sm_count(), stream);
 }
 
 }  // namespace
@@ -972,13 +973,14 @@ bool tc_fwd_supported(const Dims &dm)
     return plan_tiles(dm).ok;
 }
 
-size_t tc_fwd_workspace_bytes(const Dims &) { return 0; }
+size_t tc_fwd_workspace_bytes(const Dims &) { return 256; }  // the redo counter
 
-cudaError_t launch_tc_fwd(const FwdArgs &a, void *, unsigned int *status_word, cudaStream_t stream)
+cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word, cudaStream_t stream)
 {
     const TilePlan plan = plan_tiles(a.dims);
     if (!plan.ok) return cudaErrorInvalidValue;
-    return a.dims.d == 128 ? launch<128>(a, plan, status_word, stream) : launch<64>(a, plan, status_word, stream);
+    return a.dims.d == 128 ? launch<128>(a, plan, workspace, status_word, stream)
+                           : launch<64>(a, plan, workspace, status_word, stream);
 }
 
 }  // namespace pskv

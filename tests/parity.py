@@ -98,14 +98,18 @@ def oracle_bwd(t, scale, cand=None):
                            scale)
 
 
-def fwd_parity(w, t=None, cand=None):
-    """Forward parity for workload w (optionally only the listed candidates against the oracle)."""
+def fwd_parity(w, t=None, cand=None, strict_abs=True):
+    """Forward parity for workload w (optionally only the listed candidates against the oracle).
+
+    strict_abs: apply the absolute bar (2e-2 / 2e-3) as stated; it is meant for outputs that average
+    over hundreds of keys.  Shapes with a handful of keys give |out| up to ~4, where the bf16
+    rounding of the result alone is 8e-3, so they take the bar relative to max(1, max|ref|)."""
     if t is None:
         t = pskv_inputs.make_inputs(w)
     out, lse, _ = run_fwd_gpu(t, w.scale)
     ref_out, ref_lse = oracle_fwd(t, w.scale, cand)
     sl = slice(None) if cand is None else cand
-    s = check_tensor("out", to_f64(out[sl]), ref_out, strict_abs=True)
+    s = check_tensor("out", to_f64(out[sl]), ref_out, strict_abs=strict_abs)
     s["lse_rel"] = check_lse(to_f64(lse[sl]), ref_lse)
     return s
 
