@@ -33,6 +33,10 @@ struct BwdArgs {
 // General CUDA-core kernels (any S, P; d in {64,128}).
 cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream);
 cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream);
+// Pieces of the backward the tensor-core path reuses: D = <dout, out> per row into a.row_dot, and
+// dk_suffix / dv_suffix (needs row_dot and lse).
+cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream);
+cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
 // Recomputes the rows whose lse is NaN, if *redo_count != 0 (a device counter); `blocks` CTAs.
 cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream);
 

@@ -235,6 +235,24 @@ simt_bwd_dq_kernel(BwdArgs a)
     store_slice<D>(a.dq + (size_t)row * D, lane, acc);
 }
 
+// D = <dout, out> for every query row: one warp per row.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_row_dot_kernel(BwdArgs a)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    if (row >= (long long)a.dims.B * a.dims.Hq * a.dims.S) return;
+    float o[D / 32], g[D / 32];
+    load_slice<D>(a.out + (size_t)row * D, lane, o);
+    load_slice<D>(a.dout + (size_t)row * D, lane, g);
+    float acc = 0.f;
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) acc = fmaf(o[e], g[e], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) a.row_dot[row] = acc;
+}
+
 // Backward, key side: one warp per suffix key (b,g,t); sums over the n_rep heads of the group
 // and the rows i >= t that see the key.  Needs row_dot from the query-side kernel.
 template <int D>
@@ -321,6 +339,28 @@ cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_coun
         simt_fwd_redo_kernel<128><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(a, redo_count);
     else
         simt_fwd_redo_kernel<64><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(a, redo_count);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream)
+{
+    const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    if (a.dims.d == 128)
+        simt_row_dot_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+    else
+        simt_row_dot_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream)
+{
+    const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.S;
+    if (a.dims.d == 128)
+        simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
+    else
+        simt_bwd_dkv_kernel<64><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
     count_launches(1);
     return cudaGetLastError();
 }

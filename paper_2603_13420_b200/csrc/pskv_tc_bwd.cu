@@ -1,7 +1,734 @@
-// placeholder until the tcgen05 backward lands
+// Shared-prefix attention backward, query side, for sm_100a (tcgen05 / TMEM / TMA):
+//   dQ = scale * sum_j dS_j K_j   over the shared prefix keys and the visible suffix keys,
+//   dS = P o (dP - D),  P = exp(S - lse),  S = scale Q K^T,  dP = dO V^T,  D = <dO, O>.
+// The prefix K/V is frozen (Sec. 4.2): no gradient flows into it, so the prefix part costs three
+// contractions per block instead of five.  Tiling, operand staging and roles mirror the forward
+// kernel: 128-row tiles of the flat row list of a KV head, prefix blocks resident in shared memory
+// when they fit, one suffix block per tile with the block-diagonal causal mask.
+//
+// Persistent CTA, one per SM, 12 warps:
+//   warp 0      TMA producer: Q tile, prefix K blocks, suffix K
+//   warp 1      tcgen05.mma issuer: S = Q K^T and dP = dO V^T of every item
+//   warp 2      tcgen05.mma issuer: dQ += dS K  (owns the TMEM allocation)
+//   warp 3      TMA producer: dO tile, prefix V blocks, suffix V
+//   warps 4-7   element-wise: thread <-> query row; dS = exp2(S*sl2 - lse2) * (dP - D) as bf16
+//   warps 8-11  epilogue: dQ from tensor memory, * scale, bf16, staging, TMA store
+// Tensor memory: two 128-column S slots (dS overwrites the first half of its own slot), one dP
+// slot, and the 128 columns of dQ.  dK_suffix / dV_suffix and D are computed by the general
+// kernels around this one.  Every wait is bounded.
+#include <string.h>
+
 #include "pskv_common.cuh"
+#include "pskv_sm100.cuh"
+#include "pskv_tc_common.cuh"
+
 namespace pskv {
-bool tc_bwd_supported(const Dims &) { return false; }
-size_t tc_bwd_workspace_bytes(const Dims &) { return 0; }
-cudaError_t launch_tc_bwd(const BwdArgs &, void *, unsigned int *, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+using namespace sm100;
+
+constexpr int kSlots = 2;
+constexpr int kThreads = 384;
+constexpr int kDpCol = kSlots * kBlockN;
+constexpr int kDqCol = kDpCol + kBlockN;
+constexpr int kMaxStages = 4;
+constexpr int kPieceB = 16;  // columns per tensor-memory load of the element-wise warps
+
+enum : unsigned int {
+    kErrProdA = 0x201, kErrProdB = 0x202, kErrMmaS = 0x203, kErrMmaDq = 0x204, kErrElem = 0x205,
+    kErrEpi = 0x206, kErrAlign = 0x207
+};
+
+struct TcBwdParams {
+    const float *lse;      // [B*Hq*S] from the forward pass
+    const float *row_dot;  // [B*Hq*S] D = <dout, out>
+    unsigned int *status;
+    float sl2;             // scale * log2(e)
+    float scale;
+    int B, Hq, Hkv, S, P, n_rep;
+    int Rg, tile_rows, seg_rows, tiles_per_group, total_tiles;
+    int nblk_p, tail_rows, resident, stages, sfx_rows;
+    int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc;
+};
+
+template <int D>
+struct Cfg {
+    static constexpr int kSlabs = D / 64;
+    static constexpr int kSlabBytes = kTileM * 128;
+    static constexpr int kTileBytes = kSlabs * kSlabBytes;
+};
+
+enum {
+    kBarQFull = 0,
+    kBarQkFree,     // every S MMA of a tile completed: the Q buffer is free
+    kBarDoFull,
+    kBarDvFree,     // every dP MMA of a tile completed: dO, suffix V (and resident prefix V) are free
+    kBarSKFull,
+    kBarSVFull,
+    kBarDqFull,     // every dQ MMA of a tile completed: dQ is final, suffix K (and resident prefix K) are free
+    kBarDqFree,     // the epilogue has read dQ out (4 arrivals)
+    kBarStageFull,  // (4 arrivals)
+    kBarStageFree,
+    kBarDpFull,     // dP of an item is in tensor memory
+    kBarDpFree,     // the element-wise warps have read dP (4 arrivals)
+    kBarSFull,                        // [kSlots]
+    kBarDsReady = kBarSFull + kSlots, // [kSlots] dS written (4 arrivals)
+    kBarDqDone = kBarDsReady + kSlots, // [kSlots] the dQ MMAs of an item completed: its S slot is free
+    kBarKFull = kBarDqDone + kSlots,
+    kBarVFull = kBarKFull + kMaxStages,
+    kBarKFree = kBarVFull + kMaxStages,
+    kBarVFree = kBarKFree + kMaxStages,
+    kNumBars = kBarVFree + kMaxStages
+};
+constexpr int kBarBytes = 512;
+static_assert(kNumBars * 8 <= kBarBytes, "barrier area");
+
+__device__ __forceinline__ int prefix_block_rows(const TcBwdParams &p, int k)
+{
+    return k == p.nblk_p - 1 ? p.tail_rows : kBlockN;
 }
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
+                 const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_pk,
+                 const __grid_constant__ CUtensorMap tm_pv, const __grid_constant__ CUtensorMap tm_pk_tail,
+                 const __grid_constant__ CUtensorMap tm_pv_tail, const __grid_constant__ CUtensorMap tm_sk,
+                 const __grid_constant__ CUtensorMap tm_sv, const TcBwdParams p)
+{
+    using C = Cfg<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+    PSKV_TRACE_DECL;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + p.off_bar;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + p.off_misc + 4);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + p.off_misc);
+
+    if ((sbase & 1023u) != 0u) {
+        if (tid == 0) atomicCAS(p.status, 0u, (unsigned int)kErrAlign);
+        return;
+    }
+    // padding rows of the operand buffers must hold finite values (0 * NaN would poison dQ)
+    for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) {
+        for (int i = 0; i < kNumBars; ++i) {
+            const bool four = i == kBarDqFree || i == kBarStageFull || i == kBarDpFree ||
+                              (i >= kBarDsReady && i < kBarDsReady + kSlots);
+            mbar_init(bar(i), four ? 4u : 1u);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    fence_proxy_async();
+    __syncthreads();
+    if (warp == 2) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int t_begin = (int)((long long)blockIdx.x * p.total_tiles / gridDim.x);
+    const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
+    const int n_tiles = t_end - t_begin;
+    const int nitems = p.nblk_p + 1;
+    const int g_first = t_begin / p.tiles_per_group;
+    const int sfx_slab = p.sfx_rows * 128;
+    const int tail_slab = p.tail_rows * 128;
+    const uint32_t stages = (uint32_t)p.stages;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer: Q, K
+        if (lane == 0) {
+            prefetch_tensormap(&tm_q);
+            prefetch_tensormap(&tm_sk);
+            if (p.P > 0) { prefetch_tensormap(&tm_pk); prefetch_tensormap(&tm_pk_tail); }
+        }
+        uint32_t kload = 0;
+        bool ok = true;
+#pragma unroll 1
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdA);
+            if (!ok) break;
+            const int nseg = t.rows / p.seg_rows;
+            if (elect_one_sync()) {
+                mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
+                for (int s = 0; s < nseg; ++s) {
+                    const int R = t.R0 + s * p.seg_rows;
+                    const int b = R / p.Rg, r = R - b * p.Rg;
+                    for (int sl = 0; sl < C::kSlabs; ++sl)
+                        tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
+                                    bar(kBarQFull), sl * 64, r, t.g, b);
+                }
+            }
+            __syncwarp();
+            if (!p.resident) {
+#pragma unroll 1
+                for (int k = 0; k < p.nblk_p; ++k) {
+                    const uint32_t ks = kload % stages;
+                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / stages) & 1) ^ 1, abort_flag, p.status, kErrProdA);
+                    if (!ok) break;
+                    const bool tail = k == p.nblk_p - 1;
+                    const int slab = tail ? tail_slab : C::kSlabBytes;
+                    if (elect_one_sync()) {
+                        mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(C::kSlabs * slab));
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_3d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
+                                        bar(kBarKFull + ks), sl * 64, k * kBlockN, t.g);
+                    }
+                    __syncwarp();
+                    ++kload;
+                }
+                if (!ok) break;
+            }
+            // suffix K (and resident prefix K) are read by the dQ MMAs too: free once dQ of the
+            // previous tile is final
+            if (tl > 0) {
+                ok = mbar_wait_warp(bar(kBarDqFull), (tl - 1) & 1, abort_flag, p.status, kErrProdA);
+                if (!ok) break;
+            }
+            if (p.resident && t.first_of_g && elect_one_sync()) {
+                for (int k = 0; k < p.nblk_p; ++k) {
+                    const bool tail = k == p.nblk_p - 1;
+                    const int slab = tail ? tail_slab : C::kSlabBytes;
+                    mbar_arrive_expect_tx(bar(kBarKFull + k), (uint32_t)(C::kSlabs * slab));
+                    for (int sl = 0; sl < C::kSlabs; ++sl)
+                        tma_load_3d(sbase + p.off_pk + k * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
+                                    bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
+                }
+            }
+            __syncwarp();
+            if (elect_one_sync()) {
+                mbar_arrive_expect_tx(bar(kBarSKFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
+                for (int c = 0; c < t.nc; ++c)
+                    for (int sl = 0; sl < C::kSlabs; ++sl)
+                        tma_load_4d(sbase + p.off_sk + sl * sfx_slab + c * p.S * 128, &tm_sk, bar(kBarSKFull),
+                                    sl * 64, 0, t.g, t.b_first + c);
+            }
+            __syncwarp();
+        }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ producer: dO, V
+        if (lane == 0) {
+            prefetch_tensormap(&tm_do);
+            prefetch_tensormap(&tm_sv);
+            if (p.P > 0) { prefetch_tensormap(&tm_pv); prefetch_tensormap(&tm_pv_tail); }
+        }
+        uint32_t vload = 0;
+        bool ok = true;
+#pragma unroll 1
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            ok = mbar_wait_warp(bar(kBarDvFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdB);
+            if (!ok) break;
+            const int nseg = t.rows / p.seg_rows;
+            if (elect_one_sync()) {
+                mbar_arrive_expect_tx(bar(kBarDoFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
+                for (int s = 0; s < nseg; ++s) {
+                    const int R = t.R0 + s * p.seg_rows;
+                    const int b = R / p.Rg, r = R - b * p.Rg;
+                    for (int sl = 0; sl < C::kSlabs; ++sl)
+                        tma_load_4d(sbase + p.off_do + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_do,
+                                    bar(kBarDoFull), sl * 64, r, t.g, b);
+                }
+                if (p.resident && t.first_of_g) {
+                    for (int k = 0; k < p.nblk_p; ++k) {
+                        const bool tail = k == p.nblk_p - 1;
+                        const int slab = tail ? tail_slab : C::kSlabBytes;
+                        mbar_arrive_expect_tx(bar(kBarVFull + k), (uint32_t)(C::kSlabs * slab));
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
+                                        bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
+                    }
+                }
+                mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
+                for (int c = 0; c < t.nc; ++c)
+                    for (int sl = 0; sl < C::kSlabs; ++sl)
+                        tma_load_4d(sbase + p.off_sv + sl * sfx_slab + c * p.S * 128, &tm_sv, bar(kBarSVFull),
+                                    sl * 64, 0, t.g, t.b_first + c);
+            }
+            __syncwarp();
+            if (!p.resident) {
+#pragma unroll 1
+                for (int k = 0; k < p.nblk_p; ++k) {
+                    const uint32_t vs = vload % stages;
+                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / stages) & 1) ^ 1, abort_flag, p.status, kErrProdB);
+                    if (!ok) break;
+                    const bool tail = k == p.nblk_p - 1;
+                    const int slab = tail ? tail_slab : C::kSlabBytes;
+                    if (elect_one_sync()) {
+                        mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
+                                        bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                    }
+                    __syncwarp();
+                    ++vload;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ S = Q K^T, dP = dO V^T
+        const int total_items = n_tiles * nitems;
+        int tl = 0, k = 0;
+        uint32_t kuse = 0, vuse = 0;
+        TileInfo t = tile_info(p, t_begin, t_begin);
+        const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
+        const uint64_t do_desc = make_smem_desc(sbase + p.off_do, 0, 1024);
+        bool ok = true;
+#pragma unroll 1
+        for (int i = 0; i < total_items && ok; ++i) {
+            const int slot = i % kSlots;
+            const bool prefix = k < p.nblk_p;
+            const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
+            const int slab = prefix ? n * 128 : sfx_slab;
+            const bool last_of_tile = k == nitems - 1;
+            const bool ring = prefix && !p.resident;
+            const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
+            const uint64_t slab16 = (uint64_t)(slab >> 4);
+            // ---- S: the slot is free once the dQ MMAs of item i-2 have completed
+            ok = mbar_wait_warp(bar(kBarDqDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaS);
+            if (!ok) break;
+            if (k == 0) ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaS);
+            if (!ok) break;
+            uint32_t kaddr;
+            if (prefix) {
+                if (p.resident) {
+                    if (t.first_of_g)
+                        ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
+                    kaddr = sbase + p.off_pk + k * C::kTileBytes;
+                } else {
+                    const uint32_t ks = kuse % stages;
+                    ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / stages) & 1, abort_flag, p.status, kErrMmaS);
+                    kaddr = sbase + p.off_pk + ks * C::kTileBytes;
+                }
+            } else {
+                ok = mbar_wait_warp(bar(kBarSKFull), tl & 1, abort_flag, p.status, kErrMmaS);
+                kaddr = sbase + p.off_sk;
+            }
+            if (!ok) break;
+            tc_fence_after();
+            {
+                const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
+                const uint32_t d_tmem = tmem + slot * kBlockN;
+                if (elect_one_sync()) {
+#pragma unroll
+                    for (int ks16 = 0; ks16 < D / 16; ++ks16) {
+                        const uint64_t qoff = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
+                        const uint64_t koff = (uint64_t)(ks16 >> 2) * slab16 + (uint64_t)(((ks16 & 3) * 32) >> 4);
+                        mma_ss(d_tmem, q_desc + qoff, k_desc + koff, idesc, ks16 > 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar(kBarSFull + slot));
+                    if (last_of_tile) tc_commit(bar(kBarQkFree));
+                }
+                __syncwarp();
+            }
+            // ---- dP: its single slot is free once the element-wise warps have read item i-1
+            ok = mbar_wait_warp(bar(kBarDpFree), (i & 1) ^ 1, abort_flag, p.status, kErrMmaS);
+            if (!ok) break;
+            if (k == 0) ok = mbar_wait_warp(bar(kBarDoFull), tl & 1, abort_flag, p.status, kErrMmaS);
+            if (!ok) break;
+            uint32_t vaddr;
+            if (prefix) {
+                if (p.resident) {
+                    if (t.first_of_g)
+                        ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
+                    vaddr = sbase + p.off_pv + k * C::kTileBytes;
+                } else {
+                    const uint32_t vs = vuse % stages;
+                    ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / stages) & 1, abort_flag, p.status, kErrMmaS);
+                    vaddr = sbase + p.off_pv + vs * C::kTileBytes;
+                }
+            } else {
+                ok = mbar_wait_warp(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMmaS);
+                vaddr = sbase + p.off_sv;
+            }
+            if (!ok) break;
+            tc_fence_after();
+            {
+                const uint64_t v_desc = make_smem_desc(vaddr, 0, 1024);
+                if (elect_one_sync()) {
+#pragma unroll
+                    for (int ks16 = 0; ks16 < D / 16; ++ks16) {
+                        const uint64_t aoff = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
+                        const uint64_t voff = (uint64_t)(ks16 >> 2) * slab16 + (uint64_t)(((ks16 & 3) * 32) >> 4);
+                        mma_ss(tmem + kDpCol, do_desc + aoff, v_desc + voff, idesc, ks16 > 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar(kBarDpFull));
+                    if (ring) tc_commit(bar(kBarVFree + (vuse % stages)));
+                    if (last_of_tile) tc_commit(bar(kBarDvFree));
+                }
+                __syncwarp();
+            }
+            if (ring) { ++kuse; ++vuse; }
+            if (++k == nitems) {
+                k = 0;
+                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ dQ += dS K
+        const int total_items = n_tiles * nitems;
+        int tl = 0, k = 0;
+        uint32_t kuse = 0;
+        TileInfo t = tile_info(p, t_begin, t_begin);
+        const uint32_t idesc_dq = make_idesc_bf16(kTileM, D, 1);
+        bool ok = true;
+#pragma unroll 1
+        for (int i = 0; i < total_items && ok; ++i) {
+            const int slot = i % kSlots;
+            const bool prefix = k < p.nblk_p;
+            const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
+            const int slab = prefix ? n * 128 : sfx_slab;
+            const bool last_of_tile = k == nitems - 1;
+            const bool ring = prefix && !p.resident;
+            ok = mbar_wait_warp(bar(kBarDsReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaDq);
+            if (!ok) break;
+            if (k == 0 && tl > 0) {
+                ok = mbar_wait_warp(bar(kBarDqFree), (tl - 1) & 1, abort_flag, p.status, kErrMmaDq);
+                if (!ok) break;
+            }
+            uint32_t kaddr;
+            if (prefix) kaddr = sbase + p.off_pk + (p.resident ? (uint32_t)k : kuse % stages) * C::kTileBytes;
+            else kaddr = sbase + p.off_sk;
+            tc_fence_after();
+            const uint32_t ds_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
+            const uint64_t k_desc = make_smem_desc(kaddr, (uint32_t)slab, 1024);  // K as [keys][d]: d contiguous
+            const int nk = n >> 4;
+            const uint32_t acc0 = k > 0 ? 1u : 0u;
+            if (elect_one_sync()) {
+#pragma unroll
+                for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
+                    if (ks16 < nk)
+                        mma_ts(tmem + kDqCol, ds_tmem + ks16 * 8, k_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_dq,
+                               ks16 > 0 ? 1u : acc0);
+                }
+                tc_commit(bar(kBarDqDone + slot));
+                if (ring) tc_commit(bar(kBarKFree + (kuse % stages)));
+                if (last_of_tile) tc_commit(bar(kBarDqFull));
+            }
+            __syncwarp();
+            if (ring) ++kuse;
+            if (++k == nitems) {
+                k = 0;
+                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+            }
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------------ element-wise warps
+        const int row = 32 * (warp & 3) + lane;
+        const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+        int item = 0;
+        bool ok = true;
+#pragma unroll 1
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            const bool valid = row < t.rows;
+            const int R = t.R0 + (valid ? row : 0);
+            const int b = R / p.Rg, r = R - b * p.Rg;
+            const int sfx_lo = (b - t.b_first) * p.S;
+            const int sfx_hi = sfx_lo + (r % p.S);
+            const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
+            // padding rows: lse = +inf makes every probability (and so every dS) zero
+            const float neg_lse2 = valid ? -p.lse[grow] * kLog2e : -INFINITY;
+            const float drow = valid ? p.row_dot[grow] : 0.f;
+#pragma unroll 1
+            for (int k = 0; k < nitems && ok; ++k, ++item) {
+                const int slot = item % kSlots;
+                int n, lo, hi;
+                if (k < p.nblk_p) {
+                    n = prefix_block_rows(p, k);
+                    lo = 0;
+                    hi = min(kBlockN, p.P - k * kBlockN) - 1;
+                } else {
+                    n = t.n_sfx;
+                    lo = valid ? sfx_lo : 1;
+                    hi = valid ? sfx_hi : 0;
+                }
+                const int nh = n / kPieceB;
+                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1);
+                int h_b = 0, h_e = nh - 1;
+                if (!full) {
+                    const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
+                    const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
+                    h_b = wlo / kPieceB;
+                    h_e = min(nh - 1, whi / kPieceB);
+                }
+                const unsigned span = (unsigned)(hi - lo);
+                const bool any_col = hi >= lo;
+                const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
+                const uint32_t dp_tmem = tmem + lane_addr + kDpCol;
+
+                ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrElem);
+                if (!ok) break;
+                ok = mbar_wait_warp(bar(kBarDpFull), item & 1, abort_flag, p.status, kErrElem);
+                if (!ok) break;
+                tc_fence_after();
+
+                auto piece = [&](int h, const uint32_t (&rs)[kPieceB], const uint32_t (&rd)[kPieceB]) {
+                    uint32_t pk[kPieceB / 2];
+                    if (h >= h_b && h <= h_e) {
+                        float ds[kPieceB];
+#pragma unroll
+                        for (int c = 0; c < kPieceB; ++c) {
+                            float x = fmaf(__uint_as_float(rs[c]), p.sl2, neg_lse2);
+                            if (!full) x = (any_col && (unsigned)(h * kPieceB + c - lo) <= span) ? x : -INFINITY;
+                            ds[c] = exp2f(x) * (__uint_as_float(rd[c]) - drow);
+                        }
+#pragma unroll
+                        for (int c = 0; c < kPieceB / 2; ++c) pk[c] = pack_bf16x2(ds[2 * c], ds[2 * c + 1]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < kPieceB / 2; ++c) pk[c] = 0u;
+                    }
+                    tmem_st8(s_tmem + h * (kPieceB / 2), pk);
+                };
+                {
+                    uint32_t sa[kPieceB], sb[kPieceB], da[kPieceB], db[kPieceB];
+                    if (h_b == 0 && h_e >= 0) { tmem_ld16(s_tmem, sa); tmem_ld16(dp_tmem, da); }
+#pragma unroll 1
+                    for (int h = 0; h < nh; h += 2) {
+                        tmem_wait_ld();
+                        if (h + 1 >= h_b && h + 1 <= h_e) {
+                            tmem_ld16(s_tmem + (h + 1) * kPieceB, sb);
+                            tmem_ld16(dp_tmem + (h + 1) * kPieceB, db);
+                        }
+                        piece(h, sa, da);
+                        if (h + 1 < nh) {
+                            tmem_wait_ld();
+                            if (h + 2 >= h_b && h + 2 <= h_e) {
+                                tmem_ld16(s_tmem + (h + 2) * kPieceB, sa);
+                                tmem_ld16(dp_tmem + (h + 2) * kPieceB, da);
+                            }
+                            piece(h + 1, sb, db);
+                        }
+                    }
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar(kBarDpFree));
+                    mbar_arrive(bar(kBarDsReady + slot));
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps (8..11)
+        const int ew = warp & 3;
+        const int row = 32 * ew + lane;
+        const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
+        const uint32_t stage = sbase + p.off_stage;
+        const bool issuer = warp == 8;
+        if (issuer && lane == 0) prefetch_tensormap(&tm_dq);
+        bool ok = true;
+#pragma unroll 1
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            ok = mbar_wait_warp(bar(kBarDqFull), tl & 1, abort_flag, p.status, kErrEpi);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t ob[D / 2];
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_addr + kDqCol + ch * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                    ob[ch * 16 + c] = pack_bf16x2(__uint_as_float(o[2 * c]) * p.scale, __uint_as_float(o[2 * c + 1]) * p.scale);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarDqFree));
+            const int nseg = t.rows / p.seg_rows;
+#pragma unroll
+            for (int sl = 0; sl < C::kSlabs; ++sl) {
+                const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
+                ok = mbar_wait_warp(bar(kBarStageFree), (round & 1) ^ 1, abort_flag, p.status, kErrEpi);
+                if (!ok) break;
+                uint8_t *srow = smem + p.off_stage + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(ob[sl * 32 + 4 * c], ob[sl * 32 + 4 * c + 1], ob[sl * 32 + 4 * c + 2],
+                                   ob[sl * 32 + 4 * c + 3]);
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarStageFull));
+                if (issuer) {
+                    ok = mbar_wait_warp(bar(kBarStageFull), round & 1, abort_flag, p.status, kErrEpi);
+                    if (!ok) break;
+                    if (elect_one_sync()) {
+                        for (int s = 0; s < nseg; ++s) {
+                            const int R = t.R0 + s * p.seg_rows;
+                            const int b = R / p.Rg, r = R - b * p.Rg;
+                            tma_store_4d(&tm_dq, stage + s * p.seg_rows * 128, sl * 64, r, t.g, b);
+                        }
+                        tma_store_commit();
+                        tma_store_wait_read();
+                        mbar_arrive(bar(kBarStageFree));
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (issuer && elect_one_sync()) tma_store_wait_all();
+    }
+
+    PSKV_TRACE_FLUSH;
+    if (*abort_flag != 0) __nanosleep(20000);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------------------ host side
+
+struct BwdPlan {
+    bool ok;
+    int tile_rows, seg_rows, tiles_per_group, sfx_rows;
+    int nblk_p, tail_rows, resident, stages;
+    int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc, smem_bytes;
+};
+
+BwdPlan plan_bwd(const Dims &dm)
+{
+    BwdPlan pl;
+    memset(&pl, 0, sizeof(pl));
+    int nc_best = 0;
+    if (!pick_tile_rows(dm, &pl.tile_rows, &pl.seg_rows, &pl.tiles_per_group, &nc_best)) return pl;
+    pl.sfx_rows = round_up(nc_best * dm.S, 16);
+    pl.nblk_p = (dm.P + kBlockN - 1) / kBlockN;
+    pl.tail_rows = pl.nblk_p ? round_up(dm.P - (pl.nblk_p - 1) * kBlockN, 16) : 0;
+    const int slabs = dm.d / 64;
+    const int tile_bytes = slabs * kTileM * 128;
+    const int sfx_bytes = round_up(slabs * pl.sfx_rows * 128, 1024);
+    const int tail_bytes = round_up(slabs * pl.tail_rows * 128, 1024);
+    const int fixed = 2 * tile_bytes /*Q, dO*/ + 2 * sfx_bytes + kStagingBytes + kBarBytes + 64;
+    const int resident_bytes = pl.nblk_p ? (pl.nblk_p - 1) * tile_bytes + tail_bytes : 0;
+    int kv_bytes = 0;
+    if (pl.nblk_p <= kMaxStages && fixed + 2 * resident_bytes <= kMaxSmem) {
+        pl.resident = 1;
+        pl.stages = pl.nblk_p > 0 ? pl.nblk_p : 1;
+        kv_bytes = resident_bytes;
+    } else {
+        int st = (kMaxSmem - fixed) / (2 * tile_bytes);
+        if (st > kMaxStages) st = kMaxStages;
+        if (st < 1) return pl;
+        pl.stages = st;
+        kv_bytes = st * tile_bytes;
+    }
+    pl.off_pk = 0;
+    pl.off_pv = kv_bytes;
+    pl.off_q = 2 * kv_bytes;
+    pl.off_do = pl.off_q + tile_bytes;
+    pl.off_sk = pl.off_do + tile_bytes;
+    pl.off_sv = pl.off_sk + sfx_bytes;
+    pl.off_stage = pl.off_sv + sfx_bytes;
+    pl.off_bar = pl.off_stage + kStagingBytes;
+    pl.off_misc = pl.off_bar + kBarBytes;
+    pl.smem_bytes = pl.off_misc + 64;
+    pl.ok = pl.smem_bytes <= kMaxSmem;
+    return pl;
+}
+
+template <int D>
+cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_word, cudaStream_t stream)
+{
+    const Dims &dm = a.dims;
+    const int Rg = dm.n_rep * dm.S;
+    CUtensorMap tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail, tm_sk, tm_sv;
+    memset(&tm_pk, 0, sizeof(tm_pk));
+    memset(&tm_pv, 0, sizeof(tm_pv));
+    memset(&tm_pk_tail, 0, sizeof(tm_pk_tail));
+    memset(&tm_pv_tail, 0, sizeof(tm_pv_tail));
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Rg, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
+        cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)Rg * D * 2, (cuuint64_t)dm.Hkv * Rg * D * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)plan.seg_rows, 1, 1};
+        if (!encode_map(&tm_q, a.q, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_do, a.dout, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_dq, a.dq, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)dm.S, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
+        cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)dm.S * D * 2, (cuuint64_t)dm.Hkv * dm.S * D * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)dm.S, 1, 1};
+        if (!encode_map(&tm_sk, a.suffix_k, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_sv, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    if (dm.P > 0) {
+        cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
+        cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.P * D * 2};
+        cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
+        cuuint32_t box_tail[3] = {64, (cuuint32_t)plan.tail_rows, 1};
+        if (!encode_map(&tm_pk, a.prefix_k, 3, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_pv, a.prefix_v, 3, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_pk_tail, a.prefix_k, 3, dims, str, box_tail)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_pv_tail, a.prefix_v, 3, dims, str, box_tail)) return cudaErrorInvalidValue;
+    }
+    TcBwdParams p;
+    p.lse = a.lse;
+    p.row_dot = a.row_dot;
+    p.status = status_word;
+    p.sl2 = a.scale * kLog2e;
+    p.scale = a.scale;
+    p.B = dm.B; p.Hq = dm.Hq; p.Hkv = dm.Hkv; p.S = dm.S; p.P = dm.P; p.n_rep = dm.n_rep;
+    p.Rg = Rg;
+    p.tile_rows = plan.tile_rows;
+    p.seg_rows = plan.seg_rows;
+    p.tiles_per_group = plan.tiles_per_group;
+    p.total_tiles = plan.tiles_per_group * dm.Hkv;
+    p.nblk_p = plan.nblk_p;
+    p.tail_rows = plan.tail_rows;
+    p.resident = plan.resident;
+    p.stages = plan.stages > 0 ? plan.stages : 1;
+    p.sfx_rows = plan.sfx_rows;
+    p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_do = plan.off_do;
+    p.off_sk = plan.off_sk; p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar;
+    p.off_misc = plan.off_misc;
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    // D = <dout, out> per row, then dQ on the tensor cores, then dK_suffix / dV_suffix
+    cudaError_t e = launch_simt_row_dot(a, stream);
+    if (e != cudaSuccess) return e;
+    const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
+    tc_bwd_dq_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,
+                                                                     tm_pv_tail, tm_sk, tm_sv, p);
+    count_launches(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_simt_bwd_dkv(a, stream);
+}
+
+}  // namespace
+
+bool tc_bwd_supported(const Dims &dm)
+{
+    if (dm.d != 64 && dm.d != 128) return false;
+    if ((long long)dm.B * dm.n_rep * dm.S > 2000000000ll) return false;
+    return plan_bwd(dm).ok;
+}
+
+size_t tc_bwd_workspace_bytes(const Dims &dm) { return (size_t)dm.B * dm.Hq * dm.S * sizeof(float); }
+
+cudaError_t launch_tc_bwd(const BwdArgs &a, void *, unsigned int *status_word, cudaStream_t stream)
+{
+    const BwdPlan plan = plan_bwd(a.dims);
+    if (!plan.ok) return cudaErrorInvalidValue;
+    return a.dims.d == 128 ? launch<128>(a, plan, status_word, stream) : launch<64>(a, plan, status_word, stream);
+}
+
+}  // namespace pskv

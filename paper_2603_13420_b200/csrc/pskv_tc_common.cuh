@@ -1,0 +1,151 @@
+// Pieces shared by the tensor-core forward and backward kernels: tile geometry over the flat row
+// list of a KV-head group, the optional event trace, and the host-side TMA descriptor helpers.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pskv_common.cuh"
+
+namespace pskv {
+namespace {
+
+constexpr int kTileM = 128;    // rows of one MMA tile (tensor-memory lanes)
+constexpr int kBlockN = 128;   // keys per block
+constexpr int kStagingBytes = kTileM * 128;  // one 64-column slab of an output tile
+constexpr int kMaxSmem = 232448;             // dynamic shared memory a CTA may use on sm_100
+
+// Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
+// costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
+#ifdef PSKV_TRACE
+constexpr int kTraceWarps = 16, kTraceCap = 4096;
+__device__ long long g_trace[kTraceWarps * kTraceCap * 2];
+__device__ unsigned int g_trace_n[kTraceWarps];
+#define PSKV_TRACE_DECL unsigned int trace_i_ = 0
+#define PSKV_TRACE_EVENT(tag, val)                                                                     \
+    do {                                                                                               \
+        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0 && (threadIdx.x & 31) == 0 &&        \
+            trace_i_ < (unsigned int)kTraceCap) {                                                      \
+            long long *e_ = g_trace + ((size_t)(threadIdx.x >> 5) * kTraceCap + trace_i_) * 2;         \
+            e_[0] = clock64();                                                                         \
+            e_[1] = ((long long)(tag) << 32) | (unsigned int)(val);                                    \
+            ++trace_i_;                                                                                \
+        }                                                                                              \
+    } while (0)
+#define PSKV_TRACE_FLUSH                                                                               \
+    do {                                                                                               \
+        if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
+    } while (0)
+#else
+#define PSKV_TRACE_DECL do { } while (0)
+#define PSKV_TRACE_FLUSH do { } while (0)
+#define PSKV_TRACE_EVENT(tag, val) do { } while (0)
+#endif
+
+struct TileInfo {
+    int g, R0, rows, b_first, nc, n_sfx;  // n_sfx: suffix columns rounded up to 16
+    bool first_of_g;
+};
+
+// `Params` is any kernel parameter block with fields B, Rg, S, tile_rows, tiles_per_group.
+template <class Params>
+__device__ __forceinline__ TileInfo tile_info(const Params &p, int tile, int t_begin)
+{
+    TileInfo t;
+    t.g = tile / p.tiles_per_group;
+    const int tt = tile - t.g * p.tiles_per_group;
+    t.first_of_g = (tt == 0) || (tile == t_begin);
+    t.R0 = tt * p.tile_rows;
+    const int total = p.B * p.Rg;
+    t.rows = min(p.tile_rows, total - t.R0);
+    t.b_first = t.R0 / p.Rg;
+    const int b_last = (t.R0 + t.rows - 1) / p.Rg;
+    t.nc = b_last - t.b_first + 1;
+    t.n_sfx = (t.nc * p.S + 15) & ~15;
+    return t;
+}
+
+// ------------------------------------------------------------------------------ host side
+
+inline int gcd_int(int a, int b) { return b == 0 ? a : gcd_int(b, a % b); }
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+
+// Picks the rows per tile: the largest multiple of 8 up to 128 such that the suffix keys of all
+// candidates a tile can touch fit one 128-key block (candidates x S <= 128).  `nc_max` receives
+// that largest number of candidates.
+inline bool pick_tile_rows(const Dims &dm, int *tile_rows, int *seg_rows, int *tiles_per_group, int *nc_max_out)
+{
+    if (dm.S % 8 != 0 || dm.S > kBlockN) return false;
+    const int Rg = dm.n_rep * dm.S;
+    const long long total = (long long)dm.B * Rg;
+    for (int m = kTileM; m >= 8; m -= 8) {
+        const int seg = gcd_int(Rg, m);
+        if (seg % 8 != 0) continue;
+        // worst number of candidates a window [t*m, t*m + m) overlaps; the pattern repeats every Rg/seg tiles
+        const long long ntiles = (total + m - 1) / m;
+        const long long period = (long long)Rg / seg;
+        const long long check = ntiles < period ? ntiles : period;
+        int nc_max = 0;
+        for (long long t = 0; t < check; ++t) {
+            const long long r0 = t * m;
+            long long r1 = r0 + m;
+            if (r1 > total) r1 = total;
+            const int nc = (int)((r1 - 1) / Rg - r0 / Rg + 1);
+            if (nc > nc_max) nc_max = nc;
+        }
+        if (nc_max * dm.S > kBlockN) continue;
+        *tile_rows = m;
+        *seg_rows = seg;
+        *tiles_per_group = (int)ntiles;
+        *nc_max_out = nc_max;
+        return true;
+    }
+    return false;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// bf16 tensor, innermost dimension contiguous, 128-byte swizzle, 64-column boxes.
+inline bool encode_map(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims,
+                const cuuint64_t *strides_bytes, const cuuint32_t *box)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims,
+                    strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+inline int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    }
+    return n;
+}
+
+
+}  // namespace
+}  // namespace pskv

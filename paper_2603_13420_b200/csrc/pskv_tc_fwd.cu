@@ -23,14 +23,13 @@
 
 #include "pskv_common.cuh"
 #include "pskv_sm100.cuh"
+#include "pskv_tc_common.cuh"
 
 namespace pskv {
 namespace {
 
 using namespace sm100;
 
-constexpr int kTileM = 128;    // rows of one MMA tile (tensor-memory lanes)
-constexpr int kBlockN = 128;   // keys per block
 constexpr int kSlots = 3;      // score slots of 128 columns; an item's probabilities overwrite its own scores
 constexpr int kThreads = 512;
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
@@ -39,35 +38,6 @@ constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 constexpr float kMaxLog2 = 100.0f;
 constexpr float kMinRowSum = 7.8886090522101181e-31f;  // 2^-100
 constexpr int kMaxStages = 4;
-constexpr int kStagingBytes = kTileM * 128;  // one 64-column slab of the output tile
-constexpr int kMaxSmem = 232448;
-
-// Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
-// costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
-#ifdef PSKV_TRACE
-constexpr int kTraceWarps = 16, kTraceCap = 4096;
-__device__ long long g_trace[kTraceWarps * kTraceCap * 2];
-__device__ unsigned int g_trace_n[kTraceWarps];
-#define PSKV_TRACE_DECL unsigned int trace_i_ = 0
-#define PSKV_TRACE_EVENT(tag, val)                                                                     \
-    do {                                                                                               \
-        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0 && (threadIdx.x & 31) == 0 &&        \
-            trace_i_ < (unsigned int)kTraceCap) {                                                      \
-            long long *e_ = g_trace + ((size_t)(threadIdx.x >> 5) * kTraceCap + trace_i_) * 2;         \
-            e_[0] = clock64();                                                                         \
-            e_[1] = ((long long)(tag) << 32) | (unsigned int)(val);                                    \
-            ++trace_i_;                                                                                \
-        }                                                                                              \
-    } while (0)
-#define PSKV_TRACE_FLUSH                                                                               \
-    do {                                                                                               \
-        if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
-    } while (0)
-#else
-#define PSKV_TRACE_DECL do { } while (0)
-#define PSKV_TRACE_FLUSH do { } while (0)
-#define PSKV_TRACE_EVENT(tag, val) do { } while (0)
-#endif
 
 enum : unsigned int {
     kErrProducerK = 0x101, kErrProducerV = 0x102, kErrMmaQk = 0x103, kErrMmaPv = 0x104,
@@ -124,42 +94,11 @@ enum {
 constexpr int kBarBytes = 512;
 static_assert(kNumBars * 8 <= kBarBytes, "barrier area");
 
-struct TileInfo {
-    int g, R0, rows, b_first, nc, n_sfx;  // n_sfx: suffix columns rounded up to 16
-    bool first_of_g;
-};
-
-__device__ __forceinline__ TileInfo tile_info(const TcFwdParams &p, int tile, int t_begin)
-{
-    TileInfo t;
-    t.g = tile / p.tiles_per_group;
-    const int tt = tile - t.g * p.tiles_per_group;
-    t.first_of_g = (tt == 0) || (tile == t_begin);
-    t.R0 = tt * p.tile_rows;
-    const int total = p.B * p.Rg;
-    t.rows = min(p.tile_rows, total - t.R0);
-    t.b_first = t.R0 / p.Rg;
-    const int b_last = (t.R0 + t.rows - 1) / p.Rg;
-    t.nc = b_last - t.b_first + 1;
-    t.n_sfx = (t.nc * p.S + 15) & ~15;
-    return t;
-}
-
 // rows held (and MMA N used) by prefix block k
 __device__ __forceinline__ int prefix_block_rows(const TcFwdParams &p, int k)
 {
     return k == p.nblk_p - 1 ? p.tail_rows : kBlockN;
 }
-
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3)
-{
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(map),
-                 "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 #ifndef PSKV_PIECE
 #define PSKV_PIECE 32
@@ -755,9 +694,6 @@ struct TilePlan {
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml, smem_bytes;
 };
 
-int gcd_int(int a, int b) { return b == 0 ? a : gcd_int(b, a % b); }
-int round_up(int x, int m) { return (x + m - 1) / m * m; }
-
 // Picks the rows per tile -- the largest multiple of 8 up to 128 such that the suffix keys of all
 // candidates a tile can touch fit one 128-key block (candidates x S <= 128) -- and lays out shared
 // memory: all prefix blocks of a KV head if they fit beside the other buffers (resident mode), else
@@ -766,32 +702,8 @@ TilePlan plan_tiles(const Dims &dm)
 {
     TilePlan pl;
     memset(&pl, 0, sizeof(pl));
-    if (dm.S % 8 != 0 || dm.S > kBlockN) return pl;
-    const int Rg = dm.n_rep * dm.S;
-    const long long total = (long long)dm.B * Rg;
     int nc_best = 0;
-    for (int m = kTileM; m >= 8 && !pl.tile_rows; m -= 8) {
-        const int seg = gcd_int(Rg, m);
-        if (seg % 8 != 0) continue;
-        // worst number of candidates a window [t*m, t*m + m) overlaps; the pattern repeats every Rg/seg tiles
-        const long long ntiles = (total + m - 1) / m;
-        const long long period = (long long)Rg / seg;
-        const long long check = ntiles < period ? ntiles : period;
-        int nc_max = 0;
-        for (long long t = 0; t < check; ++t) {
-            const long long r0 = t * m;
-            long long r1 = r0 + m;
-            if (r1 > total) r1 = total;
-            const int nc = (int)((r1 - 1) / Rg - r0 / Rg + 1);
-            if (nc > nc_max) nc_max = nc;
-        }
-        if (nc_max * dm.S > kBlockN) continue;
-        pl.tile_rows = m;
-        pl.seg_rows = seg;
-        pl.tiles_per_group = (int)ntiles;
-        nc_best = nc_max;
-    }
-    if (!pl.tile_rows) return pl;
+    if (!pick_tile_rows(dm, &pl.tile_rows, &pl.seg_rows, &pl.tiles_per_group, &nc_best)) return pl;
     pl.sfx_rows = round_up(nc_best * dm.S, 16);
     pl.nblk_p = (dm.P + kBlockN - 1) / kBlockN;
     pl.tail_rows = pl.nblk_p ? round_up(dm.P - (pl.nblk_p - 1) * kBlockN, 16) : 0;
@@ -827,48 +739,6 @@ TilePlan plan_tiles(const Dims &dm)
     pl.smem_bytes = pl.off_ml + 2 * kTileM * 8;
     pl.ok = pl.smem_bytes <= kMaxSmem;
     return pl;
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-// bf16 tensor, innermost dimension contiguous, 128-byte swizzle, 64-column boxes.
-bool encode_map(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims,
-                const cuuint64_t *strides_bytes, const cuuint32_t *box)
-{
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
-    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims,
-                    strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
-int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return n;
 }
 
 template <int D>
