@@ -37,6 +37,9 @@ cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream);
 // dk_suffix / dv_suffix (needs row_dot and lse).
 cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream);
 cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
+// dk_suffix / dv_suffix on warp-level tensor-core MMAs, one CTA per (candidate, KV head); S <= 64.
+bool mma_bwd_dkv_supported(const Dims &d);
+cudaError_t launch_mma_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
 // Recomputes the rows whose lse is NaN, if *redo_count != 0 (a device counter); `blocks` CTAs.
 cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream);
 
