@@ -255,6 +255,9 @@ def run_cuda(args):
         sampler.start()
         time.sleep(0.3)
     barrier()
+    for kid in range(pskv.pskv_kernel_timing_count()):
+        pskv.pskv_kernel_timing_read(kid)  # forget launches recorded so far
+    pskv.pskv_kernel_timing_enable(True)
     launches0 = pskv.pskv_kernel_launches()
     e_start = torch.cuda.Event(enable_timing=True)
     e_stop = torch.cuda.Event(enable_timing=True)
@@ -268,6 +271,12 @@ def run_cuda(args):
     e_stop.record()
     barrier()
     launches = pskv.pskv_kernel_launches() - launches0
+    pskv.pskv_kernel_timing_enable(False)
+    kernels = {}
+    for kid in range(pskv.pskv_kernel_timing_count()):
+        ms, n = pskv.pskv_kernel_timing_read(kid)
+        if n:
+            kernels[pskv.pskv_kernel_timing_name(kid)] = {"launches": n, "total_ms": ms, "avg_us": 1e3 * ms / n}
     total_ms = e_start.elapsed_time(e_stop)
     fwd_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
     bwd_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
@@ -341,7 +350,11 @@ def run_cuda(args):
         "clocks": clocks,
         "peaks": peaks,
     }
-    line["roofline"] = roofline(w, fwd_ms, bwd_ms, peaks)
+    tot = sum(k["total_ms"] for k in kernels.values()) or 1.0
+    for k in kernels.values():
+        k["share"] = k["total_ms"] / tot
+    line["kernels"] = kernels
+    line["roofline"] = roofline(w, kernels, peaks)
 
     if world == 1 and not args.no_detail:
         line["detail"] = detail_runs(pskv, device, peaks)
@@ -352,26 +365,36 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
-def roofline(w, fwd_ms, bwd_ms, peaks):
-    """Roofline of the dominant kernel: the forward call is a single fused kernel; its algorithmic
-    bytes and flops per launch come from inputs.fwd_bytes / fwd_flops.  The binding roof is the
-    slower of bytes / HBM peak and flops / tensor peak for this workload."""
-    t_hbm = wl.fwd_bytes(w) / (peaks["hbm_gbs"] * 1e9)
-    t_mma = wl.fwd_flops(w) / (peaks["bf16_tflops"] * 1e12)
-    traffic = TRAFFIC_BYTES_PER_LAUNCH.get(w.name)
+def roofline(w, kernels, peaks):
+    """Roofline of the dominant kernel of the step: the kernel with the largest summed device time
+    in the timed region (CUDA events around each launch, on the launch stream).  Algorithmic bytes
+    and flops per launch come from inputs.kernel_work; the binding roof is the slower of
+    bytes / measured HBM peak and flops / measured bf16 peak."""
+    work = wl.kernel_work(w)
+    cands = {k: v for k, v in kernels.items() if k in work}
+    if not cands:
+        return None
+    name = max(cands, key=lambda k: cands[k]["total_ms"])
+    sec = cands[name]["avg_us"] * 1e-6
+    t_hbm = work[name]["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_mma = work[name]["flops"] / (peaks["bf16_tflops"] * 1e12)
+    traffic = TRAFFIC_BYTES_PER_LAUNCH.get((name, w.name))
+    common = {"kernel": name, "avg_us": cands[name]["avg_us"], "share_of_step": cands[name]["share"],
+              "algorithmic_bytes": work[name]["bytes"], "algorithmic_flops": work[name]["flops"],
+              "traffic": traffic}
     if t_hbm >= t_mma:
-        ach = wl.fwd_bytes(w) / (fwd_ms * 1e-3) / 1e9
-        return {"kernel": "pskv_attn_fwd", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": traffic,
-                "peak_source": peaks["source"] + ", burst copy"}
-    ach = wl.fwd_flops(w) / (fwd_ms * 1e-3) / 1e12
-    return {"kernel": "pskv_attn_fwd", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-            "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "traffic": traffic,
-            "peak_source": peaks["source"] + ", burst"}
+        ach = work[name]["bytes"] / sec / 1e9
+        common.update({"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                       "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (of measured), burst copy"})
+    else:
+        ach = work[name]["flops"] / sec / 1e12
+        common.update({"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                       "frac": ach / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (of measured), burst"})
+    return common
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the forward kernel, from the ncu
-# capture summarised under profiles/ (None until a capture exists for the workload).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/ (kernel, workload) -> bytes.
 TRAFFIC_BYTES_PER_LAUNCH = {}
 
 

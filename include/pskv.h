@@ -120,6 +120,19 @@ int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d
  */
 long long pskv_kernel_launches(void);
 
+/*
+ * Optional per-kernel device timing, for benchmarks that must report the duration of one kernel
+ * inside a call that launches several.  While enabled, every kernel the library launches is
+ * bracketed by two CUDA events on its stream (at most 8192 launches are kept).
+ * pskv_kernel_timing_read waits for the recorded launches of one kernel id, returns their summed
+ * device time in milliseconds and their count, and forgets them.  Kernel ids run from 0 to
+ * pskv_kernel_timing_count() - 1; pskv_kernel_timing_name gives the kernel's name.
+ */
+void pskv_kernel_timing_enable(int on);
+int pskv_kernel_timing_count(void);
+const char *pskv_kernel_timing_name(int kernel_id);
+pskv_status pskv_kernel_timing_read(int kernel_id, double *total_ms, long long *launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,6 +18,10 @@ from .binding import (  # noqa: F401
     pskv_attn_fwd_workspace_bytes,
     pskv_kernel_family,
     pskv_kernel_launches,
+    pskv_kernel_timing_count,
+    pskv_kernel_timing_enable,
+    pskv_kernel_timing_name,
+    pskv_kernel_timing_read,
     pskv_last_cuda_error,
     pskv_poll_device_status,
     pskv_status_string,

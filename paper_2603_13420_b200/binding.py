@@ -65,6 +65,14 @@ def lib() -> ctypes.CDLL:
         L.pskv_last_cuda_error.restype = ci
         L.pskv_version.argtypes = []
         L.pskv_version.restype = ci
+        L.pskv_kernel_timing_enable.argtypes = [ci]
+        L.pskv_kernel_timing_enable.restype = None
+        L.pskv_kernel_timing_count.argtypes = []
+        L.pskv_kernel_timing_count.restype = ci
+        L.pskv_kernel_timing_name.argtypes = [ci]
+        L.pskv_kernel_timing_name.restype = ctypes.c_char_p
+        L.pskv_kernel_timing_read.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong)]
+        L.pskv_kernel_timing_read.restype = ci
         L.pskv_kernel_launches.argtypes = []
         L.pskv_kernel_launches.restype = ctypes.c_longlong
         L.pskv_kernel_family.argtypes = [ci] + six
@@ -94,6 +102,27 @@ def _dims(q, prefix_k, suffix_k):
 
 def pskv_version() -> int:
     return int(lib().pskv_version())
+
+
+def pskv_kernel_timing_enable(on) -> None:
+    lib().pskv_kernel_timing_enable(int(bool(on)))
+
+
+def pskv_kernel_timing_count() -> int:
+    return int(lib().pskv_kernel_timing_count())
+
+
+def pskv_kernel_timing_name(kernel_id) -> str:
+    return lib().pskv_kernel_timing_name(int(kernel_id)).decode()
+
+
+def pskv_kernel_timing_read(kernel_id):
+    """(total device milliseconds, launches) of one kernel id since the last read."""
+    ms, n = ctypes.c_double(0.0), ctypes.c_longlong(0)
+    st = lib().pskv_kernel_timing_read(int(kernel_id), ctypes.byref(ms), ctypes.byref(n))
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_kernel_timing_read")
+    return ms.value, int(n.value)
 
 
 def pskv_kernel_launches() -> int:

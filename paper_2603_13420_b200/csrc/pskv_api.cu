@@ -3,6 +3,8 @@
 #include <stdio.h>
 
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "pskv_common.cuh"
 
@@ -74,9 +76,42 @@ size_t simt_bwd_workspace(const Dims &dm) { return round256((size_t)dm.B * dm.Hq
 
 std::atomic<long long> g_launches{0};
 
+// ---- optional per-kernel timing: a bounded list of (kernel id, start event, stop event)
+constexpr int kMaxTimed = 8192;
+struct TimedLaunch {
+    int id;
+    cudaEvent_t start, stop;
+};
+std::mutex g_timing_mutex;
+bool g_timing_on = false;
+std::vector<TimedLaunch> g_timed;
+const char *const kKernelNames[kKernelCount] = {
+    "tc_fwd_kernel", "simt_fwd_redo_kernel", "simt_row_dot_kernel", "tc_bwd_dq_kernel", "bwd_dkv_mma_kernel",
+    "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel"};
+
 }  // namespace
 
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+void *timing_begin(int kernel_id, cudaStream_t stream)
+{
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    if (!g_timing_on || (int)g_timed.size() >= kMaxTimed) return nullptr;
+    TimedLaunch t;
+    t.id = kernel_id;
+    if (cudaEventCreate(&t.start) != cudaSuccess) return nullptr;
+    if (cudaEventCreate(&t.stop) != cudaSuccess) { cudaEventDestroy(t.start); return nullptr; }
+    cudaEventRecord(t.start, stream);
+    g_timed.push_back(t);
+    return reinterpret_cast<void *>(g_timed.size());  // 1-based index
+}
+
+void timing_end(void *token, cudaStream_t stream)
+{
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    const size_t idx = reinterpret_cast<size_t>(token);
+    if (idx >= 1 && idx <= g_timed.size()) cudaEventRecord(g_timed[idx - 1].stop, stream);
+}
 
 }  // namespace pskv
 
@@ -87,6 +122,43 @@ extern "C" {
 int pskv_version(void) { return 100; }
 
 long long pskv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void pskv_kernel_timing_enable(int on)
+{
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    g_timing_on = on != 0;
+}
+
+int pskv_kernel_timing_count(void) { return kKernelCount; }
+
+const char *pskv_kernel_timing_name(int kernel_id)
+{
+    return (kernel_id >= 0 && kernel_id < kKernelCount) ? kKernelNames[kernel_id] : "";
+}
+
+pskv_status pskv_kernel_timing_read(int kernel_id, double *total_ms, long long *launches)
+{
+    if (!total_ms || !launches || kernel_id < 0 || kernel_id >= kKernelCount) return PSKV_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    double ms = 0.0;
+    long long n = 0;
+    std::vector<TimedLaunch> keep;
+    for (const TimedLaunch &t : g_timed) {
+        if (t.id != kernel_id) { keep.push_back(t); continue; }
+        float one = 0.f;
+        cudaError_t e = cudaEventSynchronize(t.stop);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&one, t.start, t.stop);
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+        if (e != cudaSuccess) { g_timed.swap(keep); return cuda_fail(e); }
+        ms += one;
+        ++n;
+    }
+    g_timed.swap(keep);
+    *total_ms = ms;
+    *launches = n;
+    return PSKV_OK;
+}
 
 const char *pskv_status_string(pskv_status s)
 {

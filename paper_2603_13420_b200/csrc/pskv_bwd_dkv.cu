@@ -240,6 +240,7 @@ cudaError_t launch_one(const BwdArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    KernelTiming timing(kKernelBwdDkvMma, stream);
     bwd_dkv_mma_kernel<D, TP><<<a.dims.B * a.dims.Hkv, kDkvThreads, L::kBytes, stream>>>(a);
     count_launches(1);
     return cudaGetLastError();

@@ -56,6 +56,21 @@ cudaError_t launch_tc_bwd(const BwdArgs &a, void *workspace, unsigned int *statu
 // Host-side count of kernel launches (read through pskv_kernel_launches()).
 void count_launches(int n);
 
+// Optional per-kernel device timing (pskv_kernel_timing_*): when enabled, a launch site brackets
+// its kernel with two CUDA events on the launch stream.
+enum KernelId {
+    kKernelFwdTc = 0, kKernelFwdRedo, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvMma,
+    kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCount
+};
+void *timing_begin(int kernel_id, cudaStream_t stream);  // returns nullptr when timing is off
+void timing_end(void *token, cudaStream_t stream);
+struct KernelTiming {
+    void *token;
+    cudaStream_t stream;
+    KernelTiming(int id, cudaStream_t s) : token(timing_begin(id, s)), stream(s) {}
+    ~KernelTiming() { if (token) timing_end(token, stream); }
+};
+
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 

@@ -325,6 +325,7 @@ inline unsigned int blocks_for(long long items)
 cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream)
 {
     const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    KernelTiming timing(kKernelFwdSimt, stream);
     if (a.dims.d == 128)
         simt_fwd_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
     else
@@ -335,6 +336,7 @@ cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream)
 
 cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream)
 {
+    KernelTiming timing(kKernelFwdRedo, stream);
     if (a.dims.d == 128)
         simt_fwd_redo_kernel<128><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(a, redo_count);
     else
@@ -346,6 +348,7 @@ cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_coun
 cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream)
 {
     const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    KernelTiming timing(kKernelRowDot, stream);
     if (a.dims.d == 128)
         simt_row_dot_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
     else
@@ -357,6 +360,7 @@ cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream)
 cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream)
 {
     const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.S;
+    KernelTiming timing(kKernelBwdDkvSimt, stream);
     if (a.dims.d == 128)
         simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
     else
@@ -369,12 +373,19 @@ cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream)
 {
     const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
     const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.S;
-    if (a.dims.d == 128) {
-        simt_bwd_dq_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
-        simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
-    } else {
-        simt_bwd_dq_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
-        simt_bwd_dkv_kernel<64><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
+    {
+        KernelTiming timing(kKernelBwdDqSimt, stream);
+        if (a.dims.d == 128)
+            simt_bwd_dq_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+        else
+            simt_bwd_dq_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+    }
+    {
+        KernelTiming timing(kKernelBwdDkvSimt, stream);
+        if (a.dims.d == 128)
+            simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
+        else
+            simt_bwd_dkv_kernel<64><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
     }
     count_launches(2);
     return cudaGetLastError();

@@ -705,8 +705,11 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     cudaError_t e = launch_simt_row_dot(a, stream);
     if (e != cudaSuccess) return e;
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
-    tc_bwd_dq_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,
-                                                                     tm_pv_tail, tm_sk, tm_sv, p);
+    {
+        KernelTiming timing(kKernelBwdDqTc, stream);
+        tc_bwd_dq_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,
+                                                                         tm_pv_tail, tm_sk, tm_sv, p);
+    }
     count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

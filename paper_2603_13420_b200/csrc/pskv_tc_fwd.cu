@@ -806,8 +806,11 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     cudaError_t e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), stream);
     if (e != cudaSuccess) return e;
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
-    tc_fwd_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail,
-                                                                  tm_sk, tm_sv, p);
+    {
+        KernelTiming timing(kKernelFwdTc, stream);
+        tc_fwd_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail,
+                                                                      tm_pv_tail, tm_sk, tm_sv, p);
+    }
     count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -132,3 +132,19 @@ def bwd_bytes(w: Workload) -> float:
     pkv = 2 * w.Hkv * w.P * w.d * 2
     lse = w.B * w.Hq * w.S * 4
     return float(3 * q + lse + skv + pkv + q + skv)
+
+
+def kernel_work(w: Workload) -> dict:
+    """Algorithmic flops and HBM bytes per launch of each kernel of the tensor-core path
+    (every input read once, every output written once; recomputed scores are not counted)."""
+    rows = w.B * w.Hq * w.S
+    q = rows * w.d * 2
+    skv = 2 * w.B * w.Hkv * w.S * w.d * 2
+    pkv = 2 * w.Hkv * w.P * w.d * 2
+    vis = (w.S + 1) / 2.0
+    return {
+        "tc_fwd_kernel": {"flops": fwd_flops(w), "bytes": fwd_bytes(w)},
+        "tc_bwd_dq_kernel": {"flops": rows * 6.0 * w.d * (w.P + vis), "bytes": float(3 * q + 8 * rows + skv + pkv)},
+        "bwd_dkv_mma_kernel": {"flops": rows * 4.0 * w.d * vis, "bytes": float(2 * q + 8 * rows + 2 * skv)},
+        "simt_row_dot_kernel": {"flops": rows * 2.0 * w.d, "bytes": float(2 * q + 4 * rows)},
+    }

@@ -104,5 +104,21 @@ def test_no_device_means_error_not_fallback():
     import torch
     if torch.cuda.is_available():
         pytest.skip("a CUDA device is present")
-    rc = _fwd(binding.lib(), GOOD, 0.125, (8, 4, 4, 8, 32, 64))
+    dims = (8, 4, 4, 8, 32, 64)
+    need = binding.pskv_attn_fwd_workspace_bytes(*dims)
+    assert _fwd(binding.lib(), GOOD, 0.125, dims) == (binding.PSKV_ERR_WORKSPACE if need else rc_no_device())
+    rc = _fwd(binding.lib(), GOOD, 0.125, dims, ws=0x100000, ws_bytes=max(need, 256))
     assert rc in (binding.PSKV_ERR_CUDA, binding.PSKV_ERR_UNSUPPORTED_ARCH)
+
+
+def rc_no_device():
+    return binding.PSKV_ERR_CUDA
+
+
+def test_kernel_timing_interface_without_a_device():
+    assert binding.pskv_kernel_timing_count() >= 5
+    names = [binding.pskv_kernel_timing_name(i) for i in range(binding.pskv_kernel_timing_count())]
+    assert "tc_fwd_kernel" in names and "tc_bwd_dq_kernel" in names
+    binding.pskv_kernel_timing_enable(True)
+    assert binding.pskv_kernel_timing_read(0) == (0.0, 0)
+    binding.pskv_kernel_timing_enable(False)
