@@ -91,6 +91,30 @@ pskv_status pskv_attn_bwd(const void *dout,     /* bf16 [B,Hq,S,d]  */
                           void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * pskv_attn_bwd without a workspace argument.  (The paper has no counterpart; this is a
+ * convenience of this library.)  It is for callers that cannot allocate device memory: processes
+ * in which a framework allocator owns the whole card, or loops with a fixed memory plan in which a
+ * cudaMalloc would fail or stall every stream while it synchronises the device.  The per-row
+ * scratch of the backward pass lives in a 4 MiB array inside the library image, which every GPU
+ * that loads the library holds until the process exits.
+ *   - Same arguments, results, layouts and error codes as pskv_attn_bwd; it calls no cudaMalloc,
+ *     cudaFree or other allocating routine.
+ *   - Sizes with B*Hq*S > pskv_attn_bwd_static_max_rows() (1048576) return PSKV_ERR_WORKSPACE and
+ *     launch nothing; use pskv_attn_bwd with your own workspace for those.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing needs
+ *     clearing (each call overwrites every element it later reads), but two calls that overlap
+ *     on the GPU -- different streams, or different host threads -- race on it and give wrong
+ *     gradients; serialise them.
+ */
+pskv_status pskv_attn_bwd_static(const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
+                                 const void *suffix_k, const void *suffix_v, const void *out, const float *lse,
+                                 float scale, void *dq, void *dk_suffix, void *dv_suffix,
+                                 int B, int Hq, int Hkv, int S, int P, int d, void *cuda_stream);
+long long pskv_attn_bwd_static_max_rows(void);
+
+/*
  * Synchronises `cuda_stream`, then reads and clears the device status word that
  * kernels set when one of their bounded waits gives up.  Returns PSKV_OK,
  * PSKV_ERR_DEVICE_TIMEOUT (results of the affected call are undefined) or

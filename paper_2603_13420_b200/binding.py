@@ -57,6 +57,10 @@ def lib() -> ctypes.CDLL:
         L.pskv_attn_fwd.restype = ci
         L.pskv_attn_bwd.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp, sz, vp]
         L.pskv_attn_bwd.restype = ci
+        L.pskv_attn_bwd_static.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp]
+        L.pskv_attn_bwd_static.restype = ci
+        L.pskv_attn_bwd_static_max_rows.argtypes = []
+        L.pskv_attn_bwd_static_max_rows.restype = ctypes.c_longlong
         L.pskv_poll_device_status.argtypes = [vp]
         L.pskv_poll_device_status.restype = ci
         L.pskv_status_string.argtypes = [ci]
@@ -190,6 +194,32 @@ def pskv_attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, out, lse, sca
                              _ptr(ws), ws.numel() * ws.element_size(), _stream())
     if st != PSKV_OK:
         raise PskvError(st, "pskv_attn_bwd")
+    return dq, dk_suffix, dv_suffix
+
+
+def pskv_attn_bwd_static_max_rows() -> int:
+    return int(lib().pskv_attn_bwd_static_max_rows())
+
+
+def pskv_attn_bwd_static(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, out, lse, scale,
+                         dq=None, dk_suffix=None, dv_suffix=None):
+    """pskv_attn_bwd for callers that cannot allocate device memory (a framework owns the card, or
+    a cudaMalloc would stall the device): the scratch is a fixed array inside the library, so no
+    workspace is passed.  Serves up to pskv_attn_bwd_static_max_rows() query rows (B*Hq*S); calls
+    that overlap on the GPU race on that array, so keep them on one stream.  The gradient tensors
+    are still the caller's (pass dq / dk_suffix / dv_suffix to avoid even those allocations)."""
+    dims = _dims(q, prefix_k, suffix_k)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk_suffix is None:
+        dk_suffix = torch.empty_like(suffix_k)
+    if dv_suffix is None:
+        dv_suffix = torch.empty_like(suffix_v)
+    st = lib().pskv_attn_bwd_static(_ptr(dout), _ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(suffix_k),
+                                    _ptr(suffix_v), _ptr(out), _ptr(lse), float(scale),
+                                    _ptr(dq), _ptr(dk_suffix), _ptr(dv_suffix), *dims, _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_bwd_static")
     return dq, dk_suffix, dv_suffix
 
 
