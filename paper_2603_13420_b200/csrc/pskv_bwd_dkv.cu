@@ -4,7 +4,7 @@
 // with P = exp(scale q.k - lse) on the suffix keys only and dS = P (dO.v - D).
 // One CTA per (candidate, KV head): its n_rep*S query rows and S suffix keys are contiguous in
 // memory, so everything is staged with plain coalesced copies.  The four small contractions per
-// 128-row chunk (S = Q K^T, dP = dO V^T, then P^T dO and dS^T Q) run on warp-level bf16 MMAs
+// 64-row chunk (S = Q K^T, dP = dO V^T, then P^T dO and dS^T Q) run on warp-level bf16 MMAs
 // (m16n8k16, fp32 accumulation): at 6-7 % of the backward flops and 48x192-sized operands this
 // part is bound by its memory traffic, not by tensor throughput.  Sums over the heads of a group
 // happen in registers of one CTA, so the result is deterministic and needs no atomics.
@@ -13,8 +13,9 @@
 namespace pskv {
 namespace {
 
-constexpr int kDkvThreads = 256;
-constexpr int kChunkRows = 128;
+constexpr int kDkvWarps = 4;
+constexpr int kDkvThreads = kDkvWarps * 32;
+constexpr int kChunkRows = kDkvWarps * 16;  // 64 query rows per pass: small CTAs, several per SM
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr)
 {
@@ -43,9 +44,9 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 }
 
 // Shared memory, all bf16 with 16 bytes of row padding (conflict-free ldmatrix):
-//   Qs, Gs  [128][D]      query / dout rows of the current chunk
+//   Qs, Gs  [64][D]       query / dout rows of the current chunk
 //   Ks, Vs  [TP][D]       suffix keys / values (TP = S rounded up to 16, padding rows zero)
-//   Ps, Ds  [128][TP]     probabilities / dS of the chunk
+//   Ps, Ds  [64][TP]      probabilities / dS of the chunk
 template <int D, int TP>
 struct DkvSmem {
     static constexpr int kRowD = D * 2 + 16;
@@ -90,10 +91,10 @@ bwd_dkv_mma_kernel(BwdArgs a)
         *reinterpret_cast<uint4 *>(smem + L::kOffV + t * L::kRowD + c * 16) = vv;
     }
 
-    // this warp's output tiles: all m-tiles (keys), n-tiles {2*warp, 2*warp+1} when D = 128
+    // this warp's output tiles: all m-tiles (keys) x its kNT consecutive n-tiles (8 columns each)
     constexpr int kMT = TP / 16;
-    constexpr int kNT = 2;          // n-tiles (of 8 columns) per warp; with D = 64 only warps 0-3 take part
-    const bool active = warp * kNT * 8 < D;
+    constexpr int kNT = D / 8 / kDkvWarps;
+    const bool active = true;
     float accV[kMT][kNT][4], accK[kMT][kNT][4];
 #pragma unroll
     for (int m = 0; m < kMT; ++m)

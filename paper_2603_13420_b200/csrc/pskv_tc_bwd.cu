@@ -47,7 +47,7 @@ struct TcBwdParams {
     float scale;
     int B, Hq, Hkv, S, P, n_rep;
     int Rg, tile_rows, seg_rows, tiles_per_group, total_tiles;
-    int nblk_p, tail_rows, resident, stages, sfx_rows;
+    int nblk_p, tail_rows, resident, stages_k, stages_v, sfx_rows;  // ring stages of prefix K / V (streaming mode)
     int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc;
 };
 
@@ -140,7 +140,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int g_first = t_begin / p.tiles_per_group;
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
-    const uint32_t stages = (uint32_t)p.stages;
+    const uint32_t stages_k = (uint32_t)p.stages_k, stages_v = (uint32_t)p.stages_v;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer: Q, K
@@ -171,8 +171,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!p.resident) {
 #pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
-                    const uint32_t ks = kload % stages;
-                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / stages) & 1) ^ 1, abort_flag, p.status, kErrProdA);
+                    const uint32_t ks = kload % stages_k;
+                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / stages_k) & 1) ^ 1, abort_flag, p.status, kErrProdA);
                     if (!ok) break;
                     const bool tail = k == p.nblk_p - 1;
                     const int slab = tail ? tail_slab : C::kSlabBytes;
@@ -257,8 +257,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!p.resident) {
 #pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
-                    const uint32_t vs = vload % stages;
-                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / stages) & 1) ^ 1, abort_flag, p.status, kErrProdB);
+                    const uint32_t vs = vload % stages_v;
+                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / stages_v) & 1) ^ 1, abort_flag, p.status, kErrProdB);
                     if (!ok) break;
                     const bool tail = k == p.nblk_p - 1;
                     const int slab = tail ? tail_slab : C::kSlabBytes;
@@ -304,8 +304,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
                 } else {
-                    const uint32_t ks = kuse % stages;
-                    ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / stages) & 1, abort_flag, p.status, kErrMmaS);
+                    const uint32_t ks = kuse % stages_k;
+                    ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / stages_k) & 1, abort_flag, p.status, kErrMmaS);
                     kaddr = sbase + p.off_pk + ks * C::kTileBytes;
                 }
             } else {
@@ -341,8 +341,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
                     vaddr = sbase + p.off_pv + k * C::kTileBytes;
                 } else {
-                    const uint32_t vs = vuse % stages;
-                    ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / stages) & 1, abort_flag, p.status, kErrMmaS);
+                    const uint32_t vs = vuse % stages_v;
+                    ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / stages_v) & 1, abort_flag, p.status, kErrMmaS);
                     vaddr = sbase + p.off_pv + vs * C::kTileBytes;
                 }
             } else {
@@ -361,7 +361,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         mma_ss(tmem + kDpCol, do_desc + aoff, v_desc + voff, idesc, ks16 > 0 ? 1u : 0u);
                     }
                     tc_commit(bar(kBarDpFull));
-                    if (ring) tc_commit(bar(kBarVFree + (vuse % stages)));
+                    if (ring) tc_commit(bar(kBarVFree + (vuse % stages_v)));
                     if (last_of_tile) tc_commit(bar(kBarDvFree));
                 }
                 __syncwarp();
@@ -395,7 +395,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (!ok) break;
             }
             uint32_t kaddr;
-            if (prefix) kaddr = sbase + p.off_pk + (p.resident ? (uint32_t)k : kuse % stages) * C::kTileBytes;
+            if (prefix) kaddr = sbase + p.off_pk + (p.resident ? (uint32_t)k : kuse % stages_k) * C::kTileBytes;
             else kaddr = sbase + p.off_sk;
             tc_fence_after();
             const uint32_t ds_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
@@ -410,7 +410,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                                ks16 > 0 ? 1u : acc0);
                 }
                 tc_commit(bar(kBarDqDone + slot));
-                if (ring) tc_commit(bar(kBarKFree + (kuse % stages)));
+                if (ring) tc_commit(bar(kBarKFree + (kuse % stages_k)));
                 if (last_of_tile) tc_commit(bar(kBarDqFull));
             }
             __syncwarp();
@@ -594,7 +594,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 struct BwdPlan {
     bool ok;
     int tile_rows, seg_rows, tiles_per_group, sfx_rows;
-    int nblk_p, tail_rows, resident, stages;
+    int nblk_p, tail_rows, resident, stages_k, stages_v;
     int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc, smem_bytes;
 };
 
@@ -613,21 +613,26 @@ BwdPlan plan_bwd(const Dims &dm)
     const int tail_bytes = round_up(slabs * pl.tail_rows * 128, 1024);
     const int fixed = 2 * tile_bytes /*Q, dO*/ + 2 * sfx_bytes + kStagingBytes + kBarBytes + 64;
     const int resident_bytes = pl.nblk_p ? (pl.nblk_p - 1) * tile_bytes + tail_bytes : 0;
-    int kv_bytes = 0;
+    int k_bytes = 0, v_bytes = 0;
     if (pl.nblk_p <= kMaxStages && fixed + 2 * resident_bytes <= kMaxSmem) {
         pl.resident = 1;
-        pl.stages = pl.nblk_p > 0 ? pl.nblk_p : 1;
-        kv_bytes = resident_bytes;
+        pl.stages_k = pl.stages_v = pl.nblk_p > 0 ? pl.nblk_p : 1;
+        k_bytes = v_bytes = resident_bytes;
     } else {
-        int st = (kMaxSmem - fixed) / (2 * tile_bytes);
-        if (st > kMaxStages) st = kMaxStages;
-        if (st < 1) return pl;
-        pl.stages = st;
-        kv_bytes = st * tile_bytes;
+        // ring mode: a K block lives from its score MMAs to its dQ MMAs, a V block only through its
+        // dP MMAs, so K gets the larger share of the stages that fit
+        int n = (kMaxSmem - fixed) / tile_bytes;
+        if (n > 2 * kMaxStages) n = 2 * kMaxStages;
+        if (n < 2) return pl;
+        pl.stages_v = n / 3 > 0 ? n / 3 : 1;
+        pl.stages_k = n - pl.stages_v;
+        if (pl.stages_k > kMaxStages) pl.stages_k = kMaxStages;
+        k_bytes = pl.stages_k * tile_bytes;
+        v_bytes = pl.stages_v * tile_bytes;
     }
     pl.off_pk = 0;
-    pl.off_pv = kv_bytes;
-    pl.off_q = 2 * kv_bytes;
+    pl.off_pv = k_bytes;
+    pl.off_q = k_bytes + v_bytes;
     pl.off_do = pl.off_q + tile_bytes;
     pl.off_sk = pl.off_do + tile_bytes;
     pl.off_sv = pl.off_sk + sfx_bytes;
@@ -689,7 +694,8 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.nblk_p = plan.nblk_p;
     p.tail_rows = plan.tail_rows;
     p.resident = plan.resident;
-    p.stages = plan.stages > 0 ? plan.stages : 1;
+    p.stages_k = plan.stages_k > 0 ? plan.stages_k : 1;
+    p.stages_v = plan.stages_v > 0 ? plan.stages_v : 1;
     p.sfx_rows = plan.sfx_rows;
     p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_do = plan.off_do;
     p.off_sk = plan.off_sk; p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar;
