@@ -37,6 +37,14 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// 16-byte asynchronous copy global -> shared; `valid` false writes zeros instead
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
+{
+    const int bytes = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -61,7 +69,7 @@ struct DkvSmem {
 };
 
 template <int D, int TP>
-__global__ void __launch_bounds__(kDkvThreads)
+__global__ void __launch_bounds__(kDkvThreads, 3)
 bwd_dkv_mma_kernel(BwdArgs a)
 {
     using L = DkvSmem<D, TP>;
@@ -82,13 +90,9 @@ bwd_dkv_mma_kernel(BwdArgs a)
     // suffix K / V once; padding rows zero
     for (int i = tid; i < TP * (D / 8); i += kDkvThreads) {
         const int t = i / (D / 8), c = i - t * (D / 8);
-        uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-        if (t < S) {
-            kv = __ldg(reinterpret_cast<const uint4 *>(kg + (size_t)t * D) + c);
-            vv = __ldg(reinterpret_cast<const uint4 *>(vg + (size_t)t * D) + c);
-        }
-        *reinterpret_cast<uint4 *>(smem + L::kOffK + t * L::kRowD + c * 16) = kv;
-        *reinterpret_cast<uint4 *>(smem + L::kOffV + t * L::kRowD + c * 16) = vv;
+        const int ts = t < S ? t : 0;
+        cp_async16(sb + L::kOffK + t * L::kRowD + c * 16, kg + (size_t)ts * D + c * 8, t < S);
+        cp_async16(sb + L::kOffV + t * L::kRowD + c * 16, vg + (size_t)ts * D + c * 8, t < S);
     }
 
     // this warp's output tiles: all m-tiles (keys) x its kNT consecutive n-tiles (8 columns each)
@@ -108,14 +112,11 @@ bwd_dkv_mma_kernel(BwdArgs a)
         __syncthreads();  // previous chunk fully consumed (also orders the K/V staging above)
         for (int i = tid; i < kChunkRows * (D / 8); i += kDkvThreads) {
             const int r = i / (D / 8), c = i - r * (D / 8);
-            uint4 qv = make_uint4(0, 0, 0, 0), gv = make_uint4(0, 0, 0, 0);
-            if (r < rows) {
-                qv = __ldg(reinterpret_cast<const uint4 *>(qg + (size_t)(c0 + r) * D) + c);
-                gv = __ldg(reinterpret_cast<const uint4 *>(gg + (size_t)(c0 + r) * D) + c);
-            }
-            *reinterpret_cast<uint4 *>(smem + L::kOffQ + r * L::kRowD + c * 16) = qv;
-            *reinterpret_cast<uint4 *>(smem + L::kOffG + r * L::kRowD + c * 16) = gv;
+            const int rs = r < rows ? c0 + r : 0;
+            cp_async16(sb + L::kOffQ + r * L::kRowD + c * 16, qg + (size_t)rs * D + c * 8, r < rows);
+            cp_async16(sb + L::kOffG + r * L::kRowD + c * 16, gg + (size_t)rs * D + c * 8, r < rows);
         }
+        cp_async_wait_all();
         __syncthreads();
 
         // ---- phase 1: this warp's 16 rows: S = Q K^T, dP = dO V^T, then P and dS to shared memory
