@@ -9,16 +9,17 @@
 // partial results by their log-sum-exp), probabilities go back to tensor memory as bf16 and are
 // the A operand of the P*V contraction; `out` and `lse` are written once.
 //
-// Persistent CTA, one per SM, 16 warps:
+// Persistent CTA, one per SM, 20 warps:
 //   warp 0      TMA producer, score side (Q tile, prefix K blocks, suffix K of the tile)
 //   warp 1      tcgen05.mma issuer for the score blocks  S = Q K^T
 //   warp 2      tcgen05.mma issuer for the value blocks  O += P V   (owns the TMEM allocation)
-//   warp 3      TMA producer, value side (prefix V blocks, suffix V of the tile)
-//   warps 4-11  softmax, two warpgroups on alternate items: thread <-> query row (TMEM lane)
-//   warps 12-15 epilogue: O from tensor memory, normalise, bf16, shared-memory staging, TMA store
+//   warp 3      TMA producer, value side (prefix V blocks, suffix V of the tile); TMA stores of `out`
+//   warps 4-19  softmax, four warpgroups sharing each item by 32-column pieces (thread <-> query
+//               row = TMEM lane); the same warps normalise the finished tile's O into staging
 // An "item" is one (tile, key block) pair; tensor memory holds three 128-column score slots (the
-// bf16 probabilities of an item overwrite the first half of its own slot) and the 128 columns of O.  Every wait is on an event produced by an earlier
-// item of a role that never waits on the waiter, so no wait cycle can form; every wait is bounded.
+// bf16 probabilities of an item overwrite parts of its own slot) and the 128 columns of O.  Every
+// wait is on an event produced by an earlier item of a role that never waits on the waiter, so
+// no wait cycle can form; every wait is bounded.
 #include <string.h>
 
 #include "pskv_common.cuh"
@@ -31,11 +32,12 @@ namespace {
 using namespace sm100;
 
 constexpr int kSlots = 3;      // score slots of 128 columns; an item's probabilities overwrite its own scores
-constexpr int kThreads = 512;
+constexpr int kGroups = 4;     // softmax warpgroups: one 32-column piece of every score block each
+constexpr int kThreads = 32 * (4 + 4 * kGroups);
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
-// Probabilities are 2^(s * sl2) with no max subtracted; rows whose largest exponent exceeds
-// kMaxLog2 or whose row sum falls below kMinRowSum are redone by the general kernel.
-constexpr float kMaxLog2 = 100.0f;
+// Probabilities are 2^(s * sl2) with no max subtracted; rows whose sum leaves
+// [kMinRowSum, kMaxRowSum] are redone by the general kernel.
+constexpr float kMaxRowSum = 1.2676506002282294e30f;   // 2^100
 constexpr float kMinRowSum = 7.8886090522101181e-31f;  // 2^-100
 constexpr int kMaxStages = 4;
 
@@ -60,6 +62,7 @@ struct TcFwdParams {
     int resident;         // 1 when all prefix blocks of a KV head stay in shared memory
     int stages;           // streaming mode: stages of the prefix K and V rings
     int sfx_rows;         // rows of the suffix K / V buffers (multiple of 16, <= 128)
+    int alias_stage;      // 1 when the output staging buffer shares its memory with the suffix V buffer
     // shared-memory carve-up (byte offsets from the 1024-byte aligned base)
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml;
 };
@@ -79,11 +82,11 @@ enum {
     kBarSVFull,
     kBarSVFree,      // all value MMAs of a tile completed: suffix-V buffer is free
     kBarOFull,       // O of a tile is complete in tensor memory
-    kBarOFree,       // epilogue has read O out (4 arrivals)
-    kBarStageFull,   // the epilogue warps have written a slab of the output tile (4 arrivals)
+    kBarOFree,       // epilogue has read O out (one arrival per softmax warp)
+    kBarStageFull,   // the output tile is staged (one arrival per softmax warp)
     kBarStageFree,   // the TMA stores of that slab have read it
     kBarSFull,                        // [kSlots] scores of an item are in tensor memory
-    kBarPReady = kBarSFull + kSlots,  // [kSlots] probabilities written (4 arrivals)
+    kBarPReady = kBarSFull + kSlots,  // [kSlots] probabilities written (one arrival per softmax warp)
     kBarPvDone = kBarPReady + kSlots, // [kSlots] value MMAs of an item completed
     kBarKFull = kBarPvDone + kSlots,  // [stages]
     kBarVFull = kBarKFull + kMaxStages,
@@ -100,49 +103,8 @@ __device__ __forceinline__ int prefix_block_rows(const TcFwdParams &p, int k)
     return k == p.nblk_p - 1 ? p.tail_rows : kBlockN;
 }
 
-#ifndef PSKV_PIECE
-#define PSKV_PIECE 32
-#endif
-constexpr int kPiece = PSKV_PIECE;  // score columns a softmax thread handles per tensor-memory load
-__device__ __forceinline__ void tmem_ld_piece(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld16(taddr, r); }
-__device__ __forceinline__ void tmem_ld_piece(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld32(taddr, r); }
-__device__ __forceinline__ void tmem_st_piece(uint32_t taddr, const uint32_t (&r)[8]) { tmem_st8(taddr, r); }
-__device__ __forceinline__ void tmem_st_piece(uint32_t taddr, const uint32_t (&r)[16]) { tmem_st16(taddr, r); }
-
-// ---- softmax building blocks (one thread = one row; `rr` = 32 score columns of that row) -------
-
-// max over the valid columns [lo, lo + span] of chunk `ch`
-template <bool kMasked>
-__device__ __forceinline__ void chunk_max(const uint32_t (&rr)[32], float (&m4)[4], int ch, int lo, unsigned span,
-                                          bool any_col)
-{
-#pragma unroll
-    for (int c = 0; c < 32; ++c) {
-        float v = __uint_as_float(rr[c]);
-        if (kMasked) v = (any_col && (unsigned)(ch * 32 + c - lo) <= span) ? v : -INFINITY;
-        m4[c & 3] = fmaxf(m4[c & 3], v);
-    }
-}
-
-// p = 2^(s * sl2 - m_ref) for chunk `ch`, packed to bf16 pairs; adds to the two partial row sums
-template <bool kMasked>
-__device__ __forceinline__ void chunk_exp(const uint32_t (&rr)[32], uint32_t (&pk)[16], float &ls0, float &ls1,
-                                          float sl2, float neg_m, int ch, int lo, unsigned span, bool any_col)
-{
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        float x0 = fmaf(__uint_as_float(rr[2 * c]), sl2, neg_m);
-        float x1 = fmaf(__uint_as_float(rr[2 * c + 1]), sl2, neg_m);
-        if (kMasked) {
-            x0 = (any_col && (unsigned)(ch * 32 + 2 * c - lo) <= span) ? x0 : -INFINITY;
-            x1 = (any_col && (unsigned)(ch * 32 + 2 * c + 1 - lo) <= span) ? x1 : -INFINITY;
-        }
-        const float p0 = exp2f(x0), p1 = exp2f(x1);
-        ls0 += p0;
-        ls1 += p1;
-        pk[c] = pack_bf16x2(p0, p1);
-    }
-}
+constexpr int kPiece = 32;  // score columns a softmax thread handles per tensor-memory load
+static_assert(kBlockN == 4 * kPiece, "two softmax groups x two pieces cover a score block");
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -162,8 +124,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + p.off_misc + 4);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + p.off_misc);
-    volatile int *ml_read = reinterpret_cast<volatile int *>(smem + p.off_misc + 16);  // [4] tiles read, per quadrant
-    float *ml = reinterpret_cast<float *>(smem + p.off_ml);  // partial row sums [tile parity][softmax group][128]
+    float *ml = reinterpret_cast<float *>(smem + p.off_ml);  // partial row sums [tile % 4][softmax group][128]
 
     if ((sbase & 1023u) != 0u) {  // the swizzled layouts need a 1024-byte aligned base
         if (tid == 0) atomicCAS(p.status, 0u, (unsigned int)kErrAlign);
@@ -175,11 +136,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
-            const bool four = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
-            mbar_init(bar(i), four ? 4u : 1u);
+            const bool all_sm = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
+            mbar_init(bar(i), all_sm ? (uint32_t)(4 * kGroups) : 1u);
         }
         *abort_flag = 0;
-        for (int i = 0; i < 4; ++i) ml_read[i] = 0;
         fence_barrier_init();
     }
     fence_proxy_async();
@@ -205,7 +165,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     // The producer and MMA warps run their loops with all 32 lanes (warp-uniform control flow and
     // addresses, so descriptors can live in uniform registers); one elected lane issues the
     // asynchronous instructions.
-    if (warp == 0) {
+#ifdef PSKV_SWAP23
+    const int role = warp == 2 ? 3 : warp == 3 ? 2 : warp;
+#else
+    const int role = warp;
+#endif
+    if (role == 0) {
         // ------------------------------------------------------------------ producer, score side
         if (lane == 0) {
             prefetch_tensormap(&tm_q);
@@ -274,53 +239,37 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             __syncwarp();
         }
-    } else if (warp == 3) {
+    } else if (role == 3) {
         // ------------------------------------------------------------------ producer, value side
         if (lane == 0) {
             prefetch_tensormap(&tm_sv);
+            prefetch_tensormap(&tm_out);
             if (p.P > 0) { prefetch_tensormap(&tm_pv); prefetch_tensormap(&tm_pv_tail); }
         }
         uint32_t vload = 0;
         bool ok = true;
-        for (int tl = 0; tl < n_tiles && ok; ++tl) {
-            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
-            if (p.resident) {
-                // suffix V and the resident prefix V blocks are free once every value MMA of the
-                // previous tile has completed
-                ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
-                if (!ok) break;
-                if (t.first_of_g && elect_one_sync()) {
-                    for (int k = 0; k < p.nblk_p; ++k) {
-                        const bool tail = k == p.nblk_p - 1;
-                        const int slab = tail ? tail_slab : C::kSlabBytes;
-                        mbar_arrive_expect_tx(bar(kBarVFull + k), (uint32_t)(C::kSlabs * slab));
-                        for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
-                                        bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
+        // This warp also issues the TMA stores of each finished output tile.  The staging buffer
+        // of a tile shares its shared memory with the suffix V of the tiles around it: tile t's
+        // output is staged after that tile's last value MMA has read suffix V, and suffix V of
+        // tile t+1 is fetched only once the stores of tile t have read the staging buffer.
+        const uint32_t stage = sbase + p.off_stage;
+        auto store_tile = [&](int ts) {  // StageFull of tile ts has been seen
+            const TileInfo u = tile_info(p, t_begin + ts, t_begin);
+            const int nseg = u.rows / p.seg_rows;
+            if (elect_one_sync()) {
+                for (int sl = 0; sl < C::kSlabs; ++sl)
+                    for (int s = 0; s < nseg; ++s) {
+                        const int R = u.R0 + s * p.seg_rows;
+                        const int b = R / p.Rg, r = R - b * p.Rg;
+                        tma_store_4d(&tm_out, stage + sl * kStagingBytes + s * p.seg_rows * 128, sl * 64, r, u.g, b);
                     }
-                }
-                __syncwarp();
-            } else {
-                for (int k = 0; k < p.nblk_p; ++k) {
-                    const uint32_t vs = vload % (uint32_t)p.stages;
-                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
-                                        p.status, kErrProducerV);
-                    if (!ok) break;
-                    const bool tail = k == p.nblk_p - 1;
-                    const int slab = tail ? tail_slab : C::kSlabBytes;
-                    if (elect_one_sync()) {
-                        mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
-                        for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
-                                        bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
-                    }
-                    __syncwarp();
-                    ++vload;
-                }
-                if (!ok) break;
-                ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
-                if (!ok) break;
+                tma_store_commit();
+                tma_store_wait_read();  // the staging buffer may be overwritten after this
+                mbar_arrive(bar(kBarStageFree));
             }
+            __syncwarp();
+        };
+        auto load_suffix_v = [&](const TileInfo &t) {
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
                 for (int c = 0; c < t.nc; ++c)
@@ -329,8 +278,90 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                                     sl * 64, 0, t.g, t.b_first + c);
             }
             __syncwarp();
+        };
+        for (int tl = 0; tl <= n_tiles && ok; ++tl) {
+            const bool have_tile = tl < n_tiles;
+            // Two jobs ride along with the prefix loads of tile tl: the stores of tile tl-1 (once it
+            // is staged) and the fetch of this tile's suffix V (once its buffer is free: after those
+            // stores when it doubles as the staging buffer, else after the previous tile's value MMAs).
+            bool pend_store = tl > 0, pend_sv = have_tile;
+            TileInfo t;
+            auto poll_sv = [&](bool block) -> bool {
+                if (!pend_sv || (p.alias_stage && pend_store)) return true;
+                bool ready = true;
+                if (!p.alias_stage && tl > 0) {
+                    if (block)
+                        ready = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
+                    else
+                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarSVFree), (tl & 1) ^ 1) ? 1 : 0, 0) != 0;
+                    if (block && !ready) return false;
+                }
+                if (ready) {
+                    load_suffix_v(t);
+                    pend_sv = false;
+                }
+                return true;
+            };
+            auto poll = [&](bool block) -> bool {
+                if (!p.alias_stage && !poll_sv(block)) return false;
+                if (pend_store) {
+                    bool ready;
+                    if (block)
+                        ready = mbar_wait_warp(bar(kBarStageFull), (tl - 1) & 1, abort_flag, p.status, kErrEpilogue);
+                    else
+                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarStageFull), (tl - 1) & 1) ? 1 : 0, 0) != 0;
+                    if (block && !ready) return false;
+                    if (ready) {
+                        store_tile(tl - 1);
+                        pend_store = false;
+                    }
+                }
+                return poll_sv(block);
+            };
+            if (have_tile) {
+                t = tile_info(p, t_begin + tl, t_begin);
+                if (p.resident) {
+                    // the resident prefix V blocks are free once every value MMA of the previous tile
+                    // has completed
+                    ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
+                    if (!ok) break;
+                    if (t.first_of_g && elect_one_sync()) {
+                        for (int k = 0; k < p.nblk_p; ++k) {
+                            const bool tail = k == p.nblk_p - 1;
+                            const int slab = tail ? tail_slab : C::kSlabBytes;
+                            mbar_arrive_expect_tx(bar(kBarVFull + k), (uint32_t)(C::kSlabs * slab));
+                            for (int sl = 0; sl < C::kSlabs; ++sl)
+                                tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab,
+                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
+                        }
+                    }
+                    __syncwarp();
+                } else {
+                    for (int k = 0; k < p.nblk_p; ++k) {
+                        const uint32_t vs = vload % (uint32_t)p.stages;
+                        ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
+                                            p.status, kErrProducerV);
+                        if (!ok) break;
+                        const bool tail = k == p.nblk_p - 1;
+                        const int slab = tail ? tail_slab : C::kSlabBytes;
+                        if (elect_one_sync()) {
+                            mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
+                            for (int sl = 0; sl < C::kSlabs; ++sl)
+                                tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab,
+                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                        }
+                        __syncwarp();
+                        ++vload;
+                        poll(false);
+                    }
+                    if (!ok) break;
+                }
+            }
+            ok = poll(true);
         }
-    } else if (warp == 1) {
+        if (elect_one_sync()) tma_store_wait_all();
+        __syncwarp();
+    } else if (role == 1) {
         // ------------------------------------------------------------------ score MMAs: S = Q K^T
         const int total_items = n_tiles * nitems;
         int tl = 0, k = 0;
@@ -396,7 +427,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
-    } else if (warp == 2) {
+    } else if (role == 2) {
         // ------------------------------------------------------------------ value MMAs: O += P V
         const int total_items = n_tiles * nitems;
         int tl = 0, k = 0;
@@ -447,7 +478,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll
                 for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
                     if (ks16 < nk)
-                        mma_ts(tmem + kOCol, p_tmem + ks16 * 8, v_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_pv,
+                        mma_ts(tmem + kOCol, p_tmem + (ks16 >> 1) * kPiece + (ks16 & 1) * 8, v_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_pv,
                                ks16 > 0 ? 1u : acc0);
                 }
                 tc_commit(bar(kBarPvDone + slot));
@@ -465,216 +496,180 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
-    } else if (warp < 12) {
-        // ------------------------------------------------------------------ softmax warps (4..11)
-        // Two warpgroups take alternate items (group = item parity), so
-        // that one group's tensor-memory round trips hide behind the other's exponentials.  Each
-        // thread owns one query row (tensor-memory lane) and makes one pass over a score block, a
-        // piece of columns at a time with the next piece in flight: p = 2^(s * sl2), row sum, bf16
-        // pairs into the item's probability slot.  No running max is subtracted: bf16 and fp32
-        // share an 8-bit exponent, so the quotient O / l is exact to rounding for any row whose
-        // largest s * sl2 lies within +-kMaxLog2; a row outside that range (essentially never, it
-        // means logits beyond +-69 nats) is marked through a NaN row sum and redone afterwards by
-        // the general kernel with max subtraction.  The groups share no state; their partial row
-        // sums meet in the epilogue.
+    } else {
+        // ------------------------------------------------- softmax + epilogue warps (4..19)
+        // Four warpgroups work on every item: the 128 score columns are four pieces of 32 and
+        // group j takes piece j, so that each scheduler always has four independent softmax warps
+        // to hide the others' tensor-memory and barrier latencies.  Each thread owns one query
+        // row (tensor-memory lane): p = 2^(s * sl2), row sum, bf16 pairs written over the first
+        // half of the piece they came from (a group only ever overwrites columns it has read
+        // itself).  No running max is subtracted: bf16 and fp32 share an 8-bit exponent, so the
+        // quotient O / l is exact to rounding for any row whose sum stays within [2^-100, 2^100];
+        // a row outside that range (essentially never, it means logits beyond +-69 nats) is
+        // redone afterwards by the general kernel with max subtraction.  The groups share no
+        // state; their partial row sums meet in the epilogue, which the same warps run for the
+        // previous tile (group j normalises O columns [32j, 32j+32)) right after the first item
+        // of the next one, when that tile's last value MMAs have long completed.
         const int wg = (warp - 4) >> 2;
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
         bool ok = true;
+        float lsum = 0.f;
 #pragma unroll 1
-        for (int tl = 0; tl < n_tiles && ok; ++tl) {
-            const int item0 = tl * nitems;
-            // my items of this tile: k with (item0 + k) parity == wg
-            const int k_first = ((item0 & 1) == wg) ? 0 : 1;
-            if (k_first >= nitems) continue;
-            const int k_last = k_first + ((nitems - 1 - k_first) & ~1);
-            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
-            const bool valid = row < t.rows;
-            const int R = t.R0 + (valid ? row : 0);
-            const int b = R / p.Rg, r = R - b * p.Rg;
-            const int sfx_lo = (b - t.b_first) * p.S;   // first suffix column of this row's candidate
-            const int sfx_hi = sfx_lo + (r % p.S);      // causal: suffix keys 0..i
-            float l = 0.f, smax = -INFINITY;
+        for (int tl = 0; tl <= n_tiles && ok; ++tl) {
+            const bool have_tile = tl < n_tiles;
+            TileInfo t;
+            int lo_sfx = 1, hi_sfx = 0;
+            if (have_tile) {
+                t = tile_info(p, t_begin + tl, t_begin);
+                if (row < t.rows) {
+                    const int R = t.R0 + row;
+                    const int b = R / p.Rg, r = R - b * p.Rg;
+                    lo_sfx = (b - t.b_first) * p.S;  // first suffix column of this row's candidate
+                    hi_sfx = lo_sfx + (r % p.S);     // causal: suffix keys 0..i
+                }
+                lsum = 0.f;
+            }
+            const int nk = have_tile ? nitems : 1;
 #pragma unroll 1
-            for (int k = k_first; k < nitems && ok; k += 2) {
-                const int item = item0 + k, slot = item % kSlots;
-                // scores and (over their first half, piece by piece behind the reads) probabilities
-                const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
-                const uint32_t p_tmem = s_tmem;
-                // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
-                // blocks like real rows (their scores are finite and never stored) and see no suffix key.
-                int n, lo, hi;
-                if (k < p.nblk_p) {
-                    n = prefix_block_rows(p, k);
-                    lo = 0;
-                    hi = min(kBlockN, p.P - k * kBlockN) - 1;
-                } else {
-                    n = t.n_sfx;
-                    lo = valid ? sfx_lo : 1;
-                    hi = valid ? sfx_hi : 0;
-                }
-                const int nh = (n + kPiece - 1) / kPiece;
-                // `full`: no column of any piece needs masking (also none past n in the last piece)
-                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1) && (n % kPiece == 0);
-                int h_b = 0, h_e = nh - 1;  // pieces that hold a valid column of some row of this warp
-                if (!full) {
-                    const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
-                    const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
-                    h_b = wlo / kPiece;
-                    h_e = min(nh - 1, whi / kPiece);
-                }
-                const unsigned span = (unsigned)(hi - lo);
-                const bool any_col = hi >= lo;
-
-                ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
-                if (!ok) break;
-                tc_fence_after();
-                PSKV_TRACE_EVENT(20, item);
-
-                float ls0 = 0.f, ls1 = 0.f;
-                float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                auto piece = [&](int h, const uint32_t (&rr)[kPiece]) {
-                    uint32_t pk[kPiece / 2];
-                    if (h >= h_b && h <= h_e) {
-                        float v[kPiece];
-#pragma unroll
-                        for (int c = 0; c < kPiece; ++c) {
-                            v[c] = __uint_as_float(rr[c]);
-                            if (!full) v[c] = (any_col && (unsigned)(h * kPiece + c - lo) <= span) ? v[c] : -INFINITY;
-                            m4[c & 3] = fmaxf(m4[c & 3], v[c]);
-                        }
-#pragma unroll
-                        for (int c = 0; c < kPiece / 2; ++c) {
-                            const float p0 = exp2f(v[2 * c] * p.sl2);  // -inf -> 0
-                            const float p1 = exp2f(v[2 * c + 1] * p.sl2);
-                            ls0 += p0;
-                            ls1 += p1;
-                            pk[c] = pack_bf16x2(p0, p1);
-                        }
+            for (int k = 0; k < nk && ok; ++k) {
+                if (have_tile) {
+                    const int item = tl * nitems + k, slot = item % kSlots;
+                    const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN + wg * kPiece;
+                    // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
+                    // blocks like real rows (their scores are finite and never stored) and see no
+                    // suffix key.
+                    int n, lo, hi;
+                    if (k < p.nblk_p) {
+                        n = prefix_block_rows(p, k);
+                        lo = 0;
+                        hi = min(kBlockN, p.P - k * kBlockN) - 1;
                     } else {
-#pragma unroll
-                        for (int c = 0; c < kPiece / 2; ++c) pk[c] = 0u;
+                        n = t.n_sfx;
+                        lo = lo_sfx;
+                        hi = hi_sfx;
                     }
-                    tmem_st_piece(p_tmem + h * (kPiece / 2), pk);
-                };
-                {
-                    uint32_t ra[kPiece], rb[kPiece];
-                    if (h_b == 0 && h_e >= 0) tmem_ld_piece(s_tmem, ra);
-#pragma unroll 1
-                    for (int h = 0; h < nh; h += 2) {
-                        tmem_wait_ld();
-                        if (h + 1 >= h_b && h + 1 <= h_e) tmem_ld_piece(s_tmem + (h + 1) * kPiece, rb);
-                        piece(h, ra);
-                        if (h + 1 < nh) {
-                            tmem_wait_ld();
-                            if (h + 2 >= h_b && h + 2 <= h_e) tmem_ld_piece(s_tmem + (h + 2) * kPiece, ra);
-                            piece(h + 1, rb);
-                        }
+                    const int c0 = wg * kPiece;  // first column of my piece
+                    // my piece: 0 = not read by the value MMAs, 1 = no valid column for this warp
+                    // (zeros), 2 = some columns masked, 3 = all columns valid for all rows
+                    int kind = 0;
+                    if (c0 < n) {
+                        const bool all_valid = lo <= c0 && hi >= c0 + kPiece - 1;
+                        const bool none_valid = hi < lo || hi < c0 || lo > c0 + kPiece - 1;
+                        kind = __all_sync(0xffffffffu, all_valid) ? 3 : __all_sync(0xffffffffu, none_valid) ? 1 : 2;
                     }
-                }
-                l += ls0 + ls1;
-                smax = fmaxf(smax, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
-                if (k == k_last) {
-                    // hand this group's partial row sum to the epilogue; the buffer of tile tl-2 must
-                    // have been read first
-                    if (tl >= 2) {
-                        ok = __all_sync(0xffffffffu, spin_wait_ge(ml_read + (warp & 3), tl - 1, abort_flag, p.status,
-                                                                  kErrSoftmax));
-                        if (!ok) break;
-                        __threadfence_block();
-                    }
-                    ml[((tl & 1) * 2 + wg) * kTileM + row] = (smax * p.sl2 > kMaxLog2) ? __int_as_float(0x7fc00000) : l;
-                }
-                PSKV_TRACE_EVENT(23, item);
-                tmem_wait_st();
-                tc_fence_before();
-                __threadfence_block();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPReady + slot));
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ epilogue warps (12..15)
-        const int ew = warp & 3;
-        const int row = 32 * ew + lane;
-        const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
-        const uint32_t stage = sbase + p.off_stage;
-        const bool issuer = warp == 12;  // this warp's elected lane issues the TMA stores
-        if (issuer && lane == 0) prefetch_tensormap(&tm_out);
-        bool ok = true;
-#pragma unroll 1
-        for (int tl = 0; tl < n_tiles && ok; ++tl) {
-            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
-            ok = mbar_wait_warp(bar(kBarOFull), tl & 1, abort_flag, p.status, kErrEpilogue);
-            if (!ok) break;
-            PSKV_TRACE_EVENT(30, tl);
-            tc_fence_after();
-            // row sum = the partial sums of the softmax groups that had an item in this tile
-            const int par0 = (tl * nitems) & 1;
-            float lsum = ml[((tl & 1) * 2 + par0) * kTileM + row];
-            if (nitems > 1) lsum += ml[((tl & 1) * 2 + (par0 ^ 1)) * kTileM + row];
-            __threadfence_block();
-            __syncwarp();
-            if (lane == 0) ml_read[ew] = tl + 1;  // this warp's rows of the tile's partial sums have been read
-            const bool row_ok = lsum >= kMinRowSum;  // false for NaN (marked row) and for underflow
-            const float inv = 1.f / lsum;
-            uint32_t ob[D / 2];  // the normalised row as bf16 pairs
-#pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch) {
-                uint32_t o[32];
-                tmem_ld32(tmem + lane_addr + kOCol + ch * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 16; ++c)
-                    ob[ch * 16 + c] = pack_bf16x2(__uint_as_float(o[2 * c]) * inv, __uint_as_float(o[2 * c + 1]) * inv);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarOFree));
-            const bool stored = row < t.rows;
-            if (stored) {
-                const int R = t.R0 + row;
-                const int b = R / p.Rg, r = R - b * p.Rg;
-                const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
-                p.lse[grow] = row_ok ? log2f(lsum) * kLn2 : __int_as_float(0x7fc00000);
-            }
-            const unsigned bad = __ballot_sync(0xffffffffu, stored && !row_ok);
-            if (bad != 0u && lane == 0) atomicAdd(p.redo_count, (unsigned int)__popc(bad));
-            // out: one 64-column slab at a time through the swizzled staging buffer, then TMA stores
-            const int nseg = t.rows / p.seg_rows;
-#pragma unroll
-            for (int sl = 0; sl < C::kSlabs; ++sl) {
-                const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
-                ok = mbar_wait_warp(bar(kBarStageFree), (round & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
-                if (!ok) break;
-                uint8_t *srow = smem + p.off_stage + row * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) =
-                        make_uint4(ob[sl * 32 + 4 * c], ob[sl * 32 + 4 * c + 1], ob[sl * 32 + 4 * c + 2],
-                                   ob[sl * 32 + 4 * c + 3]);
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarStageFull));
-                if (issuer) {
-                    ok = mbar_wait_warp(bar(kBarStageFull), round & 1, abort_flag, p.status, kErrEpilogue);
+                    PSKV_TRACE_EVENT(25, item);
+                    ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
                     if (!ok) break;
-                    if (elect_one_sync()) {
-                        for (int s = 0; s < nseg; ++s) {
-                            const int R = t.R0 + s * p.seg_rows;
-                            const int b = R / p.Rg, r = R - b * p.Rg;
-                            tma_store_4d(&tm_out, stage + s * p.seg_rows * 128, sl * 64, r, t.g, b);
+                    tc_fence_after();
+                    PSKV_TRACE_EVENT(20, item);
+                    if (kind != 0) {
+                        uint32_t rr[kPiece], pk[kPiece / 2];
+                        if (kind >= 2) {
+                            tmem_ld32(s_tmem, rr);
+                            tmem_wait_ld();
                         }
-                        tma_store_commit();
-                        tma_store_wait_read();  // the staging buffer may be overwritten after this
-                        mbar_arrive(bar(kBarStageFree));
+                        PSKV_TRACE_EVENT(21, item);
+                        float ls0 = 0.f, ls1 = 0.f;
+                        if (kind == 3) {
+#pragma unroll
+                            for (int c = 0; c < kPiece / 2; ++c) {
+                                const float p0 = exp2f(__uint_as_float(rr[2 * c]) * p.sl2);
+                                const float p1 = exp2f(__uint_as_float(rr[2 * c + 1]) * p.sl2);
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[c] = pack_bf16x2(p0, p1);
+                            }
+                        } else if (kind == 2) {
+                            const unsigned span = (unsigned)(hi - lo);
+                            const int base = c0 - lo;
+                            const bool any_col = hi >= lo;
+#pragma unroll
+                            for (int c = 0; c < kPiece / 2; ++c) {
+                                const bool in0 = any_col && (unsigned)(base + 2 * c) <= span;
+                                const bool in1 = any_col && (unsigned)(base + 2 * c + 1) <= span;
+                                const float p0 = in0 ? exp2f(__uint_as_float(rr[2 * c]) * p.sl2) : 0.f;
+                                const float p1 = in1 ? exp2f(__uint_as_float(rr[2 * c + 1]) * p.sl2) : 0.f;
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[c] = pack_bf16x2(p0, p1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < kPiece / 2; ++c) pk[c] = 0u;
+                        }
+                        lsum += ls0 + ls1;
+                        tmem_st16(s_tmem, pk);
                     }
+                    if (k == nitems - 1) ml[((tl & 3) * kGroups + wg) * kTileM + row] = lsum;
+                    PSKV_TRACE_EVENT(23, item);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __threadfence_block();
                     __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarPReady + slot));
+                    PSKV_TRACE_EVENT(24, item);
+                }
+                if (k == 0 && tl > 0) {
+                    // ---- epilogue of tile tl-1: O / l -> bf16 -> staging; lse; rows to redo
+                    const int te = tl - 1;
+                    const TileInfo u = tile_info(p, t_begin + te, t_begin);
+                    ok = mbar_wait_warp(bar(kBarOFull), te & 1, abort_flag, p.status, kErrEpilogue);
+                    if (!ok) break;
+                    PSKV_TRACE_EVENT(30, te);
+                    tc_fence_after();
+                    const float *mlt = ml + (te & 3) * kGroups * kTileM + row;
+                    const float l = (mlt[0] + mlt[kTileM]) + (mlt[2 * kTileM] + mlt[3 * kTileM]);
+                    const bool row_ok = l >= kMinRowSum && l <= kMaxRowSum;  // false for overflow (inf, NaN), underflow
+                    const float inv = 1.f / l;
+                    const bool mine = wg < D / kPiece;  // this group has O columns
+                    uint32_t ob[kPiece / 2];
+                    if (mine) {
+                        uint32_t o[kPiece];
+                        tmem_ld32(tmem + lane_addr + kOCol + wg * kPiece, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < kPiece / 2; ++c)
+                            ob[c] = pack_bf16x2(__uint_as_float(o[2 * c]) * inv, __uint_as_float(o[2 * c + 1]) * inv);
+                        // staged values must be finite (the buffer doubles as suffix V, whose padding
+                        // rows meet zero probabilities); rows that failed are redone anyway
+                        if (!row_ok) {
+#pragma unroll
+                            for (int c = 0; c < kPiece / 2; ++c) ob[c] = 0u;
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarOFree));
+                    if (wg == 0) {
+                        const bool stored = row < u.rows;
+                        if (stored) {
+                            const int R = u.R0 + row;
+                            const int b = R / p.Rg, r = R - b * p.Rg;
+                            const size_t grow = ((size_t)b * p.Hq + (size_t)u.g * p.n_rep) * p.S + r;
+                            p.lse[grow] = row_ok ? log2f(l) * kLn2 : __int_as_float(0x7fc00000);
+                        }
+                        const unsigned bad = __ballot_sync(0xffffffffu, stored && !row_ok);
+                        if (bad != 0u && lane == 0) atomicAdd(p.redo_count, (unsigned int)__popc(bad));
+                    }
+                    // the TMA stores of the previous tile must have read the staging buffer
+                    ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
+                    if (!ok) break;
+                    if (mine) {
+                        // 64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row
+                        uint8_t *srow = smem + p.off_stage + (wg >> 1) * kStagingBytes + row * 128;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            *reinterpret_cast<uint4 *>(srow + ((((wg & 1) * 4 + c) ^ (row & 7)) << 4)) =
+                                make_uint4(ob[4 * c], ob[4 * c + 1], ob[4 * c + 2], ob[4 * c + 3]);
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarStageFull));
+                    PSKV_TRACE_EVENT(31, te);
                 }
             }
-            PSKV_TRACE_EVENT(31, tl);
         }
-        if (issuer && elect_one_sync()) tma_store_wait_all();
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -690,7 +685,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 struct TilePlan {
     bool ok;
     int tile_rows, seg_rows, tiles_per_group, sfx_rows;
-    int nblk_p, tail_rows, resident, stages;
+    int nblk_p, tail_rows, resident, stages, alias_stage;
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml, smem_bytes;
 };
 
@@ -712,31 +707,43 @@ TilePlan plan_tiles(const Dims &dm)
     const int tile_bytes = slabs * kTileM * 128;
     const int sfx_bytes = round_up(slabs * pl.sfx_rows * 128, 1024);
     const int tail_bytes = round_up(slabs * pl.tail_rows * 128, 1024);
-    const int tail_area = 2 * kTileM * 8 /*ml*/ + 64 /*misc*/ + kBarBytes;
-    const int fixed = tile_bytes /*Q*/ + 2 * sfx_bytes + kStagingBytes + tail_area;
+    const int ml_bytes = 4 * kGroups * kTileM * 4;  // partial row sums of four tiles in flight
+    const int stage_bytes = slabs * kStagingBytes;
+    const int tail_area = ml_bytes + 64 /*misc*/ + kBarBytes;
+    // The output staging buffer gets memory of its own when that costs neither the residency of
+    // the prefix nor a ring stage; otherwise it shares the suffix V buffer (value-side producer).
+    const int fixed_own = tile_bytes /*Q*/ + 2 * sfx_bytes + stage_bytes + tail_area;
+    const int shared_sv = sfx_bytes > stage_bytes ? sfx_bytes : stage_bytes;
+    const int fixed_shared = tile_bytes + sfx_bytes + shared_sv + tail_area;
     const int resident_bytes = pl.nblk_p ? (pl.nblk_p - 1) * tile_bytes + tail_bytes : 0;
+    auto ring_stages = [&](int fixed) {
+        const int st = (kMaxSmem - fixed) / (2 * tile_bytes);
+        return st > kMaxStages ? kMaxStages : st;
+    };
     int kv_bytes = 0;  // bytes of the prefix K area (the V area has the same size)
-    if (pl.nblk_p <= kMaxStages && fixed + 2 * resident_bytes <= kMaxSmem) {
+    if (pl.nblk_p <= kMaxStages && fixed_shared + 2 * resident_bytes <= kMaxSmem) {
         pl.resident = 1;
         pl.stages = pl.nblk_p;
         kv_bytes = resident_bytes;
+        pl.alias_stage = fixed_own + 2 * resident_bytes <= kMaxSmem ? 0 : 1;
     } else {
-        int st = (kMaxSmem - fixed) / (2 * tile_bytes);
-        if (st > kMaxStages) st = kMaxStages;
-        if (st < 2) return pl;  // does not fit: the general kernels take the shape
+        const int st = ring_stages(fixed_shared);
+        if (st < 1) return pl;  // does not fit: the general kernels take the shape
         pl.stages = st;
         kv_bytes = st * tile_bytes;
+        pl.alias_stage = ring_stages(fixed_own) == st ? 0 : 1;
     }
+    const int sv_bytes = pl.alias_stage ? shared_sv : sfx_bytes;
     pl.off_pk = 0;
     pl.off_pv = pl.off_pk + kv_bytes;
     pl.off_q = pl.off_pv + kv_bytes;
     pl.off_sk = pl.off_q + tile_bytes;
     pl.off_sv = pl.off_sk + sfx_bytes;
-    pl.off_stage = pl.off_sv + sfx_bytes;
-    pl.off_bar = pl.off_stage + kStagingBytes;
+    pl.off_stage = pl.alias_stage ? pl.off_sv : pl.off_sv + sv_bytes;
+    pl.off_bar = pl.off_stage + (pl.alias_stage ? sv_bytes : stage_bytes);
     pl.off_misc = pl.off_bar + kBarBytes;
     pl.off_ml = pl.off_misc + 64;
-    pl.smem_bytes = pl.off_ml + 2 * kTileM * 8;
+    pl.smem_bytes = pl.off_ml + ml_bytes;
     pl.ok = pl.smem_bytes <= kMaxSmem;
     return pl;
 }
@@ -793,6 +800,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.resident = plan.resident;
     p.stages = plan.stages > 0 ? plan.stages : 1;
     p.sfx_rows = plan.sfx_rows;
+    p.alias_stage = plan.alias_stage;
     p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_sk = plan.off_sk;
     p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
     p.off_ml = plan.off_ml;
@@ -833,7 +841,7 @@ extern "C" int pskv_debug_read_trace(long long *host, int max_events)
     for (int w = 0; w < kTraceWarps; ++w)
         for (unsigned int i = 0; i < cnt[w] && i < (unsigned int)kTraceCap && n < max_events; ++i, ++n) {
             host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
-            host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1];
+            host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1] | ((long long)w << 24);
         }
     return n;
 }
