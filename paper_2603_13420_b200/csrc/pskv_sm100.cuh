@@ -64,16 +64,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // `code` in the device status word and returns false; the caller then leaves its role loop.
 constexpr long long kWaitBudgetCycles = 2000000000ll;  // about one second at B200 clocks
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          unsigned int *status_word, unsigned int code)
+// The polling loop is one shared out-of-line routine: the kernels' hot loops stay small enough for
+// the instruction cache, and a wait that is already satisfied costs one inlined try_wait.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                            unsigned int *status_word, unsigned int code)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     for (unsigned int spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-#ifdef PSKV_WAIT_SLEEP_NS
-        __nanosleep(PSKV_WAIT_SLEEP_NS);
-#endif
         if ((spin & 63u) == 0u) {
             if (*abort_flag != 0) return false;
             if (clock64() - start > kWaitBudgetCycles) {
@@ -83,6 +81,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             }
         }
     }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned int *status_word, unsigned int code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status_word, code);
 }
 
 // Bounded wait until a monotonically increasing shared-memory counter reaches `target`.
@@ -310,6 +315,14 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "}" ::"r"(d_tmem),
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+
+// 2^x on the special-function unit (flushes denormals; 2^-inf = 0)
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)

@@ -47,6 +47,7 @@ struct TcBwdParams {
     float scale;
     int B, Hq, Hkv, S, P, n_rep;
     int Rg, tile_rows, seg_rows, tiles_per_group, total_tiles;
+    FastDiv fd_tpg, fd_Rg, fd_S;  // divisions by tiles_per_group, Rg, S
     int nblk_p, tail_rows, resident, stages_k, stages_v, sfx_rows;  // ring stages of prefix K / V (streaming mode)
     int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc;
 };
@@ -137,7 +138,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
     const int n_tiles = t_end - t_begin;
     const int nitems = p.nblk_p + 1;
-    const int g_first = t_begin / p.tiles_per_group;
+    const int g_first = p.fd_tpg.div(t_begin);
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
     const uint32_t stages_k = (uint32_t)p.stages_k, stages_v = (uint32_t)p.stages_v;
@@ -156,12 +157,12 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdA);
             if (!ok) break;
-            const int nseg = t.rows / p.seg_rows;
+            const int nseg = t.rows / p.seg_rows;  // (once per tile)
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
                     const int R = t.R0 + s * p.seg_rows;
-                    const int b = R / p.Rg, r = R - b * p.Rg;
+                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
                                     bar(kBarQFull), sl * 64, r, t.g, b);
@@ -227,12 +228,12 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             ok = mbar_wait_warp(bar(kBarDvFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdB);
             if (!ok) break;
-            const int nseg = t.rows / p.seg_rows;
+            const int nseg = t.rows / p.seg_rows;  // (once per tile)
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarDoFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
                     const int R = t.R0 + s * p.seg_rows;
-                    const int b = R / p.Rg, r = R - b * p.Rg;
+                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + p.off_do + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_do,
                                     bar(kBarDoFull), sl * 64, r, t.g, b);
@@ -431,9 +432,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             const bool valid = row < t.rows;
             const int R = t.R0 + (valid ? row : 0);
-            const int b = R / p.Rg, r = R - b * p.Rg;
+            const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
             const int sfx_lo = (b - t.b_first) * p.S;
-            const int sfx_hi = sfx_lo + (r % p.S);
+            const int sfx_hi = sfx_lo + (r - p.fd_S.div(r) * p.S);
             const size_t grow = ((size_t)b * p.Hq + (size_t)t.g * p.n_rep) * p.S + r;
             // padding rows: lse = +inf makes every probability (and so every dS) zero
             const float neg_lse2 = valid ? -p.lse[grow] * kLog2e : -INFINITY;
@@ -547,7 +548,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarDqFree));
-            const int nseg = t.rows / p.seg_rows;
+            const int nseg = t.rows / p.seg_rows;  // (once per tile)
 #pragma unroll
             for (int sl = 0; sl < C::kSlabs; ++sl) {
                 const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
@@ -568,7 +569,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     if (elect_one_sync()) {
                         for (int s = 0; s < nseg; ++s) {
                             const int R = t.R0 + s * p.seg_rows;
-                            const int b = R / p.Rg, r = R - b * p.Rg;
+                            const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
                             tma_store_4d(&tm_dq, stage + s * p.seg_rows * 128, sl * 64, r, t.g, b);
                         }
                         tma_store_commit();
@@ -690,6 +691,9 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.tile_rows = plan.tile_rows;
     p.seg_rows = plan.seg_rows;
     p.tiles_per_group = plan.tiles_per_group;
+    p.fd_tpg.init(plan.tiles_per_group);
+    p.fd_Rg.init(Rg);
+    p.fd_S.init(dm.S);
     p.total_tiles = plan.tiles_per_group * dm.Hkv;
     p.nblk_p = plan.nblk_p;
     p.tail_rows = plan.tail_rows;

@@ -42,24 +42,43 @@ __device__ unsigned int g_trace_n[kTraceWarps];
 #define PSKV_TRACE_EVENT(tag, val) do { } while (0)
 #endif
 
+// Division by a divisor fixed at launch: one 32x32->64 multiply and a shift instead of the long
+// instruction sequence of a general integer division.  Exact for 0 <= n < 2^31, 1 <= d < 2^31:
+// with L = ceil(log2 d) and M = ceil(2^(31+L) / d), floor(n / d) = (n * M) >> (31 + L).
+struct FastDiv {
+    unsigned int mul, shift, d;
+    __host__ void init(int divisor)
+    {
+        d = (unsigned int)divisor;
+        unsigned int L = 0;
+        while ((1ull << L) < (unsigned long long)d) ++L;
+        shift = 31u + L;
+        mul = (unsigned int)(((1ull << shift) + d - 1) / d);
+    }
+    __device__ __forceinline__ int div(int n) const
+    {
+        return (int)(((unsigned long long)(unsigned int)n * mul) >> shift);
+    }
+};
+
 struct TileInfo {
     int g, R0, rows, b_first, nc, n_sfx;  // n_sfx: suffix columns rounded up to 16
     bool first_of_g;
 };
 
-// `Params` is any kernel parameter block with fields B, Rg, S, tile_rows, tiles_per_group.
+// `Params` is any kernel parameter block with fields B, Rg, S, tile_rows, tiles_per_group, fd_tpg, fd_Rg.
 template <class Params>
 __device__ __forceinline__ TileInfo tile_info(const Params &p, int tile, int t_begin)
 {
     TileInfo t;
-    t.g = tile / p.tiles_per_group;
+    t.g = p.fd_tpg.div(tile);
     const int tt = tile - t.g * p.tiles_per_group;
     t.first_of_g = (tt == 0) || (tile == t_begin);
     t.R0 = tt * p.tile_rows;
     const int total = p.B * p.Rg;
     t.rows = min(p.tile_rows, total - t.R0);
-    t.b_first = t.R0 / p.Rg;
-    const int b_last = (t.R0 + t.rows - 1) / p.Rg;
+    t.b_first = p.fd_Rg.div(t.R0);
+    const int b_last = p.fd_Rg.div(t.R0 + t.rows - 1);
     t.nc = b_last - t.b_first + 1;
     t.n_sfx = (t.nc * p.S + 15) & ~15;
     return t;

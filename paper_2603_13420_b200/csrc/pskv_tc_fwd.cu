@@ -33,7 +33,7 @@ using namespace sm100;
 
 constexpr int kSlots = 3;      // score slots of 128 columns; an item's probabilities overwrite its own scores
 constexpr int kGroups = 4;     // softmax warpgroups: one 32-column piece of every score block each
-constexpr int kThreads = 32 * (4 + 4 * kGroups);
+constexpr int kThreads = 32 * (4 + 4 * kGroups + 4);
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 // Probabilities are 2^(s * sl2) with no max subtracted; rows whose sum leaves
 // [kMinRowSum, kMaxRowSum] are redone by the general kernel.
@@ -56,6 +56,7 @@ struct TcFwdParams {
     int tile_rows;        // rows of the flat row list per tile (<= 128, multiple of seg_rows)
     int seg_rows;         // rows per Q / out TMA box: gcd(Rg, tile_rows)
     int tiles_per_group;
+    FastDiv fd_tpg, fd_Rg, fd_S;  // divisions by tiles_per_group, Rg, S
     int total_tiles;
     int nblk_p;           // prefix key blocks: ceil(P / 128)
     int tail_rows;        // rows held by the last prefix block (multiple of 16, <= 128)
@@ -136,8 +137,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
-            const bool all_sm = (i >= kBarPReady && i < kBarPReady + kSlots) || i == kBarOFree || i == kBarStageFull;
-            mbar_init(bar(i), all_sm ? (uint32_t)(4 * kGroups) : 1u);
+            const bool all_sm = i >= kBarPReady && i < kBarPReady + kSlots;
+            const bool epi = i == kBarOFree || i == kBarStageFull;
+            mbar_init(bar(i), all_sm ? (uint32_t)(4 * kGroups) : epi ? 4u : 1u);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -158,7 +160,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
     const int n_tiles = t_end - t_begin;
     const int nitems = p.nblk_p + 1;  // prefix blocks + the suffix block
-    const int g_first = t_begin / p.tiles_per_group;
+    const int g_first = p.fd_tpg.div(t_begin);
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
 
@@ -186,18 +188,23 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
             if (!ok) break;
             PSKV_TRACE_EVENT(1, tl);
-            const int nseg = t.rows / p.seg_rows;  // one box per run of seg_rows rows
+            const int nseg = t.rows / p.seg_rows;  // (once per tile)  // one box per run of seg_rows rows
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
                     const int R = t.R0 + s * p.seg_rows;
-                    const int b = R / p.Rg, r = R - b * p.Rg;
+                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
                                     bar(kBarQFull), sl * 64, r, t.g, b);
                 }
             }
             __syncwarp();
+#ifdef PSKV_TRACE_QLAND
+            PSKV_TRACE_EVENT(2, tl);
+            mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrProducerK);
+            PSKV_TRACE_EVENT(3, tl);
+#endif
             if (p.resident) {
                 if (t.first_of_g && elect_one_sync()) {
                     for (int k = 0; k < p.nblk_p; ++k) {
@@ -255,12 +262,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t stage = sbase + p.off_stage;
         auto store_tile = [&](int ts) {  // StageFull of tile ts has been seen
             const TileInfo u = tile_info(p, t_begin + ts, t_begin);
-            const int nseg = u.rows / p.seg_rows;
+            const int nseg = u.rows / p.seg_rows;  // (once per tile)
             if (elect_one_sync()) {
                 for (int sl = 0; sl < C::kSlabs; ++sl)
                     for (int s = 0; s < nseg; ++s) {
                         const int R = u.R0 + s * p.seg_rows;
-                        const int b = R / p.Rg, r = R - b * p.Rg;
+                        const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
                         tma_store_4d(&tm_out, stage + sl * kStagingBytes + s * p.seg_rows * 128, sl * 64, r, u.g, b);
                     }
                 tma_store_commit();
@@ -496,8 +503,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
-    } else {
-        // ------------------------------------------------- softmax + epilogue warps (4..19)
+    } else if (warp < 4 + 4 * kGroups) {
+        // ------------------------------------------------------------------ softmax warps (4..19)
         // Four warpgroups work on every item: the 128 score columns are four pieces of 32 and
         // group j takes piece j, so that each scheduler always has four independent softmax warps
         // to hide the others' tensor-memory and barrier latencies.  Each thread owns one query
@@ -516,24 +523,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
         float lsum = 0.f;
 #pragma unroll 1
-        for (int tl = 0; tl <= n_tiles && ok; ++tl) {
-            const bool have_tile = tl < n_tiles;
-            TileInfo t;
+        for (int tl = 0; tl < n_tiles && ok; ++tl) {
+            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             int lo_sfx = 1, hi_sfx = 0;
-            if (have_tile) {
-                t = tile_info(p, t_begin + tl, t_begin);
-                if (row < t.rows) {
-                    const int R = t.R0 + row;
-                    const int b = R / p.Rg, r = R - b * p.Rg;
-                    lo_sfx = (b - t.b_first) * p.S;  // first suffix column of this row's candidate
-                    hi_sfx = lo_sfx + (r % p.S);     // causal: suffix keys 0..i
-                }
-                lsum = 0.f;
+            if (row < t.rows) {
+                const int R = t.R0 + row;
+                const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+                lo_sfx = (b - t.b_first) * p.S;  // first suffix column of this row's candidate
+                hi_sfx = lo_sfx + (r - p.fd_S.div(r) * p.S);     // causal: suffix keys 0..i
             }
-            const int nk = have_tile ? nitems : 1;
+            lsum = 0.f;
 #pragma unroll 1
-            for (int k = 0; k < nk && ok; ++k) {
-                if (have_tile) {
+            for (int k = 0; k < nitems && ok; ++k) {
+                {
                     const int item = tl * nitems + k, slot = item % kSlots;
                     const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN + wg * kPiece;
                     // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
@@ -561,6 +563,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     PSKV_TRACE_EVENT(25, item);
                     ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
                     if (!ok) break;
+#ifdef PSKV_STAGGER
+                    if (item == 0) {
+                        const long long t0 = clock64();
+                        while (clock64() - t0 < (long long)(wg * PSKV_STAGGER)) { }
+                    }
+#endif
                     tc_fence_after();
                     PSKV_TRACE_EVENT(20, item);
                     if (kind != 0) {
@@ -571,29 +579,32 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         }
                         PSKV_TRACE_EVENT(21, item);
                         float ls0 = 0.f, ls1 = 0.f;
-                        if (kind == 3) {
+                        if (kind >= 2) {
+                            // all exponentials first (independent, so they pipeline through the
+                            // special-function unit), then sums and bf16 pairs
+                            float e[kPiece];
 #pragma unroll
-                            for (int c = 0; c < kPiece / 2; ++c) {
-                                const float p0 = exp2f(__uint_as_float(rr[2 * c]) * p.sl2);
-                                const float p1 = exp2f(__uint_as_float(rr[2 * c + 1]) * p.sl2);
-                                ls0 += p0;
-                                ls1 += p1;
-                                pk[c] = pack_bf16x2(p0, p1);
-                            }
-                        } else if (kind == 2) {
-                            const unsigned span = (unsigned)(hi - lo);
-                            const int base = c0 - lo;
-                            const bool any_col = hi >= lo;
+                            for (int c = 0; c < kPiece; ++c) e[c] = ex2_approx(__uint_as_float(rr[c]) * p.sl2);
+                            if (kind == 2) {
+                                const unsigned span = (unsigned)(hi - lo);
+                                const int base = c0 - lo;
+                                const bool any_col = hi >= lo;
 #pragma unroll
-                            for (int c = 0; c < kPiece / 2; ++c) {
-                                const bool in0 = any_col && (unsigned)(base + 2 * c) <= span;
-                                const bool in1 = any_col && (unsigned)(base + 2 * c + 1) <= span;
-                                const float p0 = in0 ? exp2f(__uint_as_float(rr[2 * c]) * p.sl2) : 0.f;
-                                const float p1 = in1 ? exp2f(__uint_as_float(rr[2 * c + 1]) * p.sl2) : 0.f;
-                                ls0 += p0;
-                                ls1 += p1;
-                                pk[c] = pack_bf16x2(p0, p1);
+                                for (int c = 0; c < kPiece; ++c)
+                                    e[c] = (any_col && (unsigned)(base + c) <= span) ? e[c] : 0.f;
                             }
+                            float ls2 = 0.f, ls3 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < kPiece / 4; ++c) {
+                                ls0 += e[4 * c];
+                                ls1 += e[4 * c + 1];
+                                ls2 += e[4 * c + 2];
+                                ls3 += e[4 * c + 3];
+                                pk[2 * c] = pack_bf16x2(e[4 * c], e[4 * c + 1]);
+                                pk[2 * c + 1] = pack_bf16x2(e[4 * c + 2], e[4 * c + 3]);
+                            }
+                            ls0 += ls2;
+                            ls1 += ls3;
                         } else {
 #pragma unroll
                             for (int c = 0; c < kPiece / 2; ++c) pk[c] = 0u;
@@ -610,65 +621,67 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (lane == 0) mbar_arrive(bar(kBarPReady + slot));
                     PSKV_TRACE_EVENT(24, item);
                 }
-                if (k == 0 && tl > 0) {
-                    // ---- epilogue of tile tl-1: O / l -> bf16 -> staging; lse; rows to redo
-                    const int te = tl - 1;
-                    const TileInfo u = tile_info(p, t_begin + te, t_begin);
-                    ok = mbar_wait_warp(bar(kBarOFull), te & 1, abort_flag, p.status, kErrEpilogue);
-                    if (!ok) break;
-                    PSKV_TRACE_EVENT(30, te);
-                    tc_fence_after();
-                    const float *mlt = ml + (te & 3) * kGroups * kTileM + row;
-                    const float l = (mlt[0] + mlt[kTileM]) + (mlt[2 * kTileM] + mlt[3 * kTileM]);
-                    const bool row_ok = l >= kMinRowSum && l <= kMaxRowSum;  // false for overflow (inf, NaN), underflow
-                    const float inv = 1.f / l;
-                    const bool mine = wg < D / kPiece;  // this group has O columns
-                    uint32_t ob[kPiece / 2];
-                    if (mine) {
-                        uint32_t o[kPiece];
-                        tmem_ld32(tmem + lane_addr + kOCol + wg * kPiece, o);
-                        tmem_wait_ld();
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps (20..23)
+        // O / l -> bf16 -> staging buffer (TMA-stored by warp 3); lse; rows to redo.  Thread <->
+        // query row; the row sum is the sum of the four softmax groups' partial sums.
+        const int ew = warp & 3;
+        const int row = 32 * ew + lane;
+        const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
+        bool ok = true;
+#pragma unroll 1
+        for (int te = 0; te < n_tiles && ok; ++te) {
+            const TileInfo u = tile_info(p, t_begin + te, t_begin);
+            ok = mbar_wait_warp(bar(kBarOFull), te & 1, abort_flag, p.status, kErrEpilogue);
+            if (!ok) break;
+            PSKV_TRACE_EVENT(30, te);
+            tc_fence_after();
+            const float *mlt = ml + (te & 3) * kGroups * kTileM + row;
+            const float l = (mlt[0] + mlt[kTileM]) + (mlt[2 * kTileM] + mlt[3 * kTileM]);
+            const bool row_ok = l >= kMinRowSum && l <= kMaxRowSum;  // false for overflow (inf, NaN), underflow
+            // staged values must be finite (the buffer may double as suffix V, whose padding rows
+            // meet zero probabilities); rows that failed are redone anyway
+            const float inv = row_ok ? 1.f / l : 0.f;
+            // the TMA stores of the previous tile must have read the staging buffer
+            ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
+            if (!ok) break;
 #pragma unroll
-                        for (int c = 0; c < kPiece / 2; ++c)
-                            ob[c] = pack_bf16x2(__uint_as_float(o[2 * c]) * inv, __uint_as_float(o[2 * c + 1]) * inv);
-                        // staged values must be finite (the buffer doubles as suffix V, whose padding
-                        // rows meet zero probabilities); rows that failed are redone anyway
-                        if (!row_ok) {
-#pragma unroll
-                            for (int c = 0; c < kPiece / 2; ++c) ob[c] = 0u;
-                        }
-                    }
+            for (int ch = 0; ch < D / kPiece; ++ch) {
+                uint32_t o[kPiece];
+                tmem_ld32(tmem + lane_addr + kOCol + ch * kPiece, o);
+                tmem_wait_ld();
+                if (ch == D / kPiece - 1) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarOFree));
-                    if (wg == 0) {
-                        const bool stored = row < u.rows;
-                        if (stored) {
-                            const int R = u.R0 + row;
-                            const int b = R / p.Rg, r = R - b * p.Rg;
-                            const size_t grow = ((size_t)b * p.Hq + (size_t)u.g * p.n_rep) * p.S + r;
-                            p.lse[grow] = row_ok ? log2f(l) * kLn2 : __int_as_float(0x7fc00000);
-                        }
-                        const unsigned bad = __ballot_sync(0xffffffffu, stored && !row_ok);
-                        if (bad != 0u && lane == 0) atomicAdd(p.redo_count, (unsigned int)__popc(bad));
-                    }
-                    // the TMA stores of the previous tile must have read the staging buffer
-                    ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
-                    if (!ok) break;
-                    if (mine) {
-                        // 64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row
-                        uint8_t *srow = smem + p.off_stage + (wg >> 1) * kStagingBytes + row * 128;
+                }
+                // 64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row
+                uint8_t *srow = smem + p.off_stage + (ch >> 1) * kStagingBytes + row * 128;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            *reinterpret_cast<uint4 *>(srow + ((((wg & 1) * 4 + c) ^ (row & 7)) << 4)) =
-                                make_uint4(ob[4 * c], ob[4 * c + 1], ob[4 * c + 2], ob[4 * c + 3]);
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(kBarStageFull));
-                    PSKV_TRACE_EVENT(31, te);
+                for (int c = 0; c < 4; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
+                    v.y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
+                    v.z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
+                    v.w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(srow + ((((ch & 1) * 4 + c) ^ (row & 7)) << 4)) = v;
                 }
             }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarStageFull));
+            const bool stored = row < u.rows;
+            if (stored) {
+                const int R = u.R0 + row;
+                const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+                const size_t grow = ((size_t)b * p.Hq + (size_t)u.g * p.n_rep) * p.S + r;
+                p.lse[grow] = row_ok ? log2f(l) * kLn2 : __int_as_float(0x7fc00000);
+            }
+            const unsigned bad = __ballot_sync(0xffffffffu, stored && !row_ok);
+            if (bad != 0u && lane == 0) atomicAdd(p.redo_count, (unsigned int)__popc(bad));
+            PSKV_TRACE_EVENT(31, te);
         }
     }
 
@@ -794,6 +807,9 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.tile_rows = plan.tile_rows;
     p.seg_rows = plan.seg_rows;
     p.tiles_per_group = plan.tiles_per_group;
+    p.fd_tpg.init(plan.tiles_per_group);
+    p.fd_Rg.init(Rg);
+    p.fd_S.init(dm.S);
     p.total_tiles = plan.tiles_per_group * dm.Hkv;
     p.nblk_p = plan.nblk_p;
     p.tail_rows = plan.tail_rows;
