@@ -47,7 +47,7 @@ struct TcBwdParams {
     float scale;
     int B, Hq, Hkv, S, P, n_rep;
     int Rg, tile_rows, seg_rows, tiles_per_group, total_tiles;
-    FastDiv fd_tpg, fd_Rg, fd_S;  // divisions by tiles_per_group, Rg, S
+    FastDiv fd_tpg, fd_Rg, fd_S, fd_seg;  // divisions by tiles_per_group, Rg, S, seg_rows
     int nblk_p, tail_rows, resident, stages_k, stages_v, sfx_rows;  // ring stages of prefix K / V (streaming mode)
     int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc;
 };
@@ -157,7 +157,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdA);
             if (!ok) break;
-            const int nseg = t.rows / p.seg_rows;  // (once per tile)
+            const int nseg = p.fd_seg.div(t.rows);
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
@@ -228,7 +228,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             ok = mbar_wait_warp(bar(kBarDvFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdB);
             if (!ok) break;
-            const int nseg = t.rows / p.seg_rows;  // (once per tile)
+            const int nseg = p.fd_seg.div(t.rows);
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarDoFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
                 for (int s = 0; s < nseg; ++s) {
@@ -548,7 +548,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarDqFree));
-            const int nseg = t.rows / p.seg_rows;  // (once per tile)
+            const int nseg = p.fd_seg.div(t.rows);
 #pragma unroll
             for (int sl = 0; sl < C::kSlabs; ++sl) {
                 const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
@@ -694,6 +694,7 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.fd_tpg.init(plan.tiles_per_group);
     p.fd_Rg.init(Rg);
     p.fd_S.init(dm.S);
+    p.fd_seg.init(plan.seg_rows);
     p.total_tiles = plan.tiles_per_group * dm.Hkv;
     p.nblk_p = plan.nblk_p;
     p.tail_rows = plan.tail_rows;

@@ -56,7 +56,7 @@ struct TcFwdParams {
     int tile_rows;        // rows of the flat row list per tile (<= 128, multiple of seg_rows)
     int seg_rows;         // rows per Q / out TMA box: gcd(Rg, tile_rows)
     int tiles_per_group;
-    FastDiv fd_tpg, fd_Rg, fd_S;  // divisions by tiles_per_group, Rg, S
+    FastDiv fd_tpg, fd_Rg, fd_S, fd_seg;  // divisions by tiles_per_group, Rg, S, seg_rows
     int total_tiles;
     int nblk_p;           // prefix key blocks: ceil(P / 128)
     int tail_rows;        // rows held by the last prefix block (multiple of 16, <= 128)
@@ -181,6 +181,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         }
         uint32_t kload = 0;  // streaming mode: prefix K blocks loaded so far
         bool ok = true;
+#pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
             // Q, suffix K and (resident mode) the prefix K blocks are free once every score MMA of
@@ -188,12 +189,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
             if (!ok) break;
             PSKV_TRACE_EVENT(1, tl);
-            const int nseg = t.rows / p.seg_rows;  // (once per tile)  // one box per run of seg_rows rows
+            const int nseg = p.fd_seg.div(t.rows);  // one box per run of seg_rows rows
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
+#pragma unroll 1
                 for (int s = 0; s < nseg; ++s) {
                     const int R = t.R0 + s * p.seg_rows;
                     const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+#pragma unroll 1
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
                                     bar(kBarQFull), sl * 64, r, t.g, b);
@@ -207,10 +210,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #endif
             if (p.resident) {
                 if (t.first_of_g && elect_one_sync()) {
+#pragma unroll 1
                     for (int k = 0; k < p.nblk_p; ++k) {
                         const bool tail = k == p.nblk_p - 1;
                         const int slab = tail ? tail_slab : C::kSlabBytes;
                         mbar_arrive_expect_tx(bar(kBarKFull + k), (uint32_t)(C::kSlabs * slab));
+#pragma unroll 1
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pk + k * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
                                         bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
@@ -218,6 +223,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
                 __syncwarp();
             } else {
+#pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const uint32_t ks = kload % (uint32_t)p.stages;
                     ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
@@ -227,6 +233,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const int slab = tail ? tail_slab : C::kSlabBytes;
                     if (elect_one_sync()) {
                         mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(C::kSlabs * slab));
+#pragma unroll 1
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
                                         bar(kBarKFull + ks), sl * 64, k * kBlockN, t.g);
@@ -239,7 +246,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // suffix K of the candidates this tile touches: one box per candidate
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarSKFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
+#pragma unroll 1
                 for (int c = 0; c < t.nc; ++c)
+#pragma unroll 1
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_4d(sbase + p.off_sk + sl * sfx_slab + c * p.S * 128, &tm_sk, bar(kBarSKFull),
                                     sl * 64, 0, t.g, t.b_first + c);
@@ -253,39 +262,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             prefetch_tensormap(&tm_out);
             if (p.P > 0) { prefetch_tensormap(&tm_pv); prefetch_tensormap(&tm_pv_tail); }
         }
+        // This warp also issues the TMA stores of each finished output tile.  The staging buffer
+        // may share its shared memory with suffix V: tile t's output is staged after that tile's
+        // last value MMA has read suffix V, and suffix V of tile t+1 is then fetched only once the
+        // stores of tile t have read the staging buffer.
+        const uint32_t stage = sbase + p.off_stage;
         uint32_t vload = 0;
         bool ok = true;
-        // This warp also issues the TMA stores of each finished output tile.  The staging buffer
-        // of a tile shares its shared memory with the suffix V of the tiles around it: tile t's
-        // output is staged after that tile's last value MMA has read suffix V, and suffix V of
-        // tile t+1 is fetched only once the stores of tile t have read the staging buffer.
-        const uint32_t stage = sbase + p.off_stage;
-        auto store_tile = [&](int ts) {  // StageFull of tile ts has been seen
-            const TileInfo u = tile_info(p, t_begin + ts, t_begin);
-            const int nseg = u.rows / p.seg_rows;  // (once per tile)
-            if (elect_one_sync()) {
-                for (int sl = 0; sl < C::kSlabs; ++sl)
-                    for (int s = 0; s < nseg; ++s) {
-                        const int R = u.R0 + s * p.seg_rows;
-                        const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
-                        tma_store_4d(&tm_out, stage + sl * kStagingBytes + s * p.seg_rows * 128, sl * 64, r, u.g, b);
-                    }
-                tma_store_commit();
-                tma_store_wait_read();  // the staging buffer may be overwritten after this
-                mbar_arrive(bar(kBarStageFree));
-            }
-            __syncwarp();
-        };
-        auto load_suffix_v = [&](const TileInfo &t) {
-            if (elect_one_sync()) {
-                mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
-                for (int c = 0; c < t.nc; ++c)
-                    for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + p.off_sv + sl * sfx_slab + c * p.S * 128, &tm_sv, bar(kBarSVFull),
-                                    sl * 64, 0, t.g, t.b_first + c);
-            }
-            __syncwarp();
-        };
+#pragma unroll 1
         for (int tl = 0; tl <= n_tiles && ok; ++tl) {
             const bool have_tile = tl < n_tiles;
             // Two jobs ride along with the prefix loads of tile tl: the stores of tile tl-1 (once it
@@ -293,38 +277,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // stores when it doubles as the staging buffer, else after the previous tile's value MMAs).
             bool pend_store = tl > 0, pend_sv = have_tile;
             TileInfo t;
-            auto poll_sv = [&](bool block) -> bool {
-                if (!pend_sv || (p.alias_stage && pend_store)) return true;
-                bool ready = true;
-                if (!p.alias_stage && tl > 0) {
-                    if (block)
-                        ready = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
-                    else
-                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarSVFree), (tl & 1) ^ 1) ? 1 : 0, 0) != 0;
-                    if (block && !ready) return false;
-                }
-                if (ready) {
-                    load_suffix_v(t);
-                    pend_sv = false;
-                }
-                return true;
-            };
-            auto poll = [&](bool block) -> bool {
-                if (!p.alias_stage && !poll_sv(block)) return false;
-                if (pend_store) {
-                    bool ready;
-                    if (block)
-                        ready = mbar_wait_warp(bar(kBarStageFull), (tl - 1) & 1, abort_flag, p.status, kErrEpilogue);
-                    else
-                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarStageFull), (tl - 1) & 1) ? 1 : 0, 0) != 0;
-                    if (block && !ready) return false;
-                    if (ready) {
-                        store_tile(tl - 1);
-                        pend_store = false;
-                    }
-                }
-                return poll_sv(block);
-            };
+            int nk = 0;  // prefix V blocks still to fetch for this tile
             if (have_tile) {
                 t = tile_info(p, t_begin + tl, t_begin);
                 if (p.resident) {
@@ -333,10 +286,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
                     if (!ok) break;
                     if (t.first_of_g && elect_one_sync()) {
+#pragma unroll 1
                         for (int k = 0; k < p.nblk_p; ++k) {
                             const bool tail = k == p.nblk_p - 1;
                             const int slab = tail ? tail_slab : C::kSlabBytes;
                             mbar_arrive_expect_tx(bar(kBarVFull + k), (uint32_t)(C::kSlabs * slab));
+#pragma unroll 1
                             for (int sl = 0; sl < C::kSlabs; ++sl)
                                 tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab,
                                             tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
@@ -344,27 +299,84 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     }
                     __syncwarp();
                 } else {
-                    for (int k = 0; k < p.nblk_p; ++k) {
-                        const uint32_t vs = vload % (uint32_t)p.stages;
-                        ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
-                                            p.status, kErrProducerV);
-                        if (!ok) break;
-                        const bool tail = k == p.nblk_p - 1;
-                        const int slab = tail ? tail_slab : C::kSlabBytes;
-                        if (elect_one_sync()) {
-                            mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
-                            for (int sl = 0; sl < C::kSlabs; ++sl)
-                                tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab,
-                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
-                        }
-                        __syncwarp();
-                        ++vload;
-                        poll(false);
-                    }
-                    if (!ok) break;
+                    nk = p.nblk_p;
                 }
             }
-            ok = poll(true);
+            int k = 0;
+#pragma unroll 1
+            while (ok && (k < nk || pend_store || pend_sv)) {
+                const bool block = k >= nk;  // nothing else left to do for this tile: wait for the jobs
+                if (k < nk) {
+                    const uint32_t vs = vload % (uint32_t)p.stages;
+                    ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
+                                        p.status, kErrProducerV);
+                    if (!ok) break;
+                    const bool tail = k == p.nblk_p - 1;
+                    const int slab = tail ? tail_slab : C::kSlabBytes;
+                    if (elect_one_sync()) {
+                        mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
+#pragma unroll 1
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
+                                        bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                    }
+                    __syncwarp();
+                    ++vload;
+                    ++k;
+                }
+                bool sv_ready = false;
+                if (pend_sv && !p.alias_stage) {
+                    if (tl == 0)
+                        sv_ready = true;
+                    else if (block)
+                        sv_ready = ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
+                    else
+                        sv_ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarSVFree), (tl & 1) ^ 1) ? 1 : 0, 0) != 0;
+                    if (!ok) break;
+                }
+                if (pend_store && !sv_ready) {
+                    bool ready;
+                    if (block)
+                        ready = ok = mbar_wait_warp(bar(kBarStageFull), (tl - 1) & 1, abort_flag, p.status, kErrEpilogue);
+                    else
+                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarStageFull), (tl - 1) & 1) ? 1 : 0, 0) != 0;
+                    if (!ok) break;
+                    if (ready) {
+                        const TileInfo u = tile_info(p, t_begin + tl - 1, t_begin);
+                        const int nseg = p.fd_seg.div(u.rows);
+                        if (elect_one_sync()) {
+#pragma unroll 1
+                            for (int sl = 0; sl < C::kSlabs; ++sl)
+#pragma unroll 1
+                                for (int s = 0; s < nseg; ++s) {
+                                    const int R = u.R0 + s * p.seg_rows;
+                                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+                                    tma_store_4d(&tm_out, stage + sl * kStagingBytes + s * p.seg_rows * 128, sl * 64, r,
+                                                 u.g, b);
+                                }
+                            tma_store_commit();
+                            tma_store_wait_read();  // the staging buffer may be overwritten after this
+                            mbar_arrive(bar(kBarStageFree));
+                        }
+                        __syncwarp();
+                        pend_store = false;
+                    }
+                }
+                if (pend_sv && p.alias_stage && !pend_store) sv_ready = true;
+                if (sv_ready) {
+                    if (elect_one_sync()) {
+                        mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
+#pragma unroll 1
+                        for (int c = 0; c < t.nc; ++c)
+#pragma unroll 1
+                            for (int sl = 0; sl < C::kSlabs; ++sl)
+                                tma_load_4d(sbase + p.off_sv + sl * sfx_slab + c * p.S * 128, &tm_sv, bar(kBarSVFull),
+                                            sl * 64, 0, t.g, t.b_first + c);
+                    }
+                    __syncwarp();
+                    pend_sv = false;
+                }
+            }
         }
         if (elect_one_sync()) tma_store_wait_all();
         __syncwarp();
@@ -563,12 +575,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     PSKV_TRACE_EVENT(25, item);
                     ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
                     if (!ok) break;
-#ifdef PSKV_STAGGER
-                    if (item == 0) {
-                        const long long t0 = clock64();
-                        while (clock64() - t0 < (long long)(wg * PSKV_STAGGER)) { }
-                    }
-#endif
                     tc_fence_after();
                     PSKV_TRACE_EVENT(20, item);
                     if (kind != 0) {
@@ -647,26 +653,38 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // the TMA stores of the previous tile must have read the staging buffer
             ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
             if (!ok) break;
-#pragma unroll
-            for (int ch = 0; ch < D / kPiece; ++ch) {
-                uint32_t o[kPiece];
-                tmem_ld32(tmem + lane_addr + kOCol + ch * kPiece, o);
+            // one 64-column slab per round; O is free for the next tile's first value MMA as soon
+            // as the last round's loads have returned
+#pragma unroll 1
+            for (int sl = 0; sl < C::kSlabs; ++sl) {
+                uint32_t o0[kPiece], o1[kPiece];
+                tmem_ld32(tmem + lane_addr + kOCol + sl * 64, o0);
+                tmem_ld32(tmem + lane_addr + kOCol + sl * 64 + kPiece, o1);
                 tmem_wait_ld();
-                if (ch == D / kPiece - 1) {
+                if (sl == C::kSlabs - 1) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarOFree));
                 }
-                // 64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row
-                uint8_t *srow = smem + p.off_stage + (ch >> 1) * kStagingBytes + row * 128;
+                // 128-byte rows, 16-byte chunks swizzled by the row
+                uint8_t *srow = smem + p.off_stage + sl * kStagingBytes + row * 128;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-                    v.y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-                    v.z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-                    v.w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-                    *reinterpret_cast<uint4 *>(srow + ((((ch & 1) * 4 + c) ^ (row & 7)) << 4)) = v;
+                    v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * inv, __uint_as_float(o0[8 * c + 1]) * inv);
+                    v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * inv, __uint_as_float(o0[8 * c + 3]) * inv);
+                    v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * inv, __uint_as_float(o0[8 * c + 5]) * inv);
+                    v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * inv, __uint_as_float(o0[8 * c + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * inv, __uint_as_float(o1[8 * c + 1]) * inv);
+                    v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * inv, __uint_as_float(o1[8 * c + 3]) * inv);
+                    v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * inv, __uint_as_float(o1[8 * c + 5]) * inv);
+                    v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * inv, __uint_as_float(o1[8 * c + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
                 }
             }
             fence_proxy_async();
@@ -810,6 +828,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.fd_tpg.init(plan.tiles_per_group);
     p.fd_Rg.init(Rg);
     p.fd_S.init(dm.S);
+    p.fd_seg.init(plan.seg_rows);
     p.total_tiles = plan.tiles_per_group * dm.Hkv;
     p.nblk_p = plan.nblk_p;
     p.tail_rows = plan.tail_rows;
