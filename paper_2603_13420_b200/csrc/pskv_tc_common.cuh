@@ -18,7 +18,7 @@ constexpr int kMaxSmem = 232448;             // dynamic shared memory a CTA may 
 // Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
 // costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
 #ifdef PSKV_TRACE
-constexpr int kTraceWarps = 16, kTraceCap = 4096;
+constexpr int kTraceWarps = 28, kTraceCap = 4096;
 __device__ long long g_trace[kTraceWarps * kTraceCap * 2];
 __device__ unsigned int g_trace_n[kTraceWarps];
 #define PSKV_TRACE_DECL unsigned int trace_i_ = 0

@@ -107,7 +107,9 @@ __device__ __forceinline__ int prefix_block_rows(const TcFwdParams &p, int k)
 constexpr int kPiece = 32;  // score columns a softmax thread handles per tensor-memory load
 static_assert(kBlockN == 4 * kPiece, "two softmax groups x two pieces cover a score block");
 
-template <int D>
+// RES: all prefix blocks of a KV head stay in shared memory (else they stream through rings); a
+// compile-time switch so that each launch carries only the code of its own mode.
+template <int D, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_out,
               const __grid_constant__ CUtensorMap tm_pk, const __grid_constant__ CUtensorMap tm_pv,
@@ -184,22 +186,54 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            // Everything the Q loads need is worked out before the wait, so that only the copy
+            // instructions themselves follow it: the Q buffer is single, and the time from "last
+            // score MMA of the previous tile done" to "Q of this tile requested" is exposed.
+            const int nseg = p.fd_seg.div(t.rows);  // one box per run of seg_rows rows
+            int qb = p.fd_Rg.div(t.R0), qr = t.R0 - qb * p.Rg;
+            const uint32_t q_bytes = (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128);
+            const uint32_t seg_bytes = (uint32_t)(p.seg_rows * 128);
+            uint32_t q_dst = sbase + p.off_q;
+#ifndef PSKV_NO_PREFETCH_Q
+            // While there is nothing else to do, ask for the NEXT tile's Q in L2: its load can only
+            // be issued a tile from now, right when it is needed, and then finds the data close by.
+            if (tl + 1 < n_tiles) {
+                const TileInfo tn = tile_info(p, t_begin + tl + 1, t_begin);
+                const int nseg_n = p.fd_seg.div(tn.rows);
+                int nb = p.fd_Rg.div(tn.R0), nr = tn.R0 - nb * p.Rg;
+                if (elect_one_sync()) {
+#pragma unroll 1
+                    for (int s = 0; s < nseg_n; ++s) {
+#pragma unroll
+                        for (int sl = 0; sl < C::kSlabs; ++sl) tma_prefetch_4d(&tm_q, sl * 64, nr, tn.g, nb);
+                        nr += p.seg_rows;
+                        if (nr >= p.Rg) {
+                            nr -= p.Rg;
+                            ++nb;
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+#endif
             // Q, suffix K and (resident mode) the prefix K blocks are free once every score MMA of
             // the previous tile has completed
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
             if (!ok) break;
             PSKV_TRACE_EVENT(1, tl);
-            const int nseg = p.fd_seg.div(t.rows);  // one box per run of seg_rows rows
             if (elect_one_sync()) {
-                mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
+                mbar_arrive_expect_tx(bar(kBarQFull), q_bytes);
 #pragma unroll 1
                 for (int s = 0; s < nseg; ++s) {
-                    const int R = t.R0 + s * p.seg_rows;
-                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
-#pragma unroll 1
+#pragma unroll
                     for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
-                                    bar(kBarQFull), sl * 64, r, t.g, b);
+                        tma_load_4d(q_dst + sl * C::kSlabBytes, &tm_q, bar(kBarQFull), sl * 64, qr, t.g, qb);
+                    q_dst += seg_bytes;
+                    qr += p.seg_rows;  // boxes never straddle a candidate: seg_rows divides Rg
+                    if (qr >= p.Rg) {
+                        qr -= p.Rg;
+                        ++qb;
+                    }
                 }
             }
             __syncwarp();
@@ -208,7 +242,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrProducerK);
             PSKV_TRACE_EVENT(3, tl);
 #endif
-            if (p.resident) {
+            if (RES) {
                 if (t.first_of_g && elect_one_sync()) {
 #pragma unroll 1
                     for (int k = 0; k < p.nblk_p; ++k) {
@@ -280,7 +314,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             int nk = 0;  // prefix V blocks still to fetch for this tile
             if (have_tile) {
                 t = tile_info(p, t_begin + tl, t_begin);
-                if (p.resident) {
+                if (RES) {
                     // the resident prefix V blocks are free once every value MMA of the previous tile
                     // has completed
                     ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
@@ -402,7 +436,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (k < p.nblk_p) {
                 n = prefix_block_rows(p, k);
                 slab = n * 128;
-                if (p.resident) {
+                if (RES) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaQk);
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
@@ -426,7 +460,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
             const uint64_t k_slab = (uint64_t)(slab >> 4);
             const bool last_of_tile = k == nitems - 1;
-            const bool free_stage = k < p.nblk_p && !p.resident;
+            const bool free_stage = k < p.nblk_p && !RES;
             if (elect_one_sync()) {
 #pragma unroll
                 for (int ks16 = 0; ks16 < D / 16; ++ks16) {
@@ -468,7 +502,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (k < p.nblk_p) {
                 n = prefix_block_rows(p, k);
                 slab = n * 128;
-                if (p.resident) {
+                if (RES) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaPv);
                     vaddr = sbase + p.off_pv + k * C::kTileBytes;
@@ -491,7 +525,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
             const int nk = n >> 4;
             const bool last_of_tile = k == nitems - 1;
-            const bool free_stage = k < p.nblk_p && !p.resident;
+            const bool free_stage = k < p.nblk_p && !RES;
             const uint32_t acc0 = k > 0 ? 1u : 0u;
             if (elect_one_sync()) {
 #pragma unroll
@@ -575,6 +609,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     PSKV_TRACE_EVENT(25, item);
                     ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
                     if (!ok) break;
+#ifdef PSKV_STAGGER
+                    if (item == 0) {
+                        const long long t0 = clock64();
+                        while (clock64() - t0 < (long long)(wg * PSKV_STAGGER)) { }
+                    }
+#endif
                     tc_fence_after();
                     PSKV_TRACE_EVENT(20, item);
                     if (kind != 0) {
@@ -840,19 +880,20 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
     p.off_ml = plan.off_ml;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    auto kernel = plan.resident ? tc_fwd_kernel<D, true> : tc_fwd_kernel<D, false>;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[plan.resident]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[plan.resident] = true;
     }
     cudaError_t e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), stream);
     if (e != cudaSuccess) return e;
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
     {
         KernelTiming timing(kKernelFwdTc, stream);
-        tc_fwd_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail,
-                                                                      tm_pv_tail, tm_sk, tm_sv, p);
+        kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail, tm_sk,
+                                                            tm_sv, p);
     }
     count_launches(1);
     e = cudaGetLastError();
