@@ -28,11 +28,12 @@ namespace {
 using namespace sm100;
 
 constexpr int kSlots = 2;
-constexpr int kThreads = 384;
+constexpr int kGroups = 4;   // element-wise warpgroups: one 32-column piece of every score block each
+constexpr int kPiece = 32;
+constexpr int kThreads = 32 * (4 + 4 * kGroups + 4);
 constexpr int kDpCol = kSlots * kBlockN;
 constexpr int kDqCol = kDpCol + kBlockN;
 constexpr int kMaxStages = 4;
-constexpr int kPieceB = 16;  // columns per tensor-memory load of the element-wise warps
 
 enum : unsigned int {
     kErrProdA = 0x201, kErrProdB = 0x202, kErrMmaS = 0x203, kErrMmaDq = 0x204, kErrElem = 0x205,
@@ -89,7 +90,9 @@ __device__ __forceinline__ int prefix_block_rows(const TcBwdParams &p, int k)
     return k == p.nblk_p - 1 ? p.tail_rows : kBlockN;
 }
 
-template <int D>
+// RES: all prefix blocks of a KV head stay in shared memory (else they stream through rings); a
+// compile-time switch so that each launch carries only the code of its own mode.
+template <int D, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                  const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_pk,
@@ -116,9 +119,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int i = tid; i < p.off_bar / 16; i += kThreads) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
-            const bool four = i == kBarDqFree || i == kBarStageFull || i == kBarDpFree ||
-                              (i >= kBarDsReady && i < kBarDsReady + kSlots);
-            mbar_init(bar(i), four ? 4u : 1u);
+            const bool epi = i == kBarDqFree || i == kBarStageFull;
+            const bool elem = i == kBarDpFree || (i >= kBarDsReady && i < kBarDsReady + kSlots);
+            mbar_init(bar(i), elem ? (uint32_t)(4 * kGroups) : epi ? 4u : 1u);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -155,21 +158,49 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            // while idle: ask for the next tile's Q in L2 (its load can only be issued a tile from
+            // now, exactly when it is needed)
+            if (tl + 1 < n_tiles) {
+                const TileInfo tn = tile_info(p, t_begin + tl + 1, t_begin);
+                const int nseg_n = p.fd_seg.div(tn.rows);
+                int nb = p.fd_Rg.div(tn.R0), nr = tn.R0 - nb * p.Rg;
+                if (elect_one_sync()) {
+#pragma unroll 1
+                    for (int s = 0; s < nseg_n; ++s) {
+#pragma unroll
+                        for (int sl = 0; sl < C::kSlabs; ++sl) tma_prefetch_4d(&tm_q, sl * 64, nr, tn.g, nb);
+                        nr += p.seg_rows;
+                        if (nr >= p.Rg) {
+                            nr -= p.Rg;
+                            ++nb;
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+            // everything the Q loads need is worked out before the wait (the Q buffer is single)
+            const int nseg = p.fd_seg.div(t.rows);
+            int qb = p.fd_Rg.div(t.R0), qr = t.R0 - qb * p.Rg;
+            uint32_t q_dst = sbase + p.off_q;
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdA);
             if (!ok) break;
-            const int nseg = p.fd_seg.div(t.rows);
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarQFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
+#pragma unroll 1
                 for (int s = 0; s < nseg; ++s) {
-                    const int R = t.R0 + s * p.seg_rows;
-                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+#pragma unroll
                     for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + p.off_q + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_q,
-                                    bar(kBarQFull), sl * 64, r, t.g, b);
+                        tma_load_4d(q_dst + sl * C::kSlabBytes, &tm_q, bar(kBarQFull), sl * 64, qr, t.g, qb);
+                    q_dst += p.seg_rows * 128;
+                    qr += p.seg_rows;  // boxes never straddle a candidate: seg_rows divides Rg
+                    if (qr >= p.Rg) {
+                        qr -= p.Rg;
+                        ++qb;
+                    }
                 }
             }
             __syncwarp();
-            if (!p.resident) {
+            if (!RES) {
 #pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const uint32_t ks = kload % stages_k;
@@ -194,7 +225,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 ok = mbar_wait_warp(bar(kBarDqFull), (tl - 1) & 1, abort_flag, p.status, kErrProdA);
                 if (!ok) break;
             }
-            if (p.resident && t.first_of_g && elect_one_sync()) {
+            if (RES && t.first_of_g && elect_one_sync()) {
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const bool tail = k == p.nblk_p - 1;
                     const int slab = tail ? tail_slab : C::kSlabBytes;
@@ -226,19 +257,44 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            if (tl + 1 < n_tiles) {  // the next tile's dO into L2, a tile ahead
+                const TileInfo tn = tile_info(p, t_begin + tl + 1, t_begin);
+                const int nseg_n = p.fd_seg.div(tn.rows);
+                int nb = p.fd_Rg.div(tn.R0), nr = tn.R0 - nb * p.Rg;
+                if (elect_one_sync()) {
+#pragma unroll 1
+                    for (int s = 0; s < nseg_n; ++s) {
+#pragma unroll
+                        for (int sl = 0; sl < C::kSlabs; ++sl) tma_prefetch_4d(&tm_do, sl * 64, nr, tn.g, nb);
+                        nr += p.seg_rows;
+                        if (nr >= p.Rg) {
+                            nr -= p.Rg;
+                            ++nb;
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+            const int nseg = p.fd_seg.div(t.rows);
+            int qb = p.fd_Rg.div(t.R0), qr = t.R0 - qb * p.Rg;
+            uint32_t do_dst = sbase + p.off_do;
             ok = mbar_wait_warp(bar(kBarDvFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProdB);
             if (!ok) break;
-            const int nseg = p.fd_seg.div(t.rows);
             if (elect_one_sync()) {
                 mbar_arrive_expect_tx(bar(kBarDoFull), (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128));
+#pragma unroll 1
                 for (int s = 0; s < nseg; ++s) {
-                    const int R = t.R0 + s * p.seg_rows;
-                    const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+#pragma unroll
                     for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + p.off_do + sl * C::kSlabBytes + s * p.seg_rows * 128, &tm_do,
-                                    bar(kBarDoFull), sl * 64, r, t.g, b);
+                        tma_load_4d(do_dst + sl * C::kSlabBytes, &tm_do, bar(kBarDoFull), sl * 64, qr, t.g, qb);
+                    do_dst += p.seg_rows * 128;
+                    qr += p.seg_rows;
+                    if (qr >= p.Rg) {
+                        qr -= p.Rg;
+                        ++qb;
+                    }
                 }
-                if (p.resident && t.first_of_g) {
+                if (RES && t.first_of_g) {
                     for (int k = 0; k < p.nblk_p; ++k) {
                         const bool tail = k == p.nblk_p - 1;
                         const int slab = tail ? tail_slab : C::kSlabBytes;
@@ -255,7 +311,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                                     sl * 64, 0, t.g, t.b_first + c);
             }
             __syncwarp();
-            if (!p.resident) {
+            if (!RES) {
 #pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const uint32_t vs = vload % stages_v;
@@ -290,7 +346,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
             const int slab = prefix ? n * 128 : sfx_slab;
             const bool last_of_tile = k == nitems - 1;
-            const bool ring = prefix && !p.resident;
+            const bool ring = prefix && !RES;
             const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
             const uint64_t slab16 = (uint64_t)(slab >> 4);
             // ---- S: the slot is free once the dQ MMAs of item i-2 have completed
@@ -300,7 +356,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) break;
             uint32_t kaddr;
             if (prefix) {
-                if (p.resident) {
+                if (RES) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
@@ -337,7 +393,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) break;
             uint32_t vaddr;
             if (prefix) {
-                if (p.resident) {
+                if (RES) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
                     vaddr = sbase + p.off_pv + k * C::kTileBytes;
@@ -388,7 +444,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
             const int slab = prefix ? n * 128 : sfx_slab;
             const bool last_of_tile = k == nitems - 1;
-            const bool ring = prefix && !p.resident;
+            const bool ring = prefix && !RES;
             ok = mbar_wait_warp(bar(kBarDsReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaDq);
             if (!ok) break;
             if (k == 0 && tl > 0) {
@@ -396,7 +452,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (!ok) break;
             }
             uint32_t kaddr;
-            if (prefix) kaddr = sbase + p.off_pk + (p.resident ? (uint32_t)k : kuse % stages_k) * C::kTileBytes;
+            if (prefix) kaddr = sbase + p.off_pk + (RES ? (uint32_t)k : kuse % stages_k) * C::kTileBytes;
             else kaddr = sbase + p.off_sk;
             tc_fence_after();
             const uint32_t ds_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
@@ -407,7 +463,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
                 for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
                     if (ks16 < nk)
-                        mma_ts(tmem + kDqCol, ds_tmem + ks16 * 8, k_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_dq,
+                        mma_ts(tmem + kDqCol, ds_tmem + (ks16 >> 1) * kPiece + (ks16 & 1) * 8, k_desc + (uint64_t)(ks16 * (2048 >> 4)), idesc_dq,
                                ks16 > 0 ? 1u : acc0);
                 }
                 tc_commit(bar(kBarDqDone + slot));
@@ -421,10 +477,17 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
-    } else if (warp < 8) {
-        // ------------------------------------------------------------------ element-wise warps
+    } else if (warp < 4 + 4 * kGroups) {
+        // ------------------------------------------------------------------ element-wise warps (4..19)
+        // Four warpgroups share every item: the 128 score columns are four pieces of 32 and group j
+        // takes piece j.  Thread <-> query row (tensor-memory lane).  Each thread pulls its piece
+        // of S and of dP into registers, hands dP back at once (the next item's dP MMAs are
+        // waiting for that buffer), then forms dS = 2^(S sl2 - lse2) (dP - D) and writes it as
+        // bf16 pairs over the first half of the S piece it came from.
+        const int wg = (warp - 4) >> 2;
         const int row = 32 * (warp & 3) + lane;
-        const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+        const int c0 = wg * kPiece;  // first column of my piece
+        const uint32_t my_tmem = tmem + ((uint32_t)(32 * (warp & 3)) << 16) + c0;
         int item = 0;
         bool ok = true;
 #pragma unroll 1
@@ -452,81 +515,71 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     lo = valid ? sfx_lo : 1;
                     hi = valid ? sfx_hi : 0;
                 }
-                const int nh = n / kPieceB;
-                const bool full = __all_sync(0xffffffffu, lo == 0 && hi >= n - 1);
-                int h_b = 0, h_e = nh - 1;
-                if (!full) {
-                    const int wlo = __reduce_min_sync(0xffffffffu, hi >= lo ? lo : 0x7fffffff);
-                    const int whi = __reduce_max_sync(0xffffffffu, hi >= lo ? hi : -1);
-                    h_b = wlo / kPieceB;
-                    h_e = min(nh - 1, whi / kPieceB);
+                // my piece: 0 = not read by the dQ MMAs, 1 = no valid column for any row of this
+                // warp (zeros), 2 = some columns masked, 3 = every column valid for every row
+                int kind = 0;
+                if (c0 < n) {
+                    const bool all_valid = lo <= c0 && hi >= c0 + kPiece - 1;
+                    const bool none_valid = hi < lo || hi < c0 || lo > c0 + kPiece - 1;
+                    kind = __all_sync(0xffffffffu, all_valid) ? 3 : __all_sync(0xffffffffu, none_valid) ? 1 : 2;
                 }
-                const unsigned span = (unsigned)(hi - lo);
-                const bool any_col = hi >= lo;
-                const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN;
-                const uint32_t dp_tmem = tmem + lane_addr + kDpCol;
+                const uint32_t s_tmem = my_tmem + slot * kBlockN;
+                const uint32_t dp_tmem = my_tmem + kDpCol;
 
                 ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrElem);
                 if (!ok) break;
                 ok = mbar_wait_warp(bar(kBarDpFull), item & 1, abort_flag, p.status, kErrElem);
                 if (!ok) break;
                 tc_fence_after();
-
-                auto piece = [&](int h, const uint32_t (&rs)[kPieceB], const uint32_t (&rd)[kPieceB]) {
-                    uint32_t pk[kPieceB / 2];
-                    if (h >= h_b && h <= h_e) {
-                        float ds[kPieceB];
+                // two halves of 16 columns; dP goes back as soon as the second half is in registers
 #pragma unroll
-                        for (int c = 0; c < kPieceB; ++c) {
-                            float x = fmaf(__uint_as_float(rs[c]), p.sl2, neg_lse2);
-                            if (!full) x = (any_col && (unsigned)(h * kPieceB + c - lo) <= span) ? x : -INFINITY;
-                            ds[c] = exp2f(x) * (__uint_as_float(rd[c]) - drow);
+                for (int hf = 0; hf < 2; ++hf) {
+                    constexpr int kHalf = kPiece / 2;
+                    uint32_t rs[kHalf], rd[kHalf], pk[kHalf / 2];
+                    if (kind >= 2) {
+                        tmem_ld16(s_tmem + hf * kHalf, rs);
+                        tmem_ld16(dp_tmem + hf * kHalf, rd);
+                        tmem_wait_ld();
+                    }
+                    if (hf == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kBarDpFree));
+                    }
+                    if (kind >= 2) {
+                        float e[kHalf];
+#pragma unroll
+                        for (int c = 0; c < kHalf; ++c) e[c] = ex2_approx(fmaf(__uint_as_float(rs[c]), p.sl2, neg_lse2));
+                        if (kind == 2) {
+                            const unsigned span = (unsigned)(hi - lo);
+                            const int base = c0 + hf * kHalf - lo;
+                            const bool any_col = hi >= lo;
+#pragma unroll
+                            for (int c = 0; c < kHalf; ++c) e[c] = (any_col && (unsigned)(base + c) <= span) ? e[c] : 0.f;
                         }
 #pragma unroll
-                        for (int c = 0; c < kPieceB / 2; ++c) pk[c] = pack_bf16x2(ds[2 * c], ds[2 * c + 1]);
+                        for (int c = 0; c < kHalf / 2; ++c)
+                            pk[c] = pack_bf16x2(e[2 * c] * (__uint_as_float(rd[2 * c]) - drow),
+                                                e[2 * c + 1] * (__uint_as_float(rd[2 * c + 1]) - drow));
                     } else {
 #pragma unroll
-                        for (int c = 0; c < kPieceB / 2; ++c) pk[c] = 0u;
+                        for (int c = 0; c < kHalf / 2; ++c) pk[c] = 0u;
                     }
-                    tmem_st8(s_tmem + h * (kPieceB / 2), pk);
-                };
-                {
-                    uint32_t sa[kPieceB], sb[kPieceB], da[kPieceB], db[kPieceB];
-                    if (h_b == 0 && h_e >= 0) { tmem_ld16(s_tmem, sa); tmem_ld16(dp_tmem, da); }
-#pragma unroll 1
-                    for (int h = 0; h < nh; h += 2) {
-                        tmem_wait_ld();
-                        if (h + 1 >= h_b && h + 1 <= h_e) {
-                            tmem_ld16(s_tmem + (h + 1) * kPieceB, sb);
-                            tmem_ld16(dp_tmem + (h + 1) * kPieceB, db);
-                        }
-                        piece(h, sa, da);
-                        if (h + 1 < nh) {
-                            tmem_wait_ld();
-                            if (h + 2 >= h_b && h + 2 <= h_e) {
-                                tmem_ld16(s_tmem + (h + 2) * kPieceB, sa);
-                                tmem_ld16(dp_tmem + (h + 2) * kPieceB, da);
-                            }
-                            piece(h + 1, sb, db);
-                        }
-                    }
+                    if (kind != 0) tmem_st8(s_tmem + hf * (kHalf / 2), pk);
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(bar(kBarDpFree));
-                    mbar_arrive(bar(kBarDsReady + slot));
-                }
+                if (lane == 0) mbar_arrive(bar(kBarDsReady + slot));
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue warps (8..11)
+        // ------------------------------------------------------------------ epilogue warps (20..23)
         const int ew = warp & 3;
         const int row = 32 * ew + lane;
         const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
         const uint32_t stage = sbase + p.off_stage;
-        const bool issuer = warp == 8;
+        const bool issuer = warp == 4 + 4 * kGroups;
         if (issuer && lane == 0) prefetch_tensormap(&tm_dq);
         bool ok = true;
 #pragma unroll 1
@@ -535,31 +588,40 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ok = mbar_wait_warp(bar(kBarDqFull), tl & 1, abort_flag, p.status, kErrEpi);
             if (!ok) break;
             tc_fence_after();
-            uint32_t ob[D / 2];
-#pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch) {
-                uint32_t o[32];
-                tmem_ld32(tmem + lane_addr + kDqCol + ch * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 16; ++c)
-                    ob[ch * 16 + c] = pack_bf16x2(__uint_as_float(o[2 * c]) * p.scale, __uint_as_float(o[2 * c + 1]) * p.scale);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarDqFree));
             const int nseg = p.fd_seg.div(t.rows);
-#pragma unroll
+#pragma unroll 1
             for (int sl = 0; sl < C::kSlabs; ++sl) {
                 const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
+                uint32_t o0[32], o1[32];
+                tmem_ld32(tmem + lane_addr + kDqCol + sl * 64, o0);
+                tmem_ld32(tmem + lane_addr + kDqCol + sl * 64 + 32, o1);
+                tmem_wait_ld();
+                if (sl == C::kSlabs - 1) {  // dQ is free for the next tile once the last slab is in registers
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarDqFree));
+                }
                 ok = mbar_wait_warp(bar(kBarStageFree), (round & 1) ^ 1, abort_flag, p.status, kErrEpi);
                 if (!ok) break;
                 uint8_t *srow = smem + p.off_stage + row * 128;
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) =
-                        make_uint4(ob[sl * 32 + 4 * c], ob[sl * 32 + 4 * c + 1], ob[sl * 32 + 4 * c + 2],
-                                   ob[sl * 32 + 4 * c + 3]);
+                for (int c = 0; c < 4; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * p.scale, __uint_as_float(o0[8 * c + 1]) * p.scale);
+                    v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * p.scale, __uint_as_float(o0[8 * c + 3]) * p.scale);
+                    v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * p.scale, __uint_as_float(o0[8 * c + 5]) * p.scale);
+                    v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * p.scale, __uint_as_float(o0[8 * c + 7]) * p.scale);
+                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * p.scale, __uint_as_float(o1[8 * c + 1]) * p.scale);
+                    v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * p.scale, __uint_as_float(o1[8 * c + 3]) * p.scale);
+                    v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * p.scale, __uint_as_float(o1[8 * c + 5]) * p.scale);
+                    v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * p.scale, __uint_as_float(o1[8 * c + 7]) * p.scale);
+                    *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
+                }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarStageFull));
@@ -698,7 +760,6 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.total_tiles = plan.tiles_per_group * dm.Hkv;
     p.nblk_p = plan.nblk_p;
     p.tail_rows = plan.tail_rows;
-    p.resident = plan.resident;
     p.stages_k = plan.stages_k > 0 ? plan.stages_k : 1;
     p.stages_v = plan.stages_v > 0 ? plan.stages_v : 1;
     p.sfx_rows = plan.sfx_rows;
@@ -706,11 +767,12 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.off_sk = plan.off_sk; p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar;
     p.off_misc = plan.off_misc;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    auto kernel = plan.resident ? tc_bwd_dq_kernel<D, true> : tc_bwd_dq_kernel<D, false>;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[plan.resident]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[plan.resident] = true;
     }
     // D = <dout, out> per row, then dQ on the tensor cores, then dK_suffix / dV_suffix
     cudaError_t e = launch_simt_row_dot(a, stream);
@@ -718,8 +780,8 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
     {
         KernelTiming timing(kKernelBwdDqTc, stream);
-        tc_bwd_dq_kernel<D><<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,
-                                                                         tm_pv_tail, tm_sk, tm_sv, p);
+        kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail,
+                                                            tm_sk, tm_sv, p);
     }
     count_launches(1);
     e = cudaGetLastError();

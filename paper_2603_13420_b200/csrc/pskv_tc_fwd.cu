@@ -120,7 +120,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31;
-    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
+    const int phys_warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
+#ifdef PSKV_SERVICE_HIGH
+    // role index: physical warps 0-15 are the softmax warps (roles 4-19), 16-19 the producers and MMA
+    // issuers (roles 0-3), 20-23 the epilogue; the quadrant (index mod 4) is the same either way
+    const int warp = phys_warp < 16 ? phys_warp + 4 : phys_warp < 20 ? phys_warp - 16 : phys_warp;
+#else
+    const int warp = phys_warp;
+#endif
     PSKV_TRACE_DECL;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + p.off_bar;
@@ -393,6 +400,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                             mbar_arrive(bar(kBarStageFree));
                         }
                         __syncwarp();
+                        PSKV_TRACE_EVENT(4, tl - 1);
                         pend_store = false;
                     }
                 }
@@ -408,6 +416,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                                             sl * 64, 0, t.g, t.b_first + c);
                     }
                     __syncwarp();
+                    PSKV_TRACE_EVENT(5, tl);
                     pend_sv = false;
                 }
             }
@@ -494,6 +503,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (!ok) break;
             if (k == 0 && tl > 0) {
                 // O of the previous tile must have been read out by the epilogue warps
+                PSKV_TRACE_EVENT(15, i);
                 ok = mbar_wait_warp(bar(kBarOFree), (tl - 1) & 1, abort_flag, p.status, kErrMmaPv);
                 if (!ok) break;
             }
@@ -515,6 +525,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             } else {
                 n = t.n_sfx;
                 slab = sfx_slab;
+                PSKV_TRACE_EVENT(14, i);
                 ok = mbar_wait_warp(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMmaPv);
                 vaddr = sbase + p.off_sv;
             }
