@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kDkvWarps = 4;
 constexpr int kDkvThreads = kDkvWarps * 32;
-constexpr int kChunkRows = kDkvWarps * 16;  // 64 query rows per pass: small CTAs, several per SM
+constexpr int kChunkRows = kDkvWarps * 16;  // 64 query rows per pass
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr)
 {
@@ -44,6 +44,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool v
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_group1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
@@ -52,16 +54,17 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 }
 
 // Shared memory, all bf16 with 16 bytes of row padding (conflict-free ldmatrix):
-//   Qs, Gs  [64][D]       query / dout rows of the current chunk
+//   Qs, Gs  [2][64][D]    query / dout rows of the current chunk and of the next one (two stages)
 //   Ks, Vs  [TP][D]       suffix keys / values (TP = S rounded up to 16, padding rows zero)
 //   Ps, Ds  [64][TP]      probabilities / dS of the chunk
 template <int D, int TP>
 struct DkvSmem {
     static constexpr int kRowD = D * 2 + 16;
     static constexpr int kRowT = TP * 2 + 16;
-    static constexpr int kOffQ = 0;
+    static constexpr int kStage = 2 * kChunkRows * kRowD;  // one stage: Q rows, then dout rows
+    static constexpr int kOffQ = 0;                        // stage 0; stage 1 follows
     static constexpr int kOffG = kOffQ + kChunkRows * kRowD;
-    static constexpr int kOffK = kOffG + kChunkRows * kRowD;
+    static constexpr int kOffK = kOffQ + 2 * kStage;
     static constexpr int kOffV = kOffK + TP * kRowD;
     static constexpr int kOffP = kOffV + TP * kRowD;
     static constexpr int kOffS = kOffP + kChunkRows * kRowT;
@@ -69,36 +72,56 @@ struct DkvSmem {
 };
 
 template <int D, int TP>
-__global__ void __launch_bounds__(kDkvThreads, 3)
+__global__ void __launch_bounds__(kDkvThreads, 2)
 bwd_dkv_mma_kernel(BwdArgs a)
 {
     using L = DkvSmem<D, TP>;
     extern __shared__ __align__(16) uint8_t smem[];
     const Dims dm = a.dims;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bg = blockIdx.x;  // b * Hkv + g
-    const int b = bg / dm.Hkv, g = bg - b * dm.Hkv;
     const int S = dm.S, Rg = dm.n_rep * S;
-    const size_t row0 = ((size_t)b * dm.Hq + (size_t)g * dm.n_rep) * S;  // first query row of the group
-    const __nv_bfloat16 *qg = a.q + row0 * D;
-    const __nv_bfloat16 *gg = a.dout + row0 * D;
-    const __nv_bfloat16 *kg = a.suffix_k + (size_t)bg * S * D;
-    const __nv_bfloat16 *vg = a.suffix_v + (size_t)bg * S * D;
+    const int nchunk = (Rg + kChunkRows - 1) / kChunkRows;
+    const int total_bg = dm.B * dm.Hkv;
     const uint32_t sb = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
     const float sl2 = a.scale * kLog2e;
 
-    // suffix K / V once; padding rows zero
-    for (int i = tid; i < TP * (D / 8); i += kDkvThreads) {
-        const int t = i / (D / 8), c = i - t * (D / 8);
-        const int ts = t < S ? t : 0;
-        cp_async16(sb + L::kOffK + t * L::kRowD + c * 16, kg + (size_t)ts * D + c * 8, t < S);
-        cp_async16(sb + L::kOffV + t * L::kRowD + c * 16, vg + (size_t)ts * D + c * 8, t < S);
-    }
+    // The CTA walks over its (candidate, KV head) groups, a chunk of 64 query rows at a time; the
+    // copies of the next chunk (of this group or the next) are in flight while this one is computed.
+    // unit u = (group index within this CTA, chunk)
+    const int my_groups = blockIdx.x < total_bg ? (total_bg - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+    const int total_units = my_groups * nchunk;
+
+    auto issue_qg = [&](int u) {  // asynchronous copies of unit u's query / dout rows into stage u & 1
+        const int gi = u / nchunk, c = u - gi * nchunk;
+        const int bg = blockIdx.x + gi * gridDim.x;
+        const int b = bg / dm.Hkv, g = bg - b * dm.Hkv;
+        const size_t row0 = ((size_t)b * dm.Hq + (size_t)g * dm.n_rep) * S + (size_t)c * kChunkRows;
+        const __nv_bfloat16 *qg = a.q + row0 * D;
+        const __nv_bfloat16 *gg = a.dout + row0 * D;
+        const int rows = min(kChunkRows, Rg - c * kChunkRows);
+        const uint32_t st = sb + (u & 1) * L::kStage;
+        for (int i = tid; i < kChunkRows * (D / 8); i += kDkvThreads) {
+            const int r = i / (D / 8), cc = i - r * (D / 8);
+            const int rs = r < rows ? r : 0;
+            cp_async16(st + L::kOffQ + r * L::kRowD + cc * 16, qg + (size_t)rs * D + cc * 8, r < rows);
+            cp_async16(st + L::kOffG + r * L::kRowD + cc * 16, gg + (size_t)rs * D + cc * 8, r < rows);
+        }
+    };
+    auto issue_kv = [&](int gi) {  // suffix K / V of group gi; padding rows zero
+        const int bg = blockIdx.x + gi * gridDim.x;
+        const __nv_bfloat16 *kg = a.suffix_k + (size_t)bg * S * D;
+        const __nv_bfloat16 *vg = a.suffix_v + (size_t)bg * S * D;
+        for (int i = tid; i < TP * (D / 8); i += kDkvThreads) {
+            const int t = i / (D / 8), c = i - t * (D / 8);
+            const int ts = t < S ? t : 0;
+            cp_async16(sb + L::kOffK + t * L::kRowD + c * 16, kg + (size_t)ts * D + c * 8, t < S);
+            cp_async16(sb + L::kOffV + t * L::kRowD + c * 16, vg + (size_t)ts * D + c * 8, t < S);
+        }
+    };
 
     // this warp's output tiles: all m-tiles (keys) x its kNT consecutive n-tiles (8 columns each)
     constexpr int kMT = TP / 16;
     constexpr int kNT = D / 8 / kDkvWarps;
-    const bool active = true;
     float accV[kMT][kNT][4], accK[kMT][kNT][4];
 #pragma unroll
     for (int m = 0; m < kMT; ++m)
@@ -107,16 +130,27 @@ bwd_dkv_mma_kernel(BwdArgs a)
 #pragma unroll
             for (int e = 0; e < 4; ++e) { accV[m][n][e] = 0.f; accK[m][n][e] = 0.f; }
 
-    for (int c0 = 0; c0 < Rg; c0 += kChunkRows) {
+    if (total_units > 0) {
+        issue_kv(0);
+        issue_qg(0);
+    }
+    cp_async_commit();
+
+#pragma unroll 1
+    for (int u = 0; u < total_units; ++u) {
+        const int gi = u / nchunk, c = u - gi * nchunk;
+        const int bg = blockIdx.x + gi * gridDim.x;
+        const int b = bg / dm.Hkv, g = bg - b * dm.Hkv;
+        const size_t row0 = ((size_t)b * dm.Hq + (size_t)g * dm.n_rep) * S;  // first query row of the group
+        const int c0 = c * kChunkRows;
         const int rows = min(kChunkRows, Rg - c0);
-        __syncthreads();  // previous chunk fully consumed (also orders the K/V staging above)
-        for (int i = tid; i < kChunkRows * (D / 8); i += kDkvThreads) {
-            const int r = i / (D / 8), c = i - r * (D / 8);
-            const int rs = r < rows ? c0 + r : 0;
-            cp_async16(sb + L::kOffQ + r * L::kRowD + c * 16, qg + (size_t)rs * D + c * 8, r < rows);
-            cp_async16(sb + L::kOffG + r * L::kRowD + c * 16, gg + (size_t)rs * D + c * 8, r < rows);
-        }
-        cp_async_wait_all();
+        const uint32_t st = sb + (u & 1) * L::kStage;
+        const bool last_chunk = c == nchunk - 1;
+
+        // the next unit's rows go into the other stage (free since the barrier that ended unit u-1)
+        if (u + 1 < total_units) issue_qg(u + 1);
+        cp_async_commit();
+        cp_async_wait_group1();  // everything but the copies just issued has landed: unit u (and its K / V)
         __syncthreads();
 
         // ---- phase 1: this warp's 16 rows: S = Q K^T, dP = dO V^T, then P and dS to shared memory
@@ -131,8 +165,8 @@ bwd_dkv_mma_kernel(BwdArgs a)
             for (int k0 = 0; k0 < D; k0 += 16) {
                 uint32_t aq[4], ag[4];
                 const uint32_t arow = (uint32_t)(r_base + (lane & 15)) * L::kRowD + (uint32_t)(k0 + (lane >> 4) * 8) * 2;
-                ldsm_x4(aq, sb + L::kOffQ + arow);
-                ldsm_x4(ag, sb + L::kOffG + arow);
+                ldsm_x4(aq, st + L::kOffQ + arow);
+                ldsm_x4(ag, st + L::kOffG + arow);
 #pragma unroll
                 for (int n = 0; n < TP / 16; ++n) {
                     // two key tiles (16 keys) per ldmatrix.x4: lanes 0-7 keys +0..7 @k0, 8-15 same keys @k0+8,
@@ -175,10 +209,13 @@ bwd_dkv_mma_kernel(BwdArgs a)
             }
         }
         __syncthreads();
+        // suffix K / V are not read after phase 1: fetch the next group's while phase 2 runs
+        if (last_chunk && gi + 1 < my_groups) issue_kv(gi + 1);
+        cp_async_commit();  // its own group (possibly empty), so that the wait above covers it next time round
 
         // ---- phase 2: dV += P^T dO, dK += dS^T Q over the chunk's rows (contraction index = row)
 #pragma unroll 1
-        for (int k0 = 0; k0 < kChunkRows && active; k0 += 16) {
+        for (int k0 = 0; k0 < kChunkRows; k0 += 16) {
             if (k0 >= rows) break;  // rows past `rows` inside a started 16-row step are zero
             uint32_t bg_[kNT][2], bq_[kNT][2];
 #pragma unroll
@@ -187,9 +224,9 @@ bwd_dkv_mma_kernel(BwdArgs a)
                 const uint32_t off = (uint32_t)(k0 + (lane & 7) + ((lane >> 3) & 1) * 8) * L::kRowD +
                                      (uint32_t)((warp * kNT + n) * 8 + (lane >> 4) * 8) * 2;
                 uint32_t t4[4];
-                ldsm_x4_trans(t4, sb + L::kOffG + off);
+                ldsm_x4_trans(t4, st + L::kOffG + off);
                 bg_[n][0] = t4[0]; bg_[n][1] = t4[1]; bg_[n + 1][0] = t4[2]; bg_[n + 1][1] = t4[3];
-                ldsm_x4_trans(t4, sb + L::kOffQ + off);
+                ldsm_x4_trans(t4, st + L::kOffQ + off);
                 bq_[n][0] = t4[0]; bq_[n][1] = t4[1]; bq_[n + 1][0] = t4[2]; bq_[n + 1][1] = t4[3];
             }
 #pragma unroll
@@ -208,27 +245,44 @@ bwd_dkv_mma_kernel(BwdArgs a)
                 }
             }
         }
-    }
 
-    // ---- store: accumulator element e: key = m*16 + lane/4 + 8*(e/2), column = n-tile*8 + 2*(lane%4) + (e%2)
-    __nv_bfloat16 *dkg = a.dk_suffix + (size_t)bg * S * D;
-    __nv_bfloat16 *dvg = a.dv_suffix + (size_t)bg * S * D;
+        if (last_chunk) {
+            // ---- store: accumulator element e: key = m*16 + lane/4 + 8*(e/2), column = n-tile*8 + 2*(lane%4) + (e%2)
+            __nv_bfloat16 *dkg = a.dk_suffix + (size_t)bg * S * D;
+            __nv_bfloat16 *dvg = a.dv_suffix + (size_t)bg * S * D;
 #pragma unroll
-    for (int m = 0; m < kMT; ++m)
+            for (int m = 0; m < kMT; ++m)
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int t = m * 16 + (lane >> 2) + 8 * half;
-            if (t < S && active) {
+                for (int half = 0; half < 2; ++half) {
+                    const int t = m * 16 + (lane >> 2) + 8 * half;
 #pragma unroll
-                for (int n = 0; n < kNT; ++n) {
-                    const int col = (warp * kNT + n) * 8 + 2 * (lane & 3);
-                    *reinterpret_cast<uint32_t *>(dvg + (size_t)t * D + col) =
-                        pack2(accV[m][n][2 * half], accV[m][n][2 * half + 1]);
-                    *reinterpret_cast<uint32_t *>(dkg + (size_t)t * D + col) =
-                        pack2(accK[m][n][2 * half] * a.scale, accK[m][n][2 * half + 1] * a.scale);
+                    for (int n = 0; n < kNT; ++n) {
+                        if (t < S) {
+                            const int col = (warp * kNT + n) * 8 + 2 * (lane & 3);
+                            *reinterpret_cast<uint32_t *>(dvg + (size_t)t * D + col) =
+                                pack2(accV[m][n][2 * half], accV[m][n][2 * half + 1]);
+                            *reinterpret_cast<uint32_t *>(dkg + (size_t)t * D + col) =
+                                pack2(accK[m][n][2 * half] * a.scale, accK[m][n][2 * half + 1] * a.scale);
+                        }
+                        accV[m][n][2 * half] = 0.f; accV[m][n][2 * half + 1] = 0.f;
+                        accK[m][n][2 * half] = 0.f; accK[m][n][2 * half + 1] = 0.f;
+                    }
                 }
-            }
         }
+        __syncthreads();  // this unit's stage, P and dS are free for the next units
+    }
+    cp_async_wait_all();
+}
+
+inline int sm_count_dkv()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    }
+    return n;
 }
 
 template <int D, int TP>
@@ -243,7 +297,9 @@ cudaError_t launch_one(const BwdArgs &a, cudaStream_t stream)
         attr_set = true;
     }
     KernelTiming timing(kKernelBwdDkvMma, stream);
-    bwd_dkv_mma_kernel<D, TP><<<a.dims.B * a.dims.Hkv, kDkvThreads, L::kBytes, stream>>>(a);
+    const int total_bg = a.dims.B * a.dims.Hkv;
+    const int max_ctas = 2 * sm_count_dkv();  // two resident CTAs per SM, each walking over its groups
+    bwd_dkv_mma_kernel<D, TP><<<total_bg < max_ctas ? total_bg : max_ctas, kDkvThreads, L::kBytes, stream>>>(a);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -334,6 +334,38 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
+// Two-wide fp32 arithmetic (one instruction for a pair of values): (a, b) *= s and (a, b) += (c, d)
+__device__ __forceinline__ void mul_f32x2(float &a, float &b, float s)
+{
+    asm("{\n\t.reg .b64 x, y;\n\tmov.b64 x, {%0, %1};\n\tmov.b64 y, {%2, %2};\n\tmul.f32x2 x, x, y;\n\t"
+        "mov.b64 {%0, %1}, x;\n\t}"
+        : "+f"(a), "+f"(b)
+        : "f"(s));
+}
+// (a, b) = (a, b) * s + t
+__device__ __forceinline__ void fma_f32x2(float &a, float &b, float s, float t)
+{
+    asm("{\n\t.reg .b64 x, y, z;\n\tmov.b64 x, {%0, %1};\n\tmov.b64 y, {%2, %2};\n\tmov.b64 z, {%3, %3};\n\t"
+        "fma.rn.f32x2 x, x, y, z;\n\tmov.b64 {%0, %1}, x;\n\t}"
+        : "+f"(a), "+f"(b)
+        : "f"(s), "f"(t));
+}
+// (a, b) *= (c, d)
+__device__ __forceinline__ void mul_f32x2(float &a, float &b, float c, float d)
+{
+    asm("{\n\t.reg .b64 x, y;\n\tmov.b64 x, {%0, %1};\n\tmov.b64 y, {%2, %3};\n\tmul.f32x2 x, x, y;\n\t"
+        "mov.b64 {%0, %1}, x;\n\t}"
+        : "+f"(a), "+f"(b)
+        : "f"(c), "f"(d));
+}
+__device__ __forceinline__ void add_f32x2(float &a, float &b, float c, float d)
+{
+    asm("{\n\t.reg .b64 x, y;\n\tmov.b64 x, {%0, %1};\n\tmov.b64 y, {%2, %3};\n\tadd.f32x2 x, x, y;\n\t"
+        "mov.b64 {%0, %1}, x;\n\t}"
+        : "+f"(a), "+f"(b)
+        : "f"(c), "f"(d));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     uint32_t r;

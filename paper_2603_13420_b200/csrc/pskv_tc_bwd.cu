@@ -549,7 +549,12 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     if (kind >= 2) {
                         float e[kHalf];
 #pragma unroll
-                        for (int c = 0; c < kHalf; ++c) e[c] = ex2_approx(fmaf(__uint_as_float(rs[c]), p.sl2, neg_lse2));
+                        for (int c = 0; c < kHalf; c += 2) {
+                            float x0 = __uint_as_float(rs[c]), x1 = __uint_as_float(rs[c + 1]);
+                            fma_f32x2(x0, x1, p.sl2, neg_lse2);
+                            e[c] = ex2_approx(x0);
+                            e[c + 1] = ex2_approx(x1);
+                        }
                         if (kind == 2) {
                             const unsigned span = (unsigned)(hi - lo);
                             const int base = c0 + hf * kHalf - lo;
@@ -558,9 +563,12 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                             for (int c = 0; c < kHalf; ++c) e[c] = (any_col && (unsigned)(base + c) <= span) ? e[c] : 0.f;
                         }
 #pragma unroll
-                        for (int c = 0; c < kHalf / 2; ++c)
-                            pk[c] = pack_bf16x2(e[2 * c] * (__uint_as_float(rd[2 * c]) - drow),
-                                                e[2 * c + 1] * (__uint_as_float(rd[2 * c + 1]) - drow));
+                        for (int c = 0; c < kHalf / 2; ++c) {
+                            float d0 = __uint_as_float(rd[2 * c]), d1 = __uint_as_float(rd[2 * c + 1]);
+                            add_f32x2(d0, d1, -drow, -drow);
+                            mul_f32x2(d0, d1, e[2 * c], e[2 * c + 1]);
+                            pk[c] = pack_bf16x2(d0, d1);
+                        }
                     } else {
 #pragma unroll
                         for (int c = 0; c < kHalf / 2; ++c) pk[c] = 0u;

@@ -641,7 +641,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                             // special-function unit), then sums and bf16 pairs
                             float e[kPiece];
 #pragma unroll
-                            for (int c = 0; c < kPiece; ++c) e[c] = ex2_approx(__uint_as_float(rr[c]) * p.sl2);
+                            for (int c = 0; c < kPiece; c += 2) {
+                                float x0 = __uint_as_float(rr[c]), x1 = __uint_as_float(rr[c + 1]);
+                                mul_f32x2(x0, x1, p.sl2);
+                                e[c] = ex2_approx(x0);
+                                e[c + 1] = ex2_approx(x1);
+                            }
                             if (kind == 2) {
                                 const unsigned span = (unsigned)(hi - lo);
                                 const int base = c0 - lo;
@@ -653,10 +658,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                             float ls2 = 0.f, ls3 = 0.f;
 #pragma unroll
                             for (int c = 0; c < kPiece / 4; ++c) {
-                                ls0 += e[4 * c];
-                                ls1 += e[4 * c + 1];
-                                ls2 += e[4 * c + 2];
-                                ls3 += e[4 * c + 3];
+                                add_f32x2(ls0, ls1, e[4 * c], e[4 * c + 1]);
+                                add_f32x2(ls2, ls3, e[4 * c + 2], e[4 * c + 3]);
                                 pk[2 * c] = pack_bf16x2(e[4 * c], e[4 * c + 1]);
                                 pk[2 * c + 1] = pack_bf16x2(e[4 * c + 2], e[4 * c + 3]);
                             }
