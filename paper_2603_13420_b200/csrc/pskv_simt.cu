@@ -235,22 +235,47 @@ simt_bwd_dq_kernel(BwdArgs a)
     store_slice<D>(a.dq + (size_t)row * D, lane, acc);
 }
 
-// D = <dout, out> for every query row: one warp per row.
+// D = <dout, out> for every query row.  A pure streaming pass over two tensors, so it is laid out
+// for bytes in flight: D/8 lanes share a row with one 16-byte load each per tensor, so a warp-wide
+// load covers 2 rows (d = 128) or 4 (d = 64), and every thread keeps kRowDotUnroll such loads of
+// both tensors outstanding.
+constexpr int kRowDotUnroll = 4;
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 simt_row_dot_kernel(BwdArgs a)
 {
+    constexpr int kLanesPerRow = D / 8;             // 16 (d = 128) or 8 (d = 64)
+    constexpr int kRowsPerLoad = 32 / kLanesPerRow;  // rows one warp-wide load covers
+    constexpr int kRowsPerWarp = kRowsPerLoad * kRowDotUnroll;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * kWarpsPerBlock + warp;
-    if (row >= (long long)a.dims.B * a.dims.Hq * a.dims.S) return;
-    float o[D / 32], g[D / 32];
-    load_slice<D>(a.out + (size_t)row * D, lane, o);
-    load_slice<D>(a.dout + (size_t)row * D, lane, g);
-    float acc = 0.f;
+    const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
+    const long long first = ((long long)blockIdx.x * kWarpsPerBlock + warp) * kRowsPerWarp;
+    if (first >= rows) return;
+    const int sub = lane / kLanesPerRow, col = (lane % kLanesPerRow) * 8;
+    uint4 o[kRowDotUnroll], g[kRowDotUnroll];
 #pragma unroll
-    for (int e = 0; e < D / 32; ++e) acc = fmaf(o[e], g[e], acc);
-    acc = warp_sum(acc);
-    if (lane == 0) a.row_dot[row] = acc;
+    for (int u = 0; u < kRowDotUnroll; ++u) {
+        const long long row = first + u * kRowsPerLoad + sub;
+        const long long rc = row < rows ? row : rows - 1;  // clamp: the value is dropped below
+        o[u] = *reinterpret_cast<const uint4 *>(a.out + (size_t)rc * D + col);
+        g[u] = *reinterpret_cast<const uint4 *>(a.dout + (size_t)rc * D + col);
+    }
+#pragma unroll
+    for (int u = 0; u < kRowDotUnroll; ++u) {
+        const __nv_bfloat162 *ob = reinterpret_cast<const __nv_bfloat162 *>(&o[u]);
+        const __nv_bfloat162 *gb = reinterpret_cast<const __nv_bfloat162 *>(&g[u]);
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 x = __bfloat1622float2(ob[e]), y = __bfloat1622float2(gb[e]);
+            acc = fmaf(x.x, y.x, acc);
+            acc = fmaf(x.y, y.y, acc);
+        }
+#pragma unroll
+        for (int off = kLanesPerRow / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        const long long row = first + u * kRowsPerLoad + sub;
+        if (lane % kLanesPerRow == 0 && row < rows) a.row_dot[row] = acc;
+    }
 }
 
 // Backward, key side: one warp per suffix key (b,g,t); sums over the n_rep heads of the group
@@ -350,9 +375,11 @@ cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream)
     const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
     KernelTiming timing(kKernelRowDot, stream);
     if (a.dims.d == 128)
-        simt_row_dot_kernel<128><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+        simt_row_dot_kernel<128><<<blocks_for((rows + 2 * kRowDotUnroll - 1) / (2 * kRowDotUnroll)), kWarpsPerBlock * 32, 0,
+                                   stream>>>(a);
     else
-        simt_row_dot_kernel<64><<<blocks_for(rows), kWarpsPerBlock * 32, 0, stream>>>(a);
+        simt_row_dot_kernel<64><<<blocks_for((rows + 4 * kRowDotUnroll - 1) / (4 * kRowDotUnroll)), kWarpsPerBlock * 32, 0,
+                                  stream>>>(a);
     count_launches(1);
     return cudaGetLastError();
 }
