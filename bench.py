@@ -396,9 +396,10 @@ def roofline(w, kernels, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (kernel, workload) -> bytes.
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("tc_fwd_kernel", "C2"): 475.2e6,       # profiles/tc_fwd_kernel_C2.md
-    ("tc_bwd_dq_kernel", "C2"): 690.6e6,    # profiles/tc_bwd_dq_kernel_C2.md
-    ("bwd_dkv_mma_kernel", "C2"): 596.7e6,  # profiles/bwd_dkv_mma_kernel_C2.md
+    ("tc_fwd_kernel", "C2"): 473.4e6,        # profiles/tc_fwd_kernel_C2.md
+    ("tc_bwd_dq_kernel", "C2"): 694.7e6,     # profiles/tc_bwd_dq_kernel_C2.md
+    ("bwd_dkv_mma_kernel", "C2"): 592.7e6,   # profiles/bwd_dkv_mma_kernel_C2.md
+    ("simt_row_dot_kernel", "C2"): 408.8e6,  # profiles/simt_row_dot_kernel_C2.md
 }
 
 
