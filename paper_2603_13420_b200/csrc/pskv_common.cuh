@@ -40,6 +40,8 @@ cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
 // dk_suffix / dv_suffix on warp-level tensor-core MMAs, one CTA per (candidate, KV head); S <= 64.
 bool mma_bwd_dkv_supported(const Dims &d);
 cudaError_t launch_mma_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
+bool tc_bwd_dkv_supported(const Dims &d);
+cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream);
 // Recomputes the rows whose lse is NaN, if *redo_count != 0 (a device counter); `blocks` CTAs.
 cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream);
 
@@ -59,7 +61,7 @@ void count_launches(int n);
 // Optional per-kernel device timing (pskv_kernel_timing_*): when enabled, a launch site brackets
 // its kernel with two CUDA events on the launch stream.
 enum KernelId {
-    kKernelFwdTc = 0, kKernelFwdRedo, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvMma,
+    kKernelFwdTc = 0, kKernelFwdRedo, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvTc, kKernelBwdDkvMma,
     kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCount
 };
 void *timing_begin(int kernel_id, cudaStream_t stream);  // returns nullptr when timing is off

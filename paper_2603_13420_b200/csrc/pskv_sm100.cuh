@@ -298,6 +298,13 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int b_mn_ma
            (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// The same with either operand's major-ness given: *_mn_major = 1 when that operand is stored with
+// its M (A) or N (B) index contiguous instead of K.
+__host__ __device__ constexpr uint32_t make_idesc_bf16_ab(int M, int N, int a_mn_major, int b_mn_major)
+{
+    return make_idesc_bf16(M, N, b_mn_major) | (static_cast<uint32_t>(a_mn_major) << 15);
+}
+
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate)

@@ -794,6 +794,7 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (tc_bwd_dkv_supported(dm)) return launch_tc_bwd_dkv(a, status_word, stream);
     return mma_bwd_dkv_supported(dm) ? launch_mma_bwd_dkv(a, stream) : launch_simt_bwd_dkv(a, stream);
 }
 
