@@ -90,9 +90,11 @@ __device__ __forceinline__ int prefix_block_rows(const TcBwdParams &p, int k)
     return k == p.nblk_p - 1 ? p.tail_rows : kBlockN;
 }
 
-// RES: all prefix blocks of a KV head stay in shared memory (else they stream through rings); a
-// compile-time switch so that each launch carries only the code of its own mode.
-template <int D, bool RES>
+// MODE bit 0: the prefix K blocks of a KV head stay in shared memory; bit 1: the prefix V blocks do
+// (else they stream through rings).  A K block is needed through a whole item (the dQ MMA reads it
+// after the element-wise stage), a V block only for its dP MMA, so when not both fit it is K that
+// stays.  Compile-time, so that each launch carries only the code of its own mode.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                  const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_pk,
@@ -101,6 +103,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                  const __grid_constant__ CUtensorMap tm_sv, const TcBwdParams p)
 {
     using C = Cfg<D>;
+    constexpr bool RK = (MODE & 1) != 0, RV = (MODE & 2) != 0;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
@@ -200,7 +203,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
             }
             __syncwarp();
-            if (!RES) {
+            if (!RK) {
 #pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const uint32_t ks = kload % stages_k;
@@ -225,7 +228,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 ok = mbar_wait_warp(bar(kBarDqFull), (tl - 1) & 1, abort_flag, p.status, kErrProdA);
                 if (!ok) break;
             }
-            if (RES && t.first_of_g && elect_one_sync()) {
+            if (RK && t.first_of_g && elect_one_sync()) {
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const bool tail = k == p.nblk_p - 1;
                     const int slab = tail ? tail_slab : C::kSlabBytes;
@@ -294,7 +297,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         ++qb;
                     }
                 }
-                if (RES && t.first_of_g) {
+                if (RV && t.first_of_g) {
                     for (int k = 0; k < p.nblk_p; ++k) {
                         const bool tail = k == p.nblk_p - 1;
                         const int slab = tail ? tail_slab : C::kSlabBytes;
@@ -311,7 +314,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                                     sl * 64, 0, t.g, t.b_first + c);
             }
             __syncwarp();
-            if (!RES) {
+            if (!RV) {
 #pragma unroll 1
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const uint32_t vs = vload % stages_v;
@@ -346,7 +349,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
             const int slab = prefix ? n * 128 : sfx_slab;
             const bool last_of_tile = k == nitems - 1;
-            const bool ring = prefix && !RES;
+            const bool ring_k = prefix && !RK, ring_v = prefix && !RV;
             const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
             const uint64_t slab16 = (uint64_t)(slab >> 4);
             // ---- S: the slot is free once the dQ MMAs of item i-2 have completed
@@ -356,7 +359,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) break;
             uint32_t kaddr;
             if (prefix) {
-                if (RES) {
+                if (RK) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
@@ -393,7 +396,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) break;
             uint32_t vaddr;
             if (prefix) {
-                if (RES) {
+                if (RV) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
                     vaddr = sbase + p.off_pv + k * C::kTileBytes;
@@ -418,12 +421,13 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         mma_ss(tmem + kDpCol, do_desc + aoff, v_desc + voff, idesc, ks16 > 0 ? 1u : 0u);
                     }
                     tc_commit(bar(kBarDpFull));
-                    if (ring) tc_commit(bar(kBarVFree + (vuse % stages_v)));
+                    if (ring_v) tc_commit(bar(kBarVFree + (vuse % stages_v)));
                     if (last_of_tile) tc_commit(bar(kBarDvFree));
                 }
                 __syncwarp();
             }
-            if (ring) { ++kuse; ++vuse; }
+            if (ring_k) ++kuse;
+            if (ring_v) ++vuse;
             if (++k == nitems) {
                 k = 0;
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
@@ -444,7 +448,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
             const int slab = prefix ? n * 128 : sfx_slab;
             const bool last_of_tile = k == nitems - 1;
-            const bool ring = prefix && !RES;
+            const bool ring = prefix && !RK;
             ok = mbar_wait_warp(bar(kBarDsReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaDq);
             if (!ok) break;
             if (k == 0 && tl > 0) {
@@ -452,7 +456,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (!ok) break;
             }
             uint32_t kaddr;
-            if (prefix) kaddr = sbase + p.off_pk + (RES ? (uint32_t)k : kuse % stages_k) * C::kTileBytes;
+            if (prefix) kaddr = sbase + p.off_pk + (RK ? (uint32_t)k : kuse % stages_k) * C::kTileBytes;
             else kaddr = sbase + p.off_sk;
             tc_fence_after();
             const uint32_t ds_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
@@ -686,16 +690,24 @@ BwdPlan plan_bwd(const Dims &dm)
     const int resident_bytes = pl.nblk_p ? (pl.nblk_p - 1) * tile_bytes + tail_bytes : 0;
     int k_bytes = 0, v_bytes = 0;
     if (pl.nblk_p <= kMaxStages && fixed + 2 * resident_bytes <= kMaxSmem) {
-        pl.resident = 1;
+        pl.resident = 3;  // K and V resident
         pl.stages_k = pl.stages_v = pl.nblk_p > 0 ? pl.nblk_p : 1;
         k_bytes = v_bytes = resident_bytes;
+    } else if (pl.nblk_p <= kMaxStages && fixed + resident_bytes + tile_bytes <= kMaxSmem) {
+        // K resident, V through a ring: a K block is needed through a whole item (its dQ MMA comes
+        // after the element-wise stage), a V block only for its dP MMA
+        pl.resident = 1;
+        pl.stages_k = pl.nblk_p;
+        int nv = (kMaxSmem - fixed - resident_bytes) / tile_bytes;
+        pl.stages_v = nv > kMaxStages ? kMaxStages : nv;
+        k_bytes = resident_bytes;
+        v_bytes = pl.stages_v * tile_bytes;
     } else {
-        // ring mode: a K block lives from its score MMAs to its dQ MMAs, a V block only through its
-        // dP MMAs, so K gets the larger share of the stages that fit
+        // ring mode: K gets the larger share of the stages that fit, for the same reason
         int n = (kMaxSmem - fixed) / tile_bytes;
         if (n > 2 * kMaxStages) n = 2 * kMaxStages;
         if (n < 2) return pl;
-        pl.stages_v = n / 3 > 0 ? n / 3 : 1;
+        pl.stages_v = n >= 6 ? 2 : 1;
         pl.stages_k = n - pl.stages_v;
         if (pl.stages_k > kMaxStages) pl.stages_k = kMaxStages;
         k_bytes = pl.stages_k * tile_bytes;
@@ -775,8 +787,8 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.off_sk = plan.off_sk; p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar;
     p.off_misc = plan.off_misc;
 
-    auto kernel = plan.resident ? tc_bwd_dq_kernel<D, true> : tc_bwd_dq_kernel<D, false>;
-    static bool attr_set[2] = {false, false};
+    auto kernel = plan.resident == 3 ? tc_bwd_dq_kernel<D, 3> : plan.resident == 1 ? tc_bwd_dq_kernel<D, 1> : tc_bwd_dq_kernel<D, 0>;
+    static bool attr_set[4] = {false, false, false, false};
     if (!attr_set[plan.resident]) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
