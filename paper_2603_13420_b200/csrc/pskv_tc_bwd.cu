@@ -334,13 +334,12 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ S = Q K^T, dP = dO V^T
+        // ------------------------------------------------------------------ S = Q K^T
         const int total_items = n_tiles * nitems;
         int tl = 0, k = 0;
-        uint32_t kuse = 0, vuse = 0;
+        uint32_t kuse = 0;
         TileInfo t = tile_info(p, t_begin, t_begin);
         const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
-        const uint64_t do_desc = make_smem_desc(sbase + p.off_do, 0, 1024);
         bool ok = true;
 #pragma unroll 1
         for (int i = 0; i < total_items && ok; ++i) {
@@ -349,7 +348,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
             const int slab = prefix ? n * 128 : sfx_slab;
             const bool last_of_tile = k == nitems - 1;
-            const bool ring_k = prefix && !RK, ring_v = prefix && !RV;
+            const bool ring_k = prefix && !RK;
             const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
             const uint64_t slab16 = (uint64_t)(slab >> 4);
             // ---- S: the slot is free once the dQ MMAs of item i-2 have completed
@@ -389,60 +388,91 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
                 __syncwarp();
             }
-            // ---- dP: its single slot is free once the element-wise warps have read item i-1
-            ok = mbar_wait_warp(bar(kBarDpFree), (i & 1) ^ 1, abort_flag, p.status, kErrMmaS);
-            if (!ok) break;
-            if (k == 0) ok = mbar_wait_warp(bar(kBarDoFull), tl & 1, abort_flag, p.status, kErrMmaS);
-            if (!ok) break;
-            uint32_t vaddr;
-            if (prefix) {
-                if (RV) {
-                    if (t.first_of_g)
-                        ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
-                    vaddr = sbase + p.off_pv + k * C::kTileBytes;
-                } else {
-                    const uint32_t vs = vuse % stages_v;
-                    ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / stages_v) & 1, abort_flag, p.status, kErrMmaS);
-                    vaddr = sbase + p.off_pv + vs * C::kTileBytes;
-                }
-            } else {
-                ok = mbar_wait_warp(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMmaS);
-                vaddr = sbase + p.off_sv;
-            }
-            if (!ok) break;
-            tc_fence_after();
-            {
-                const uint64_t v_desc = make_smem_desc(vaddr, 0, 1024);
-                if (elect_one_sync()) {
-#pragma unroll
-                    for (int ks16 = 0; ks16 < D / 16; ++ks16) {
-                        const uint64_t aoff = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
-                        const uint64_t voff = (uint64_t)(ks16 >> 2) * slab16 + (uint64_t)(((ks16 & 3) * 32) >> 4);
-                        mma_ss(tmem + kDpCol, do_desc + aoff, v_desc + voff, idesc, ks16 > 0 ? 1u : 0u);
-                    }
-                    tc_commit(bar(kBarDpFull));
-                    if (ring_v) tc_commit(bar(kBarVFree + (vuse % stages_v)));
-                    if (last_of_tile) tc_commit(bar(kBarDvFree));
-                }
-                __syncwarp();
-            }
             if (ring_k) ++kuse;
-            if (ring_v) ++vuse;
             if (++k == nitems) {
                 k = 0;
                 if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
             }
         }
     } else if (warp == 2) {
-        // ------------------------------------------------------------------ dQ += dS K
+        // ------------------------------------------------------------------ dP = dO V^T, dQ += dS K
+        // This warp alternates: dP of item i+1 (its buffer comes free early in the element-wise
+        // stage of item i), then dQ of item i (whose dS comes at the end of that stage).  The score
+        // MMAs of warp 1 run beside both, so two threads keep the tensor pipe fed.
         const int total_items = n_tiles * nitems;
         int tl = 0, k = 0;
         uint32_t kuse = 0;
         TileInfo t = tile_info(p, t_begin, t_begin);
         const uint32_t idesc_dq = make_idesc_bf16(kTileM, D, 1);
+        const uint64_t do_desc = make_smem_desc(sbase + p.off_do, 0, 1024);
         bool ok = true;
+        // cursor of the dP stream
+        int ptl = 0, pk = 0;
+        uint32_t vuse = 0;
+        TileInfo pt = t;
+        auto issue_dp = [&](int i) -> bool {
+            const int tl = ptl, k = pk;
+            const TileInfo &t = pt;
+            const bool prefix = k < p.nblk_p;
+            const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
+            const int slab = prefix ? n * 128 : sfx_slab;
+            const bool last_of_tile = k == nitems - 1;
+            const bool ring_v = prefix && !RV;
+            const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
+            const uint64_t slab16 = (uint64_t)(slab >> 4);
+            bool ok = true;
+                // ---- dP: its single slot is free once the element-wise warps have read item i-1
+                ok = mbar_wait_warp(bar(kBarDpFree), (i & 1) ^ 1, abort_flag, p.status, kErrMmaDq);
+                if (!ok) return false;
+                if (k == 0) ok = mbar_wait_warp(bar(kBarDoFull), tl & 1, abort_flag, p.status, kErrMmaDq);
+                if (!ok) return false;
+                uint32_t vaddr;
+                if (prefix) {
+                    if (RV) {
+                        if (t.first_of_g)
+                            ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaDq);
+                        vaddr = sbase + p.off_pv + k * C::kTileBytes;
+                    } else {
+                        const uint32_t vs = vuse % stages_v;
+                        ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / stages_v) & 1, abort_flag, p.status, kErrMmaDq);
+                        vaddr = sbase + p.off_pv + vs * C::kTileBytes;
+                    }
+                } else {
+                    ok = mbar_wait_warp(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMmaDq);
+                    vaddr = sbase + p.off_sv;
+                }
+                if (!ok) return false;
+                tc_fence_after();
+                {
+                    const uint64_t v_desc = make_smem_desc(vaddr, 0, 1024);
+                    if (elect_one_sync()) {
+#pragma unroll
+                        for (int ks16 = 0; ks16 < D / 16; ++ks16) {
+                            const uint64_t aoff = (uint64_t)(((ks16 >> 2) * C::kSlabBytes + (ks16 & 3) * 32) >> 4);
+                            const uint64_t voff = (uint64_t)(ks16 >> 2) * slab16 + (uint64_t)(((ks16 & 3) * 32) >> 4);
+                            mma_ss(tmem + kDpCol, do_desc + aoff, v_desc + voff, idesc, ks16 > 0 ? 1u : 0u);
+                        }
+                        tc_commit(bar(kBarDpFull));
+                        if (ring_v) tc_commit(bar(kBarVFree + (vuse % stages_v)));
+                        if (last_of_tile) tc_commit(bar(kBarDvFree));
+                    }
+                    __syncwarp();
+                }
+            if (!ok) return false;
+            if (ring_v) ++vuse;
+            if (++pk == nitems) {
+                pk = 0;
+                if (++ptl < n_tiles) pt = tile_info(p, t_begin + ptl, t_begin);
+            }
+            return true;
+        };
+        if (total_items > 0) ok = issue_dp(0);
 #pragma unroll 1
         for (int i = 0; i < total_items && ok; ++i) {
+            if (i + 1 < total_items) {
+                ok = issue_dp(i + 1);
+                if (!ok) break;
+            }
             const int slot = i % kSlots;
             const bool prefix = k < p.nblk_p;
             const int n = prefix ? prefix_block_rows(p, k) : t.n_sfx;
