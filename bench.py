@@ -359,7 +359,7 @@ def run_cuda(args):
     if world == 1 and not args.no_detail:
         line["detail"] = detail_runs(pskv, device, peaks)
     if world == 1 and not args.no_cpu:
-        line["cpu_baseline"] = cpu_baseline(w, args.ref_candidates)
+        line["cpu_baseline"] = cpu_baseline(w, args.cpu_candidates)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -396,9 +396,9 @@ def roofline(w, kernels, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (kernel, workload) -> bytes.
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("tc_fwd_kernel", "C2"): 473.4e6,        # profiles/tc_fwd_kernel_C2.md
-    ("tc_bwd_dq_kernel", "C2"): 694.7e6,     # profiles/tc_bwd_dq_kernel_C2.md
-    ("bwd_dkv_mma_kernel", "C2"): 592.7e6,   # profiles/bwd_dkv_mma_kernel_C2.md
+    ("tc_fwd_kernel", "C2"): 474.0e6,        # profiles/tc_fwd_kernel_C2.md
+    ("tc_bwd_dq_kernel", "C2"): 691.0e6,     # profiles/tc_bwd_dq_kernel_C2.md
+    ("tc_bwd_dkv_kernel", "C2"): 595.2e6,    # profiles/tc_bwd_dkv_kernel_C2.md
     ("simt_row_dot_kernel", "C2"): 408.8e6,  # profiles/simt_row_dot_kernel_C2.md
 }
 
@@ -465,7 +465,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-candidates", type=int, default=32,
-                    help="candidates per step of the CPU oracle sample")
+                    help="candidates per step of the CPU oracle sample (--impl reference)")
+    ap.add_argument("--cpu-candidates", type=int, default=256,
+                    help="candidates of the one-off CPU oracle sample reported as cpu_baseline")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     args = ap.parse_args()
