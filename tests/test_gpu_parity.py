@@ -72,6 +72,9 @@ EDGE = [
     (3, 2, 2, 72, 50, 128),   # rows per candidate (72) force 72-row tiles
     (40, 4, 4, 8, 16, 128),   # sixteen candidates share one tile
     (37, 2, 1, 40, 129, 128), # ragged last tile, prefix one key past a block
+    (2, 8, 2, 64, 64, 128),   # 256 rows per group: two full row tiles of the suffix-gradient kernel, 64 keys
+    (2, 8, 1, 40, 32, 128),   # 320 rows per group: two and a half row tiles, n_rep = 8
+    (300, 4, 4, 16, 48, 128), # more groups than SMs: every persistent CTA walks over several groups
 ]
 
 
@@ -90,7 +93,8 @@ def test_backward_edge_shapes(shape):
 
 
 def test_outlier_key_channels_and_large_scores():
-    """Large score spread (outlier channels x8 and a 4x scale) exercises the running-max rescale."""
+    """Large score spread (outlier channels x8 and a 4x scale): exponents far from zero without any
+    max subtraction in the tensor-core kernel."""
     w = wl("C2", B=3)
     t = make_inputs(w)
     out, lse, _ = parity.run_fwd_gpu(t, 4 * w.scale)
