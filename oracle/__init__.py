@@ -47,6 +47,12 @@ def _load():
         lib.pskv_oracle_attn_fwd.restype = ctypes.c_int
         lib.pskv_oracle_attn_bwd.argtypes = [dp] * 6 + [ctypes.c_double] + [dp] * 3 + ints
         lib.pskv_oracle_attn_bwd.restype = ctypes.c_int
+        ip = ctypes.POINTER(ctypes.c_int)
+        ints7 = [ctypes.c_int] * 7
+        lib.pskv_oracle_attn_fwd_multi.argtypes = [dp] * 3 + [ip] + [dp] * 2 + [ctypes.c_double] + [dp] * 2 + ints7
+        lib.pskv_oracle_attn_fwd_multi.restype = ctypes.c_int
+        lib.pskv_oracle_attn_bwd_multi.argtypes = [dp] * 4 + [ip] + [dp] * 2 + [ctypes.c_double] + [dp] * 3 + ints7
+        lib.pskv_oracle_attn_bwd_multi.restype = ctypes.c_int
         lib.pskv_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -109,4 +115,62 @@ def attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, scale):
                                       B, Hq, Hkv, S, P, d)
     if rc != 0:
         raise RuntimeError("pskv_oracle_attn_bwd failed with code %d" % rc)
+    return dq, dk, dv
+
+
+def _mask_i32(mask, Bp, Pmax):
+    m = np.ascontiguousarray(np.asarray(mask, dtype=np.int32))
+    if m.shape != (Bp, Pmax):
+        raise ValueError("expected mask shape %s, got %s" % ((Bp, Pmax), m.shape))
+    return m
+
+
+def left_padding_mask(prefix_len, Pmax):
+    """Prefix attention mask of left-padded prefixes: 1 on the last prefix_len[i] positions."""
+    lens = np.asarray(prefix_len, dtype=np.int64)
+    return (np.arange(Pmax)[None, :] >= (Pmax - lens)[:, None]).astype(np.int32)
+
+
+def attn_fwd_multi(q, prefix_k, prefix_v, mask, suffix_k, suffix_v, scale):
+    """Batched multi-instruction forward (Sec. 4.3): prefix_k / prefix_v [Bp,Hkv,Pmax,d], mask
+    [Bp,Pmax] (1 = real prefix token), candidate b uses instruction b // (B // Bp)."""
+    q = np.asarray(q)
+    B, Hq, S, d = q.shape
+    Bp, Hkv, Pmax = np.asarray(prefix_k).shape[:3]
+    q = _f64(q, (B, Hq, S, d))
+    pk = _f64(prefix_k, (Bp, Hkv, Pmax, d))
+    pv = _f64(prefix_v, (Bp, Hkv, Pmax, d))
+    sk = _f64(suffix_k, (B, Hkv, S, d))
+    sv = _f64(suffix_v, (B, Hkv, S, d))
+    m = _mask_i32(mask, Bp, Pmax)
+    out = np.empty((B, Hq, S, d), dtype=np.float64)
+    lse = np.empty((B, Hq, S), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_fwd_multi(_ptr(q), _ptr(pk), _ptr(pv), m.ctypes.data_as(ctypes.POINTER(ctypes.c_int)),
+                                            _ptr(sk), _ptr(sv), float(scale), _ptr(out), _ptr(lse),
+                                            B, Bp, Hq, Hkv, S, Pmax, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_fwd_multi failed with code %d" % rc)
+    return out, lse
+
+
+def attn_bwd_multi(dout, q, prefix_k, prefix_v, mask, suffix_k, suffix_v, scale):
+    """dq, dk_suffix, dv_suffix (fp64) of the multi-instruction forward; prefix caches frozen."""
+    q = np.asarray(q)
+    B, Hq, S, d = q.shape
+    Bp, Hkv, Pmax = np.asarray(prefix_k).shape[:3]
+    do = _f64(dout, (B, Hq, S, d))
+    q = _f64(q, (B, Hq, S, d))
+    pk = _f64(prefix_k, (Bp, Hkv, Pmax, d))
+    pv = _f64(prefix_v, (Bp, Hkv, Pmax, d))
+    sk = _f64(suffix_k, (B, Hkv, S, d))
+    sv = _f64(suffix_v, (B, Hkv, S, d))
+    m = _mask_i32(mask, Bp, Pmax)
+    dq = np.empty((B, Hq, S, d), dtype=np.float64)
+    dk = np.empty((B, Hkv, S, d), dtype=np.float64)
+    dv = np.empty((B, Hkv, S, d), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_bwd_multi(_ptr(do), _ptr(q), _ptr(pk), _ptr(pv),
+                                            m.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), _ptr(sk), _ptr(sv),
+                                            float(scale), _ptr(dq), _ptr(dk), _ptr(dv), B, Bp, Hq, Hkv, S, Pmax, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_bwd_multi failed with code %d" % rc)
     return dq, dk, dv

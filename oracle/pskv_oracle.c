@@ -198,3 +198,142 @@ int pskv_oracle_attn_bwd(const double *dout, const double *q,
     }
     return failed ? 2 : 0;
 }
+
+/*
+ * Batched multi-instruction variant (Sec. 4.3, suffix-centric alignment; appendix on
+ * position consistency under padding).  There are Bp prefix caches of padded
+ * length Pmax, prefix_k / prefix_v [Bp][Hkv][Pmax][d], and a prefix attention
+ * mask m[Bp][Pmax] (1 on real prefix tokens, 0 on padding: "padding tokens are
+ * excluded from attention").  Candidate b belongs to instruction b / (B / Bp):
+ * each cache is reused by its B / Bp candidates.  The keys a query row sees are
+ * the real prefix tokens of its instruction, in order, followed by the
+ * candidate's own suffix keys 0..i -- exactly the unpadded sequence.  Here that
+ * is written out literally: the masked rows are gathered into a per-candidate
+ * K/V copy and ordinary attention (Eq. 2) runs on it.  Any 0/1 mask is
+ * accepted, not only left padding.
+ */
+static int gather_prefix(const double *prefix, const int *mask, double *full, int inst, int g,
+                         int Hkv, int Pmax, int d)
+{
+    int n = 0;
+    for (int j = 0; j < Pmax; ++j) {
+        if (mask[(size_t)inst * Pmax + j]) {
+            memcpy(full + (size_t)n * d, prefix + (((size_t)inst * Hkv + g) * Pmax + j) * d, sizeof(double) * (size_t)d);
+            ++n;
+        }
+    }
+    return n;
+}
+
+int pskv_oracle_attn_fwd_multi(const double *q, const double *prefix_k, const double *prefix_v,
+                               const int *mask, const double *suffix_k, const double *suffix_v,
+                               double scale, double *out, double *lse,
+                               int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d)
+{
+    if (B < 1 || Bp < 1 || B % Bp != 0 || Hq < 1 || Hkv < 1 || S < 1 || Pmax < 0 || d < 1 || Hq % Hkv != 0) return 1;
+    const int n_rep = Hq / Hkv, Kq = B / Bp;
+    const int T = Pmax + S;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int inst = b / Kq;
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        if (!Kf || !Vf || !p) {
+            failed = 1;
+        } else {
+            for (int g = 0; g < Hkv; ++g) {
+                const int n = gather_prefix(prefix_k, mask, Kf, inst, g, Hkv, Pmax, d);
+                gather_prefix(prefix_v, mask, Vf, inst, g, Hkv, Pmax, d);
+                memcpy(Kf + (size_t)n * d, suffix_k + ((size_t)b * Hkv + g) * S * d, sizeof(double) * (size_t)S * d);
+                memcpy(Vf + (size_t)n * d, suffix_v + ((size_t)b * Hkv + g) * S * d, sizeof(double) * (size_t)S * d);
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < S; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * S + i;
+                        const int n_vis = n + i + 1;
+                        lse[row] = softmax_row(q + row * d, Kf, n_vis, d, scale, p);
+                        double *o = out + row * d;
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+    }
+    return failed ? 2 : 0;
+}
+
+/* Backward of the multi-instruction forward: the closed form of pskv_oracle_attn_bwd on the
+ * gathered keys; prefix caches are frozen, only dq, dk_suffix, dv_suffix are produced. */
+int pskv_oracle_attn_bwd_multi(const double *dout, const double *q, const double *prefix_k,
+                               const double *prefix_v, const int *mask, const double *suffix_k,
+                               const double *suffix_v, double scale, double *dq, double *dk_suffix,
+                               double *dv_suffix, int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d)
+{
+    if (B < 1 || Bp < 1 || B % Bp != 0 || Hq < 1 || Hkv < 1 || S < 1 || Pmax < 0 || d < 1 || Hq % Hkv != 0) return 1;
+    const int n_rep = Hq / Hkv, Kq = B / Bp;
+    const int T = Pmax + S;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int inst = b / Kq;
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        double *o = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!Kf || !Vf || !p || !o) {
+            failed = 1;
+        } else {
+            for (int g = 0; g < Hkv; ++g) {
+                const int n = gather_prefix(prefix_k, mask, Kf, inst, g, Hkv, Pmax, d);
+                gather_prefix(prefix_v, mask, Vf, inst, g, Hkv, Pmax, d);
+                memcpy(Kf + (size_t)n * d, suffix_k + ((size_t)b * Hkv + g) * S * d, sizeof(double) * (size_t)S * d);
+                memcpy(Vf + (size_t)n * d, suffix_v + ((size_t)b * Hkv + g) * S * d, sizeof(double) * (size_t)S * d);
+                double *dKs = dk_suffix + ((size_t)b * Hkv + g) * S * d;
+                double *dVs = dv_suffix + ((size_t)b * Hkv + g) * S * d;
+                for (size_t e = 0; e < (size_t)S * d; ++e) { dKs[e] = 0.0; dVs[e] = 0.0; }
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < S; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * S + i;
+                        const int n_vis = n + i + 1;
+                        const double *qr = q + row * d;
+                        const double *go = dout + row * d;
+                        softmax_row(qr, Kf, n_vis, d, scale, p);
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                        double D = 0.0;
+                        for (int c = 0; c < d; ++c) D += go[c] * o[c];
+                        double *dqr = dq + row * d;
+                        for (int c = 0; c < d; ++c) dqr[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j) {
+                            double dp = 0.0;
+                            for (int c = 0; c < d; ++c) dp += go[c] * Vf[(size_t)j * d + c];
+                            const double ds = p[j] * (dp - D);
+                            for (int c = 0; c < d; ++c) dqr[c] += scale * ds * Kf[(size_t)j * d + c];
+                            if (j >= n) {
+                                const int t = j - n;
+                                for (int c = 0; c < d; ++c) {
+                                    dKs[(size_t)t * d + c] += scale * ds * qr[c];
+                                    dVs[(size_t)t * d + c] += p[j] * go[c];
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+        free(o);
+    }
+    return failed ? 2 : 0;
+}
