@@ -14,6 +14,7 @@ rank runs the same step on its own B candidates against its own replica of the p
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -440,6 +441,41 @@ def detail_runs(pskv, device, peaks):
                                "candidates_per_s": w.B / ms * 1e3}
     del layers
     torch.cuda.empty_cache()
+    # Batched multi-instruction variant (Sec. 4.3) at the C2 shape: 8 instructions x 64 candidates, one
+    # left-padded prefix cache per instruction, true lengths 144..256
+    lens = [256, 240, 224, 208, 192, 176, 160, 144]
+    Bp, Pmax = len(lens), w.P
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(w.seed + 500)
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16).to(device)
+
+    q, sk, sv, do = draw(w.B, w.Hq, w.S, w.d), draw(w.B, w.Hkv, w.S, w.d), draw(w.B, w.Hkv, w.S, w.d), draw(w.B, w.Hq, w.S, w.d)
+    pk, pv = draw(Bp, w.Hkv, Pmax, w.d), draw(Bp, w.Hkv, Pmax, w.d)
+    out = torch.empty_like(q)
+    lse = torch.empty((w.B, w.Hq, w.S), dtype=torch.float32, device=device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(sk), torch.empty_like(sv)
+    mdims = (w.B, Bp, w.Hq, w.Hkv, w.S, Pmax, w.d)
+    ws_f = torch.empty(max(pskv.pskv_attn_fwd_multi_workspace_bytes(*mdims), 256), dtype=torch.uint8, device=device)
+    ws_b = torch.empty(max(pskv.pskv_attn_bwd_multi_workspace_bytes(*mdims), 256), dtype=torch.uint8, device=device)
+
+    def mfwd():
+        pskv.pskv_attn_fwd_multi(q, pk, pv, lens, sk, sv, w.scale, out=out, lse=lse, workspace=ws_f)
+
+    def mbwd():
+        pskv.pskv_attn_bwd_multi(do, q, pk, pv, lens, sk, sv, out, lse, w.scale, dq=dq, dk_suffix=dk, dv_suffix=dv,
+                                 workspace=ws_b)
+
+    mfwd()
+    kq = w.B // Bp
+    fl_f = sum(wl.fwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
+    fl_b = sum(wl.bwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
+    ms_f = time_calls(mfwd, 20, 3)
+    ms_b = time_calls(mbwd, 20, 3)
+    res["C2_multi_8x64"] = {"prefix_len": lens,
+                            "fwd": {"ms": ms_f, "tflops": fl_f / ms_f / 1e9, "candidates_per_s": w.B / ms_f * 1e3},
+                            "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
     return res
 
 

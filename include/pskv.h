@@ -115,6 +115,39 @@ pskv_status pskv_attn_bwd_static(const void *dout, const void *q, const void *pr
 long long pskv_attn_bwd_static_max_rows(void);
 
 /*
+ * Several instructions per call: the batched multi-instruction layout of Sec. 4.3 (suffix-centric
+ * alignment) with the position rules of the appendix on position consistency under padding.
+ * There are Bp prefix caches, one per instruction, stored left-padded to a common length Pmax:
+ *   prefix_k, prefix_v   bf16 [Bp,Hkv,Pmax,d]; the real tokens of instruction i are its LAST
+ *                        prefix_len[i] rows (0 <= prefix_len[i] <= Pmax); padding rows are never read
+ *   prefix_len           HOST array of Bp ints (read before the call returns)
+ * The B candidates are grouped by instruction: candidate b belongs to instruction b / (B / Bp), so B
+ * must be a multiple of Bp and each cache is reused by its B / Bp candidates.  Everything else (q,
+ * suffix_k, suffix_v, out, lse, dout, dq, dk_suffix, dv_suffix; scale; causal rule; error codes) is as
+ * in pskv_attn_fwd / pskv_attn_bwd, with P replaced per candidate by the true prefix length of its
+ * instruction.  The work is enqueued on `cuda_stream` as one pass per instruction.
+ */
+size_t pskv_attn_fwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d);
+pskv_status pskv_attn_fwd_multi(const void *q,        /* bf16 [B,Hq,S,d] */
+                                const void *prefix_k, /* bf16 [Bp,Hkv,Pmax,d] (may be NULL when Pmax == 0) */
+                                const void *prefix_v, /* bf16 [Bp,Hkv,Pmax,d] */
+                                const int *prefix_len, /* host, [Bp] */
+                                const void *suffix_k, /* bf16 [B,Hkv,S,d] */
+                                const void *suffix_v, /* bf16 [B,Hkv,S,d] */
+                                float scale,
+                                void *out,            /* bf16 [B,Hq,S,d] */
+                                float *lse,           /* fp32 [B,Hq,S] */
+                                int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+size_t pskv_attn_bwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d);
+pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
+                                const int *prefix_len, const void *suffix_k, const void *suffix_v,
+                                const void *out, const float *lse, float scale,
+                                void *dq, void *dk_suffix, void *dv_suffix,
+                                int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then reads and clears the device status word that
  * kernels set when one of their bounded waits gives up.  Returns PSKV_OK,
  * PSKV_ERR_DEVICE_TIMEOUT (results of the affected call are undefined) or

@@ -57,6 +57,15 @@ def lib() -> ctypes.CDLL:
         L.pskv_attn_fwd.restype = ci
         L.pskv_attn_bwd.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp, sz, vp]
         L.pskv_attn_bwd.restype = ci
+        seven = [ci] * 7
+        L.pskv_attn_fwd_multi_workspace_bytes.argtypes = seven
+        L.pskv_attn_fwd_multi_workspace_bytes.restype = sz
+        L.pskv_attn_bwd_multi_workspace_bytes.argtypes = seven
+        L.pskv_attn_bwd_multi_workspace_bytes.restype = sz
+        L.pskv_attn_fwd_multi.argtypes = [vp] * 6 + [cf] + [vp] * 2 + seven + [vp, sz, vp]
+        L.pskv_attn_fwd_multi.restype = ci
+        L.pskv_attn_bwd_multi.argtypes = [vp] * 9 + [cf] + [vp] * 3 + seven + [vp, sz, vp]
+        L.pskv_attn_bwd_multi.restype = ci
         L.pskv_attn_bwd_static.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp]
         L.pskv_attn_bwd_static.restype = ci
         L.pskv_attn_bwd_static_max_rows.argtypes = []
@@ -194,6 +203,68 @@ def pskv_attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, out, lse, sca
                              _ptr(ws), ws.numel() * ws.element_size(), _stream())
     if st != PSKV_OK:
         raise PskvError(st, "pskv_attn_bwd")
+    return dq, dk_suffix, dv_suffix
+
+
+def _multi_dims(q, prefix_k, suffix_k, prefix_len):
+    B, Hq, S, d = q.shape
+    Hkv = suffix_k.shape[1]
+    Bp = len(prefix_len)
+    Pmax = 0 if prefix_k is None else prefix_k.shape[2]
+    return [int(B), int(Bp), int(Hq), int(Hkv), int(S), int(Pmax), int(d)]
+
+
+def _host_lens(prefix_len):
+    arr = (ctypes.c_int * len(prefix_len))(*[int(x) for x in prefix_len])
+    return arr
+
+
+def pskv_attn_fwd_multi_workspace_bytes(B, Bp, Hq, Hkv, S, Pmax, d) -> int:
+    return int(lib().pskv_attn_fwd_multi_workspace_bytes(B, Bp, Hq, Hkv, S, Pmax, d))
+
+
+def pskv_attn_bwd_multi_workspace_bytes(B, Bp, Hq, Hkv, S, Pmax, d) -> int:
+    return int(lib().pskv_attn_bwd_multi_workspace_bytes(B, Bp, Hq, Hkv, S, Pmax, d))
+
+
+def pskv_attn_fwd_multi(q, prefix_k, prefix_v, prefix_len, suffix_k, suffix_v, scale, out=None, lse=None,
+                        workspace=None):
+    """Forward with one left-padded prefix cache per instruction: prefix_k / prefix_v are
+    [Bp, Hkv, Pmax, d], prefix_len (host ints) the true lengths, candidate b uses instruction
+    b // (B // Bp)."""
+    dims = _multi_dims(q, prefix_k, suffix_k, prefix_len)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    ws = _workspace(max(256, pskv_attn_fwd_multi_workspace_bytes(*dims)), q.device, workspace)
+    lens = _host_lens(prefix_len)
+    st = lib().pskv_attn_fwd_multi(_ptr(q), _ptr(prefix_k), _ptr(prefix_v), ctypes.cast(lens, ctypes.c_void_p),
+                                   _ptr(suffix_k), _ptr(suffix_v), float(scale), _ptr(out), _ptr(lse), *dims,
+                                   _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_fwd_multi")
+    return out, lse
+
+
+def pskv_attn_bwd_multi(dout, q, prefix_k, prefix_v, prefix_len, suffix_k, suffix_v, out, lse, scale,
+                        dq=None, dk_suffix=None, dv_suffix=None, workspace=None):
+    """Backward of pskv_attn_fwd_multi: dq, dk_suffix, dv_suffix; the prefix caches get no gradient."""
+    dims = _multi_dims(q, prefix_k, suffix_k, prefix_len)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk_suffix is None:
+        dk_suffix = torch.empty_like(suffix_k)
+    if dv_suffix is None:
+        dv_suffix = torch.empty_like(suffix_v)
+    ws = _workspace(pskv_attn_bwd_multi_workspace_bytes(*dims), q.device, workspace)
+    lens = _host_lens(prefix_len)
+    st = lib().pskv_attn_bwd_multi(_ptr(dout), _ptr(q), _ptr(prefix_k), _ptr(prefix_v),
+                                   ctypes.cast(lens, ctypes.c_void_p), _ptr(suffix_k), _ptr(suffix_v), _ptr(out),
+                                   _ptr(lse), float(scale), _ptr(dq), _ptr(dk_suffix), _ptr(dv_suffix), *dims,
+                                   _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_bwd_multi")
     return dq, dk_suffix, dv_suffix
 
 

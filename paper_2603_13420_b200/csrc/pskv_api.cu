@@ -40,6 +40,7 @@ pskv_status check_dims(int B, int Hq, int Hkv, int S, int P, int d, Dims *dm)
     const double rows = (double)B * Hq * S;
     if (rows * d > 1.0e12 || (double)Hkv * P * d > 1.0e12) return PSKV_ERR_UNSUPPORTED_SHAPE;
     dm->B = B; dm->Hq = Hq; dm->Hkv = Hkv; dm->S = S; dm->P = P; dm->d = d; dm->n_rep = Hq / Hkv;
+    dm->Pstride = P;
     return PSKV_OK;
 }
 
@@ -280,6 +281,140 @@ pskv_status pskv_attn_bwd(const void *dout, const void *q, const void *prefix_k,
     cudaError_t e = tc_bwd_supported(dm) ? launch_tc_bwd(a, workspace, status_word, stream)
                                          : launch_simt_bwd(a, stream);
     return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
+}
+
+// ---- several instructions per call (suffix-centric alignment, Sec. 4.3) --------------------------
+
+size_t pskv_attn_fwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d)
+{
+    Dims dm;
+    if (Bp < 1 || B < Bp || B % Bp != 0 || check_dims(B / Bp, Hq, Hkv, S, Pmax, d, &dm) != PSKV_OK) return 0;
+    return 256;  // the per-call scratch of the single-prefix forward, reused by every instruction's part
+}
+
+size_t pskv_attn_bwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d)
+{
+    Dims dm;
+    if (Bp < 1 || B < Bp || B % Bp != 0 || check_dims(B / Bp, Hq, Hkv, S, Pmax, d, &dm) != PSKV_OK) return 0;
+    // one fp32 per query row; each instruction's part gets its own 256-byte aligned slice
+    const size_t part = round256((size_t)(B / Bp) * Hq * S * sizeof(float));
+    return part * (size_t)Bp;
+}
+
+namespace {
+// checks shared by the two multi-instruction calls; fills the per-instruction geometry
+pskv_status check_multi(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d, const int *prefix_len)
+{
+    if (Bp < 1 || B < Bp || B % Bp != 0 || !prefix_len) return PSKV_ERR_INVALID_ARG;
+    Dims dm;
+    pskv_status st = check_dims(B / Bp, Hq, Hkv, S, Pmax, d, &dm);
+    if (st != PSKV_OK) return st;
+    for (int i = 0; i < Bp; ++i)
+        if (prefix_len[i] < 0 || prefix_len[i] > Pmax) return PSKV_ERR_INVALID_ARG;
+    return PSKV_OK;
+}
+}  // namespace
+
+pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void *prefix_v, const int *prefix_len,
+                                const void *suffix_k, const void *suffix_v, float scale, void *out, float *lse,
+                                int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream)
+{
+    pskv_status st = check_multi(B, Bp, Hq, Hkv, S, Pmax, d, prefix_len);
+    if (st != PSKV_OK) return st;
+    if (!q || !suffix_k || !suffix_v || !out || !lse) return PSKV_ERR_INVALID_ARG;
+    if (Pmax > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) || !aligned16(suffix_k) ||
+        !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse))
+        return PSKV_ERR_INVALID_ARG;
+    if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < 256 || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
+
+    unsigned int *status_word = nullptr;
+    st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+
+    const int Kq = B / Bp;  // candidates per instruction, contiguous in the candidate dimension
+    const size_t q_part = (size_t)Kq * Hq * S * d, s_part = (size_t)Kq * Hkv * S * d, l_part = (size_t)Kq * Hq * S;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (int i = 0; i < Bp; ++i) {
+        Dims dm;
+        st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
+        if (st != PSKV_OK) return st;
+        dm.Pstride = Pmax;
+        // the real tokens of a left-padded prefix are its last prefix_len[i] rows
+        const size_t p_off = ((size_t)i * Hkv * Pmax + (size_t)(Pmax - prefix_len[i])) * d;
+        FwdArgs a;
+        a.q = static_cast<const __nv_bfloat16 *>(q) + i * q_part;
+        a.prefix_k = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_k) + p_off : nullptr;
+        a.prefix_v = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_v) + p_off : nullptr;
+        a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k) + i * s_part;
+        a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v) + i * s_part;
+        a.out = static_cast<__nv_bfloat16 *>(out) + i * q_part;
+        a.lse = lse + i * l_part;
+        a.scale = scale;
+        a.dims = dm;
+        cudaError_t e = tc_fwd_supported(dm) ? launch_tc_fwd(a, workspace, status_word, stream)
+                                             : launch_simt_fwd(a, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return PSKV_OK;
+}
+
+pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
+                                const int *prefix_len, const void *suffix_k, const void *suffix_v, const void *out,
+                                const float *lse, float scale, void *dq, void *dk_suffix, void *dv_suffix, int B,
+                                int Bp, int Hq, int Hkv, int S, int Pmax, int d, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream)
+{
+    pskv_status st = check_multi(B, Bp, Hq, Hkv, S, Pmax, d, prefix_len);
+    if (st != PSKV_OK) return st;
+    if (!dout || !q || !suffix_k || !suffix_v || !out || !lse || !dq || !dk_suffix || !dv_suffix)
+        return PSKV_ERR_INVALID_ARG;
+    if (Pmax > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
+    if (!aligned16(dout) || !aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) ||
+        !aligned16(suffix_k) || !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse) ||
+        !aligned16(dq) || !aligned16(dk_suffix) || !aligned16(dv_suffix))
+        return PSKV_ERR_INVALID_ARG;
+    if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
+    const size_t need = pskv_attn_bwd_multi_workspace_bytes(B, Bp, Hq, Hkv, S, Pmax, d);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
+
+    unsigned int *status_word = nullptr;
+    st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+
+    const int Kq = B / Bp;
+    const size_t q_part = (size_t)Kq * Hq * S * d, s_part = (size_t)Kq * Hkv * S * d, l_part = (size_t)Kq * Hq * S;
+    const size_t ws_part = need / (size_t)Bp;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (int i = 0; i < Bp; ++i) {
+        Dims dm;
+        st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
+        if (st != PSKV_OK) return st;
+        dm.Pstride = Pmax;
+        const size_t p_off = ((size_t)i * Hkv * Pmax + (size_t)(Pmax - prefix_len[i])) * d;
+        void *ws = static_cast<char *>(workspace) + i * ws_part;
+        BwdArgs a;
+        a.dout = static_cast<const __nv_bfloat16 *>(dout) + i * q_part;
+        a.q = static_cast<const __nv_bfloat16 *>(q) + i * q_part;
+        a.prefix_k = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_k) + p_off : nullptr;
+        a.prefix_v = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_v) + p_off : nullptr;
+        a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k) + i * s_part;
+        a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v) + i * s_part;
+        a.out = static_cast<const __nv_bfloat16 *>(out) + i * q_part;
+        a.lse = lse + i * l_part;
+        a.dq = static_cast<__nv_bfloat16 *>(dq) + i * q_part;
+        a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix) + i * s_part;
+        a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix) + i * s_part;
+        a.row_dot = static_cast<float *>(ws);
+        a.scale = scale;
+        a.dims = dm;
+        cudaError_t e = tc_bwd_supported(dm) ? launch_tc_bwd(a, ws, status_word, stream)
+                                             : launch_simt_bwd(a, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return PSKV_OK;
 }
 
 pskv_status pskv_poll_device_status(void *cuda_stream)

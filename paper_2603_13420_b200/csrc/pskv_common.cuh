@@ -8,9 +8,11 @@
 
 namespace pskv {
 
-// Dimensions of one call; `n_rep` = Hq / Hkv query heads per KV head.
+// Dimensions of one call; `n_rep` = Hq / Hkv query heads per KV head.  `Pstride` is the distance, in
+// rows, between the prefix blocks of consecutive KV heads (P for a dense prefix cache; the padded
+// length when the call works on the real tokens of a left-padded cache).
 struct Dims {
-    int B, Hq, Hkv, S, P, d, n_rep;
+    int B, Hq, Hkv, S, P, d, n_rep, Pstride;
 };
 
 struct FwdArgs {

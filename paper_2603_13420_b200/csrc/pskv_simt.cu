@@ -94,8 +94,8 @@ __device__ __forceinline__ void fwd_row(const FwdArgs &a, long long row, float *
     const int h = (int)((row / dm.S) % dm.Hq);
     const int b = (int)(row / ((long long)dm.S * dm.Hq));
     const int g = h / dm.n_rep;
-    const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.P * D;
-    const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.P * D;
+    const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.Pstride * D;
+    const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.Pstride * D;
     const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
     const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
 
@@ -186,8 +186,8 @@ simt_bwd_dq_kernel(BwdArgs a)
     const int h = (int)((row / dm.S) % dm.Hq);
     const int b = (int)(row / ((long long)dm.S * dm.Hq));
     const int g = h / dm.n_rep;
-    const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.P * D;
-    const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.P * D;
+    const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.Pstride * D;
+    const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.Pstride * D;
     const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
     const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
 

@@ -372,6 +372,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 kaddr = sbase + p.off_sk;
             }
             if (!ok) break;
+            PSKV_TRACE_EVENT(10, i);
             tc_fence_after();
             {
                 const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
@@ -442,6 +443,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     vaddr = sbase + p.off_sv;
                 }
                 if (!ok) return false;
+                PSKV_TRACE_EVENT(12, i);
                 tc_fence_after();
                 {
                     const uint64_t v_desc = make_smem_desc(vaddr, 0, 1024);
@@ -488,6 +490,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             uint32_t kaddr;
             if (prefix) kaddr = sbase + p.off_pk + (RK ? (uint32_t)k : kuse % stages_k) * C::kTileBytes;
             else kaddr = sbase + p.off_sk;
+            PSKV_TRACE_EVENT(11, i);
             tc_fence_after();
             const uint32_t ds_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
             const uint64_t k_desc = make_smem_desc(kaddr, (uint32_t)slab, 1024);  // K as [keys][d]: d contiguous
@@ -564,6 +567,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (!ok) break;
                 ok = mbar_wait_warp(bar(kBarDpFull), item & 1, abort_flag, p.status, kErrElem);
                 if (!ok) break;
+                PSKV_TRACE_EVENT(20, item);
                 tc_fence_after();
                 // two halves of 16 columns; dP goes back as soon as the second half is in registers
 #pragma unroll
@@ -613,6 +617,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarDsReady + slot));
+                PSKV_TRACE_EVENT(24, item);
             }
         }
     } else {
@@ -784,7 +789,7 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     }
     if (dm.P > 0) {
         cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
-        cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.P * D * 2};
+        cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.Pstride * D * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
         cuuint32_t box_tail[3] = {64, (cuuint32_t)plan.tail_rows, 1};
         if (!encode_map(&tm_pk, a.prefix_k, 3, dims, str, box)) return cudaErrorInvalidValue;
@@ -841,6 +846,25 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
 }
 
 }  // namespace
+
+#ifdef PSKV_TRACE
+// Debug builds only: copies this kernel's event trace of CTA 0 to the host.
+extern "C" int pskv_debug_read_trace_dq(long long *host, int max_events)
+{
+    static long long buf[kTraceWarps * kTraceCap * 2];
+    unsigned int cnt[kTraceWarps];
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(cnt, g_trace_n, sizeof(cnt));
+    cudaMemcpyFromSymbol(buf, g_trace, sizeof(buf));
+    int n = 0;
+    for (int w = 0; w < kTraceWarps; ++w)
+        for (unsigned int i = 0; i < cnt[w] && i < (unsigned int)kTraceCap && n < max_events; ++i, ++n) {
+            host[2 * n] = buf[((size_t)w * kTraceCap + i) * 2];
+            host[2 * n + 1] = buf[((size_t)w * kTraceCap + i) * 2 + 1] | ((long long)w << 24);
+        }
+    return n;
+}
+#endif
 
 bool tc_bwd_supported(const Dims &dm)
 {

@@ -861,7 +861,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     }
     if (dm.P > 0) {
         cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
-        cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.P * D * 2};
+        cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.Pstride * D * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
         cuuint32_t box_tail[3] = {64, (cuuint32_t)plan.tail_rows, 1};
         if (!encode_map(&tm_pk, a.prefix_k, 3, dims, str, box)) return cudaErrorInvalidValue;

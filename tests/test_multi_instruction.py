@@ -1,0 +1,99 @@
+"""Batched multi-instruction variant (Sec. 4.3): one left-padded prefix cache per instruction, reused
+by that instruction's candidates.  GPU parity against the fp64 oracle (which gathers the unmasked
+prefix rows per candidate and runs plain attention), plus host-side argument checks."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_13420_b200 as pskv
+import parity
+
+SEED = 260313420 + 77
+
+
+def make(B, Bp, Hq, Hkv, S, Pmax, d, lens, seed=SEED):
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed + B + 7 * Bp + 13 * S + Pmax)
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+
+    t = dict(q=draw(B, Hq, S, d), prefix_k=draw(Bp, Hkv, Pmax, d), prefix_v=draw(Bp, Hkv, Pmax, d),
+             suffix_k=draw(B, Hkv, S, d), suffix_v=draw(B, Hkv, S, d), dout=draw(B, Hq, S, d))
+    # padding rows hold large garbage: they must never be read
+    for i, n in enumerate(lens):
+        t["prefix_k"][i, :, : Pmax - n] = 3.0e4
+        t["prefix_v"][i, :, : Pmax - n] = -3.0e4
+    return t
+
+
+CASES = [
+    # B, Bp, Hq, Hkv, S, Pmax, d, lens
+    (12, 3, 8, 2, 16, 300, 128, (300, 129, 40)),   # tensor-core path, ragged prefixes, GQA
+    (8, 2, 4, 4, 40, 160, 128, (160, 96)),         # MHA, 40-token suffix
+    (6, 3, 4, 2, 8, 64, 64, (0, 64, 17)),          # head dim 64, an empty prefix, odd length
+    (4, 4, 2, 1, 5, 33, 128, (33, 1, 20, 7)),      # general kernels (S not a multiple of 8)
+    (64, 2, 32, 8, 48, 256, 128, (256, 200)),      # the GQA layer shape, two instructions
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", CASES)
+def test_forward_and_backward_match_the_oracle(case):
+    B, Bp, Hq, Hkv, S, Pmax, d, lens = case
+    t = make(*case)
+    scale = 1.0 / np.sqrt(d)
+    dev = {k: v.cuda() for k, v in t.items()}
+    out = parity.Guarded((B, Hq, S, d), torch.bfloat16, "cuda")
+    lse = parity.Guarded((B, Hq, S), torch.float32, "cuda")
+    pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"], dev["suffix_v"],
+                             scale, out=out.view, lse=lse.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    out.check("out"); lse.check("lse")
+    f = {k: parity.to_f64(v) for k, v in t.items()}
+    mask = oracle.left_padding_mask(lens, Pmax)
+    ref_out, ref_lse = oracle.attn_fwd_multi(f["q"], f["prefix_k"], f["prefix_v"], mask, f["suffix_k"], f["suffix_v"], scale)
+    parity.check_tensor("out", parity.to_f64(out.view), ref_out, strict_abs=(min(lens) + S >= 128))
+    parity.check_lse(parity.to_f64(lse.view), ref_lse)
+
+    dq = parity.Guarded((B, Hq, S, d), torch.bfloat16, "cuda")
+    dk = parity.Guarded((B, Hkv, S, d), torch.bfloat16, "cuda")
+    dv = parity.Guarded((B, Hkv, S, d), torch.bfloat16, "cuda")
+    pskv.pskv_attn_bwd_multi(dev["dout"], dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
+                             dev["suffix_v"], out.view, lse.view, scale, dq=dq.view, dk_suffix=dk.view,
+                             dv_suffix=dv.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    dq.check("dq"); dk.check("dk_suffix"); dv.check("dv_suffix")
+    rq, rk, rv = oracle.attn_bwd_multi(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], mask, f["suffix_k"],
+                                       f["suffix_v"], scale)
+    parity.check_tensor("dq", parity.to_f64(dq.view), rq)
+    parity.check_tensor("dk_suffix", parity.to_f64(dk.view), rk)
+    parity.check_tensor("dv_suffix", parity.to_f64(dv.view), rv)
+
+
+@pytest.mark.gpu
+def test_one_unpadded_instruction_equals_the_single_prefix_call_bit_for_bit():
+    B, Hq, Hkv, S, P, d = 16, 8, 2, 16, 200, 128
+    t = make(B, 1, Hq, Hkv, S, P, d, (P,))
+    dev = {k: v.cuda() for k, v in t.items()}
+    scale = 1.0 / np.sqrt(d)
+    o1, l1 = pskv.pskv_attn_fwd(dev["q"], dev["prefix_k"][0], dev["prefix_v"][0], dev["suffix_k"], dev["suffix_v"], scale)
+    o2, l2 = pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], (P,), dev["suffix_k"],
+                                      dev["suffix_v"], scale)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+
+
+def test_multi_arguments_are_checked_on_the_host():
+    L = pskv.binding.lib()
+    lens = (ctypes.c_int * 2)(4, 9)
+    fake = ctypes.c_void_p(4096)
+    args = lambda B, Bp, Pmax, ln: L.pskv_attn_fwd_multi(fake, fake, fake, ctypes.cast(ln, ctypes.c_void_p), fake, fake,
+                                                          ctypes.c_float(0.1), fake, fake, B, Bp, 4, 4, 8, Pmax, 128, fake, 256, None)
+    assert args(7, 2, 16, lens) == pskv.PSKV_ERR_INVALID_ARG          # B not a multiple of Bp
+    assert args(8, 2, 8, lens) == pskv.PSKV_ERR_INVALID_ARG           # a length beyond Pmax
+    assert args(8, 2, 16, None) == pskv.PSKV_ERR_INVALID_ARG          # no length array
+    assert pskv.pskv_attn_bwd_multi_workspace_bytes(8, 2, 4, 4, 8, 16, 128) >= 8 * 4 * 8 * 4
+    assert pskv.pskv_attn_fwd_multi_workspace_bytes(7, 2, 4, 4, 8, 16, 128) == 0
