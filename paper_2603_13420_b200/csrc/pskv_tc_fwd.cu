@@ -120,14 +120,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31;
-    const int phys_warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
-#ifdef PSKV_SERVICE_HIGH
-    // role index: physical warps 0-15 are the softmax warps (roles 4-19), 16-19 the producers and MMA
-    // issuers (roles 0-3), 20-23 the epilogue; the quadrant (index mod 4) is the same either way
-    const int warp = phys_warp < 16 ? phys_warp + 4 : phys_warp < 20 ? phys_warp - 16 : phys_warp;
-#else
-    const int warp = phys_warp;
-#endif
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
     PSKV_TRACE_DECL;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + p.off_bar;
@@ -176,11 +169,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     // The producer and MMA warps run their loops with all 32 lanes (warp-uniform control flow and
     // addresses, so descriptors can live in uniform registers); one elected lane issues the
     // asynchronous instructions.
-#ifdef PSKV_SWAP23
-    const int role = warp == 2 ? 3 : warp == 3 ? 2 : warp;
-#else
     const int role = warp;
-#endif
     if (role == 0) {
         // ------------------------------------------------------------------ producer, score side
         if (lane == 0) {
@@ -201,7 +190,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint32_t q_bytes = (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128);
             const uint32_t seg_bytes = (uint32_t)(p.seg_rows * 128);
             uint32_t q_dst = sbase + p.off_q;
-#ifndef PSKV_NO_PREFETCH_Q
             // While there is nothing else to do, ask for the NEXT tile's Q in L2: its load can only
             // be issued a tile from now, right when it is needed, and then finds the data close by.
             if (tl + 1 < n_tiles) {
@@ -222,7 +210,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
                 __syncwarp();
             }
-#endif
             // Q, suffix K and (resident mode) the prefix K blocks are free once every score MMA of
             // the previous tile has completed
             ok = mbar_wait_warp(bar(kBarQkFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerK);
@@ -244,11 +231,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
             }
             __syncwarp();
-#ifdef PSKV_TRACE_QLAND
-            PSKV_TRACE_EVENT(2, tl);
-            mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrProducerK);
-            PSKV_TRACE_EVENT(3, tl);
-#endif
             if (RES) {
                 if (t.first_of_g && elect_one_sync()) {
 #pragma unroll 1
@@ -620,12 +602,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     PSKV_TRACE_EVENT(25, item);
                     ok = mbar_wait_warp(bar(kBarSFull + slot), (item / kSlots) & 1, abort_flag, p.status, kErrSoftmax);
                     if (!ok) break;
-#ifdef PSKV_STAGGER
-                    if (item == 0) {
-                        const long long t0 = clock64();
-                        while (clock64() - t0 < (long long)(wg * PSKV_STAGGER)) { }
-                    }
-#endif
                     tc_fence_after();
                     PSKV_TRACE_EVENT(20, item);
                     if (kind != 0) {
