@@ -53,6 +53,10 @@ def _load():
         lib.pskv_oracle_attn_fwd_multi.restype = ctypes.c_int
         lib.pskv_oracle_attn_bwd_multi.argtypes = [dp] * 4 + [ip] + [dp] * 2 + [ctypes.c_double] + [dp] * 3 + ints7
         lib.pskv_oracle_attn_bwd_multi.restype = ctypes.c_int
+        lib.pskv_oracle_attn_fwd_decode.argtypes = [dp] * 5 + [ip] + [ctypes.c_double] + [dp] * 2 + ints7
+        lib.pskv_oracle_attn_fwd_decode.restype = ctypes.c_int
+        lib.pskv_oracle_attn_bwd_decode.argtypes = [dp] * 6 + [ip] + [ctypes.c_double] + [dp] * 3 + ints7
+        lib.pskv_oracle_attn_bwd_decode.restype = ctypes.c_int
         lib.pskv_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -173,4 +177,60 @@ def attn_bwd_multi(dout, q, prefix_k, prefix_v, mask, suffix_k, suffix_v, scale)
                                             float(scale), _ptr(dq), _ptr(dk), _ptr(dv), B, Bp, Hq, Hkv, S, Pmax, d)
     if rc != 0:
         raise RuntimeError("pskv_oracle_attn_bwd_multi failed with code %d" % rc)
+    return dq, dk, dv
+
+
+def _len_i32(suffix_len, B):
+    if suffix_len is None:
+        return None, None
+    a = np.ascontiguousarray(np.asarray(suffix_len, dtype=np.int32))
+    if a.shape != (B,):
+        raise ValueError("expected suffix_len shape %s, got %s" % ((B,), a.shape))
+    return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_int))
+
+
+def attn_fwd_decode(q, prefix_k, prefix_v, suffix_k, suffix_v, scale, suffix_len=None):
+    """Decode-shaped forward: q [B,Hq,Sq,d] are the LAST Sq of each candidate's suffix_len[b]
+    cached suffix tokens (suffix_k / suffix_v [B,Hkv,Skv,d], rows past suffix_len[b] ignored;
+    None = all Skv rows real).  Returns out [B,Hq,Sq,d], lse [B,Hq,Sq]."""
+    q = np.asarray(q)
+    B, Hq, Sq, d = q.shape
+    Hkv, P = np.asarray(prefix_k).shape[:2]
+    Skv = np.asarray(suffix_k).shape[2]
+    q = _f64(q, (B, Hq, Sq, d))
+    pk = _f64(prefix_k, (Hkv, P, d))
+    pv = _f64(prefix_v, (Hkv, P, d))
+    sk = _f64(suffix_k, (B, Hkv, Skv, d))
+    sv = _f64(suffix_v, (B, Hkv, Skv, d))
+    keep, lp = _len_i32(suffix_len, B)
+    out = np.empty((B, Hq, Sq, d), dtype=np.float64)
+    lse = np.empty((B, Hq, Sq), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_fwd_decode(_ptr(q), _ptr(pk), _ptr(pv), _ptr(sk), _ptr(sv), lp, float(scale),
+                                             _ptr(out), _ptr(lse), B, Hq, Hkv, Sq, Skv, P, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_fwd_decode failed with code %d" % rc)
+    return out, lse
+
+
+def attn_bwd_decode(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, scale, suffix_len=None):
+    """dq [B,Hq,Sq,d], dk_suffix, dv_suffix [B,Hkv,Skv,d] (fp64) of the decode-shaped forward;
+    rows past suffix_len[b] of the key-side gradients are zero; prefix K/V frozen."""
+    q = np.asarray(q)
+    B, Hq, Sq, d = q.shape
+    Hkv, P = np.asarray(prefix_k).shape[:2]
+    Skv = np.asarray(suffix_k).shape[2]
+    do = _f64(dout, (B, Hq, Sq, d))
+    q = _f64(q, (B, Hq, Sq, d))
+    pk = _f64(prefix_k, (Hkv, P, d))
+    pv = _f64(prefix_v, (Hkv, P, d))
+    sk = _f64(suffix_k, (B, Hkv, Skv, d))
+    sv = _f64(suffix_v, (B, Hkv, Skv, d))
+    keep, lp = _len_i32(suffix_len, B)
+    dq = np.empty((B, Hq, Sq, d), dtype=np.float64)
+    dk = np.empty((B, Hkv, Skv, d), dtype=np.float64)
+    dv = np.empty((B, Hkv, Skv, d), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_bwd_decode(_ptr(do), _ptr(q), _ptr(pk), _ptr(pv), _ptr(sk), _ptr(sv), lp,
+                                             float(scale), _ptr(dq), _ptr(dk), _ptr(dv), B, Hq, Hkv, Sq, Skv, P, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_bwd_decode failed with code %d" % rc)
     return dq, dk, dv

@@ -337,3 +337,141 @@ int pskv_oracle_attn_bwd_multi(const double *dout, const double *q, const double
     }
     return failed ? 2 : 0;
 }
+
+/*
+ * Decode-shaped variant: token-by-token growth of the suffix (the beam-search and
+ * sampling-based attacks of the related-work discussion extend every candidate by a few
+ * tokens per step on top of what is already cached).  Each candidate b has a suffix cache
+ * buffer of Skv rows of which the first len[b] are real (Sq <= len[b] <= Skv; rows past
+ * len[b] are ignored whatever they hold), and only the LAST Sq of those len[b] suffix
+ * tokens are queries: query i is suffix token len[b] - Sq + i, so by Eq. 2's causal mask
+ * it sees the P prefix keys and suffix keys 0 .. len[b] - Sq + i.  With Sq == Skv == len[b]
+ * this is pskv_oracle_attn_fwd.  Written out literally: the candidate's real keys are
+ * copied behind its own copy of the prefix and each query row runs Eq. 2 on what it sees.
+ *
+ * Layouts: q, out, dout, dq [B][Hq][Sq][d]; suffix_k, suffix_v, dk_suffix, dv_suffix
+ * [B][Hkv][Skv][d]; lse [B][Hq][Sq]; len [B] (NULL = every candidate uses all Skv rows).
+ */
+static int decode_args_ok(const int *len, int B, int Hq, int Hkv, int Sq, int Skv, int P, int d)
+{
+    if (B < 1 || Hq < 1 || Hkv < 1 || Sq < 1 || Skv < Sq || P < 0 || d < 1 || Hq % Hkv != 0) return 0;
+    if (len)
+        for (int b = 0; b < B; ++b)
+            if (len[b] < Sq || len[b] > Skv) return 0;
+    return 1;
+}
+
+int pskv_oracle_attn_fwd_decode(const double *q, const double *prefix_k, const double *prefix_v,
+                                const double *suffix_k, const double *suffix_v, const int *len,
+                                double scale, double *out, double *lse,
+                                int B, int Hq, int Hkv, int Sq, int Skv, int P, int d)
+{
+    if (!decode_args_ok(len, B, Hq, Hkv, Sq, Skv, P, d)) return 1;
+    const int n_rep = Hq / Hkv;
+    const int T = P + Skv;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int L = len ? len[b] : Skv;
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        if (!Kf || !Vf || !p) {
+            failed = 1;
+        } else {
+            for (int g = 0; g < Hkv; ++g) {
+                memcpy(Kf, prefix_k + (size_t)g * P * d, sizeof(double) * (size_t)P * d);
+                memcpy(Vf, prefix_v + (size_t)g * P * d, sizeof(double) * (size_t)P * d);
+                memcpy(Kf + (size_t)P * d, suffix_k + ((size_t)b * Hkv + g) * Skv * d, sizeof(double) * (size_t)L * d);
+                memcpy(Vf + (size_t)P * d, suffix_v + ((size_t)b * Hkv + g) * Skv * d, sizeof(double) * (size_t)L * d);
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < Sq; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * Sq + i;
+                        const int pos = L - Sq + i;          /* suffix position of this query */
+                        const int n_vis = P + pos + 1;
+                        lse[row] = softmax_row(q + row * d, Kf, n_vis, d, scale, p);
+                        double *o = out + row * d;
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+    }
+    return failed ? 2 : 0;
+}
+
+/* Backward of the decode-shaped forward: the closed form of pskv_oracle_attn_bwd with the
+ * shifted causal mask.  Every real suffix key (also those older than the queries) receives a
+ * gradient; rows past len[b] of dk_suffix / dv_suffix are zero.  The prefix stays frozen. */
+int pskv_oracle_attn_bwd_decode(const double *dout, const double *q, const double *prefix_k,
+                                const double *prefix_v, const double *suffix_k, const double *suffix_v,
+                                const int *len, double scale, double *dq, double *dk_suffix,
+                                double *dv_suffix, int B, int Hq, int Hkv, int Sq, int Skv, int P, int d)
+{
+    if (!decode_args_ok(len, B, Hq, Hkv, Sq, Skv, P, d)) return 1;
+    const int n_rep = Hq / Hkv;
+    const int T = P + Skv;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int L = len ? len[b] : Skv;
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        double *o = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!Kf || !Vf || !p || !o) {
+            failed = 1;
+        } else {
+            for (int g = 0; g < Hkv; ++g) {
+                memcpy(Kf, prefix_k + (size_t)g * P * d, sizeof(double) * (size_t)P * d);
+                memcpy(Vf, prefix_v + (size_t)g * P * d, sizeof(double) * (size_t)P * d);
+                memcpy(Kf + (size_t)P * d, suffix_k + ((size_t)b * Hkv + g) * Skv * d, sizeof(double) * (size_t)L * d);
+                memcpy(Vf + (size_t)P * d, suffix_v + ((size_t)b * Hkv + g) * Skv * d, sizeof(double) * (size_t)L * d);
+                double *dKs = dk_suffix + ((size_t)b * Hkv + g) * Skv * d;
+                double *dVs = dv_suffix + ((size_t)b * Hkv + g) * Skv * d;
+                for (size_t e = 0; e < (size_t)Skv * d; ++e) { dKs[e] = 0.0; dVs[e] = 0.0; }
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < Sq; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * Sq + i;
+                        const int n_vis = P + (L - Sq + i) + 1;
+                        const double *qr = q + row * d;
+                        const double *go = dout + row * d;
+                        softmax_row(qr, Kf, n_vis, d, scale, p);
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                        double D = 0.0;
+                        for (int c = 0; c < d; ++c) D += go[c] * o[c];
+                        double *dqr = dq + row * d;
+                        for (int c = 0; c < d; ++c) dqr[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j) {
+                            double dp = 0.0;
+                            for (int c = 0; c < d; ++c) dp += go[c] * Vf[(size_t)j * d + c];
+                            const double ds = p[j] * (dp - D);
+                            for (int c = 0; c < d; ++c) dqr[c] += scale * ds * Kf[(size_t)j * d + c];
+                            if (j >= P) {
+                                const int t = j - P;
+                                for (int c = 0; c < d; ++c) {
+                                    dKs[(size_t)t * d + c] += scale * ds * qr[c];
+                                    dVs[(size_t)t * d + c] += p[j] * go[c];
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+        free(o);
+    }
+    return failed ? 2 : 0;
+}
