@@ -148,6 +148,45 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Decode-shaped variant: the suffix grows token by token (beam-search and sampling-based attacks
+ * extend every candidate by a few tokens per step on top of what is already cached), so only the
+ * newest tokens of each candidate are queries.  Each candidate b owns a suffix cache buffer of Skv
+ * rows, suffix_k / suffix_v [B,Hkv,Skv,d], whose first suffix_len[b] rows are cached suffix tokens
+ * (the K/V of the new tokens already appended); the Sq query rows q[b,:,i,:] are the LAST Sq of
+ * them: query i is suffix token suffix_len[b] - Sq + i and, by the causal rule of Eq. 2, sees all P
+ * prefix keys and suffix keys 0 .. suffix_len[b] - Sq + i.  With Sq == Skv and no suffix_len this is
+ * pskv_attn_fwd / pskv_attn_bwd.
+ *   suffix_len   DEVICE array of B ints, 4-byte aligned, or NULL (= every candidate has Skv tokens).
+ *                Values must lie in [Sq, Skv]; the kernels force them into that range, so a bad
+ *                value gives wrong numbers for that candidate but never an out-of-range access.
+ *   Rows of suffix_k / suffix_v at or past suffix_len[b] take no part in the result, but they are
+ *   loaded and multiplied by a zero probability, so they must hold finite numbers (clear the
+ *   buffer once when it is allocated).
+ *   Backward: dq [B,Hq,Sq,d]; dk_suffix, dv_suffix [B,Hkv,Skv,d] cover every cached token (also
+ *   those older than the queries); rows at or past suffix_len[b] are written as zeros.
+ * Everything else (layouts, scale, lse, error codes, stream semantics) is as in the calls above.
+ */
+size_t pskv_attn_fwd_decode_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int P, int d);
+pskv_status pskv_attn_fwd_decode(const void *q,        /* bf16 [B,Hq,Sq,d] */
+                                 const void *prefix_k, /* bf16 [Hkv,P,d] (may be NULL when P == 0) */
+                                 const void *prefix_v, /* bf16 [Hkv,P,d] */
+                                 const void *suffix_k, /* bf16 [B,Hkv,Skv,d] */
+                                 const void *suffix_v, /* bf16 [B,Hkv,Skv,d] */
+                                 const int *suffix_len, /* device, [B], or NULL */
+                                 float scale,
+                                 void *out,            /* bf16 [B,Hq,Sq,d] */
+                                 float *lse,           /* fp32 [B,Hq,Sq] */
+                                 int B, int Hq, int Hkv, int Sq, int Skv, int P, int d,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+size_t pskv_attn_bwd_decode_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int P, int d);
+pskv_status pskv_attn_bwd_decode(const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
+                                 const void *suffix_k, const void *suffix_v, const int *suffix_len,
+                                 const void *out, const float *lse, float scale,
+                                 void *dq, void *dk_suffix, void *dv_suffix,
+                                 int B, int Hq, int Hkv, int Sq, int Skv, int P, int d,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then reads and clears the device status word that
  * kernels set when one of their bounded waits gives up.  Returns PSKV_OK,
  * PSKV_ERR_DEVICE_TIMEOUT (results of the affected call are undefined) or

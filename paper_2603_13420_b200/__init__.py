@@ -13,12 +13,16 @@ from .binding import (  # noqa: F401
     PSKV_OK,
     PskvError,
     pskv_attn_bwd,
+    pskv_attn_bwd_decode,
+    pskv_attn_bwd_decode_workspace_bytes,
     pskv_attn_bwd_multi,
     pskv_attn_bwd_multi_workspace_bytes,
     pskv_attn_bwd_static,
     pskv_attn_bwd_static_max_rows,
     pskv_attn_bwd_workspace_bytes,
     pskv_attn_fwd,
+    pskv_attn_fwd_decode,
+    pskv_attn_fwd_decode_workspace_bytes,
     pskv_attn_fwd_multi,
     pskv_attn_fwd_multi_workspace_bytes,
     pskv_attn_fwd_workspace_bytes,

@@ -66,6 +66,14 @@ def lib() -> ctypes.CDLL:
         L.pskv_attn_fwd_multi.restype = ci
         L.pskv_attn_bwd_multi.argtypes = [vp] * 9 + [cf] + [vp] * 3 + seven + [vp, sz, vp]
         L.pskv_attn_bwd_multi.restype = ci
+        L.pskv_attn_fwd_decode_workspace_bytes.argtypes = seven
+        L.pskv_attn_fwd_decode_workspace_bytes.restype = sz
+        L.pskv_attn_bwd_decode_workspace_bytes.argtypes = seven
+        L.pskv_attn_bwd_decode_workspace_bytes.restype = sz
+        L.pskv_attn_fwd_decode.argtypes = [vp] * 6 + [cf] + [vp] * 2 + seven + [vp, sz, vp]
+        L.pskv_attn_fwd_decode.restype = ci
+        L.pskv_attn_bwd_decode.argtypes = [vp] * 9 + [cf] + [vp] * 3 + seven + [vp, sz, vp]
+        L.pskv_attn_bwd_decode.restype = ci
         L.pskv_attn_bwd_static.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp]
         L.pskv_attn_bwd_static.restype = ci
         L.pskv_attn_bwd_static_max_rows.argtypes = []
@@ -265,6 +273,67 @@ def pskv_attn_bwd_multi(dout, q, prefix_k, prefix_v, prefix_len, suffix_k, suffi
                                    _ptr(ws), ws.numel() * ws.element_size(), _stream())
     if st != PSKV_OK:
         raise PskvError(st, "pskv_attn_bwd_multi")
+    return dq, dk_suffix, dv_suffix
+
+
+def _decode_dims(q, prefix_k, suffix_k):
+    B, Hq, Sq, d = q.shape
+    Hkv, Skv = suffix_k.shape[1], suffix_k.shape[2]
+    P = 0 if prefix_k is None else prefix_k.shape[1]
+    return [int(B), int(Hq), int(Hkv), int(Sq), int(Skv), int(P), int(d)]
+
+
+def _len_ptr(suffix_len, B):
+    if suffix_len is None:
+        return None
+    if suffix_len.dtype != torch.int32 or tuple(suffix_len.shape) != (B,):
+        raise ValueError("suffix_len must be an int32 CUDA tensor of shape [B]")
+    return _ptr(suffix_len)
+
+
+def pskv_attn_fwd_decode_workspace_bytes(B, Hq, Hkv, Sq, Skv, P, d) -> int:
+    return int(lib().pskv_attn_fwd_decode_workspace_bytes(B, Hq, Hkv, Sq, Skv, P, d))
+
+
+def pskv_attn_bwd_decode_workspace_bytes(B, Hq, Hkv, Sq, Skv, P, d) -> int:
+    return int(lib().pskv_attn_bwd_decode_workspace_bytes(B, Hq, Hkv, Sq, Skv, P, d))
+
+
+def pskv_attn_fwd_decode(q, prefix_k, prefix_v, suffix_k, suffix_v, suffix_len, scale, out=None, lse=None,
+                         workspace=None):
+    """Decode-shaped forward: q [B,Hq,Sq,d] are the last Sq of each candidate's suffix_len[b] cached
+    suffix tokens (suffix_k / suffix_v [B,Hkv,Skv,d]; suffix_len an int32 CUDA tensor [B] or None)."""
+    dims = _decode_dims(q, prefix_k, suffix_k)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    ws = _workspace(pskv_attn_fwd_decode_workspace_bytes(*dims), q.device, workspace)
+    st = lib().pskv_attn_fwd_decode(_ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(suffix_k), _ptr(suffix_v),
+                                    _len_ptr(suffix_len, dims[0]), float(scale), _ptr(out), _ptr(lse), *dims,
+                                    _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_fwd_decode")
+    return out, lse
+
+
+def pskv_attn_bwd_decode(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, suffix_len, out, lse, scale,
+                         dq=None, dk_suffix=None, dv_suffix=None, workspace=None):
+    """Backward of pskv_attn_fwd_decode: dq [B,Hq,Sq,d], dk_suffix / dv_suffix [B,Hkv,Skv,d]."""
+    dims = _decode_dims(q, prefix_k, suffix_k)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk_suffix is None:
+        dk_suffix = torch.empty_like(suffix_k)
+    if dv_suffix is None:
+        dv_suffix = torch.empty_like(suffix_v)
+    ws = _workspace(pskv_attn_bwd_decode_workspace_bytes(*dims), q.device, workspace)
+    st = lib().pskv_attn_bwd_decode(_ptr(dout), _ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(suffix_k),
+                                    _ptr(suffix_v), _len_ptr(suffix_len, dims[0]), _ptr(out), _ptr(lse),
+                                    float(scale), _ptr(dq), _ptr(dk_suffix), _ptr(dv_suffix), *dims,
+                                    _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_bwd_decode")
     return dq, dk_suffix, dv_suffix
 
 

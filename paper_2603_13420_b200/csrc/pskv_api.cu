@@ -41,6 +41,20 @@ pskv_status check_dims(int B, int Hq, int Hkv, int S, int P, int d, Dims *dm)
     if (rows * d > 1.0e12 || (double)Hkv * P * d > 1.0e12) return PSKV_ERR_UNSUPPORTED_SHAPE;
     dm->B = B; dm->Hq = Hq; dm->Hkv = Hkv; dm->S = S; dm->P = P; dm->d = d; dm->n_rep = Hq / Hkv;
     dm->Pstride = P;
+    dm->Skv = S;
+    dm->ragged = 0;
+    return PSKV_OK;
+}
+
+// The decode-shaped operator: S query rows per candidate against a suffix cache of Skv >= S rows.
+pskv_status check_dims_decode(int B, int Hq, int Hkv, int Sq, int Skv, int P, int d, bool ragged, Dims *dm)
+{
+    pskv_status st = check_dims(B, Hq, Hkv, Sq, P, d, dm);
+    if (st != PSKV_OK) return st;
+    if (Skv < Sq) return PSKV_ERR_INVALID_ARG;
+    if ((double)B * Hkv * Skv * d > 1.0e12) return PSKV_ERR_UNSUPPORTED_SHAPE;
+    dm->Skv = Skv;
+    dm->ragged = ragged ? 1 : 0;
     return PSKV_OK;
 }
 
@@ -200,26 +214,26 @@ size_t pskv_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d
     return tc_bwd_supported(dm) ? round256(tc_bwd_workspace_bytes(dm)) : simt_bwd_workspace(dm);
 }
 
-pskv_status pskv_attn_fwd(const void *q, const void *prefix_k, const void *prefix_v,
-                          const void *suffix_k, const void *suffix_v, float scale,
-                          void *out, float *lse, int B, int Hq, int Hkv, int S, int P, int d,
-                          void *workspace, size_t workspace_bytes, void *cuda_stream)
+namespace {
+
+// Pointer, scale and workspace checks plus the launch, shared by the full-suffix and the
+// decode-shaped forward; `dm` has passed check_dims / check_dims_decode.
+pskv_status fwd_checked(const Dims &dm, const void *q, const void *prefix_k, const void *prefix_v,
+                        const void *suffix_k, const void *suffix_v, const int *suffix_len, float scale, void *out,
+                        float *lse, size_t need, void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
-    Dims dm;
-    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
-    if (st != PSKV_OK) return st;
     if (!q || !suffix_k || !suffix_v || !out || !lse) return PSKV_ERR_INVALID_ARG;
-    if (P > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
+    if (dm.P > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) || !aligned16(suffix_k) ||
         !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse))
         return PSKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(suffix_len) & 3u) != 0) return PSKV_ERR_INVALID_ARG;
     if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
-    const size_t need = pskv_attn_fwd_workspace_bytes(B, Hq, Hkv, S, P, d);
     if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace)))
         return PSKV_ERR_WORKSPACE;
 
     unsigned int *status_word = nullptr;
-    st = check_device(&status_word);
+    pskv_status st = check_device(&status_word);
     if (st != PSKV_OK) return st;
 
     FwdArgs a;
@@ -230,6 +244,7 @@ pskv_status pskv_attn_fwd(const void *q, const void *prefix_k, const void *prefi
     a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v);
     a.out = static_cast<__nv_bfloat16 *>(out);
     a.lse = lse;
+    a.suffix_len = suffix_len;
     a.scale = scale;
     a.dims = dm;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -238,28 +253,24 @@ pskv_status pskv_attn_fwd(const void *q, const void *prefix_k, const void *prefi
     return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
 }
 
-pskv_status pskv_attn_bwd(const void *dout, const void *q, const void *prefix_k,
-                          const void *prefix_v, const void *suffix_k, const void *suffix_v,
-                          const void *out, const float *lse, float scale, void *dq,
-                          void *dk_suffix, void *dv_suffix, int B, int Hq, int Hkv, int S, int P,
-                          int d, void *workspace, size_t workspace_bytes, void *cuda_stream)
+pskv_status bwd_checked(const Dims &dm, const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
+                        const void *suffix_k, const void *suffix_v, const int *suffix_len, const void *out,
+                        const float *lse, float scale, void *dq, void *dk_suffix, void *dv_suffix, size_t need,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
-    Dims dm;
-    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
-    if (st != PSKV_OK) return st;
     if (!dout || !q || !suffix_k || !suffix_v || !out || !lse || !dq || !dk_suffix || !dv_suffix)
         return PSKV_ERR_INVALID_ARG;
-    if (P > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
+    if (dm.P > 0 && (!prefix_k || !prefix_v)) return PSKV_ERR_INVALID_ARG;
     if (!aligned16(dout) || !aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) ||
         !aligned16(suffix_k) || !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse) ||
         !aligned16(dq) || !aligned16(dk_suffix) || !aligned16(dv_suffix))
         return PSKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(suffix_len) & 3u) != 0) return PSKV_ERR_INVALID_ARG;
     if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
-    const size_t need = pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d);
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
 
     unsigned int *status_word = nullptr;
-    st = check_device(&status_word);
+    pskv_status st = check_device(&status_word);
     if (st != PSKV_OK) return st;
 
     BwdArgs a;
@@ -275,12 +286,82 @@ pskv_status pskv_attn_bwd(const void *dout, const void *q, const void *prefix_k,
     a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix);
     a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix);
     a.row_dot = static_cast<float *>(workspace);
+    a.suffix_len = suffix_len;
     a.scale = scale;
     a.dims = dm;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = tc_bwd_supported(dm) ? launch_tc_bwd(a, workspace, status_word, stream)
                                          : launch_simt_bwd(a, stream);
     return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+pskv_status pskv_attn_fwd(const void *q, const void *prefix_k, const void *prefix_v,
+                          const void *suffix_k, const void *suffix_v, float scale,
+                          void *out, float *lse, int B, int Hq, int Hkv, int S, int P, int d,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return st;
+    return fwd_checked(dm, q, prefix_k, prefix_v, suffix_k, suffix_v, nullptr, scale, out, lse,
+                       pskv_attn_fwd_workspace_bytes(B, Hq, Hkv, S, P, d), workspace, workspace_bytes, cuda_stream);
+}
+
+pskv_status pskv_attn_bwd(const void *dout, const void *q, const void *prefix_k,
+                          const void *prefix_v, const void *suffix_k, const void *suffix_v,
+                          const void *out, const float *lse, float scale, void *dq,
+                          void *dk_suffix, void *dv_suffix, int B, int Hq, int Hkv, int S, int P,
+                          int d, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return st;
+    return bwd_checked(dm, dout, q, prefix_k, prefix_v, suffix_k, suffix_v, nullptr, out, lse, scale, dq, dk_suffix,
+                       dv_suffix, pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d), workspace, workspace_bytes,
+                       cuda_stream);
+}
+
+// ---- decode-shaped variant: the last Sq of each candidate's cached suffix tokens are the queries ------
+
+size_t pskv_attn_fwd_decode_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int P, int d)
+{
+    Dims dm;
+    if (check_dims_decode(B, Hq, Hkv, Sq, Skv, P, d, true, &dm) != PSKV_OK) return 0;
+    return 256;  // the redo counter of the tensor-core forward (whether or not suffix_len is given)
+}
+
+size_t pskv_attn_bwd_decode_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int P, int d)
+{
+    Dims dm;
+    if (check_dims_decode(B, Hq, Hkv, Sq, Skv, P, d, true, &dm) != PSKV_OK) return 0;
+    return simt_bwd_workspace(dm);  // one fp32 per query row
+}
+
+pskv_status pskv_attn_fwd_decode(const void *q, const void *prefix_k, const void *prefix_v, const void *suffix_k,
+                                 const void *suffix_v, const int *suffix_len, float scale, void *out, float *lse,
+                                 int B, int Hq, int Hkv, int Sq, int Skv, int P, int d, void *workspace,
+                                 size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims_decode(B, Hq, Hkv, Sq, Skv, P, d, suffix_len != nullptr, &dm);
+    if (st != PSKV_OK) return st;
+    return fwd_checked(dm, q, prefix_k, prefix_v, suffix_k, suffix_v, suffix_len, scale, out, lse, 256, workspace,
+                       workspace_bytes, cuda_stream);
+}
+
+pskv_status pskv_attn_bwd_decode(const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
+                                 const void *suffix_k, const void *suffix_v, const int *suffix_len, const void *out,
+                                 const float *lse, float scale, void *dq, void *dk_suffix, void *dv_suffix, int B,
+                                 int Hq, int Hkv, int Sq, int Skv, int P, int d, void *workspace,
+                                 size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims_decode(B, Hq, Hkv, Sq, Skv, P, d, suffix_len != nullptr, &dm);
+    if (st != PSKV_OK) return st;
+    return bwd_checked(dm, dout, q, prefix_k, prefix_v, suffix_k, suffix_v, suffix_len, out, lse, scale, dq, dk_suffix,
+                       dv_suffix, simt_bwd_workspace(dm), workspace, workspace_bytes, cuda_stream);
 }
 
 // ---- several instructions per call (suffix-centric alignment, Sec. 4.3) --------------------------
@@ -352,6 +433,7 @@ pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void 
         a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v) + i * s_part;
         a.out = static_cast<__nv_bfloat16 *>(out) + i * q_part;
         a.lse = lse + i * l_part;
+        a.suffix_len = nullptr;
         a.scale = scale;
         a.dims = dm;
         cudaError_t e = tc_fwd_supported(dm) ? launch_tc_fwd(a, workspace, status_word, stream)
@@ -408,6 +490,7 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix) + i * s_part;
         a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix) + i * s_part;
         a.row_dot = static_cast<float *>(ws);
+        a.suffix_len = nullptr;
         a.scale = scale;
         a.dims = dm;
         cudaError_t e = tc_bwd_supported(dm) ? launch_tc_bwd(a, ws, status_word, stream)

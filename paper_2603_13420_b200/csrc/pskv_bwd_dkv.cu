@@ -308,6 +308,7 @@ cudaError_t launch_one(const BwdArgs &a, cudaStream_t stream)
 
 bool mma_bwd_dkv_supported(const Dims &dm)
 {
+    if (dm.Skv != dm.S || dm.ragged) return false;  // full-suffix operator only
     return (dm.d == 64 || dm.d == 128) && dm.S >= 1 && dm.S <= 64 && (long long)dm.B * dm.Hkv < 2000000000ll;
 }
 

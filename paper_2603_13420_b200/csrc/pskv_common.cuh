@@ -10,15 +10,28 @@ namespace pskv {
 
 // Dimensions of one call; `n_rep` = Hq / Hkv query heads per KV head.  `Pstride` is the distance, in
 // rows, between the prefix blocks of consecutive KV heads (P for a dense prefix cache; the padded
-// length when the call works on the real tokens of a left-padded cache).
+// length when the call works on the real tokens of a left-padded cache).  `S` counts the query rows
+// per candidate and `Skv` the rows of its suffix K/V buffer: equal for the full-suffix operator,
+// Skv >= S for the decode-shaped one, where the queries are the last S of the candidate's cached
+// suffix tokens.  `ragged` is 1 when a per-candidate count of cached tokens (suffix_len) is given.
 struct Dims {
-    int B, Hq, Hkv, S, P, d, n_rep, Pstride;
+    int B, Hq, Hkv, S, P, d, n_rep, Pstride, Skv, ragged;
 };
+
+// Cached suffix tokens of candidate b, forced into [S, Skv] so that no value can index outside the
+// buffers; query i of the candidate is suffix token suffix_tokens(...) - S + i.
+__device__ __forceinline__ int suffix_tokens(const int *suffix_len, int b, int S, int Skv)
+{
+    if (!suffix_len) return Skv;
+    const int L = suffix_len[b];
+    return L < S ? S : (L > Skv ? Skv : L);
+}
 
 struct FwdArgs {
     const __nv_bfloat16 *q, *prefix_k, *prefix_v, *suffix_k, *suffix_v;
     __nv_bfloat16 *out;
     float *lse;
+    const int *suffix_len;  // device, [B], or nullptr: every candidate has Skv cached suffix tokens
     float scale;
     Dims dims;
 };
@@ -28,11 +41,12 @@ struct BwdArgs {
     const float *lse;
     __nv_bfloat16 *dq, *dk_suffix, *dv_suffix;
     float *row_dot;  // workspace: D[b,h,i] = <dout, out>, fp32 [B*Hq*S]
+    const int *suffix_len;  // as in FwdArgs
     float scale;
     Dims dims;
 };
 
-// General CUDA-core kernels (any S, P; d in {64,128}).
+// General CUDA-core kernels (any S, Skv, P; d in {64,128}; ragged or not).
 cudaError_t launch_simt_fwd(const FwdArgs &a, cudaStream_t stream);
 cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream);
 // Pieces of the backward the tensor-core path reuses: D = <dout, out> per row into a.row_dot, and

@@ -96,14 +96,15 @@ __device__ __forceinline__ void fwd_row(const FwdArgs &a, long long row, float *
     const int g = h / dm.n_rep;
     const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.Pstride * D;
     const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.Pstride * D;
-    const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
-    const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
+    const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.Skv * D;
+    const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.Skv * D;
 
     stage_row<D>(q_s, a.q + (size_t)row * D, lane);
     __syncwarp();
 
     const float scale2 = a.scale * kLog2e;
-    const int n_vis = dm.P + i + 1;
+    // the query is suffix token L - S + i of its candidate: it sees the prefix and suffix keys up to itself
+    const int n_vis = dm.P + suffix_tokens(a.suffix_len, b, dm.S, dm.Skv) - dm.S + i + 1;
     float m = -INFINITY, l = 0.f;
     float acc[D / 32];
 #pragma unroll
@@ -188,8 +189,8 @@ simt_bwd_dq_kernel(BwdArgs a)
     const int g = h / dm.n_rep;
     const __nv_bfloat16 *pk = a.prefix_k + (size_t)g * dm.Pstride * D;
     const __nv_bfloat16 *pv = a.prefix_v + (size_t)g * dm.Pstride * D;
-    const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.S * D;
-    const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.S * D;
+    const __nv_bfloat16 *sk = a.suffix_k + ((size_t)b * dm.Hkv + g) * dm.Skv * D;
+    const __nv_bfloat16 *sv = a.suffix_v + ((size_t)b * dm.Hkv + g) * dm.Skv * D;
 
     stage_row<D>(q_s[warp], a.q + (size_t)row * D, lane);
     stage_row<D>(do_s[warp], a.dout + (size_t)row * D, lane);
@@ -204,7 +205,7 @@ simt_bwd_dq_kernel(BwdArgs a)
 
     const float scale2 = a.scale * kLog2e;
     const float lse2 = a.lse[row] * kLog2e;
-    const int n_vis = dm.P + i + 1;
+    const int n_vis = dm.P + suffix_tokens(a.suffix_len, b, dm.S, dm.Skv) - dm.S + i + 1;
     float acc[D / 32];
 #pragma unroll
     for (int e = 0; e < D / 32; ++e) acc[e] = 0.f;
@@ -279,7 +280,7 @@ simt_row_dot_kernel(BwdArgs a)
 }
 
 // Backward, key side: one warp per suffix key (b,g,t); sums over the n_rep heads of the group
-// and the rows i >= t that see the key.  Needs row_dot from the query-side kernel.
+// and the query rows that see the key.  Needs row_dot from the query-side kernel.
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 simt_bwd_dkv_kernel(BwdArgs a)
@@ -289,17 +290,28 @@ simt_bwd_dkv_kernel(BwdArgs a)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Dims dm = a.dims;
     const long long key = (long long)blockIdx.x * kWarpsPerBlock + warp;
-    if (key >= (long long)dm.B * dm.Hkv * dm.S) return;
-    const int t = (int)(key % dm.S);
-    const int g = (int)((key / dm.S) % dm.Hkv);
-    const int b = (int)(key / ((long long)dm.S * dm.Hkv));
+    if (key >= (long long)dm.B * dm.Hkv * dm.Skv) return;
+    const int t = (int)(key % dm.Skv);
+    const int g = (int)((key / dm.Skv) % dm.Hkv);
+    const int b = (int)(key / ((long long)dm.Skv * dm.Hkv));
+    const int L = suffix_tokens(a.suffix_len, b, dm.S, dm.Skv);
+    if (t >= L) {  // not a cached token: no query sees it
+        float z[D / 32];
+#pragma unroll
+        for (int e = 0; e < D / 32; ++e) z[e] = 0.f;
+        store_slice<D>(a.dk_suffix + (size_t)key * D, lane, z);
+        store_slice<D>(a.dv_suffix + (size_t)key * D, lane, z);
+        return;
+    }
 
     stage_row<D>(k_s[warp], a.suffix_k + (size_t)key * D, lane);
     stage_row<D>(v_s[warp], a.suffix_v + (size_t)key * D, lane);
     __syncwarp();
 
     const float scale2 = a.scale * kLog2e;
-    const int per_head = dm.S - t;            // rows i = t .. S-1
+    // query i is suffix token L - S + i: the key is seen by rows i >= t - (L - S)
+    const int i_min = max(0, t - (L - dm.S));
+    const int per_head = dm.S - i_min;        // rows i = i_min .. S-1
     const int n_rows = dm.n_rep * per_head;
     float dk[D / 32], dv[D / 32];
 #pragma unroll
@@ -310,7 +322,7 @@ simt_bwd_dkv_kernel(BwdArgs a)
         float p = 0.f, ds = 0.f;
         if (r < n_rows) {
             const int h = g * dm.n_rep + r / per_head;
-            const int i = t + r % per_head;
+            const int i = i_min + r % per_head;
             const size_t row = ((size_t)b * dm.Hq + h) * dm.S + i;
             p = exp2f(scale2 * dot_row<D>(k_s[warp], a.q + row * D) - a.lse[row] * kLog2e);
             const float dp = dot_row<D>(v_s[warp], a.dout + row * D);
@@ -322,7 +334,7 @@ simt_bwd_dkv_kernel(BwdArgs a)
             const float dsu = __shfl_sync(0xffffffffu, ds, u);
             const int rr = r0 + u;
             const int h = g * dm.n_rep + rr / per_head;
-            const int i = t + rr % per_head;
+            const int i = i_min + rr % per_head;
             const size_t row = ((size_t)b * dm.Hq + h) * dm.S + i;
             float qv[D / 32], gv[D / 32];
             load_slice<D>(a.q + row * D, lane, qv);
@@ -386,7 +398,7 @@ cudaError_t launch_simt_row_dot(const BwdArgs &a, cudaStream_t stream)
 
 cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream)
 {
-    const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.S;
+    const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.Skv;
     KernelTiming timing(kKernelBwdDkvSimt, stream);
     if (a.dims.d == 128)
         simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
@@ -399,7 +411,7 @@ cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream)
 cudaError_t launch_simt_bwd(const BwdArgs &a, cudaStream_t stream)
 {
     const long long rows = (long long)a.dims.B * a.dims.Hq * a.dims.S;
-    const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.S;
+    const long long keys = (long long)a.dims.B * a.dims.Hkv * a.dims.Skv;
     {
         KernelTiming timing(kKernelBwdDqSimt, stream);
         if (a.dims.d == 128)

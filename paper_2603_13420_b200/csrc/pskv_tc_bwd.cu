@@ -868,6 +868,7 @@ extern "C" int pskv_debug_read_trace_dq(long long *host, int max_events)
 
 bool tc_bwd_supported(const Dims &dm)
 {
+    if (dm.Skv != dm.S || dm.ragged) return false;  // full-suffix operator only
     if (dm.d != 64 && dm.d != 128) return false;
     if ((long long)dm.B * dm.n_rep * dm.S > 2000000000ll) return false;
     return plan_bwd(dm).ok;

@@ -448,6 +448,7 @@ extern "C" int pskv_debug_read_trace_dkv(long long *host, int max_events)
 
 bool tc_bwd_dkv_supported(const Dims &dm)
 {
+    if (dm.Skv != dm.S || dm.ragged) return false;  // full-suffix operator only
     return dm.d == kD && dm.S >= 1 && dm.S <= 64 && (long long)dm.B * dm.Hkv < 2000000000ll &&
            (long long)dm.n_rep * dm.S < 2000000000ll && get_encode_fn() != nullptr;
 }

@@ -915,6 +915,7 @@ extern "C" int pskv_debug_read_trace(long long *host, int max_events)
 
 bool tc_fwd_supported(const Dims &dm)
 {
+    if (dm.Skv != dm.S || dm.ragged) return false;  // full-suffix operator only
     if (dm.d != 64 && dm.d != 128) return false;
     if ((long long)dm.B * dm.n_rep * dm.S > 2000000000ll) return false;  // flat row index fits an int
     return plan_tiles(dm).ok;

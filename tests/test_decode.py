@@ -1,0 +1,133 @@
+"""Decode-shaped variant: only the last Sq of each candidate's suffix_len[b] cached suffix tokens are
+queries (token-by-token suffix growth).  GPU parity against the fp64 oracle on seeded inputs whose
+unused cache rows hold large finite garbage, plus host-side argument checks."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_13420_b200 as pskv
+import parity
+
+SEED = 260313420 + 99
+
+
+def make(B, Hq, Hkv, Sq, Skv, P, d, ragged, seed=SEED):
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed + B + 7 * Sq + 13 * Skv + P)
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+
+    t = dict(q=draw(B, Hq, Sq, d), prefix_k=draw(Hkv, P, d), prefix_v=draw(Hkv, P, d),
+             suffix_k=draw(B, Hkv, Skv, d), suffix_v=draw(B, Hkv, Skv, d), dout=draw(B, Hq, Sq, d))
+    lens = None
+    if ragged:
+        lens = torch.randint(Sq, Skv + 1, (B,), generator=gen, dtype=torch.int32)
+        lens[0] = Sq           # the shortest legal cache: the queries are all there is
+        lens[B - 1] = Skv      # and a full one
+        for b in range(B):     # rows past the cached tokens must not matter
+            t["suffix_k"][b, :, int(lens[b]):] = 3.0e4
+            t["suffix_v"][b, :, int(lens[b]):] = -3.0e4
+    return t, lens
+
+
+CASES = [
+    # B, Hq, Hkv, Sq, Skv, P, d, ragged
+    (64, 32, 8, 1, 48, 256, 128, False),    # one new token per candidate, the GQA layer shape
+    (130, 32, 8, 1, 48, 256, 128, True),    # ragged lengths; candidate count leaves a partial last tile
+    (32, 8, 2, 8, 40, 300, 128, True),      # a few new tokens, prefix with a ragged last block
+    (16, 4, 4, 4, 20, 160, 128, True),      # MHA
+    (12, 4, 2, 3, 7, 33, 64, True),         # head dim 64, odd sizes
+    (6, 4, 2, 2, 150, 64, 128, True),       # suffix cache longer than one key block
+    (9, 8, 2, 2, 24, 0, 128, True),         # no prefix
+    (20, 16, 4, 16, 64, 700, 128, False),   # prefix streamed in several blocks
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", CASES)
+def test_decode_forward_and_backward_match_the_oracle(case):
+    B, Hq, Hkv, Sq, Skv, P, d, ragged = case
+    t, lens = make(*case)
+    scale = 1.0 / np.sqrt(d)
+    dev = {k: v.cuda() for k, v in t.items()}
+    dlens = None if lens is None else lens.cuda()
+    pk = dev["prefix_k"] if P > 0 else None
+    pv = dev["prefix_v"] if P > 0 else None
+    out = parity.Guarded((B, Hq, Sq, d), torch.bfloat16, "cuda")
+    lse = parity.Guarded((B, Hq, Sq), torch.float32, "cuda")
+    pskv.pskv_attn_fwd_decode(dev["q"], pk, pv, dev["suffix_k"], dev["suffix_v"], dlens, scale,
+                              out=out.view, lse=lse.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    out.check("out"); lse.check("lse")
+    f = {k: parity.to_f64(v) for k, v in t.items()}
+    nl = None if lens is None else lens.numpy()
+    ref_out, ref_lse = oracle.attn_fwd_decode(f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"],
+                                              scale, nl)
+    parity.check_tensor("out", parity.to_f64(out.view), ref_out, strict_abs=(P + 1 >= 128))
+    parity.check_lse(parity.to_f64(lse.view), ref_lse)
+
+    dq = parity.Guarded((B, Hq, Sq, d), torch.bfloat16, "cuda")
+    dk = parity.Guarded((B, Hkv, Skv, d), torch.bfloat16, "cuda")
+    dv = parity.Guarded((B, Hkv, Skv, d), torch.bfloat16, "cuda")
+    pskv.pskv_attn_bwd_decode(dev["dout"], dev["q"], pk, pv, dev["suffix_k"], dev["suffix_v"], dlens, out.view,
+                              lse.view, scale, dq=dq.view, dk_suffix=dk.view, dv_suffix=dv.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    dq.check("dq"); dk.check("dk_suffix"); dv.check("dv_suffix")
+    rq, rk, rv = oracle.attn_bwd_decode(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"],
+                                        f["suffix_v"], scale, nl)
+    parity.check_tensor("dq", parity.to_f64(dq.view), rq)
+    parity.check_tensor("dk_suffix", parity.to_f64(dk.view), rk)
+    parity.check_tensor("dv_suffix", parity.to_f64(dv.view), rv)
+    if lens is not None:   # gradients of rows that are not cached tokens are exactly zero
+        for b in range(B):
+            assert not dk.view[b, :, int(lens[b]):].any() and not dv.view[b, :, int(lens[b]):].any()
+
+
+@pytest.mark.gpu
+def test_all_tokens_as_queries_equals_the_full_suffix_call_bit_for_bit():
+    B, Hq, Hkv, S, P, d = 16, 8, 2, 16, 200, 128
+    t, _ = make(B, Hq, Hkv, S, S, P, d, False)
+    dev = {k: v.cuda() for k, v in t.items()}
+    scale = 1.0 / np.sqrt(d)
+    o1, l1 = pskv.pskv_attn_fwd(dev["q"], dev["prefix_k"], dev["prefix_v"], dev["suffix_k"], dev["suffix_v"], scale)
+    o2, l2 = pskv.pskv_attn_fwd_decode(dev["q"], dev["prefix_k"], dev["prefix_v"], dev["suffix_k"], dev["suffix_v"],
+                                       None, scale)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+
+
+@pytest.mark.gpu
+def test_growing_the_suffix_token_by_token_reproduces_the_full_evaluation():
+    """Three decode steps of one token each give the last three rows of a full-suffix call."""
+    B, Hq, Hkv, S, P, d = 24, 8, 2, 16, 256, 128
+    t, _ = make(B, Hq, Hkv, S, S, P, d, False)
+    dev = {k: v.cuda() for k, v in t.items()}
+    scale = 1.0 / np.sqrt(d)
+    o_full, l_full = pskv.pskv_attn_fwd(dev["q"], dev["prefix_k"], dev["prefix_v"], dev["suffix_k"], dev["suffix_v"],
+                                        scale)
+    for step, L in enumerate((S - 2, S - 1, S)):
+        lens = torch.full((B,), L, dtype=torch.int32, device="cuda")
+        q1 = dev["q"][:, :, L - 1:L].contiguous()
+        o1, l1 = pskv.pskv_attn_fwd_decode(q1, dev["prefix_k"], dev["prefix_v"], dev["suffix_k"], dev["suffix_v"],
+                                           lens, scale)
+        assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+        err = (o1.float() - o_full[:, :, L - 1:L].float()).abs().max().item()
+        assert err <= 2e-2, (step, err)
+        assert (l1 - l_full[:, :, L - 1:L]).abs().max().item() <= 1e-3 * max(1.0, l_full.abs().max().item())
+
+
+def test_decode_arguments_are_checked_on_the_host():
+    L = pskv.binding.lib()
+    fake = ctypes.c_void_p(4096)
+    call = lambda Sq, Skv, lens=None, ws=256: L.pskv_attn_fwd_decode(
+        fake, fake, fake, fake, fake, lens, ctypes.c_float(0.1), fake, fake, 8, 4, 4, Sq, Skv, 16, 128, fake, ws, None)
+    assert call(9, 8) == pskv.PSKV_ERR_INVALID_ARG                       # more queries than cache rows
+    assert call(0, 8) == pskv.PSKV_ERR_INVALID_ARG
+    assert call(1, 8, ctypes.c_void_p(4098)) == pskv.PSKV_ERR_INVALID_ARG  # misaligned length array
+    assert call(1, 8, None, 16) == pskv.PSKV_ERR_WORKSPACE
+    assert pskv.pskv_attn_fwd_decode_workspace_bytes(8, 4, 4, 1, 8, 16, 128) == 256
+    assert pskv.pskv_attn_fwd_decode_workspace_bytes(8, 4, 4, 9, 8, 16, 128) == 0
+    assert pskv.pskv_attn_bwd_decode_workspace_bytes(8, 4, 4, 2, 8, 16, 128) >= 8 * 4 * 2 * 4
