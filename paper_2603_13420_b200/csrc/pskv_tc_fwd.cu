@@ -64,6 +64,12 @@ struct TcFwdParams {
     int stages;           // streaming mode: stages of the prefix K and V rings
     int sfx_rows;         // rows of the suffix K / V buffers (multiple of 16, <= 128)
     int alias_stage;      // 1 when the output staging buffer shares its memory with the suffix V buffer
+    // suffix-ring mode (tiles of whole candidates, suffix keys in blocks through the K/V rings)
+    const int *suffix_len;  // cached suffix tokens per candidate, or nullptr (= Skv)
+    int Skv;              // rows of a candidate's suffix K/V buffer (S counts its query rows)
+    int Spad;             // Skv rounded up to 8: rows a candidate takes inside a suffix block
+    int cpb;              // candidates per suffix block: 128 / Spad
+    FastDiv fd_cpb;
     // shared-memory carve-up (byte offsets from the 1024-byte aligned base)
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml;
 };
@@ -107,9 +113,24 @@ __device__ __forceinline__ int prefix_block_rows(const TcFwdParams &p, int k)
 constexpr int kPiece = 32;  // score columns a softmax thread handles per tensor-memory load
 static_assert(kBlockN == 4 * kPiece, "two softmax groups x two pieces cover a score block");
 
-// RES: all prefix blocks of a KV head stay in shared memory (else they stream through rings); a
-// compile-time switch so that each launch carries only the code of its own mode.
-template <int D, bool RES>
+// Suffix-ring mode: candidates [first, first + count) of a tile that suffix block j holds, and the
+// MMA N (rows rounded up to 16) of that block.
+__device__ __forceinline__ int sfx_block_cands(const TcFwdParams &p, int nc, int j)
+{
+    return min(p.cpb, nc - j * p.cpb);
+}
+__device__ __forceinline__ int sfx_block_rows(const TcFwdParams &p, int nc, int j)
+{
+    return (sfx_block_cands(p, nc, j) * p.Spad + 15) & ~15;
+}
+
+// MODE 1: all prefix blocks of a KV head stay in shared memory; MODE 0: they stream through rings,
+// and the suffix keys of a tile sit in one block with buffers of its own; MODE 2 (suffix-ring): a
+// tile is a run of whole candidates and their suffix keys follow the prefix through the same rings
+// in as many blocks as it takes -- the mode of the decode-shaped operator, where a 128-row tile
+// spans many candidates, and of full-suffix shapes the other two modes cannot tile.  A compile-time
+// switch so that each launch carries only the code of its own mode.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_out,
               const __grid_constant__ CUtensorMap tm_pk, const __grid_constant__ CUtensorMap tm_pv,
@@ -118,6 +139,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
               const TcFwdParams p)
 {
     using C = Cfg<D>;
+    constexpr bool RES = MODE == 1;
+    constexpr bool SR = MODE == 2;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
@@ -161,7 +184,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int t_begin = (int)((long long)blockIdx.x * p.total_tiles / gridDim.x);
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
     const int n_tiles = t_end - t_begin;
-    const int nitems = p.nblk_p + 1;  // prefix blocks + the suffix block
+    // items of a tile: prefix blocks + the suffix block(s)
+    auto items_of = [&](const TileInfo &t) { return p.nblk_p + (SR ? p.fd_cpb.div(t.nc + p.cpb - 1) : 1); };
     const int g_first = p.fd_tpg.div(t_begin);
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
@@ -185,7 +209,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // Everything the Q loads need is worked out before the wait, so that only the copy
             // instructions themselves follow it: the Q buffer is single, and the time from "last
             // score MMA of the previous tile done" to "Q of this tile requested" is exposed.
-            const int nseg = p.fd_seg.div(t.rows);  // one box per run of seg_rows rows
+            // (Suffix-ring mode: one box per slab holds the tile's whole candidates; a box reaching
+            // past the last candidate is filled with zeros and still counts its full size.)
+            const int nseg = SR ? 1 : p.fd_seg.div(t.rows);  // one box per run of seg_rows rows
             int qb = p.fd_Rg.div(t.R0), qr = t.R0 - qb * p.Rg;
             const uint32_t q_bytes = (uint32_t)(nseg * C::kSlabs * p.seg_rows * 128);
             const uint32_t seg_bytes = (uint32_t)(p.seg_rows * 128);
@@ -194,7 +220,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // be issued a tile from now, right when it is needed, and then finds the data close by.
             if (tl + 1 < n_tiles) {
                 const TileInfo tn = tile_info(p, t_begin + tl + 1, t_begin);
-                const int nseg_n = p.fd_seg.div(tn.rows);
+                const int nseg_n = SR ? 1 : p.fd_seg.div(tn.rows);
                 int nb = p.fd_Rg.div(tn.R0), nr = tn.R0 - nb * p.Rg;
                 if (elect_one_sync()) {
 #pragma unroll 1
@@ -266,17 +292,44 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
                 if (!ok) break;
             }
-            // suffix K of the candidates this tile touches: one box per candidate
-            if (elect_one_sync()) {
-                mbar_arrive_expect_tx(bar(kBarSKFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
+            if (SR) {
+                // suffix K of the tile's candidates, block by block through the ring: one box of
+                // Skv rows per candidate, candidates Spad rows apart inside a block
+                const int nbs = items_of(t) - p.nblk_p;
 #pragma unroll 1
-                for (int c = 0; c < t.nc; ++c)
+                for (int j = 0; j < nbs; ++j) {
+                    const uint32_t ks = kload % (uint32_t)p.stages;
+                    ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
+                                        p.status, kErrProducerK);
+                    if (!ok) break;
+                    const int ncb = sfx_block_cands(p, t.nc, j);
+                    const int slab = sfx_block_rows(p, t.nc, j) * 128;
+                    if (elect_one_sync()) {
+                        mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(ncb * C::kSlabs * p.Skv * 128));
 #pragma unroll 1
-                    for (int sl = 0; sl < C::kSlabs; ++sl)
-                        tma_load_4d(sbase + p.off_sk + sl * sfx_slab + c * p.S * 128, &tm_sk, bar(kBarSKFull),
-                                    sl * 64, 0, t.g, t.b_first + c);
+                        for (int c = 0; c < ncb; ++c)
+#pragma unroll 1
+                            for (int sl = 0; sl < C::kSlabs; ++sl)
+                                tma_load_4d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab + c * p.Spad * 128, &tm_sk,
+                                            bar(kBarKFull + ks), sl * 64, 0, t.g, t.b_first + j * p.cpb + c);
+                    }
+                    __syncwarp();
+                    ++kload;
+                }
+                if (!ok) break;
+            } else {
+                // suffix K of the candidates this tile touches: one box per candidate
+                if (elect_one_sync()) {
+                    mbar_arrive_expect_tx(bar(kBarSKFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
+#pragma unroll 1
+                    for (int c = 0; c < t.nc; ++c)
+#pragma unroll 1
+                        for (int sl = 0; sl < C::kSlabs; ++sl)
+                            tma_load_4d(sbase + p.off_sk + sl * sfx_slab + c * p.S * 128, &tm_sk, bar(kBarSKFull),
+                                        sl * 64, 0, t.g, t.b_first + c);
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
     } else if (role == 3) {
         // ------------------------------------------------------------------ producer, value side
@@ -298,9 +351,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // Two jobs ride along with the prefix loads of tile tl: the stores of tile tl-1 (once it
             // is staged) and the fetch of this tile's suffix V (once its buffer is free: after those
             // stores when it doubles as the staging buffer, else after the previous tile's value MMAs).
-            bool pend_store = tl > 0, pend_sv = have_tile;
+            bool pend_store = tl > 0, pend_sv = have_tile && !SR;
             TileInfo t;
-            int nk = 0;  // prefix V blocks still to fetch for this tile
+            int nk = 0;  // V blocks still to fetch through the ring for this tile
             if (have_tile) {
                 t = tile_info(p, t_begin + tl, t_begin);
                 if (RES) {
@@ -322,7 +375,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     }
                     __syncwarp();
                 } else {
-                    nk = p.nblk_p;
+                    nk = SR ? items_of(t) : p.nblk_p;
                 }
             }
             int k = 0;
@@ -334,14 +387,30 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
                                         p.status, kErrProducerV);
                     if (!ok) break;
-                    const bool tail = k == p.nblk_p - 1;
-                    const int slab = tail ? tail_slab : C::kSlabBytes;
-                    if (elect_one_sync()) {
-                        mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
+                    if (SR && k >= p.nblk_p) {
+                        // a suffix V block: one box of Skv rows per candidate, Spad rows apart
+                        const int j = k - p.nblk_p;
+                        const int ncb = sfx_block_cands(p, t.nc, j);
+                        const int slab = sfx_block_rows(p, t.nc, j) * 128;
+                        if (elect_one_sync()) {
+                            mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(ncb * C::kSlabs * p.Skv * 128));
 #pragma unroll 1
-                        for (int sl = 0; sl < C::kSlabs; ++sl)
-                            tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
-                                        bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                            for (int c = 0; c < ncb; ++c)
+#pragma unroll 1
+                                for (int sl = 0; sl < C::kSlabs; ++sl)
+                                    tma_load_4d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab + c * p.Spad * 128,
+                                                &tm_sv, bar(kBarVFull + vs), sl * 64, 0, t.g, t.b_first + j * p.cpb + c);
+                        }
+                    } else {
+                        const bool tail = k == p.nblk_p - 1;
+                        const int slab = tail ? tail_slab : C::kSlabBytes;
+                        if (elect_one_sync()) {
+                            mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
+#pragma unroll 1
+                            for (int sl = 0; sl < C::kSlabs; ++sl)
+                                tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab,
+                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                        }
                     }
                     __syncwarp();
                     ++vload;
@@ -366,7 +435,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (!ok) break;
                     if (ready) {
                         const TileInfo u = tile_info(p, t_begin + tl - 1, t_begin);
-                        const int nseg = p.fd_seg.div(u.rows);
+                        const int nseg = SR ? 1 : p.fd_seg.div(u.rows);  // (one box of whole candidates)
                         if (elect_one_sync()) {
 #pragma unroll 1
                             for (int sl = 0; sl < C::kSlabs; ++sl)
@@ -407,13 +476,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         __syncwarp();
     } else if (role == 1) {
         // ------------------------------------------------------------------ score MMAs: S = Q K^T
-        const int total_items = n_tiles * nitems;
         int tl = 0, k = 0;
-        uint32_t kuse = 0;  // streaming mode: prefix K blocks consumed
+        uint32_t kuse = 0;  // streaming mode: K blocks consumed from the ring
         TileInfo t = tile_info(p, t_begin, t_begin);
+        int nitems = items_of(t);
         const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
         bool ok = true;
-        for (int i = 0; i < total_items && ok; ++i) {
+        for (int i = 0; tl < n_tiles && ok; ++i) {
             const int slot = i % kSlots;
             // the slot is free once the value MMAs of item i-3 (which read P from it) have completed
             ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
@@ -424,8 +493,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             uint32_t kaddr;
             int n, slab;
-            if (k < p.nblk_p) {
-                n = prefix_block_rows(p, k);
+            if (k < p.nblk_p || SR) {
+                n = k < p.nblk_p ? prefix_block_rows(p, k) : sfx_block_rows(p, t.nc, k - p.nblk_p);
                 slab = n * 128;
                 if (RES) {
                     if (t.first_of_g)
@@ -451,7 +520,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
             const uint64_t k_slab = (uint64_t)(slab >> 4);
             const bool last_of_tile = k == nitems - 1;
-            const bool free_stage = k < p.nblk_p && !RES;
+            const bool free_stage = (k < p.nblk_p || SR) && !RES;
             if (elect_one_sync()) {
 #pragma unroll
                 for (int ks16 = 0; ks16 < D / 16; ++ks16) {
@@ -468,18 +537,21 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (free_stage) ++kuse;
             if (++k == nitems) {
                 k = 0;
-                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+                if (++tl < n_tiles) {
+                    t = tile_info(p, t_begin + tl, t_begin);
+                    nitems = items_of(t);
+                }
             }
         }
     } else if (role == 2) {
         // ------------------------------------------------------------------ value MMAs: O += P V
-        const int total_items = n_tiles * nitems;
         int tl = 0, k = 0;
         uint32_t vuse = 0;
         TileInfo t = tile_info(p, t_begin, t_begin);
+        int nitems = items_of(t);
         const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
         bool ok = true;
-        for (int i = 0; i < total_items && ok; ++i) {
+        for (int i = 0; tl < n_tiles && ok; ++i) {
             const int slot = i % kSlots;
             ok = mbar_wait_warp(bar(kBarPReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaPv);
             if (!ok) break;
@@ -491,8 +563,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             uint32_t vaddr;
             int n, slab;
-            if (k < p.nblk_p) {
-                n = prefix_block_rows(p, k);
+            if (k < p.nblk_p || SR) {
+                n = k < p.nblk_p ? prefix_block_rows(p, k) : sfx_block_rows(p, t.nc, k - p.nblk_p);
                 slab = n * 128;
                 if (RES) {
                     if (t.first_of_g)
@@ -518,7 +590,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
             const int nk = n >> 4;
             const bool last_of_tile = k == nitems - 1;
-            const bool free_stage = k < p.nblk_p && !RES;
+            const bool free_stage = (k < p.nblk_p || SR) && !RES;
             const uint32_t acc0 = k > 0 ? 1u : 0u;
             if (elect_one_sync()) {
 #pragma unroll
@@ -539,7 +611,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (free_stage) ++vuse;
             if (++k == nitems) {
                 k = 0;
-                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+                if (++tl < n_tiles) {
+                    t = tile_info(p, t_begin + tl, t_begin);
+                    nitems = items_of(t);
+                }
             }
         }
     } else if (warp < 4 + 4 * kGroups) {
@@ -561,21 +636,33 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
         bool ok = true;
         float lsum = 0.f;
+        int item = 0;  // items handled so far
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
             const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            const int nitems = items_of(t);
             int lo_sfx = 1, hi_sfx = 0;
+            int k_own = p.nblk_p;  // suffix-ring mode: the item that holds this row's candidate
             if (row < t.rows) {
                 const int R = t.R0 + row;
                 const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
-                lo_sfx = (b - t.b_first) * p.S;  // first suffix column of this row's candidate
-                hi_sfx = lo_sfx + (r - p.fd_S.div(r) * p.S);     // causal: suffix keys 0..i
+                const int i = r - p.fd_S.div(r) * p.S;  // query index inside the candidate
+                if (SR) {
+                    // query i is suffix token L - S + i of its candidate: suffix keys 0 .. L - S + i
+                    const int c = b - t.b_first, j = p.fd_cpb.div(c);
+                    k_own += j;
+                    lo_sfx = (c - j * p.cpb) * p.Spad;
+                    hi_sfx = lo_sfx + suffix_tokens(p.suffix_len, b, p.S, p.Skv) - p.S + i;
+                } else {
+                    lo_sfx = (b - t.b_first) * p.S;  // first suffix column of this row's candidate
+                    hi_sfx = lo_sfx + i;             // causal: suffix keys 0..i
+                }
             }
             lsum = 0.f;
 #pragma unroll 1
-            for (int k = 0; k < nitems && ok; ++k) {
+            for (int k = 0; k < nitems && ok; ++k, ++item) {
                 {
-                    const int item = tl * nitems + k, slot = item % kSlots;
+                    const int slot = item % kSlots;
                     const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN + wg * kPiece;
                     // valid columns of this row: [lo, hi].  Padding rows of a tile take part in prefix
                     // blocks like real rows (their scores are finite and never stored) and see no
@@ -585,6 +672,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         n = prefix_block_rows(p, k);
                         lo = 0;
                         hi = min(kBlockN, p.P - k * kBlockN) - 1;
+                    } else if (SR) {
+                        n = sfx_block_rows(p, t.nc, k - p.nblk_p);
+                        lo = k == k_own ? lo_sfx : 1;  // other candidates' blocks: nothing visible
+                        hi = k == k_own ? hi_sfx : 0;
                     } else {
                         n = t.n_sfx;
                         lo = lo_sfx;
@@ -745,6 +836,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 
 struct TilePlan {
     bool ok;
+    int mode;   // kernel template MODE: 0 rings, 1 resident prefix, 2 suffix-ring
+    int cbox, Spad, cpb;  // suffix-ring mode: candidates per tile, rows per candidate in a block, candidates per block
     int tile_rows, seg_rows, tiles_per_group, sfx_rows;
     int nblk_p, tail_rows, resident, stages, alias_stage;
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml, smem_bytes;
@@ -754,7 +847,44 @@ struct TilePlan {
 // candidates a tile can touch fit one 128-key block (candidates x S <= 128) -- and lays out shared
 // memory: all prefix blocks of a KV head if they fit beside the other buffers (resident mode), else
 // rings of 2..4 block stages.
-TilePlan plan_tiles(const Dims &dm)
+// Suffix-ring mode: a tile is the largest run of whole candidates with at most 128 rows; the
+// suffix keys follow the prefix blocks through K/V rings, 128 / Spad candidates per block.
+TilePlan plan_suffix_ring(const Dims &dm)
+{
+    TilePlan pl;
+    memset(&pl, 0, sizeof(pl));
+    const int Rg = dm.n_rep * dm.S;
+    if (Rg > kTileM || dm.Skv > kBlockN) return pl;
+    pl.mode = 2;
+    pl.Spad = round_up(dm.Skv, 8);
+    pl.cpb = kBlockN / pl.Spad;
+    pl.cbox = kTileM / Rg < dm.B ? kTileM / Rg : dm.B;
+    pl.tile_rows = pl.seg_rows = Rg * pl.cbox;
+    pl.tiles_per_group = (dm.B + pl.cbox - 1) / pl.cbox;
+    pl.nblk_p = (dm.P + kBlockN - 1) / kBlockN;
+    pl.tail_rows = pl.nblk_p ? round_up(dm.P - (pl.nblk_p - 1) * kBlockN, 16) : 0;
+    const int slabs = dm.d / 64;
+    const int tile_bytes = slabs * kTileM * 128;
+    const int ml_bytes = 4 * kGroups * kTileM * 4;
+    const int stage_bytes = slabs * kStagingBytes;
+    const int fixed = tile_bytes /*Q*/ + stage_bytes + ml_bytes + 64 + kBarBytes;
+    int st = (kMaxSmem - fixed) / (2 * tile_bytes);
+    if (st > kMaxStages) st = kMaxStages;
+    if (st < 1) return pl;
+    pl.stages = st;
+    pl.off_pk = 0;
+    pl.off_pv = st * tile_bytes;
+    pl.off_q = 2 * st * tile_bytes;
+    pl.off_sk = pl.off_sv = pl.off_stage = pl.off_q + tile_bytes;  // no suffix buffers of their own
+    pl.off_bar = pl.off_stage + stage_bytes;
+    pl.off_misc = pl.off_bar + kBarBytes;
+    pl.off_ml = pl.off_misc + 64;
+    pl.smem_bytes = pl.off_ml + ml_bytes;
+    pl.ok = pl.smem_bytes <= kMaxSmem;
+    return pl;
+}
+
+TilePlan plan_base(const Dims &dm)
 {
     TilePlan pl;
     memset(&pl, 0, sizeof(pl));
@@ -806,7 +936,19 @@ TilePlan plan_tiles(const Dims &dm)
     pl.off_ml = pl.off_misc + 64;
     pl.smem_bytes = pl.off_ml + ml_bytes;
     pl.ok = pl.smem_bytes <= kMaxSmem;
+    pl.mode = pl.resident ? 1 : 0;
     return pl;
+}
+
+// The full-suffix operator takes the tiling with the suffix in one block when it has one; the
+// decode-shaped operator, and full-suffix shapes that tiling cannot take, go to suffix-ring mode.
+TilePlan plan_tiles(const Dims &dm)
+{
+    if (dm.Skv == dm.S && !dm.ragged) {
+        const TilePlan pl = plan_base(dm);
+        if (pl.ok) return pl;
+    }
+    return plan_suffix_ring(dm);
 }
 
 template <int D>
@@ -825,13 +967,17 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
         cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Rg, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
         cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)Rg * D * 2, (cuuint64_t)dm.Hkv * Rg * D * 2};
         cuuint32_t box[4] = {64, (cuuint32_t)plan.seg_rows, 1, 1};
+        if (plan.mode == 2) {  // one box = the whole candidates of a tile
+            box[1] = (cuuint32_t)Rg;
+            box[3] = (cuuint32_t)plan.cbox;
+        }
         if (!encode_map(&tm_q, a.q, 4, dims, str, box)) return cudaErrorInvalidValue;
         if (!encode_map(&tm_out, a.out, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
     {
-        cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)dm.S, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
-        cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)dm.S * D * 2, (cuuint64_t)dm.Hkv * dm.S * D * 2};
-        cuuint32_t box[4] = {64, (cuuint32_t)dm.S, 1, 1};
+        cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)dm.Skv, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
+        cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)dm.Skv * D * 2, (cuuint64_t)dm.Hkv * dm.Skv * D * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)dm.Skv, 1, 1};
         if (!encode_map(&tm_sk, a.suffix_k, 4, dims, str, box)) return cudaErrorInvalidValue;
         if (!encode_map(&tm_sv, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
@@ -866,16 +1012,21 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.stages = plan.stages > 0 ? plan.stages : 1;
     p.sfx_rows = plan.sfx_rows;
     p.alias_stage = plan.alias_stage;
+    p.suffix_len = a.suffix_len;
+    p.Skv = dm.Skv;
+    p.Spad = plan.Spad > 0 ? plan.Spad : 8;
+    p.cpb = plan.cpb > 0 ? plan.cpb : 1;
+    p.fd_cpb.init(p.cpb);
     p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_sk = plan.off_sk;
     p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
     p.off_ml = plan.off_ml;
 
-    auto kernel = plan.resident ? tc_fwd_kernel<D, true> : tc_fwd_kernel<D, false>;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[plan.resident]) {
+    auto kernel = plan.mode == 1 ? tc_fwd_kernel<D, 1> : plan.mode == 2 ? tc_fwd_kernel<D, 2> : tc_fwd_kernel<D, 0>;
+    static bool attr_set[3] = {false, false, false};
+    if (!attr_set[plan.mode]) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
-        attr_set[plan.resident] = true;
+        attr_set[plan.mode] = true;
     }
     cudaError_t e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), stream);
     if (e != cudaSuccess) return e;
@@ -915,7 +1066,6 @@ extern "C" int pskv_debug_read_trace(long long *host, int max_events)
 
 bool tc_fwd_supported(const Dims &dm)
 {
-    if (dm.Skv != dm.S || dm.ragged) return false;  // full-suffix operator only
     if (dm.d != 64 && dm.d != 128) return false;
     if ((long long)dm.B * dm.n_rep * dm.S > 2000000000ll) return false;  // flat row index fits an int
     return plan_tiles(dm).ok;
