@@ -476,6 +476,37 @@ def detail_runs(pskv, device, peaks):
     res["C2_multi_8x64"] = {"prefix_len": lens,
                             "fwd": {"ms": ms_f, "tflops": fl_f / ms_f / 1e9, "candidates_per_s": w.B / ms_f * 1e3},
                             "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
+    del q, sk, sv, do, pk, pv, out, lse, dq, dk, dv
+    torch.cuda.empty_cache()
+    # Decode-shaped variant at the C2 layer shape: one new token per candidate on top of a suffix cache of
+    # up to 48 tokens (uniform ragged lengths), forward only (the attacks that grow suffixes token by token
+    # are gradient-free).  The call is bound by reading each candidate's suffix K/V once, so it is reported
+    # against the HBM roofline; four input sets are rotated so that every call reads from HBM, not L2.
+    for tag, Bd in (("C2_decode_1of48_B512", 512), ("C2_decode_1of48_B2048", 2048)):
+        Sq, Skv = 1, 48
+        sets = []
+        for i in range(4):
+            sets.append((draw(Bd, w.Hq, Sq, w.d), draw(Bd, w.Hkv, Skv, w.d), draw(Bd, w.Hkv, Skv, w.d),
+                         torch.randint(Sq, Skv + 1, (Bd,), generator=gen, dtype=torch.int32).to(device)))
+        pk, pv = draw(w.Hkv, w.P, w.d), draw(w.Hkv, w.P, w.d)
+        out = torch.empty_like(sets[0][0])
+        lse = torch.empty((Bd, w.Hq, Sq), dtype=torch.float32, device=device)
+        ws = torch.empty(256, dtype=torch.uint8, device=device)
+        turn = [0]
+
+        def dfwd():
+            qd, skd, svd, ln = sets[turn[0] % 4]
+            turn[0] += 1
+            pskv.pskv_attn_fwd_decode(qd, pk, pv, skd, svd, ln, w.scale, out=out, lse=lse, workspace=ws)
+
+        dfwd()
+        ms = time_calls(dfwd, 40, 4)
+        nbytes = (2 * Bd * w.Hq * Sq * w.d + 2 * Bd * w.Hkv * Skv * w.d + 2 * w.Hkv * w.P * w.d) * 2 + Bd * w.Hq * Sq * 4
+        res[tag] = {"Sq": Sq, "Skv": Skv, "B": Bd,
+                    "fwd": {"ms": ms, "candidates_per_s": Bd / ms * 1e3, "hbm_gbs": nbytes / ms / 1e6,
+                            "pct_hbm_peak": 100 * nbytes / ms / 1e6 / peaks["hbm_gbs"]}}
+        del sets, pk, pv, out, lse
+        torch.cuda.empty_cache()
     return res
 
 
