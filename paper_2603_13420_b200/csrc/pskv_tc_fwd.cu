@@ -70,6 +70,8 @@ struct TcFwdParams {
     int Spad;             // Skv rounded up to 8: rows a candidate takes inside a suffix block
     int cpb;              // candidates per suffix block: 128 / Spad
     FastDiv fd_cpb;
+    int long_sfx;         // 1: a tile lies inside ONE candidate and that candidate's suffix keys come in
+                          //    128-key blocks (suffix caches or row groups beyond 128); 0: whole-candidate tiles
     // shared-memory carve-up (byte offsets from the 1024-byte aligned base)
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml;
 };
@@ -122,6 +124,22 @@ __device__ __forceinline__ int sfx_block_cands(const TcFwdParams &p, int nc, int
 __device__ __forceinline__ int sfx_block_rows(const TcFwdParams &p, int nc, int j)
 {
     return (sfx_block_cands(p, nc, j) * p.Spad + 15) & ~15;
+}
+
+// Suffix-ring mode with long suffixes: the tile's rows belong to one candidate; it needs that
+// candidate's suffix keys up to the last one any of its rows may see, in blocks of 128.
+__device__ __forceinline__ int sfx_blocks_long(const TcFwdParams &p, const TileInfo &t)
+{
+    const int r0 = t.R0 - t.b_first * p.Rg;
+    const int s0 = r0 - p.fd_S.div(r0) * p.S;  // query index of the tile's first row
+    const int s_max = (s0 + t.rows > p.S) ? p.S - 1 : s0 + t.rows - 1;  // rows wrap into the next head
+    const int pos = suffix_tokens(p.suffix_len, t.b_first, p.S, p.Skv) - p.S + s_max;
+    return (pos >> 7) + 1;
+}
+// MMA N of long-suffix block j (its 128-row box is zero-filled past the end of the cache)
+__device__ __forceinline__ int sfx_long_rows(const TcFwdParams &p, int j)
+{
+    return min(kBlockN, (p.Skv - j * kBlockN + 15) & ~15);
 }
 
 // MODE 1: all prefix blocks of a KV head stay in shared memory; MODE 0: they stream through rings,
@@ -185,7 +203,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
     const int n_tiles = t_end - t_begin;
     // items of a tile: prefix blocks + the suffix block(s)
-    auto items_of = [&](const TileInfo &t) { return p.nblk_p + (SR ? p.fd_cpb.div(t.nc + p.cpb - 1) : 1); };
+    auto items_of = [&](const TileInfo &t) {
+        return p.nblk_p + (!SR ? 1 : p.long_sfx ? sfx_blocks_long(p, t) : p.fd_cpb.div(t.nc + p.cpb - 1));
+    };
     const int g_first = p.fd_tpg.div(t_begin);
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
@@ -302,16 +322,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
                                         p.status, kErrProducerK);
                     if (!ok) break;
-                    const int ncb = sfx_block_cands(p, t.nc, j);
-                    const int slab = sfx_block_rows(p, t.nc, j) * 128;
-                    if (elect_one_sync()) {
-                        mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(ncb * C::kSlabs * p.Skv * 128));
-#pragma unroll 1
-                        for (int c = 0; c < ncb; ++c)
+                    if (p.long_sfx) {
+                        // keys [128 j, 128 j + 128) of the tile's candidate; rows past the cache are zero-filled
+                        if (elect_one_sync()) {
+                            mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)C::kTileBytes);
 #pragma unroll 1
                             for (int sl = 0; sl < C::kSlabs; ++sl)
-                                tma_load_4d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab + c * p.Spad * 128, &tm_sk,
-                                            bar(kBarKFull + ks), sl * 64, 0, t.g, t.b_first + j * p.cpb + c);
+                                tma_load_4d(sbase + p.off_pk + ks * C::kTileBytes + sl * C::kSlabBytes, &tm_sk,
+                                            bar(kBarKFull + ks), sl * 64, j * kBlockN, t.g, t.b_first);
+                        }
+                    } else {
+                        const int ncb = sfx_block_cands(p, t.nc, j);
+                        const int slab = sfx_block_rows(p, t.nc, j) * 128;
+                        if (elect_one_sync()) {
+                            mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(ncb * C::kSlabs * p.Skv * 128));
+#pragma unroll 1
+                            for (int c = 0; c < ncb; ++c)
+#pragma unroll 1
+                                for (int sl = 0; sl < C::kSlabs; ++sl)
+                                    tma_load_4d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab + c * p.Spad * 128,
+                                                &tm_sk, bar(kBarKFull + ks), sl * 64, 0, t.g, t.b_first + j * p.cpb + c);
+                        }
                     }
                     __syncwarp();
                     ++kload;
@@ -390,16 +421,27 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (SR && k >= p.nblk_p) {
                         // a suffix V block: one box of Skv rows per candidate, Spad rows apart
                         const int j = k - p.nblk_p;
-                        const int ncb = sfx_block_cands(p, t.nc, j);
-                        const int slab = sfx_block_rows(p, t.nc, j) * 128;
-                        if (elect_one_sync()) {
-                            mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(ncb * C::kSlabs * p.Skv * 128));
-#pragma unroll 1
-                            for (int c = 0; c < ncb; ++c)
+                        if (p.long_sfx) {
+                            if (elect_one_sync()) {
+                                mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)C::kTileBytes);
 #pragma unroll 1
                                 for (int sl = 0; sl < C::kSlabs; ++sl)
-                                    tma_load_4d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab + c * p.Spad * 128,
-                                                &tm_sv, bar(kBarVFull + vs), sl * 64, 0, t.g, t.b_first + j * p.cpb + c);
+                                    tma_load_4d(sbase + p.off_pv + vs * C::kTileBytes + sl * C::kSlabBytes, &tm_sv,
+                                                bar(kBarVFull + vs), sl * 64, j * kBlockN, t.g, t.b_first);
+                            }
+                        } else {
+                            const int ncb = sfx_block_cands(p, t.nc, j);
+                            const int slab = sfx_block_rows(p, t.nc, j) * 128;
+                            if (elect_one_sync()) {
+                                mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(ncb * C::kSlabs * p.Skv * 128));
+#pragma unroll 1
+                                for (int c = 0; c < ncb; ++c)
+#pragma unroll 1
+                                    for (int sl = 0; sl < C::kSlabs; ++sl)
+                                        tma_load_4d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab + c * p.Spad * 128,
+                                                    &tm_sv, bar(kBarVFull + vs), sl * 64, 0, t.g,
+                                                    t.b_first + j * p.cpb + c);
+                            }
                         }
                     } else {
                         const bool tail = k == p.nblk_p - 1;
@@ -494,8 +536,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             uint32_t kaddr;
             int n, slab;
             if (k < p.nblk_p || SR) {
-                n = k < p.nblk_p ? prefix_block_rows(p, k) : sfx_block_rows(p, t.nc, k - p.nblk_p);
-                slab = n * 128;
+                n = k < p.nblk_p ? prefix_block_rows(p, k)
+                    : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
+                slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
                 if (RES) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaQk);
@@ -564,8 +607,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             uint32_t vaddr;
             int n, slab;
             if (k < p.nblk_p || SR) {
-                n = k < p.nblk_p ? prefix_block_rows(p, k) : sfx_block_rows(p, t.nc, k - p.nblk_p);
-                slab = n * 128;
+                n = k < p.nblk_p ? prefix_block_rows(p, k)
+                    : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
+                slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
                 if (RES) {
                     if (t.first_of_g)
                         ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaPv);
@@ -649,10 +693,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int i = r - p.fd_S.div(r) * p.S;  // query index inside the candidate
                 if (SR) {
                     // query i is suffix token L - S + i of its candidate: suffix keys 0 .. L - S + i
-                    const int c = b - t.b_first, j = p.fd_cpb.div(c);
-                    k_own += j;
-                    lo_sfx = (c - j * p.cpb) * p.Spad;
-                    hi_sfx = lo_sfx + suffix_tokens(p.suffix_len, b, p.S, p.Skv) - p.S + i;
+                    const int pos = suffix_tokens(p.suffix_len, b, p.S, p.Skv) - p.S + i;
+                    if (p.long_sfx) {
+                        lo_sfx = 0;
+                        hi_sfx = pos;  // counted from the candidate's first key; block j starts at 128 j
+                    } else {
+                        const int c = b - t.b_first, j = p.fd_cpb.div(c);
+                        k_own += j;
+                        lo_sfx = (c - j * p.cpb) * p.Spad;
+                        hi_sfx = lo_sfx + pos;
+                    }
                 } else {
                     lo_sfx = (b - t.b_first) * p.S;  // first suffix column of this row's candidate
                     hi_sfx = lo_sfx + i;             // causal: suffix keys 0..i
@@ -672,6 +722,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         n = prefix_block_rows(p, k);
                         lo = 0;
                         hi = min(kBlockN, p.P - k * kBlockN) - 1;
+                    } else if (SR && p.long_sfx) {
+                        n = sfx_long_rows(p, k - p.nblk_p);
+                        lo = lo_sfx;  // 0 for a real row, 1 (with hi 0 - ...: nothing visible) for padding
+                        hi = lo_sfx == 0 ? hi_sfx - (k - p.nblk_p) * kBlockN : 0;
                     } else if (SR) {
                         n = sfx_block_rows(p, t.nc, k - p.nblk_p);
                         lo = k == k_own ? lo_sfx : 1;  // other candidates' blocks: nothing visible
@@ -838,6 +892,7 @@ struct TilePlan {
     bool ok;
     int mode;   // kernel template MODE: 0 rings, 1 resident prefix, 2 suffix-ring
     int cbox, Spad, cpb;  // suffix-ring mode: candidates per tile, rows per candidate in a block, candidates per block
+    int long_sfx;         // suffix-ring mode: tiles inside one candidate, its suffix keys in 128-key blocks
     int tile_rows, seg_rows, tiles_per_group, sfx_rows;
     int nblk_p, tail_rows, resident, stages, alias_stage;
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml, smem_bytes;
@@ -854,13 +909,29 @@ TilePlan plan_suffix_ring(const Dims &dm)
     TilePlan pl;
     memset(&pl, 0, sizeof(pl));
     const int Rg = dm.n_rep * dm.S;
-    if (Rg > kTileM || dm.Skv > kBlockN) return pl;
     pl.mode = 2;
-    pl.Spad = round_up(dm.Skv, 8);
-    pl.cpb = kBlockN / pl.Spad;
-    pl.cbox = kTileM / Rg < dm.B ? kTileM / Rg : dm.B;
-    pl.tile_rows = pl.seg_rows = Rg * pl.cbox;
-    pl.tiles_per_group = (dm.B + pl.cbox - 1) / pl.cbox;
+    if (Rg > kTileM || dm.Skv > kBlockN) {
+        // long suffixes: a tile is a run of rows inside one candidate (the largest divisor of its
+        // row count that fits a tile), the candidate's suffix keys come in blocks of 128
+        int rows = 0;
+        for (int m = kTileM; m >= 16 && !rows; --m)
+            if (Rg % m == 0) rows = m;
+        if (!rows && Rg <= kTileM) rows = Rg;
+        if (!rows) return pl;  // no usable divisor: the general kernels take the shape
+        if ((long long)dm.B * (Rg / rows) > 2000000000ll) return pl;
+        pl.long_sfx = 1;
+        pl.Spad = 8;
+        pl.cpb = 1;
+        pl.cbox = 1;
+        pl.tile_rows = pl.seg_rows = rows;
+        pl.tiles_per_group = dm.B * (Rg / rows);
+    } else {
+        pl.Spad = round_up(dm.Skv, 8);
+        pl.cpb = kBlockN / pl.Spad;
+        pl.cbox = kTileM / Rg < dm.B ? kTileM / Rg : dm.B;
+        pl.tile_rows = pl.seg_rows = Rg * pl.cbox;
+        pl.tiles_per_group = (dm.B + pl.cbox - 1) / pl.cbox;
+    }
     pl.nblk_p = (dm.P + kBlockN - 1) / kBlockN;
     pl.tail_rows = pl.nblk_p ? round_up(dm.P - (pl.nblk_p - 1) * kBlockN, 16) : 0;
     const int slabs = dm.d / 64;
@@ -967,8 +1038,8 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
         cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Rg, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
         cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)Rg * D * 2, (cuuint64_t)dm.Hkv * Rg * D * 2};
         cuuint32_t box[4] = {64, (cuuint32_t)plan.seg_rows, 1, 1};
-        if (plan.mode == 2) {  // one box = the whole candidates of a tile
-            box[1] = (cuuint32_t)Rg;
+        if (plan.mode == 2) {  // one box = the whole candidates of a tile, or the tile's rows of one candidate
+            box[1] = (cuuint32_t)(plan.long_sfx ? plan.tile_rows : Rg);
             box[3] = (cuuint32_t)plan.cbox;
         }
         if (!encode_map(&tm_q, a.q, 4, dims, str, box)) return cudaErrorInvalidValue;
@@ -977,7 +1048,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     {
         cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)dm.Skv, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
         cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)dm.Skv * D * 2, (cuuint64_t)dm.Hkv * dm.Skv * D * 2};
-        cuuint32_t box[4] = {64, (cuuint32_t)dm.Skv, 1, 1};
+        cuuint32_t box[4] = {64, (cuuint32_t)(plan.long_sfx ? kBlockN : dm.Skv), 1, 1};
         if (!encode_map(&tm_sk, a.suffix_k, 4, dims, str, box)) return cudaErrorInvalidValue;
         if (!encode_map(&tm_sv, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
@@ -1017,6 +1088,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.Spad = plan.Spad > 0 ? plan.Spad : 8;
     p.cpb = plan.cpb > 0 ? plan.cpb : 1;
     p.fd_cpb.init(p.cpb);
+    p.long_sfx = plan.long_sfx;
     p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_sk = plan.off_sk;
     p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
     p.off_ml = plan.off_ml;

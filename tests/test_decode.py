@@ -44,6 +44,9 @@ CASES = [
     (6, 4, 2, 2, 150, 64, 128, True),       # suffix cache longer than one key block
     (9, 8, 2, 2, 24, 0, 128, True),         # no prefix
     (20, 16, 4, 16, 64, 700, 128, False),   # prefix streamed in several blocks
+    (4, 8, 2, 16, 300, 64, 128, True),      # long suffix cache: several 128-key blocks per candidate
+    (6, 32, 8, 48, 64, 256, 128, True),     # more than 128 query rows per candidate and KV head
+    (3, 8, 8, 24, 200, 0, 64, True),        # head dim 64, long cache, no prefix
 ]
 
 

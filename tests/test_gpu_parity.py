@@ -75,6 +75,10 @@ EDGE = [
     (2, 8, 2, 64, 64, 128),   # 256 rows per group: two full row tiles of the suffix-gradient kernel, 64 keys
     (2, 8, 1, 40, 32, 128),   # 320 rows per group: two and a half row tiles, n_rep = 8
     (300, 4, 4, 16, 48, 128), # more groups than SMs: every persistent CTA walks over several groups
+    # suffixes beyond one key block (forward: tiles inside one candidate, suffix keys in 128-key blocks)
+    (2, 8, 2, 256, 100, 128), # 1024 rows per group, two suffix blocks, causal limit inside each
+    (1, 8, 2, 512, 0, 128),   # one sequence, no prefix: plain causal self-attention (a prefix prefill)
+    (2, 4, 4, 131, 20, 128),  # a prime row count per group: no tiling, general kernels
 ]
 
 
