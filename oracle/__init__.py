@@ -47,6 +47,8 @@ def _load():
         lib.pskv_oracle_attn_fwd.restype = ctypes.c_int
         lib.pskv_oracle_attn_bwd.argtypes = [dp] * 6 + [ctypes.c_double] + [dp] * 3 + ints
         lib.pskv_oracle_attn_bwd.restype = ctypes.c_int
+        lib.pskv_oracle_attn_bwd_lse.argtypes = [dp] * 7 + [ctypes.c_double] + [dp] * 3 + ints
+        lib.pskv_oracle_attn_bwd_lse.restype = ctypes.c_int
         ip = ctypes.POINTER(ctypes.c_int)
         ints7 = [ctypes.c_int] * 7
         lib.pskv_oracle_attn_fwd_multi.argtypes = [dp] * 3 + [ip] + [dp] * 2 + [ctypes.c_double] + [dp] * 2 + ints7
@@ -119,6 +121,26 @@ def attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, scale):
                                       B, Hq, Hkv, S, P, d)
     if rc != 0:
         raise RuntimeError("pskv_oracle_attn_bwd failed with code %d" % rc)
+    return dq, dk, dv
+
+
+def attn_bwd_lse(dout, dlse, q, prefix_k, prefix_v, suffix_k, suffix_v, scale):
+    """dq, dk_suffix, dv_suffix (fp64) of L = sum(out * dout) + sum(lse * dlse); prefix K/V frozen."""
+    B, Hq, Hkv, S, P, d = _dims(q, prefix_k, suffix_k)
+    do = _f64(dout, (B, Hq, S, d))
+    dl = _f64(dlse, (B, Hq, S))
+    q = _f64(q, (B, Hq, S, d))
+    pk = _f64(prefix_k, (Hkv, P, d))
+    pv = _f64(prefix_v, (Hkv, P, d))
+    sk = _f64(suffix_k, (B, Hkv, S, d))
+    sv = _f64(suffix_v, (B, Hkv, S, d))
+    dq = np.empty((B, Hq, S, d), dtype=np.float64)
+    dk = np.empty((B, Hkv, S, d), dtype=np.float64)
+    dv = np.empty((B, Hkv, S, d), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_bwd_lse(_ptr(do), _ptr(dl), _ptr(q), _ptr(pk), _ptr(pv), _ptr(sk), _ptr(sv),
+                                          float(scale), _ptr(dq), _ptr(dk), _ptr(dv), B, Hq, Hkv, S, P, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_bwd_lse failed with code %d" % rc)
     return dq, dk, dv
 
 

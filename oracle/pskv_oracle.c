@@ -134,7 +134,7 @@ int pskv_oracle_attn_fwd(const double *q, const double *prefix_k, const double *
  * suffix side are needed), so contributions to prefix keys are discarded.
  * The forward quantities (p, out) are recomputed here in fp64.
  */
-int pskv_oracle_attn_bwd(const double *dout, const double *q,
+static int attn_bwd_impl(const double *dout, const double *dlse, const double *q,
                          const double *prefix_k, const double *prefix_v,
                          const double *suffix_k, const double *suffix_v, double scale,
                          double *dq, double *dk_suffix, double *dv_suffix,
@@ -172,12 +172,13 @@ int pskv_oracle_attn_bwd(const double *dout, const double *q,
                             for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
                         double D = 0.0;
                         for (int c = 0; c < d; ++c) D += go[c] * o[c];
+                        const double gl = dlse ? dlse[row] : 0.0;  /* d lse / d s_j = p_j */
                         double *dqr = dq + row * d;
                         for (int c = 0; c < d; ++c) dqr[c] = 0.0;
                         for (int j = 0; j < n_vis; ++j) {
                             double dp = 0.0;
                             for (int c = 0; c < d; ++c) dp += go[c] * Vf[(size_t)j * d + c];
-                            const double ds = p[j] * (dp - D);
+                            const double ds = p[j] * (dp - D + gl);
                             for (int c = 0; c < d; ++c) dqr[c] += scale * ds * Kf[(size_t)j * d + c];
                             if (j >= P) {
                                 const int t = j - P;
@@ -197,6 +198,34 @@ int pskv_oracle_attn_bwd(const double *dout, const double *q,
         free(o);
     }
     return failed ? 2 : 0;
+}
+
+int pskv_oracle_attn_bwd(const double *dout, const double *q,
+                         const double *prefix_k, const double *prefix_v,
+                         const double *suffix_k, const double *suffix_v, double scale,
+                         double *dq, double *dk_suffix, double *dv_suffix,
+                         int B, int Hq, int Hkv, int S, int P, int d)
+{
+    return attn_bwd_impl(dout, NULL, q, prefix_k, prefix_v, suffix_k, suffix_v, scale, dq, dk_suffix,
+                         dv_suffix, B, Hq, Hkv, S, P, d);
+}
+
+/*
+ * Backward of L = sum(out * dout) + sum(lse * dlse): the log-sum-exp is a second output of the
+ * forward pass, and a caller that uses it (to merge this call's result with another partial
+ * attention result, or in a loss) sends a gradient back through it.  Since lse = ln sum_j exp(s_j),
+ * d lse / d s_j = p_j, so the only change to the closed form above is ds_j = p_j (dp_j - D + dlse);
+ * dV receives nothing from lse.  dlse is [B][Hq][S].
+ */
+int pskv_oracle_attn_bwd_lse(const double *dout, const double *dlse, const double *q,
+                             const double *prefix_k, const double *prefix_v,
+                             const double *suffix_k, const double *suffix_v, double scale,
+                             double *dq, double *dk_suffix, double *dv_suffix,
+                             int B, int Hq, int Hkv, int S, int P, int d)
+{
+    if (!dlse) return 1;
+    return attn_bwd_impl(dout, dlse, q, prefix_k, prefix_v, suffix_k, suffix_v, scale, dq, dk_suffix,
+                         dv_suffix, B, Hq, Hkv, S, P, d);
 }
 
 /*
