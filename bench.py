@@ -508,6 +508,24 @@ def detail_runs(pskv, device, peaks):
                             "pct_hbm_peak": 100 * nbytes / ms / 1e6 / peaks["hbm_gbs"]}}
         del sets, pk, pv, out, lse
         torch.cuda.empty_cache()
+    # Prefix prefill, attention step: the causal self-attention of one 2048-token sequence (B = 1, P = 0, the
+    # sequence's K/V passed as the suffix), i.e. what produces a C3-sized prefix cache in the first place.
+    w3 = wl.WORKLOADS["C3"]
+    Sp = w3.P
+    qp, kp, vp = draw(1, w3.Hq, Sp, w3.d), draw(1, w3.Hkv, Sp, w3.d), draw(1, w3.Hkv, Sp, w3.d)
+    outp = torch.empty_like(qp)
+    lsep = torch.empty((1, w3.Hq, Sp), dtype=torch.float32, device=device)
+    wsp = torch.empty(256, dtype=torch.uint8, device=device)
+
+    def prefill():
+        pskv.pskv_attn_fwd(qp, None, None, kp, vp, w3.scale, out=outp, lse=lsep, workspace=wsp)
+
+    prefill()
+    ms = time_calls(prefill, 40, 4)
+    fl = 4.0 * w3.d * ((Sp + 1) / 2) * w3.Hq * Sp
+    res["prefix_prefill_P%d" % Sp] = {"fwd": {"ms": ms, "tflops": fl / ms / 1e9,
+                                              "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
+                                              "kernel_family": pskv.pskv_kernel_family(0, 1, w3.Hq, w3.Hkv, Sp, 0, w3.d)}}
     return res
 
 

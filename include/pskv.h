@@ -51,6 +51,9 @@ size_t pskv_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d
  *   lse[b,h,i]   = ln sum_j exp(s_j)                      (natural log, scale included)
  *   out[b,h,i,:] = sum_j exp(s_j - lse) V_j                (rounded to bf16)
  * Inputs are read-only; out and lse are fully overwritten.  Accumulation is fp32.
+ * Any S is legal.  With B = 1 and P = 0 the call is the causal self-attention of one sequence whose
+ * keys and values are passed as suffix_k / suffix_v: the attention step of the prefill that produces a
+ * prefix cache in the first place.
  */
 pskv_status pskv_attn_fwd(const void *q,        /* bf16 [B,Hq,S,d]  */
                           const void *prefix_k, /* bf16 [Hkv,P,d]   (may be NULL when P == 0) */
@@ -75,7 +78,8 @@ size_t pskv_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d
  *   dk_suffix[b,g,t,:] = scale * sum over heads h of g and rows i >= t of ds_{P+t} q[b,h,i,:]
  *   dv_suffix[b,g,t,:] =         sum over the same (h, i) of p_{P+t} dout[b,h,i,:]
  * `out` and `lse` are the forward results for the same inputs.  No gradient is
- * produced for prefix_k / prefix_v, and lse carries no incoming gradient.
+ * produced for prefix_k / prefix_v, and lse carries no incoming gradient here (pskv_attn_bwd_lse
+ * takes one).
  * The three outputs are fully overwritten.
  */
 pskv_status pskv_attn_bwd(const void *dout,     /* bf16 [B,Hq,S,d]  */
@@ -89,6 +93,24 @@ pskv_status pskv_attn_bwd(const void *dout,     /* bf16 [B,Hq,S,d]  */
                           void *dv_suffix,      /* bf16 [B,Hkv,S,d] */
                           int B, int Hq, int Hkv, int S, int P, int d,
                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * pskv_attn_bwd with a gradient arriving on the log-sum-exp as well: the backward of
+ * L = sum(out * dout) + sum(lse * dlse).  lse is a second output of the forward call; a caller that
+ * merges this call's result with another partial attention result by their log-sum-exps, or that uses
+ * lse in a loss, sends a gradient back through it.  Since d lse / d s_j = p_j, the formulas of
+ * pskv_attn_bwd hold with ds_j = p_j (<dout, V_j> - D + dlse[b,h,i]); dv_suffix is unaffected.
+ * dlse is fp32 [B,Hq,S], device, 16-byte aligned, read-only, and must not be NULL (use pskv_attn_bwd).
+ * Everything else -- arguments, workspace size, error codes -- is as in pskv_attn_bwd.
+ */
+pskv_status pskv_attn_bwd_lse(const void *dout,   /* bf16 [B,Hq,S,d] */
+                              const float *dlse,  /* fp32 [B,Hq,S]   */
+                              const void *q, const void *prefix_k, const void *prefix_v,
+                              const void *suffix_k, const void *suffix_v,
+                              const void *out, const float *lse, float scale,
+                              void *dq, void *dk_suffix, void *dv_suffix,
+                              int B, int Hq, int Hkv, int S, int P, int d,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * pskv_attn_bwd without a workspace argument.  (The paper has no counterpart; this is a

@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.pskv_attn_fwd.restype = ci
         L.pskv_attn_bwd.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp, sz, vp]
         L.pskv_attn_bwd.restype = ci
+        L.pskv_attn_bwd_lse.argtypes = [vp] * 9 + [cf] + [vp] * 3 + six + [vp, sz, vp]
+        L.pskv_attn_bwd_lse.restype = ci
         seven = [ci] * 7
         L.pskv_attn_fwd_multi_workspace_bytes.argtypes = seven
         L.pskv_attn_fwd_multi_workspace_bytes.restype = sz
@@ -211,6 +213,28 @@ def pskv_attn_bwd(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, out, lse, sca
                              _ptr(ws), ws.numel() * ws.element_size(), _stream())
     if st != PSKV_OK:
         raise PskvError(st, "pskv_attn_bwd")
+    return dq, dk_suffix, dv_suffix
+
+
+def pskv_attn_bwd_lse(dout, dlse, q, prefix_k, prefix_v, suffix_k, suffix_v, out, lse, scale,
+                      dq=None, dk_suffix=None, dv_suffix=None, workspace=None):
+    """Backward of L = sum(out * dout) + sum(lse * dlse): pskv_attn_bwd with a gradient on lse (fp32 [B,Hq,S])."""
+    dims = _dims(q, prefix_k, suffix_k)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk_suffix is None:
+        dk_suffix = torch.empty_like(suffix_k)
+    if dv_suffix is None:
+        dv_suffix = torch.empty_like(suffix_v)
+    if dlse is None or dlse.dtype != torch.float32 or tuple(dlse.shape) != tuple(q.shape[:3]):
+        raise ValueError("dlse must be a float32 CUDA tensor of shape [B,Hq,S]")
+    ws = _workspace(pskv_attn_bwd_workspace_bytes(*dims), q.device, workspace)
+    st = lib().pskv_attn_bwd_lse(_ptr(dout), _ptr(dlse), _ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(suffix_k),
+                                 _ptr(suffix_v), _ptr(out), _ptr(lse), float(scale),
+                                 _ptr(dq), _ptr(dk_suffix), _ptr(dv_suffix), *dims,
+                                 _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_bwd_lse")
     return dq, dk_suffix, dv_suffix
 
 

@@ -253,9 +253,9 @@ pskv_status fwd_checked(const Dims &dm, const void *q, const void *prefix_k, con
     return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
 }
 
-pskv_status bwd_checked(const Dims &dm, const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
-                        const void *suffix_k, const void *suffix_v, const int *suffix_len, const void *out,
-                        const float *lse, float scale, void *dq, void *dk_suffix, void *dv_suffix, size_t need,
+pskv_status bwd_checked(const Dims &dm, const void *dout, const float *dlse, const void *q, const void *prefix_k,
+                        const void *prefix_v, const void *suffix_k, const void *suffix_v, const int *suffix_len,
+                        const void *out, const float *lse, float scale, void *dq, void *dk_suffix, void *dv_suffix, size_t need,
                         void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     if (!dout || !q || !suffix_k || !suffix_v || !out || !lse || !dq || !dk_suffix || !dv_suffix)
@@ -265,7 +265,7 @@ pskv_status bwd_checked(const Dims &dm, const void *dout, const void *q, const v
         !aligned16(suffix_k) || !aligned16(suffix_v) || !aligned16(out) || !aligned16(lse) ||
         !aligned16(dq) || !aligned16(dk_suffix) || !aligned16(dv_suffix))
         return PSKV_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(suffix_len) & 3u) != 0) return PSKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(suffix_len) & 3u) != 0 || !aligned16(dlse)) return PSKV_ERR_INVALID_ARG;
     if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
 
@@ -286,6 +286,7 @@ pskv_status bwd_checked(const Dims &dm, const void *dout, const void *q, const v
     a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix);
     a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix);
     a.row_dot = static_cast<float *>(workspace);
+    a.dlse = dlse;
     a.suffix_len = suffix_len;
     a.scale = scale;
     a.dims = dm;
@@ -318,9 +319,23 @@ pskv_status pskv_attn_bwd(const void *dout, const void *q, const void *prefix_k,
     Dims dm;
     pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
     if (st != PSKV_OK) return st;
-    return bwd_checked(dm, dout, q, prefix_k, prefix_v, suffix_k, suffix_v, nullptr, out, lse, scale, dq, dk_suffix,
-                       dv_suffix, pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d), workspace, workspace_bytes,
-                       cuda_stream);
+    return bwd_checked(dm, dout, nullptr, q, prefix_k, prefix_v, suffix_k, suffix_v, nullptr, out, lse, scale, dq,
+                       dk_suffix, dv_suffix, pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d), workspace,
+                       workspace_bytes, cuda_stream);
+}
+
+pskv_status pskv_attn_bwd_lse(const void *dout, const float *dlse, const void *q, const void *prefix_k,
+                              const void *prefix_v, const void *suffix_k, const void *suffix_v, const void *out,
+                              const float *lse, float scale, void *dq, void *dk_suffix, void *dv_suffix, int B, int Hq,
+                              int Hkv, int S, int P, int d, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return st;
+    if (!dlse) return PSKV_ERR_INVALID_ARG;
+    return bwd_checked(dm, dout, dlse, q, prefix_k, prefix_v, suffix_k, suffix_v, nullptr, out, lse, scale, dq,
+                       dk_suffix, dv_suffix, pskv_attn_bwd_workspace_bytes(B, Hq, Hkv, S, P, d), workspace,
+                       workspace_bytes, cuda_stream);
 }
 
 // ---- decode-shaped variant: the last Sq of each candidate's cached suffix tokens are the queries ------
@@ -360,8 +375,8 @@ pskv_status pskv_attn_bwd_decode(const void *dout, const void *q, const void *pr
     Dims dm;
     pskv_status st = check_dims_decode(B, Hq, Hkv, Sq, Skv, P, d, suffix_len != nullptr, &dm);
     if (st != PSKV_OK) return st;
-    return bwd_checked(dm, dout, q, prefix_k, prefix_v, suffix_k, suffix_v, suffix_len, out, lse, scale, dq, dk_suffix,
-                       dv_suffix, simt_bwd_workspace(dm), workspace, workspace_bytes, cuda_stream);
+    return bwd_checked(dm, dout, nullptr, q, prefix_k, prefix_v, suffix_k, suffix_v, suffix_len, out, lse, scale, dq,
+                       dk_suffix, dv_suffix, simt_bwd_workspace(dm), workspace, workspace_bytes, cuda_stream);
 }
 
 // ---- several instructions per call (suffix-centric alignment, Sec. 4.3) --------------------------
@@ -490,6 +505,7 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix) + i * s_part;
         a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix) + i * s_part;
         a.row_dot = static_cast<float *>(ws);
+        a.dlse = nullptr;
         a.suffix_len = nullptr;
         a.scale = scale;
         a.dims = dm;

@@ -40,7 +40,8 @@ struct BwdArgs {
     const __nv_bfloat16 *dout, *q, *prefix_k, *prefix_v, *suffix_k, *suffix_v, *out;
     const float *lse;
     __nv_bfloat16 *dq, *dk_suffix, *dv_suffix;
-    float *row_dot;  // workspace: D[b,h,i] = <dout, out>, fp32 [B*Hq*S]
+    float *row_dot;  // workspace: D[b,h,i] = <dout, out> - dlse[b,h,i], fp32 [B*Hq*S]
+    const float *dlse;  // gradient arriving on lse, fp32 [B*Hq*S], or nullptr (none)
     const int *suffix_len;  // as in FwdArgs
     float scale;
     Dims dims;

@@ -200,7 +200,8 @@ simt_bwd_dq_kernel(BwdArgs a)
     float dsum = 0.f;
 #pragma unroll
     for (int e = 0; e < D / 32; ++e) dsum = fmaf(o[e], do_s[warp][lane * (D / 32) + e], dsum);
-    const float Drow = warp_sum(dsum);
+    // d lse / d s_j = p_j, so a gradient on lse enters every ds_j = p_j (dp_j - D) as -D += dlse
+    const float Drow = warp_sum(dsum) - (a.dlse ? a.dlse[row] : 0.f);
     if (lane == 0) a.row_dot[row] = Drow;
 
     const float scale2 = a.scale * kLog2e;
@@ -236,7 +237,7 @@ simt_bwd_dq_kernel(BwdArgs a)
     store_slice<D>(a.dq + (size_t)row * D, lane, acc);
 }
 
-// D = <dout, out> for every query row.  A pure streaming pass over two tensors, so it is laid out
+// D = <dout, out> (minus the gradient arriving on lse, if any) for every query row.  A pure streaming pass over two tensors, so it is laid out
 // for bytes in flight: D/8 lanes share a row with one 16-byte load each per tensor, so a warp-wide
 // load covers 2 rows (d = 128) or 4 (d = 64), and every thread keeps kRowDotUnroll such loads of
 // both tensors outstanding.
@@ -275,7 +276,7 @@ simt_row_dot_kernel(BwdArgs a)
 #pragma unroll
         for (int off = kLanesPerRow / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         const long long row = first + u * kRowsPerLoad + sub;
-        if (lane % kLanesPerRow == 0 && row < rows) a.row_dot[row] = acc;
+        if (lane % kLanesPerRow == 0 && row < rows) a.row_dot[row] = acc - (a.dlse ? a.dlse[row] : 0.f);
     }
 }
 
