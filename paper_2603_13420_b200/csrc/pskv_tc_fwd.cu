@@ -70,6 +70,7 @@ struct TcFwdParams {
     int Spad;             // Skv rounded up to 8: rows a candidate takes inside a suffix block
     int cpb;              // candidates per suffix block: 128 / Spad
     FastDiv fd_cpb;
+    int deal_by_cost;     // long suffixes: hand tiles to CTAs by cost rank instead of in contiguous ranges
     int long_sfx;         // 1: a tile lies inside ONE candidate and that candidate's suffix keys come in
                           //    128-key blocks (suffix caches or row groups beyond 128); 0: whole-candidate tiles
     // shared-memory carve-up (byte offsets from the 1024-byte aligned base)
@@ -198,10 +199,29 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // contiguous range of tiles for this CTA (tiles are ordered KV head major)
+    // Tiles of this CTA.  Normally a contiguous range (tiles are ordered KV head major, so the
+    // resident prefix of a head serves a whole run).  With long suffixes a tile's cost grows with the
+    // position of its rows inside the suffix (causal block skipping), so there -- when tiles do not
+    // straddle heads and the suffix K/V of all candidates stays in L2 anyway -- the tiles are dealt out by cost: ranked from the last (longest) suffix
+    // position down, round r hands ranks r*G .. r*G+G-1 to the CTAs in alternating direction (the
+    // longest-first rule in closed form).
     const int t_begin = (int)((long long)blockIdx.x * p.total_tiles / gridDim.x);
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
-    const int n_tiles = t_end - t_begin;
+    const int G = (int)gridDim.x;
+    const int n_sp = (SR && p.deal_by_cost) ? p.S / p.tile_rows : 1;  // tiles per head
+    const bool dealt = n_sp > 1;
+    auto rank_at = [&](int tl) { return tl * G + ((tl & 1) ? G - 1 - (int)blockIdx.x : (int)blockIdx.x); };
+    auto tile_at = [&](int tl) {
+        if (!dealt) return t_begin + tl;
+        // rank -> (suffix position from the end, candidate, KV head, head inside the group)
+        const int rank = rank_at(tl), M = p.B * p.Hkv * p.n_rep;
+        const int spr = rank / M, m = rank - spr * M;
+        const int b = m / (p.Hkv * p.n_rep), gh = m - b * (p.Hkv * p.n_rep);
+        const int g = gh / p.n_rep, hr = gh - g * p.n_rep;
+        return g * p.tiles_per_group + (b * p.n_rep + hr) * n_sp + (n_sp - 1 - spr);
+    };
+    const int n_rounds = (p.total_tiles + G - 1) / G;
+    const int n_tiles = !dealt ? t_end - t_begin : (n_rounds - 1) + (rank_at(n_rounds - 1) < p.total_tiles ? 1 : 0);
     // items of a tile: prefix blocks + the suffix block(s)
     auto items_of = [&](const TileInfo &t) {
         return p.nblk_p + (!SR ? 1 : p.long_sfx ? sfx_blocks_long(p, t) : p.fd_cpb.div(t.nc + p.cpb - 1));
@@ -225,7 +245,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
-            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            const TileInfo t = tile_info(p, tile_at(tl), t_begin);
             // Everything the Q loads need is worked out before the wait, so that only the copy
             // instructions themselves follow it: the Q buffer is single, and the time from "last
             // score MMA of the previous tile done" to "Q of this tile requested" is exposed.
@@ -239,7 +259,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // While there is nothing else to do, ask for the NEXT tile's Q in L2: its load can only
             // be issued a tile from now, right when it is needed, and then finds the data close by.
             if (tl + 1 < n_tiles) {
-                const TileInfo tn = tile_info(p, t_begin + tl + 1, t_begin);
+                const TileInfo tn = tile_info(p, tile_at(tl + 1), t_begin);
                 const int nseg_n = SR ? 1 : p.fd_seg.div(tn.rows);
                 int nb = p.fd_Rg.div(tn.R0), nr = tn.R0 - nb * p.Rg;
                 if (elect_one_sync()) {
@@ -386,7 +406,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             TileInfo t;
             int nk = 0;  // V blocks still to fetch through the ring for this tile
             if (have_tile) {
-                t = tile_info(p, t_begin + tl, t_begin);
+                t = tile_info(p, tile_at(tl), t_begin);
                 if (RES) {
                     // the resident prefix V blocks are free once every value MMA of the previous tile
                     // has completed
@@ -476,7 +496,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarStageFull), (tl - 1) & 1) ? 1 : 0, 0) != 0;
                     if (!ok) break;
                     if (ready) {
-                        const TileInfo u = tile_info(p, t_begin + tl - 1, t_begin);
+                        const TileInfo u = tile_info(p, tile_at(tl - 1), t_begin);
                         const int nseg = SR ? 1 : p.fd_seg.div(u.rows);  // (one box of whole candidates)
                         if (elect_one_sync()) {
 #pragma unroll 1
@@ -520,7 +540,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         // ------------------------------------------------------------------ score MMAs: S = Q K^T
         int tl = 0, k = 0;
         uint32_t kuse = 0;  // streaming mode: K blocks consumed from the ring
-        TileInfo t = tile_info(p, t_begin, t_begin);
+        TileInfo t = tile_info(p, tile_at(0), t_begin);
         int nitems = items_of(t);
         const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
         bool ok = true;
@@ -581,7 +601,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (++k == nitems) {
                 k = 0;
                 if (++tl < n_tiles) {
-                    t = tile_info(p, t_begin + tl, t_begin);
+                    t = tile_info(p, tile_at(tl), t_begin);
                     nitems = items_of(t);
                 }
             }
@@ -590,7 +610,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         // ------------------------------------------------------------------ value MMAs: O += P V
         int tl = 0, k = 0;
         uint32_t vuse = 0;
-        TileInfo t = tile_info(p, t_begin, t_begin);
+        TileInfo t = tile_info(p, tile_at(0), t_begin);
         int nitems = items_of(t);
         const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
         bool ok = true;
@@ -656,7 +676,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (++k == nitems) {
                 k = 0;
                 if (++tl < n_tiles) {
-                    t = tile_info(p, t_begin + tl, t_begin);
+                    t = tile_info(p, tile_at(tl), t_begin);
                     nitems = items_of(t);
                 }
             }
@@ -683,7 +703,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         int item = 0;  // items handled so far
 #pragma unroll 1
         for (int tl = 0; tl < n_tiles && ok; ++tl) {
-            const TileInfo t = tile_info(p, t_begin + tl, t_begin);
+            const TileInfo t = tile_info(p, tile_at(tl), t_begin);
             const int nitems = items_of(t);
             int lo_sfx = 1, hi_sfx = 0;
             int k_own = p.nblk_p;  // suffix-ring mode: the item that holds this row's candidate
@@ -814,7 +834,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
 #pragma unroll 1
         for (int te = 0; te < n_tiles && ok; ++te) {
-            const TileInfo u = tile_info(p, t_begin + te, t_begin);
+            const TileInfo u = tile_info(p, tile_at(te), t_begin);
             ok = mbar_wait_warp(bar(kBarOFull), te & 1, abort_flag, p.status, kErrEpilogue);
             if (!ok) break;
             PSKV_TRACE_EVENT(30, te);
@@ -1089,6 +1109,10 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.cpb = plan.cpb > 0 ? plan.cpb : 1;
     p.fd_cpb.init(p.cpb);
     p.long_sfx = plan.long_sfx;
+    // Dealing by cost balances the causal skew but lets every CTA touch every candidate's suffix K/V
+    // at several times; it pays when those tensors stay in L2 between the touches.
+    p.deal_by_cost = plan.long_sfx && dm.S % plan.tile_rows == 0 && dm.S / plan.tile_rows > 1 &&
+                     4.0 * dm.B * dm.Hkv * dm.Skv * D <= 48.0e6;
     p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_sk = plan.off_sk;
     p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
     p.off_ml = plan.off_ml;
