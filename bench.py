@@ -479,38 +479,57 @@ def detail_runs(pskv, device, peaks):
                             "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
     del q, sk, sv, do, pk, pv, out, lse, dq, dk, dv
     torch.cuda.empty_cache()
-    # Decode-shaped variant at the C2 layer shape: one new token per candidate on top of a suffix cache of
-    # up to 48 tokens (uniform ragged lengths), forward only (the attacks that grow suffixes token by token
-    # are gradient-free).  The call is bound by reading each candidate's suffix K/V once, so it is reported
-    # against the HBM roofline; four input sets are rotated so that every call reads from HBM, not L2.
-    for tag, Bd in (("C2_decode_1of48_B512", 512), ("C2_decode_1of48_B2048", 2048)):
-        Sq, Skv = 1, 48
-        sets = []
-        for i in range(4):
-            sets.append((draw(Bd, w.Hq, Sq, w.d), draw(Bd, w.Hkv, Skv, w.d), draw(Bd, w.Hkv, Skv, w.d),
-                         torch.randint(Sq, Skv + 1, (Bd,), generator=gen, dtype=torch.int32).to(device)))
-        pk, pv = draw(w.Hkv, w.P, w.d), draw(w.Hkv, w.P, w.d)
-        out = torch.empty_like(sets[0][0])
-        lse = torch.empty((Bd, w.Hq, Sq), dtype=torch.float32, device=device)
-        ws = torch.empty(256, dtype=torch.uint8, device=device)
-        turn = [0]
+    for Bd in (512, 2048):
+        res["C2_decode_1of48_B%d" % Bd] = decode_run(pskv, device, peaks, Bd, 40, 4)
+    res["prefix_prefill_P%d" % wl.WORKLOADS["C3"].P] = prefill_run(pskv, device, peaks, 40, 4)
+    return res
 
-        def dfwd():
-            qd, skd, svd, ln = sets[turn[0] % 4]
-            turn[0] += 1
-            pskv.pskv_attn_fwd_decode(qd, pk, pv, skd, svd, ln, w.scale, out=out, lse=lse, workspace=ws)
 
-        dfwd()
-        ms = time_calls(dfwd, 40, 4)
-        nbytes = (2 * Bd * w.Hq * Sq * w.d + 2 * Bd * w.Hkv * Skv * w.d + 2 * w.Hkv * w.P * w.d) * 2 + Bd * w.Hq * Sq * 4
-        res[tag] = {"Sq": Sq, "Skv": Skv, "B": Bd,
-                    "fwd": {"ms": ms, "candidates_per_s": Bd / ms * 1e3, "hbm_gbs": nbytes / ms / 1e6,
-                            "pct_hbm_peak": 100 * nbytes / ms / 1e6 / peaks["hbm_gbs"]}}
-        del sets, pk, pv, out, lse
-        torch.cuda.empty_cache()
-    # Prefix prefill, attention step: the causal self-attention of one 2048-token sequence (B = 1, P = 0, the
-    # sequence's K/V passed as the suffix), i.e. what produces a C3-sized prefix cache in the first place.
+def _draw_on(device, seed):
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16).to(device)
+
+    return draw, gen
+
+
+def decode_run(pskv, device, peaks, Bd, iters, warmup):
+    """Decode-shaped variant at the C2 layer shape: one new token per candidate on top of a suffix cache of up
+    to 48 tokens (uniform ragged lengths), forward only (the attacks that grow suffixes token by token are
+    gradient-free).  The call is bound by reading each candidate's suffix K/V once, so it is reported
+    against the HBM roofline; four input sets are rotated so that every call reads from HBM, not L2."""
+    w = wl.WORKLOADS["C2"]
+    draw, gen = _draw_on(device, w.seed + 600 + Bd)
+    Sq, Skv = 1, 48
+    sets = []
+    for i in range(4):
+        sets.append((draw(Bd, w.Hq, Sq, w.d), draw(Bd, w.Hkv, Skv, w.d), draw(Bd, w.Hkv, Skv, w.d),
+                     torch.randint(Sq, Skv + 1, (Bd,), generator=gen, dtype=torch.int32).to(device)))
+    pk, pv = draw(w.Hkv, w.P, w.d), draw(w.Hkv, w.P, w.d)
+    out = torch.empty_like(sets[0][0])
+    lse = torch.empty((Bd, w.Hq, Sq), dtype=torch.float32, device=device)
+    ws = torch.empty(256, dtype=torch.uint8, device=device)
+    turn = [0]
+
+    def dfwd():
+        qd, skd, svd, ln = sets[turn[0] % 4]
+        turn[0] += 1
+        pskv.pskv_attn_fwd_decode(qd, pk, pv, skd, svd, ln, w.scale, out=out, lse=lse, workspace=ws)
+
+    ms = time_calls(dfwd, iters, warmup)
+    nbytes = (2 * Bd * w.Hq * Sq * w.d + 2 * Bd * w.Hkv * Skv * w.d + 2 * w.Hkv * w.P * w.d) * 2 + Bd * w.Hq * Sq * 4
+    return {"Sq": Sq, "Skv": Skv, "B": Bd, "algorithmic_bytes": nbytes,
+            "fwd": {"ms": ms, "candidates_per_s": Bd / ms * 1e3, "hbm_gbs": nbytes / ms / 1e6,
+                    "pct_hbm_peak": 100 * nbytes / ms / 1e6 / peaks["hbm_gbs"]}}
+
+
+def prefill_run(pskv, device, peaks, iters, warmup):
+    """Prefix prefill, attention step: the causal self-attention of one 2048-token sequence (B = 1, P = 0, the
+    sequence's K/V passed as the suffix), i.e. what produces a C3-sized prefix cache in the first place."""
     w3 = wl.WORKLOADS["C3"]
+    draw, _ = _draw_on(device, w3.seed + 700)
     Sp = w3.P
     qp, kp, vp = draw(1, w3.Hq, Sp, w3.d), draw(1, w3.Hkv, Sp, w3.d), draw(1, w3.Hkv, Sp, w3.d)
     outp = torch.empty_like(qp)
@@ -520,13 +539,28 @@ def detail_runs(pskv, device, peaks):
     def prefill():
         pskv.pskv_attn_fwd(qp, None, None, kp, vp, w3.scale, out=outp, lse=lsep, workspace=wsp)
 
-    prefill()
-    ms = time_calls(prefill, 40, 4)
+    ms = time_calls(prefill, iters, warmup)
     fl = 4.0 * w3.d * ((Sp + 1) / 2) * w3.Hq * Sp
-    res["prefix_prefill_P%d" % Sp] = {"fwd": {"ms": ms, "tflops": fl / ms / 1e9,
-                                              "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
-                                              "kernel_family": pskv.pskv_kernel_family(0, 1, w3.Hq, w3.Hkv, Sp, 0, w3.d)}}
-    return res
+    return {"fwd": {"ms": ms, "tflops": fl / ms / 1e9, "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
+                    "kernel_family": pskv.pskv_kernel_family(0, 1, w3.Hq, w3.Hkv, Sp, 0, w3.d)}}
+
+
+def run_variant(args):
+    """One variant's timing loop alone (for profiling it without the rest of the benchmark)."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    import paper_2603_13420_b200 as pskv
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peaks = load_peaks()
+    if args.variant == "prefill":
+        res = prefill_run(pskv, device, peaks, args.steps, max(args.warmup, 3))
+    else:
+        res = decode_run(pskv, device, peaks, int(args.variant.split("_B")[1]), args.steps, max(args.warmup, 3))
+    status = pskv.pskv_poll_device_status()
+    if status != pskv.PSKV_OK:
+        raise SystemExit("device status: %s" % pskv.pskv_status_string(status))
+    print(json.dumps({"variant": args.variant, "steps": args.steps, **res}))
 
 
 def cpu_baseline(w, cand):
@@ -556,9 +590,13 @@ def main():
                     help="candidates of the one-off CPU oracle sample reported as cpu_baseline")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill"],
+                    help="time only this variant of the detail runs (1 GPU) and print its entry")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.variant:
+        run_variant(args)
     else:
         run_cuda(args)
 
