@@ -59,6 +59,8 @@ def _load():
         lib.pskv_oracle_attn_fwd_decode.restype = ctypes.c_int
         lib.pskv_oracle_attn_bwd_decode.argtypes = [dp] * 6 + [ip] + [ctypes.c_double] + [dp] * 3 + ints7
         lib.pskv_oracle_attn_bwd_decode.restype = ctypes.c_int
+        lib.pskv_oracle_target_ce_fwd.argtypes = [dp, dp, ip, dp, dp, dp, dp] + [ctypes.c_int] * 4
+        lib.pskv_oracle_target_ce_fwd.restype = ctypes.c_int
         lib.pskv_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -256,3 +258,25 @@ def attn_bwd_decode(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, scale, suff
     if rc != 0:
         raise RuntimeError("pskv_oracle_attn_bwd_decode failed with code %d" % rc)
     return dq, dk, dv
+
+
+def target_ce_fwd(hidden, weight, target, mask):
+    """Masked target cross-entropy on top of the vocabulary projection: hidden [N,Lr,Dm], weight [V,Dm],
+    target [N,Lr] ints, mask [N,Lr] loss weights.  Returns nll [N,Lr], lse [N,Lr], loss [N] (fp64)."""
+    hidden = np.asarray(hidden)
+    N, Lr, Dm = hidden.shape
+    V = np.asarray(weight).shape[0]
+    h = _f64(hidden, (N, Lr, Dm))
+    w = _f64(weight, (V, Dm))
+    t = np.ascontiguousarray(np.asarray(target, dtype=np.int32))
+    if t.shape != (N, Lr):
+        raise ValueError("expected target shape %s, got %s" % ((N, Lr), t.shape))
+    m = _f64(mask, (N, Lr))
+    nll = np.empty((N, Lr), dtype=np.float64)
+    lse = np.empty((N, Lr), dtype=np.float64)
+    loss = np.empty((N,), dtype=np.float64)
+    rc = _load().pskv_oracle_target_ce_fwd(_ptr(h), _ptr(w), t.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), _ptr(m),
+                                           _ptr(nll), _ptr(lse), _ptr(loss), N, Lr, Dm, V)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_target_ce_fwd failed with code %d" % rc)
+    return nll, lse, loss

@@ -504,3 +504,57 @@ int pskv_oracle_attn_bwd_decode(const double *dout, const double *q, const doubl
     }
     return failed ? 2 : 0;
 }
+
+/*
+ * Masked target cross-entropy on top of the vocabulary projection (appendix on the loss:
+ * L = sum m^tar CE(logits, z) / sum m^tar, the loss mask being one only on the target-response
+ * span).  For N candidates of Lr scored positions each:
+ *   logits[r, v] = <hidden[r, :], weight[v, :]>                (the output head, no bias)
+ *   lse[r]       = ln sum_v exp(logits[r, v])
+ *   nll[r]       = mask[r] * (lse[r] - logits[r, target[r]])   (CE of position r against its token)
+ *   loss[c]      = sum_{r in candidate c} nll[r] / sum_{r in c} mask[r]    (0 if the candidate has
+ *                  no weighted position): the masked average, per candidate, which is what ranks
+ *                  the candidates of one search step; the paper's scalar is the same ratio over all
+ *                  candidates and instructions.
+ * Written out literally: the full logits row is formed and reduced.  Layouts: hidden [N*Lr][Dm],
+ * weight [V][Dm], target [N*Lr] (ints in [0, V) wherever mask != 0), mask [N*Lr].
+ */
+int pskv_oracle_target_ce_fwd(const double *hidden, const double *weight, const int *target,
+                              const double *mask, double *nll, double *lse, double *loss,
+                              int N, int Lr, int Dm, int V)
+{
+    if (N < 1 || Lr < 1 || Dm < 1 || V < 1) return 1;
+    const long long R = (long long)N * Lr;
+    for (long long r = 0; r < R; ++r)
+        if (mask[r] != 0.0 && (target[r] < 0 || target[r] >= V)) return 1;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int c = 0; c < N; ++c) {
+        double *z = (double *)malloc(sizeof(double) * (size_t)V);
+        if (!z) {
+            failed = 1;
+        } else {
+            double num = 0.0, den = 0.0;
+            for (int i = 0; i < Lr; ++i) {
+                const long long r = (long long)c * Lr + i;
+                const double *h = hidden + r * Dm;
+                double m = -INFINITY;
+                for (int v = 0; v < V; ++v) {
+                    double acc = 0.0;
+                    for (int k = 0; k < Dm; ++k) acc += h[k] * weight[(size_t)v * Dm + k];
+                    z[v] = acc;
+                    if (acc > m) m = acc;
+                }
+                double l = 0.0;
+                for (int v = 0; v < V; ++v) l += exp(z[v] - m);
+                lse[r] = m + log(l);
+                nll[r] = mask[r] != 0.0 ? mask[r] * (lse[r] - z[target[r]]) : 0.0;
+                num += nll[r];
+                den += mask[r];
+            }
+            loss[c] = den != 0.0 ? num / den : 0.0;
+        }
+        free(z);
+    }
+    return failed ? 2 : 0;
+}
