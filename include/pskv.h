@@ -209,6 +209,32 @@ pskv_status pskv_attn_bwd_decode(const void *dout, const void *q, const void *pr
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Masked target cross-entropy fused with the vocabulary projection (loss appendix: the objective is
+ * the masked average of CE(logits, target token) over the target-response span; the logits tensor
+ * [candidates x positions x vocabulary] is the memory high-water mark the paper reports for a search
+ * step).  For N candidates with Lr scored positions each (rows r = c * Lr + i):
+ *   logits[r, v] = <hidden[r, :], weight[v, :]>          (output head without bias; never stored)
+ *   lse[r]       = ln sum_v exp(logits[r, v])
+ *   nll[r]       = mask[r] * (lse[r] - logits[r, target[r]])      (0 where mask[r] == 0)
+ *   loss[c]      = sum_i nll[c*Lr + i] / sum_i mask[c*Lr + i]      (0 for a candidate without weight)
+ * The paper's scalar objective is sum_c loss[c] * (weight of c) / (total weight); loss[c] itself is what
+ * ranks the candidates of a search step.  Products are exact in fp32 and accumulated in fp32; the
+ * logits are never rounded to bf16.
+ *   hidden  bf16 [N*Lr, Dm]   final hidden state of every scored position (position r-1 predicts token r)
+ *   weight  bf16 [V, Dm]      output-head matrix
+ *   target  int32 [N*Lr]      token ids; must lie in [0, V) wherever mask != 0 (else that nll is NaN)
+ *   mask    fp32 [N*Lr]       loss weights m^tar (0/1, or any non-negative weight)
+ *   nll, lse fp32 [N*Lr], loss fp32 [N]: fully overwritten
+ * All pointers are device pointers, 16-byte aligned.  Dm must be a multiple of 8 (else
+ * PSKV_ERR_UNSUPPORTED_SHAPE); any N, Lr, V.  Forward only: a search step ranks its candidates by
+ * this loss without differentiating through it.
+ */
+size_t pskv_target_ce_fwd_workspace_bytes(int N, int Lr, int Dm, int V);
+pskv_status pskv_target_ce_fwd(const void *hidden, const void *weight, const int *target, const float *mask,
+                               float *nll, float *lse, float *loss, int N, int Lr, int Dm, int V,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then reads and clears the device status word that
  * kernels set when one of their bounded waits gives up.  Returns PSKV_OK,
  * PSKV_ERR_DEVICE_TIMEOUT (results of the affected call are undefined) or

@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.pskv_attn_fwd_decode.restype = ci
         L.pskv_attn_bwd_decode.argtypes = [vp] * 9 + [cf] + [vp] * 3 + seven + [vp, sz, vp]
         L.pskv_attn_bwd_decode.restype = ci
+        L.pskv_target_ce_fwd_workspace_bytes.argtypes = [ci] * 4
+        L.pskv_target_ce_fwd_workspace_bytes.restype = sz
+        L.pskv_target_ce_fwd.argtypes = [vp] * 7 + [ci] * 4 + [vp, sz, vp]
+        L.pskv_target_ce_fwd.restype = ci
         L.pskv_attn_bwd_static.argtypes = [vp] * 8 + [cf] + [vp] * 3 + six + [vp]
         L.pskv_attn_bwd_static.restype = ci
         L.pskv_attn_bwd_static_max_rows.argtypes = []
@@ -359,6 +363,31 @@ def pskv_attn_bwd_decode(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, suffix
     if st != PSKV_OK:
         raise PskvError(st, "pskv_attn_bwd_decode")
     return dq, dk_suffix, dv_suffix
+
+
+def pskv_target_ce_fwd_workspace_bytes(N, Lr, Dm, V) -> int:
+    return int(lib().pskv_target_ce_fwd_workspace_bytes(N, Lr, Dm, V))
+
+
+def pskv_target_ce_fwd(hidden, weight, target, mask, nll=None, lse=None, loss=None, workspace=None):
+    """Masked target cross-entropy fused with the vocabulary projection: hidden bf16 [N,Lr,Dm], weight
+    bf16 [V,Dm], target int32 [N,Lr], mask fp32 [N,Lr].  Returns nll [N,Lr], lse [N,Lr], loss [N] (fp32)."""
+    N, Lr, Dm = (int(x) for x in hidden.shape)
+    V = int(weight.shape[0])
+    if target.dtype != torch.int32 or mask.dtype != torch.float32:
+        raise ValueError("target must be int32 and mask float32")
+    if tuple(target.shape) != (N, Lr) or tuple(mask.shape) != (N, Lr) or int(weight.shape[1]) != Dm:
+        raise ValueError("shape mismatch")
+    f32 = dict(dtype=torch.float32, device=hidden.device)
+    nll = torch.empty((N, Lr), **f32) if nll is None else nll
+    lse = torch.empty((N, Lr), **f32) if lse is None else lse
+    loss = torch.empty((N,), **f32) if loss is None else loss
+    ws = _workspace(pskv_target_ce_fwd_workspace_bytes(N, Lr, Dm, V), hidden.device, workspace)
+    st = lib().pskv_target_ce_fwd(_ptr(hidden), _ptr(weight), _ptr(target), _ptr(mask), _ptr(nll), _ptr(lse),
+                                  _ptr(loss), N, Lr, Dm, V, _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_target_ce_fwd")
+    return nll, lse, loss
 
 
 def pskv_attn_bwd_static_max_rows() -> int:

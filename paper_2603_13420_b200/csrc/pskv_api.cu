@@ -103,7 +103,7 @@ std::vector<TimedLaunch> g_timed;
 const char *const kKernelNames[kKernelCount] = {
     "tc_fwd_kernel", "simt_fwd_redo_kernel", "simt_row_dot_kernel", "tc_bwd_dq_kernel", "tc_bwd_dkv_kernel",
     "bwd_dkv_mma_kernel",
-    "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel"};
+    "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel", "ce_fwd_kernel", "ce_finalize_kernel"};
 
 }  // namespace
 
@@ -514,6 +514,37 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return PSKV_OK;
+}
+
+// ---- masked target cross-entropy fused with the vocabulary projection ---------------------------------
+
+size_t pskv_target_ce_fwd_workspace_bytes(int N, int Lr, int Dm, int V)
+{
+    return ce_fwd_supported(N, Lr, Dm, V) ? round256(ce_fwd_workspace_bytes(N, Lr, Dm, V)) : 0;
+}
+
+pskv_status pskv_target_ce_fwd(const void *hidden, const void *weight, const int *target, const float *mask,
+                               float *nll, float *lse, float *loss, int N, int Lr, int Dm, int V, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream)
+{
+    if (N < 1 || Lr < 1 || Dm < 1 || V < 1) return PSKV_ERR_INVALID_ARG;
+    if (!ce_fwd_supported(N, Lr, Dm, V)) return PSKV_ERR_UNSUPPORTED_SHAPE;
+    if (!hidden || !weight || !target || !mask || !nll || !lse || !loss) return PSKV_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(weight) || !aligned16(target) || !aligned16(mask) || !aligned16(nll) ||
+        !aligned16(lse) || !aligned16(loss))
+        return PSKV_ERR_INVALID_ARG;
+    const size_t need = pskv_target_ce_fwd_workspace_bytes(N, Lr, Dm, V);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
+    unsigned int *status_word = nullptr;
+    pskv_status st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+    CeArgs a;
+    a.hidden = static_cast<const __nv_bfloat16 *>(hidden);
+    a.weight = static_cast<const __nv_bfloat16 *>(weight);
+    a.target = target; a.mask = mask; a.nll = nll; a.lse = lse; a.loss = loss;
+    a.N = N; a.Lr = Lr; a.Dm = Dm; a.V = V;
+    cudaError_t e = launch_ce_fwd(a, workspace, status_word, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
 }
 
 pskv_status pskv_poll_device_status(void *cuda_stream)

@@ -72,6 +72,18 @@ size_t tc_bwd_workspace_bytes(const Dims &d);
 cudaError_t launch_tc_bwd(const BwdArgs &a, void *workspace, unsigned int *status_word,
                           cudaStream_t stream);
 
+// Masked target cross-entropy fused with the vocabulary projection (tcgen05 GEMM whose logits stay on chip).
+struct CeArgs {
+    const __nv_bfloat16 *hidden, *weight;  // [N*Lr, Dm], [V, Dm]
+    const int *target;                     // [N*Lr]
+    const float *mask;                     // [N*Lr] loss weights
+    float *nll, *lse, *loss;               // [N*Lr], [N*Lr], [N]
+    int N, Lr, Dm, V;
+};
+bool ce_fwd_supported(int N, int Lr, int Dm, int V);
+size_t ce_fwd_workspace_bytes(int N, int Lr, int Dm, int V);
+cudaError_t launch_ce_fwd(const CeArgs &a, void *workspace, unsigned int *status_word, cudaStream_t stream);
+
 // Host-side count of kernel launches (read through pskv_kernel_launches()).
 void count_launches(int n);
 
@@ -79,7 +91,7 @@ void count_launches(int n);
 // its kernel with two CUDA events on the launch stream.
 enum KernelId {
     kKernelFwdTc = 0, kKernelFwdRedo, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvTc, kKernelBwdDkvMma,
-    kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCount
+    kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCeFwd, kKernelCeFinalize, kKernelCount
 };
 void *timing_begin(int kernel_id, cudaStream_t stream);  // returns nullptr when timing is off
 void timing_end(void *token, cudaStream_t stream);
