@@ -482,6 +482,7 @@ def detail_runs(pskv, device, peaks):
     for Bd in (512, 2048):
         res["C2_decode_1of48_B%d" % Bd] = decode_run(pskv, device, peaks, Bd, 40, 4)
     res["prefix_prefill_P%d" % wl.WORKLOADS["C3"].P] = prefill_run(pskv, device, peaks, 40, 4)
+    res["target_ce_512x20_Dm4096_V128256"] = ce_run(pskv, device, peaks, 5, 3)
     return res
 
 
@@ -545,6 +546,44 @@ def prefill_run(pskv, device, peaks, iters, warmup):
                     "kernel_family": pskv.pskv_kernel_family(0, 1, w3.Hq, w3.Hkv, Sp, 0, w3.d)}}
 
 
+def ce_run(pskv, device, peaks, iters, warmup, with_library=True):
+    """Masked target cross-entropy fused with the vocabulary projection at the Llama-3-8B head (hidden 4096,
+    vocabulary 128256), 512 candidates x 20 target positions.  A dense contraction: reported against the
+    bf16 tensor peak (sustained figure: the launch runs for milliseconds under the power cap).  For context
+    the library pipeline on the same inputs: one bf16 GEMM that writes the logits, then float cross-entropy."""
+    import math
+    N, Lr, Dm, V = 512, 20, 4096, 128256
+    gen = torch.Generator(device=device)
+    gen.manual_seed(wl.WORKLOADS["C2"].seed + 800)
+    h = torch.randn((N, Lr, Dm), generator=gen, device=device).to(torch.bfloat16)
+    wt = (torch.randn((V, Dm), generator=gen, device=device) / math.sqrt(Dm)).to(torch.bfloat16)
+    t = torch.randint(0, V, (N, Lr), generator=gen, device=device, dtype=torch.int32)
+    m = (torch.rand((N, Lr), generator=gen, device=device) < 0.8).to(torch.float32)
+    f32 = dict(dtype=torch.float32, device=device)
+    nll, lse, loss = torch.empty((N, Lr), **f32), torch.empty((N, Lr), **f32), torch.empty((N,), **f32)
+    ws = torch.empty(pskv.pskv_target_ce_fwd_workspace_bytes(N, Lr, Dm, V), dtype=torch.uint8, device=device)
+
+    def fused():
+        pskv.pskv_target_ce_fwd(h, wt, t, m, nll=nll, lse=lse, loss=loss, workspace=ws)
+
+    ms = time_calls(fused, iters, warmup)
+    fl = 2.0 * N * Lr * Dm * V
+    out = {"N": N, "Lr": Lr, "Dm": Dm, "V": V, "algorithmic_flops": fl,
+           "fwd": {"ms": ms, "tflops": fl / ms / 1e9, "candidates_per_s": N / ms * 1e3,
+                   "pct_bf16_peak_sustained": 100 * fl / ms / 1e9 / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                   "pct_bf16_peak_burst": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
+                   "logits_bytes_never_written": 2.0 * N * Lr * V}}
+    if with_library:
+        tl = t.view(-1).long()
+
+        def library():
+            logits = h.view(-1, Dm) @ wt.T
+            return torch.nn.functional.cross_entropy(logits.float(), tl, reduction="none")
+
+        out["library_gemm_plus_ce_ms"] = time_calls(library, 3, 2)
+    return out
+
+
 def run_variant(args):
     """One variant's timing loop alone (for profiling it without the rest of the benchmark)."""
     if not torch.cuda.is_available():
@@ -555,6 +594,8 @@ def run_variant(args):
     peaks = load_peaks()
     if args.variant == "prefill":
         res = prefill_run(pskv, device, peaks, args.steps, max(args.warmup, 3))
+    elif args.variant == "target_ce":
+        res = ce_run(pskv, device, peaks, args.steps, max(args.warmup, 3), with_library=False)
     else:
         res = decode_run(pskv, device, peaks, int(args.variant.split("_B")[1]), args.steps, max(args.warmup, 3))
     status = pskv.pskv_poll_device_status()
@@ -590,7 +631,7 @@ def main():
                     help="candidates of the one-off CPU oracle sample reported as cpu_baseline")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
-    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill"],
+    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill", "target_ce"],
                     help="time only this variant of the detail runs (1 GPU) and print its entry")
     args = ap.parse_args()
     if args.impl == "reference":

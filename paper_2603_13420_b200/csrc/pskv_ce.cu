@@ -8,10 +8,11 @@
 // (max, sum) per row and pick out the target's logit while the tensor cores already work on the next
 // block in the other half of tensor memory.
 //
-// Work units are (vocabulary panel of 8 blocks, 128-row tile), numbered row tile fastest, and CTA c
-// takes units c, c + G, c + 2G, ...: the CTAs running at any moment work on the same one or two
-// weight panels (16 MB each, L2 resident) against different row tiles, so the weight matrix is
-// fetched from HBM about once.  Each unit leaves one partial (max, sum) per row; a small second
+// Work units are (vocabulary panel of 8 blocks, 128-row tile).  Row tiles are taken in groups of a
+// quarter of the CTA count; inside a group the units are numbered panel-major, row tile fastest, and
+// CTA c takes units c, c + G, c + 2G, ...: the CTAs running at any moment work on about four weight
+// panels (16 MB each) against one group of row tiles (1 MB each), a working set that stays in L2, so
+// the weight matrix comes from HBM once per row group and the hidden states once.  Each unit leaves one partial (max, sum) per row; a small second
 // kernel merges the partials of a row, forms nll = mask * (lse - target logit) and the masked
 // average per candidate.
 //
@@ -49,8 +50,24 @@ struct CeParams {
     unsigned int *status;
     int R, Rpad, Dm, V;
     int nrt, nvb, npanel, units, ksteps;
-    FastDiv fd_nrt;
+    int rg;                // row tiles per group
 };
+
+// unit -> (panel, row tile): groups of rg row tiles, panel-major inside a group, the last group smaller
+__device__ __forceinline__ void ce_unit(const CeParams &p, int u, int &pn, int &rt)
+{
+    const int per_group = p.rg * p.npanel;
+    const int nfull = p.nrt / p.rg;
+    if (u < nfull * per_group) {
+        const int gi = u / per_group, rem = u - gi * per_group;
+        pn = rem / p.rg;
+        rt = gi * p.rg + (rem - pn * p.rg);
+    } else {
+        const int tail = p.nrt - nfull * p.rg, rem = u - nfull * per_group;
+        pn = rem / tail;
+        rt = nfull * p.rg + (rem - pn * tail);
+    }
+}
 
 __global__ void __launch_bounds__(kCeThreads, 1)
 ce_fwd_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w, const CeParams p)
@@ -96,7 +113,8 @@ ce_fwd_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ 
 #pragma unroll 1
         for (int tl = 0; tl < n_units && ok; ++tl) {
             const int u = (int)blockIdx.x + tl * (int)gridDim.x;
-            const int pn = p.fd_nrt.div(u), rt = u - pn * p.nrt;
+            int pn, rt;
+            ce_unit(p, u, pn, rt);
             const int vb_end = min(p.nvb, (pn + 1) * kCePanel);
 #pragma unroll 1
             for (int vb = pn * kCePanel; vb < vb_end && ok; ++vb) {
@@ -126,7 +144,8 @@ ce_fwd_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ 
 #pragma unroll 1
         for (int tl = 0; tl < n_units && ok; ++tl) {
             const int u = (int)blockIdx.x + tl * (int)gridDim.x;
-            const int pn = p.fd_nrt.div(u);
+            int pn, rt;
+            ce_unit(p, u, pn, rt);
             const int vb_end = min(p.nvb, (pn + 1) * kCePanel);
 #pragma unroll 1
             for (int vb = pn * kCePanel; vb < vb_end && ok; ++vb, ++blk) {
@@ -165,7 +184,8 @@ ce_fwd_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ 
 #pragma unroll 1
         for (int tl = 0; tl < n_units && ok; ++tl) {
             const int u = (int)blockIdx.x + tl * (int)gridDim.x;
-            const int pn = p.fd_nrt.div(u), rt = u - pn * p.nrt;
+            int pn, rt;
+            ce_unit(p, u, pn, rt);
             const int vb_end = min(p.nvb, (pn + 1) * kCePanel);
             const int grow = rt * kCeM + row;
             const bool valid = grow < p.R;
@@ -321,7 +341,8 @@ cudaError_t launch_ce_fwd(const CeArgs &a, void *workspace, unsigned int *status
     p.status = status_word;
     p.R = (int)R; p.Rpad = pl.Rpad; p.Dm = a.Dm; p.V = a.V;
     p.nrt = pl.nrt; p.nvb = pl.nvb; p.npanel = pl.npanel; p.units = pl.npanel * pl.nrt; p.ksteps = pl.ksteps;
-    p.fd_nrt.init(pl.nrt);
+    p.rg = sm_count() / 4 < 1 ? 1 : sm_count() / 4;
+    if (p.rg > pl.nrt) p.rg = pl.nrt;
     const int smem_bytes = kCeStages * kCeStageBytes + 8 * kCeNumBars + 64;
     static bool attr_set = false;
     if (!attr_set) {

@@ -61,6 +61,25 @@ def test_fused_cross_entropy_matches_the_oracle(case):
 
 
 @pytest.mark.gpu
+def test_full_size_head_on_sampled_candidates():
+    """512 candidates x 20 positions against a 4096 x 32000 head (the launch shape of the bench line, with the
+    smaller of the two vocabularies so that the fp64 copy of the head fits the host): four candidates, the
+    first and last among them, are checked against the oracle; every lse must also be finite and at least
+    the largest logit bound ln(V) - |min| cannot beat, i.e. >= the target logit (nll >= 0)."""
+    N, Lr, Dm, V = 512, 20, 4096, 32000
+    h, w, t, m = make(N, Lr, Dm, V, seed=1234)
+    nll, lse, loss = pskv.pskv_target_ce_fwd(h.cuda(), w.cuda(), t.cuda(), m.cuda())
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    assert torch.isfinite(lse).all() and torch.isfinite(nll).all() and (nll >= 0).all()
+    cand = [0, 1, 255, 511]
+    rn, rl, rs = oracle.target_ce_fwd(parity.to_f64(h[cand]), parity.to_f64(w), t[cand].numpy(),
+                                      m[cand].numpy().astype(np.float64))
+    assert np.max(np.abs(parity.to_f64(lse[cand]) - rl) / np.maximum(np.abs(rl), 1.0)) <= 1e-3
+    assert np.max(np.abs(parity.to_f64(nll[cand]) - rn) / np.maximum(np.abs(rn), 1.0)) <= 1e-3
+    assert np.max(np.abs(parity.to_f64(loss[cand]) - rs) / np.maximum(np.abs(rs), 1.0)) <= 1e-3
+
+
+@pytest.mark.gpu
 def test_large_logits_need_the_running_maximum():
     """Hidden states x12: logits of +-40 and more, far outside what exp() without a max can take in the sum."""
     N, Lr, Dm, V = 8, 6, 256, 3000
