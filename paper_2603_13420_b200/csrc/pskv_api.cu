@@ -392,9 +392,7 @@ size_t pskv_attn_bwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S
 {
     Dims dm;
     if (Bp < 1 || B < Bp || B % Bp != 0 || check_dims(B / Bp, Hq, Hkv, S, Pmax, d, &dm) != PSKV_OK) return 0;
-    // one fp32 per query row; each instruction's part gets its own 256-byte aligned slice
-    const size_t part = round256((size_t)(B / Bp) * Hq * S * sizeof(float));
-    return part * (size_t)Bp;
+    return round256((size_t)B * Hq * S * sizeof(float));  // one fp32 per query row, all instructions in one array
 }
 
 namespace {
@@ -483,34 +481,63 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
 
     const int Kq = B / Bp;
     const size_t q_part = (size_t)Kq * Hq * S * d, s_part = (size_t)Kq * Hkv * S * d, l_part = (size_t)Kq * Hq * S;
-    const size_t ws_part = need / (size_t)Bp;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    auto fill = [&](BwdArgs &a, int first, const Dims &dm, size_t p_off) {
+        // arguments of the candidates [first*Kq, ...) with the prefix cache of one instruction
+        a.dout = static_cast<const __nv_bfloat16 *>(dout) + first * q_part;
+        a.q = static_cast<const __nv_bfloat16 *>(q) + first * q_part;
+        a.prefix_k = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_k) + p_off : nullptr;
+        a.prefix_v = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_v) + p_off : nullptr;
+        a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k) + first * s_part;
+        a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v) + first * s_part;
+        a.out = static_cast<const __nv_bfloat16 *>(out) + first * q_part;
+        a.lse = lse + first * l_part;
+        a.dq = static_cast<__nv_bfloat16 *>(dq) + first * q_part;
+        a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix) + first * s_part;
+        a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix) + first * s_part;
+        a.row_dot = static_cast<float *>(workspace) + first * l_part;  // one contiguous [B*Hq*S] array
+        a.dlse = nullptr;
+        a.suffix_len = nullptr;
+        a.scale = scale;
+        a.dims = dm;
+    };
+    // The row statistic D = <dout, out> and the suffix gradients do not involve the prefix: when every
+    // instruction's part runs on the tensor-core kernels they are done once over all B candidates, and
+    // only the dQ step runs once per instruction.
+    bool all_tc = true;
+    for (int i = 0; i < Bp && all_tc; ++i) {
+        Dims dm;
+        st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
+        if (st != PSKV_OK) return st;
+        all_tc = tc_bwd_supported(dm);
+    }
+    Dims whole;
+    st = check_dims(B, Hq, Hkv, S, prefix_len[0], d, &whole);
+    if (st != PSKV_OK) return st;
+    all_tc = all_tc && tc_bwd_supported(whole);
+    if (all_tc) {
+        BwdArgs a;
+        fill(a, 0, whole, 0);
+        cudaError_t e = launch_tc_bwd(a, workspace, status_word, stream, kBwdPartRowDot);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     for (int i = 0; i < Bp; ++i) {
         Dims dm;
         st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
         if (st != PSKV_OK) return st;
         dm.Pstride = Pmax;
         const size_t p_off = ((size_t)i * Hkv * Pmax + (size_t)(Pmax - prefix_len[i])) * d;
-        void *ws = static_cast<char *>(workspace) + i * ws_part;
         BwdArgs a;
-        a.dout = static_cast<const __nv_bfloat16 *>(dout) + i * q_part;
-        a.q = static_cast<const __nv_bfloat16 *>(q) + i * q_part;
-        a.prefix_k = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_k) + p_off : nullptr;
-        a.prefix_v = Pmax > 0 ? static_cast<const __nv_bfloat16 *>(prefix_v) + p_off : nullptr;
-        a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k) + i * s_part;
-        a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v) + i * s_part;
-        a.out = static_cast<const __nv_bfloat16 *>(out) + i * q_part;
-        a.lse = lse + i * l_part;
-        a.dq = static_cast<__nv_bfloat16 *>(dq) + i * q_part;
-        a.dk_suffix = static_cast<__nv_bfloat16 *>(dk_suffix) + i * s_part;
-        a.dv_suffix = static_cast<__nv_bfloat16 *>(dv_suffix) + i * s_part;
-        a.row_dot = static_cast<float *>(ws);
-        a.dlse = nullptr;
-        a.suffix_len = nullptr;
-        a.scale = scale;
-        a.dims = dm;
-        cudaError_t e = tc_bwd_supported(dm) ? launch_tc_bwd(a, ws, status_word, stream)
-                                             : launch_simt_bwd(a, stream);
+        fill(a, i, dm, p_off);
+        cudaError_t e = all_tc ? launch_tc_bwd(a, a.row_dot, status_word, stream, kBwdPartDq)
+                               : tc_bwd_supported(dm) ? launch_tc_bwd(a, a.row_dot, status_word, stream)
+                                                      : launch_simt_bwd(a, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (all_tc) {
+        BwdArgs a;
+        fill(a, 0, whole, 0);
+        cudaError_t e = launch_tc_bwd(a, workspace, status_word, stream, kBwdPartDkv);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return PSKV_OK;

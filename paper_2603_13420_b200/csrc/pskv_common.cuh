@@ -69,8 +69,12 @@ cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *statu
                           cudaStream_t stream);
 bool tc_bwd_supported(const Dims &d);
 size_t tc_bwd_workspace_bytes(const Dims &d);
+// `parts` selects which of the three steps run (all by default): the row statistic D and the suffix
+// gradients do not involve the prefix, so a caller with several prefixes runs them once over all
+// candidates and the dQ step once per prefix.
+enum { kBwdPartRowDot = 1, kBwdPartDq = 2, kBwdPartDkv = 4, kBwdPartAll = 7 };
 cudaError_t launch_tc_bwd(const BwdArgs &a, void *workspace, unsigned int *status_word,
-                          cudaStream_t stream);
+                          cudaStream_t stream, int parts = kBwdPartAll);
 
 // Masked target cross-entropy fused with the vocabulary projection (tcgen05 GEMM whose logits stay on chip).
 struct CeArgs {

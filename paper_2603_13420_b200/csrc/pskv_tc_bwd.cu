@@ -763,7 +763,7 @@ BwdPlan plan_bwd(const Dims &dm)
 }
 
 template <int D>
-cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_word, cudaStream_t stream)
+cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_word, cudaStream_t stream, int parts)
 {
     const Dims &dm = a.dims;
     const int Rg = dm.n_rep * dm.S;
@@ -830,17 +830,23 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
         attr_set[plan.resident] = true;
     }
     // D = <dout, out> per row, then dQ on the tensor cores, then dK_suffix / dV_suffix
-    cudaError_t e = launch_simt_row_dot(a, stream);
-    if (e != cudaSuccess) return e;
-    const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
-    {
-        KernelTiming timing(kKernelBwdDqTc, stream);
-        kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail,
-                                                            tm_sk, tm_sv, p);
+    cudaError_t e = cudaSuccess;
+    if (parts & kBwdPartRowDot) {
+        e = launch_simt_row_dot(a, stream);
+        if (e != cudaSuccess) return e;
     }
-    count_launches(1);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (parts & kBwdPartDq) {
+        const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
+        {
+            KernelTiming timing(kKernelBwdDqTc, stream);
+            kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,
+                                                                tm_pv_tail, tm_sk, tm_sv, p);
+        }
+        count_launches(1);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    if (!(parts & kBwdPartDkv)) return cudaSuccess;
     if (tc_bwd_dkv_supported(dm)) return launch_tc_bwd_dkv(a, status_word, stream);
     return mma_bwd_dkv_supported(dm) ? launch_mma_bwd_dkv(a, stream) : launch_simt_bwd_dkv(a, stream);
 }
@@ -876,11 +882,12 @@ bool tc_bwd_supported(const Dims &dm)
 
 size_t tc_bwd_workspace_bytes(const Dims &dm) { return (size_t)dm.B * dm.Hq * dm.S * sizeof(float); }
 
-cudaError_t launch_tc_bwd(const BwdArgs &a, void *, unsigned int *status_word, cudaStream_t stream)
+cudaError_t launch_tc_bwd(const BwdArgs &a, void *, unsigned int *status_word, cudaStream_t stream, int parts)
 {
     const BwdPlan plan = plan_bwd(a.dims);
     if (!plan.ok) return cudaErrorInvalidValue;
-    return a.dims.d == 128 ? launch<128>(a, plan, status_word, stream) : launch<64>(a, plan, status_word, stream);
+    return a.dims.d == 128 ? launch<128>(a, plan, status_word, stream, parts)
+                           : launch<64>(a, plan, status_word, stream, parts);
 }
 
 }  // namespace pskv
