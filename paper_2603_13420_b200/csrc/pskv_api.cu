@@ -101,7 +101,7 @@ std::mutex g_timing_mutex;
 bool g_timing_on = false;
 std::vector<TimedLaunch> g_timed;
 const char *const kKernelNames[kKernelCount] = {
-    "tc_fwd_kernel", "simt_fwd_redo_kernel", "simt_row_dot_kernel", "tc_bwd_dq_kernel", "tc_bwd_dkv_kernel",
+    "tc_fwd_kernel", "simt_row_dot_kernel", "tc_bwd_dq_kernel", "tc_bwd_dkv_kernel",
     "bwd_dkv_mma_kernel",
     "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel", "ce_fwd_kernel", "ce_finalize_kernel"};
 

@@ -59,8 +59,6 @@ bool mma_bwd_dkv_supported(const Dims &d);
 cudaError_t launch_mma_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
 bool tc_bwd_dkv_supported(const Dims &d);
 cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream);
-// Recomputes the rows whose lse is NaN, if *redo_count != 0 (a device counter); `blocks` CTAs.
-cudaError_t launch_simt_fwd_redo(const FwdArgs &a, const unsigned int *redo_count, int blocks, cudaStream_t stream);
 
 // tcgen05/TMEM kernels.  `status_word` is the device status flag that bounded waits set.
 bool tc_fwd_supported(const Dims &d);
@@ -94,7 +92,7 @@ void count_launches(int n);
 // Optional per-kernel device timing (pskv_kernel_timing_*): when enabled, a launch site brackets
 // its kernel with two CUDA events on the launch stream.
 enum KernelId {
-    kKernelFwdTc = 0, kKernelFwdRedo, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvTc, kKernelBwdDkvMma,
+    kKernelFwdTc = 0, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvTc, kKernelBwdDkvMma,
     kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCeFwd, kKernelCeFinalize, kKernelCount
 };
 void *timing_begin(int kernel_id, cudaStream_t stream);  // returns nullptr when timing is off

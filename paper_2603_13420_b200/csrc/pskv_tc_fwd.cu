@@ -23,6 +23,7 @@
 #include <string.h>
 
 #include "pskv_common.cuh"
+#include "pskv_rows.cuh"
 #include "pskv_sm100.cuh"
 #include "pskv_tc_common.cuh"
 
@@ -36,7 +37,7 @@ constexpr int kGroups = 4;     // softmax warpgroups: one 32-column piece of eve
 constexpr int kThreads = 32 * (4 + 4 * kGroups + 4);
 constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 // Probabilities are 2^(s * sl2) with no max subtracted; rows whose sum leaves
-// [kMinRowSum, kMaxRowSum] are redone by the general kernel.
+// [kMinRowSum, kMaxRowSum] are redone with max subtraction at the end of the kernel.
 constexpr float kMaxRowSum = 1.2676506002282294e30f;   // 2^100
 constexpr float kMinRowSum = 7.8886090522101181e-31f;  // 2^-100
 constexpr int kMaxStages = 4;
@@ -49,7 +50,7 @@ enum : unsigned int {
 struct TcFwdParams {
     float *lse;
     unsigned int *status;
-    unsigned int *redo_count;  // rows marked for the general kernel (zeroed before the launch)
+    FwdArgs args;         // the call's raw arguments, for the rows that are redone row by row
     float sl2;            // scale * log2(e)
     int B, Hq, Hkv, S, P, n_rep;
     int Rg;               // rows per candidate in one KV-head group: n_rep * S
@@ -169,6 +170,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + p.off_misc + 4);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + p.off_misc);
+    int *cta_redo = reinterpret_cast<int *>(smem + p.off_misc + 8);  // rows of this CTA's tiles to redo
     float *ml = reinterpret_cast<float *>(smem + p.off_ml);  // partial row sums [tile % 4][softmax group][128]
 
     if ((sbase & 1023u) != 0u) {  // the swizzled layouts need a 1024-byte aligned base
@@ -186,6 +188,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             mbar_init(bar(i), all_sm ? (uint32_t)(4 * kGroups) : epi ? 4u : 1u);
         }
         *abort_flag = 0;
+        *cta_redo = 0;
         fence_barrier_init();
     }
     fence_proxy_async();
@@ -691,7 +694,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         // itself).  No running max is subtracted: bf16 and fp32 share an 8-bit exponent, so the
         // quotient O / l is exact to rounding for any row whose sum stays within [2^-100, 2^100];
         // a row outside that range (essentially never, it means logits beyond +-69 nats) is
-        // redone afterwards by the general kernel with max subtraction.  The groups share no
+        // redone with max subtraction by this CTA once its tiles are finished.  The groups share no
         // state; their partial row sums meet in the epilogue, which the same warps run for the
         // previous tile (group j normalises O columns [32j, 32j+32)) right after the first item
         // of the next one, when that tile's last value MMAs have long completed.
@@ -893,7 +896,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 p.lse[grow] = row_ok ? log2f(l) * kLn2 : __int_as_float(0x7fc00000);
             }
             const unsigned bad = __ballot_sync(0xffffffffu, stored && !row_ok);
-            if (bad != 0u && lane == 0) atomicAdd(p.redo_count, (unsigned int)__popc(bad));
+            if (bad != 0u && lane == 0) atomicAdd(cta_redo, __popc(bad));
             PSKV_TRACE_EVENT(31, te);
         }
     }
@@ -904,6 +907,25 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == 2) tmem_dealloc(tmem, 512);
+    // Rows whose sum left the safe range carry a NaN lse (and zeros in `out`): all warps of the CTA
+    // now walk over its tiles and recompute those rows one warp per row with a running maximum.
+    // Every role has finished, the stores of `out` have completed, so the data area of shared
+    // memory is free: each warp stages its query row there.
+    if (*cta_redo > 0 && *abort_flag == 0) {
+        float *q_s = reinterpret_cast<float *>(smem) + warp * D;
+#pragma unroll 1
+        for (int tl = 0; tl < n_tiles; ++tl) {
+            const TileInfo t = tile_info(p, tile_at(tl), t_begin);
+#pragma unroll 1
+            for (int r = warp; r < t.rows; r += kThreads / 32) {
+                const int R = t.R0 + r;
+                const int b = p.fd_Rg.div(R), rr = R - b * p.Rg;
+                const long long grow = ((long long)b * p.Hq + (long long)t.g * p.n_rep) * p.S + rr;
+                const float v = p.lse[grow];
+                if (v != v) fwd_row<D>(p.args, grow, q_s, lane);
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -1085,7 +1107,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     TcFwdParams p;
     p.lse = a.lse;
     p.status = status_word;
-    p.redo_count = static_cast<unsigned int *>(workspace);
+    p.args = a;
     p.sl2 = a.scale * kLog2e;
     p.B = dm.B; p.Hq = dm.Hq; p.Hkv = dm.Hkv; p.S = dm.S; p.P = dm.P; p.n_rep = dm.n_rep;
     p.Rg = Rg;
@@ -1124,8 +1146,6 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
         if (e != cudaSuccess) return e;
         attr_set[plan.mode] = true;
     }
-    cudaError_t e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), stream);
-    if (e != cudaSuccess) return e;
     const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
     {
         KernelTiming timing(kKernelFwdTc, stream);
@@ -1133,10 +1153,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
                                                             tm_sv, p);
     }
     count_launches(1);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    // rows the tensor-core kernel marked (NaN lse) are recomputed with max subtraction
-    return launch_simt_fwd_redo(a, p.redo_count, sm_count(), stream);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -1167,7 +1184,7 @@ bool tc_fwd_supported(const Dims &dm)
     return plan_tiles(dm).ok;
 }
 
-size_t tc_fwd_workspace_bytes(const Dims &) { return 256; }  // the redo counter
+size_t tc_fwd_workspace_bytes(const Dims &) { return 0; }
 
 cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word, cudaStream_t stream)
 {
