@@ -6,16 +6,18 @@
 // kernel: 128-row tiles of the flat row list of a KV head, prefix blocks resident in shared memory
 // when they fit, one suffix block per tile with the block-diagonal causal mask.
 //
-// Persistent CTA, one per SM, 12 warps:
+// Persistent CTA, one per SM, 24 warps:
 //   warp 0      TMA producer: Q tile, prefix K blocks, suffix K
-//   warp 1      tcgen05.mma issuer: S = Q K^T and dP = dO V^T of every item
-//   warp 2      tcgen05.mma issuer: dQ += dS K  (owns the TMEM allocation)
+//   warp 1      tcgen05.mma issuer: S = Q K^T of every item
+//   warp 2      tcgen05.mma issuer: dP = dO V^T of the next item, then dQ += dS K of the current one
+//               (owns the TMEM allocation)
 //   warp 3      TMA producer: dO tile, prefix V blocks, suffix V
-//   warps 4-7   element-wise: thread <-> query row; dS = exp2(S*sl2 - lse2) * (dP - D) as bf16
-//   warps 8-11  epilogue: dQ from tensor memory, * scale, bf16, staging, TMA store
+//   warps 4-19  element-wise, four warpgroups sharing each item by 32-column pieces (thread <->
+//               query row): dS = exp2(S*sl2 - lse2) * (dP - D) as bf16
+//   warps 20-23 epilogue: dQ from tensor memory, * scale, bf16, staging, TMA store
 // Tensor memory: two 128-column S slots (dS overwrites the first half of its own slot), one dP
-// slot, and the 128 columns of dQ.  dK_suffix / dV_suffix and D are computed by the general
-// kernels around this one.  Every wait is bounded.
+// slot, and the 128 columns of dQ.  D comes from a streaming pre-pass, dK_suffix / dV_suffix from
+// a kernel of their own behind this one.  Every wait is bounded.
 #include <string.h>
 
 #include "pskv_common.cuh"

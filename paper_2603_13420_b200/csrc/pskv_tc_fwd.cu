@@ -9,17 +9,24 @@
 // partial results by their log-sum-exp), probabilities go back to tensor memory as bf16 and are
 // the A operand of the P*V contraction; `out` and `lse` are written once.
 //
-// Persistent CTA, one per SM, 20 warps:
+// Persistent CTA, one per SM, 24 warps:
 //   warp 0      TMA producer, score side (Q tile, prefix K blocks, suffix K of the tile)
 //   warp 1      tcgen05.mma issuer for the score blocks  S = Q K^T
 //   warp 2      tcgen05.mma issuer for the value blocks  O += P V   (owns the TMEM allocation)
 //   warp 3      TMA producer, value side (prefix V blocks, suffix V of the tile); TMA stores of `out`
 //   warps 4-19  softmax, four warpgroups sharing each item by 32-column pieces (thread <-> query
-//               row = TMEM lane); the same warps normalise the finished tile's O into staging
+//               row = TMEM lane)
+//   warps 20-23 epilogue: O / row sum -> bf16 -> staging buffer, lse
 // An "item" is one (tile, key block) pair; tensor memory holds three 128-column score slots (the
 // bf16 probabilities of an item overwrite parts of its own slot) and the 128 columns of O.  Every
 // wait is on an event produced by an earlier item of a role that never waits on the waiter, so
 // no wait cycle can form; every wait is bounded.
+//
+// Three instantiations share this code (see the comment at the kernel): prefix streamed through
+// rings, prefix resident in shared memory, and the suffix-ring mode, in which a tile is a run of
+// whole candidates (or of rows inside one candidate) and the suffix keys follow the prefix through
+// the same rings in as many blocks as it takes -- the mode of the decode-shaped operator, of
+// suffixes beyond one key block and of the causal self-attention of a single sequence.
 #include <string.h>
 
 #include "pskv_common.cuh"
