@@ -147,7 +147,10 @@ long long pskv_attn_bwd_static_max_rows(void);
  * must be a multiple of Bp and each cache is reused by its B / Bp candidates.  Everything else (q,
  * suffix_k, suffix_v, out, lse, dout, dq, dk_suffix, dv_suffix; scale; causal rule; error codes) is as
  * in pskv_attn_fwd / pskv_attn_bwd, with P replaced per candidate by the true prefix length of its
- * instruction.  The work is enqueued on `cuda_stream` as one pass per instruction.
+ * instruction.  The work is one pass per instruction; the passes are independent, so every other one
+ * is enqueued on a stream of the library's own that forks from `cuda_stream` at the start of the call
+ * and joins it again before the call returns (to the caller everything is ordered as if it had run on
+ * `cuda_stream`, also under stream capture).
  */
 size_t pskv_attn_fwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d);
 pskv_status pskv_attn_fwd_multi(const void *q,        /* bf16 [B,Hq,S,d] */

@@ -396,6 +396,35 @@ size_t pskv_attn_bwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S
 }
 
 namespace {
+// The passes of different instructions are independent, and each one fills the GPU with one
+// persistent CTA per SM, so back to back on one stream every pass pays its ramp-up, its uneven last
+// round and the launch gap in full.  Alternating the passes between the caller's stream and one
+// internal stream lets the CTAs of the next pass move onto SMs as the previous pass drains.  The
+// internal stream and the two events are created once per device; the mutex keeps the
+// fork / enqueue / join sequence of concurrent host threads apart.
+struct SideStream {
+    cudaStream_t stream;
+    cudaEvent_t fork, join;
+    int state;  // 0 = not created yet, 1 = usable, -1 = creation failed (passes then stay on the caller's stream)
+};
+SideStream g_side[kMaxDevices];
+std::mutex g_side_mutex;
+
+SideStream *side_stream()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    SideStream &ss = g_side[dev];
+    if (ss.state == 0) {
+        ss.state = -1;
+        if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) == cudaSuccess)
+            ss.state = 1;
+    }
+    return ss.state == 1 ? &ss : nullptr;
+}
+
 // checks shared by the two multi-instruction calls; fills the per-instruction geometry
 pskv_status check_multi(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d, const int *prefix_len)
 {
@@ -431,11 +460,24 @@ pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void 
     const int Kq = B / Bp;  // candidates per instruction, contiguous in the candidate dimension
     const size_t q_part = (size_t)Kq * Hq * S * d, s_part = (size_t)Kq * Hkv * S * d, l_part = (size_t)Kq * Hq * S;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    for (int i = 0; i < Bp; ++i) {
+    for (int i = 0; i < Bp; ++i) {  // all sizes are checked before anything is enqueued
         Dims dm;
         st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
         if (st != PSKV_OK) return st;
+    }
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    SideStream *side = Bp > 1 ? side_stream() : nullptr;
+    if (side) {
+        cudaError_t e = cudaEventRecord(side->fork, stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    pskv_status result = PSKV_OK;
+    for (int i = 0; i < Bp && result == PSKV_OK; ++i) {
+        Dims dm;
+        check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
         dm.Pstride = Pmax;
+        cudaStream_t pass_stream = (side && (i & 1)) ? side->stream : stream;
         // the real tokens of a left-padded prefix are its last prefix_len[i] rows
         const size_t p_off = ((size_t)i * Hkv * Pmax + (size_t)(Pmax - prefix_len[i])) * d;
         FwdArgs a;
@@ -449,11 +491,16 @@ pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void 
         a.suffix_len = nullptr;
         a.scale = scale;
         a.dims = dm;
-        cudaError_t e = tc_fwd_supported(dm) ? launch_tc_fwd(a, workspace, status_word, stream)
-                                             : launch_simt_fwd(a, stream);
-        if (e != cudaSuccess) return cuda_fail(e);
+        cudaError_t e = tc_fwd_supported(dm) ? launch_tc_fwd(a, workspace, status_word, pass_stream)
+                                             : launch_simt_fwd(a, pass_stream);
+        if (e != cudaSuccess) result = cuda_fail(e);
     }
-    return PSKV_OK;
+    if (side) {  // the caller's stream waits for the passes that ran beside it (also after an error)
+        cudaError_t e = cudaEventRecord(side->join, side->stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join, 0);
+        if (e != cudaSuccess && result == PSKV_OK) result = cuda_fail(e);
+    }
+    return result;
 }
 
 pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *prefix_k, const void *prefix_v,
@@ -521,19 +568,35 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         cudaError_t e = launch_tc_bwd(a, workspace, status_word, stream, kBwdPartRowDot);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    for (int i = 0; i < Bp; ++i) {
-        Dims dm;
-        st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
-        if (st != PSKV_OK) return st;
-        dm.Pstride = Pmax;
-        const size_t p_off = ((size_t)i * Hkv * Pmax + (size_t)(Pmax - prefix_len[i])) * d;
-        BwdArgs a;
-        fill(a, i, dm, p_off);
-        cudaError_t e = all_tc ? launch_tc_bwd(a, a.row_dot, status_word, stream, kBwdPartDq)
-                               : tc_bwd_supported(dm) ? launch_tc_bwd(a, a.row_dot, status_word, stream)
-                                                      : launch_simt_bwd(a, stream);
+    // the dQ passes of different instructions alternate between the caller's stream and the internal one
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    SideStream *side = (all_tc && Bp > 1) ? side_stream() : nullptr;
+    if (side) {
+        cudaError_t e = cudaEventRecord(side->fork, stream);  // behind the D pre-pass
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
         if (e != cudaSuccess) return cuda_fail(e);
     }
+    pskv_status result = PSKV_OK;
+    for (int i = 0; i < Bp && result == PSKV_OK; ++i) {
+        Dims dm;
+        st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
+        if (st != PSKV_OK) { result = st; break; }
+        dm.Pstride = Pmax;
+        const size_t p_off = ((size_t)i * Hkv * Pmax + (size_t)(Pmax - prefix_len[i])) * d;
+        cudaStream_t pass_stream = (side && (i & 1)) ? side->stream : stream;
+        BwdArgs a;
+        fill(a, i, dm, p_off);
+        cudaError_t e = all_tc ? launch_tc_bwd(a, a.row_dot, status_word, pass_stream, kBwdPartDq)
+                               : tc_bwd_supported(dm) ? launch_tc_bwd(a, a.row_dot, status_word, stream)
+                                                      : launch_simt_bwd(a, stream);
+        if (e != cudaSuccess) result = cuda_fail(e);
+    }
+    if (side) {
+        cudaError_t e = cudaEventRecord(side->join, side->stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join, 0);
+        if (e != cudaSuccess && result == PSKV_OK) result = cuda_fail(e);
+    }
+    if (result != PSKV_OK) return result;
     if (all_tc) {
         BwdArgs a;
         fill(a, 0, whole, 0);
