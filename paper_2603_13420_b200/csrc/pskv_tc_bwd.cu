@@ -879,7 +879,8 @@ bool tc_bwd_supported(const Dims &dm)
     if (dm.Skv != dm.S || dm.ragged) return false;  // full-suffix operator only
     if (dm.d != 64 && dm.d != 128) return false;
     if ((long long)dm.B * dm.n_rep * dm.S > 2000000000ll) return false;
-    return plan_bwd(dm).ok;
+    const BwdPlan pl = plan_bwd(dm);
+    return pl.ok && (long long)pl.tiles_per_group * dm.Hkv <= 2000000000ll;
 }
 
 size_t tc_bwd_workspace_bytes(const Dims &dm) { return (size_t)dm.B * dm.Hq * dm.S * sizeof(float); }

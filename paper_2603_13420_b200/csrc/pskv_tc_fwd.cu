@@ -1188,7 +1188,8 @@ bool tc_fwd_supported(const Dims &dm)
 {
     if (dm.d != 64 && dm.d != 128) return false;
     if ((long long)dm.B * dm.n_rep * dm.S > 2000000000ll) return false;  // flat row index fits an int
-    return plan_tiles(dm).ok;
+    const TilePlan pl = plan_tiles(dm);
+    return pl.ok && (long long)pl.tiles_per_group * dm.Hkv <= 2000000000ll;  // ... and so does the tile index
 }
 
 size_t tc_fwd_workspace_bytes(const Dims &) { return 0; }
