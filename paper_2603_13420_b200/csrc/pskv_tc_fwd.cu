@@ -823,11 +823,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         lsum += ls0 + ls1;
                         tmem_st16(s_tmem, pk);
                     }
-                    if (k == nitems - 1) ml[((tl & 3) * kGroups + wg) * kTileM + row] = lsum;
+                    if (k == nitems - 1) {
+                        // the tile's partial row sums go to the epilogue warps through shared memory
+                        ml[((tl & 3) * kGroups + wg) * kTileM + row] = lsum;
+                        __threadfence_block();
+                    }
                     PSKV_TRACE_EVENT(23, item);
                     tmem_wait_st();
                     tc_fence_before();
-                    __threadfence_block();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarPReady + slot));
                     PSKV_TRACE_EVENT(24, item);
