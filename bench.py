@@ -523,7 +523,11 @@ def decode_run(pskv, device, peaks, Bd, iters, warmup):
     nbytes = (2 * Bd * w.Hq * Sq * w.d + 2 * Bd * w.Hkv * Skv * w.d + 2 * w.Hkv * w.P * w.d) * 2 + Bd * w.Hq * Sq * 4
     return {"Sq": Sq, "Skv": Skv, "B": Bd, "algorithmic_bytes": nbytes,
             "fwd": {"ms": ms, "candidates_per_s": Bd / ms * 1e3, "hbm_gbs": nbytes / ms / 1e6,
-                    "pct_hbm_peak": 100 * nbytes / ms / 1e6 / peaks["hbm_gbs"]}}
+                    "pct_hbm_peak": 100 * nbytes / ms / 1e6 / peaks["hbm_gbs"]},
+            "roofline": {"kernel": "tc_fwd_kernel<128, 2>", "bound": "hbm", "achieved": nbytes / ms / 1e6,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": nbytes / ms / 1e6 / peaks["hbm_gbs"],
+                         "traffic": 449.3e6 if Bd == 2048 else None,  # profiles/tc_fwd_kernel_decode_B2048.md
+                         "note": "whole call timed with CUDA events (one kernel launch); peak = measured copy bandwidth"}}
 
 
 def prefill_run(pskv, device, peaks, iters, warmup):
@@ -543,7 +547,10 @@ def prefill_run(pskv, device, peaks, iters, warmup):
     ms = time_calls(prefill, iters, warmup)
     fl = 4.0 * w3.d * ((Sp + 1) / 2) * w3.Hq * Sp
     return {"fwd": {"ms": ms, "tflops": fl / ms / 1e9, "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
-                    "kernel_family": pskv.pskv_kernel_family(0, 1, w3.Hq, w3.Hkv, Sp, 0, w3.d)}}
+                    "kernel_family": pskv.pskv_kernel_family(0, 1, w3.Hq, w3.Hkv, Sp, 0, w3.d)},
+            "roofline": {"kernel": "tc_fwd_kernel<128, 2>", "bound": "tensor", "achieved": fl / ms / 1e9,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fl / ms / 1e9 / peaks["bf16_tflops"],
+                         "traffic": None, "note": "causal-visible flops; inputs (34 MB) are L2 resident as in use"}}
 
 
 def ce_run(pskv, device, peaks, iters, warmup, with_library=True):
@@ -572,7 +579,11 @@ def ce_run(pskv, device, peaks, iters, warmup, with_library=True):
            "fwd": {"ms": ms, "tflops": fl / ms / 1e9, "candidates_per_s": N / ms * 1e3,
                    "pct_bf16_peak_sustained": 100 * fl / ms / 1e9 / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
                    "pct_bf16_peak_burst": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
-                   "logits_bytes_never_written": 2.0 * N * Lr * V}}
+                   "logits_bytes_never_written": 2.0 * N * Lr * V},
+           "roofline": {"kernel": "ce_fwd_kernel", "bound": "tensor", "achieved": fl / ms / 1e9, "peak": peaks["bf16_tflops"],
+                        "unit": "TFLOP/s", "frac": fl / ms / 1e9 / peaks["bf16_tflops"],
+                        "traffic": 3.65e9,  # profiles/ce_fwd_kernel_512x20_V128256.md (algorithmic 1.13 GB)
+                        "note": "call = GEMM kernel + a 40 us finalize kernel; peak = measured bf16 burst (a library GEMM)"}}
     if with_library:
         tl = t.view(-1).long()
 
