@@ -49,6 +49,8 @@ def _load():
         lib.pskv_oracle_attn_bwd.restype = ctypes.c_int
         lib.pskv_oracle_attn_bwd_lse.argtypes = [dp] * 7 + [ctypes.c_double] + [dp] * 3 + ints
         lib.pskv_oracle_attn_bwd_lse.restype = ctypes.c_int
+        lib.pskv_oracle_attn_bwd_prefix.argtypes = [dp] * 7 + [ctypes.c_double] + [dp] * 2 + ints
+        lib.pskv_oracle_attn_bwd_prefix.restype = ctypes.c_int
         ip = ctypes.POINTER(ctypes.c_int)
         ints7 = [ctypes.c_int] * 7
         lib.pskv_oracle_attn_fwd_multi.argtypes = [dp] * 3 + [ip] + [dp] * 2 + [ctypes.c_double] + [dp] * 2 + ints7
@@ -144,6 +146,26 @@ def attn_bwd_lse(dout, dlse, q, prefix_k, prefix_v, suffix_k, suffix_v, scale):
     if rc != 0:
         raise RuntimeError("pskv_oracle_attn_bwd_lse failed with code %d" % rc)
     return dq, dk, dv
+
+
+def attn_bwd_prefix(dout, q, prefix_k, prefix_v, suffix_k, suffix_v, scale, dlse=None):
+    """dk_prefix, dv_prefix [Hkv,P,d] (fp64) of L = sum(out * dout) (+ sum(lse * dlse)): the gradients of the
+    shared prefix cache, summed over all candidates."""
+    B, Hq, Hkv, S, P, d = _dims(q, prefix_k, suffix_k)
+    do = _f64(dout, (B, Hq, S, d))
+    q = _f64(q, (B, Hq, S, d))
+    pk = _f64(prefix_k, (Hkv, P, d))
+    pv = _f64(prefix_v, (Hkv, P, d))
+    sk = _f64(suffix_k, (B, Hkv, S, d))
+    sv = _f64(suffix_v, (B, Hkv, S, d))
+    dl = None if dlse is None else _f64(dlse, (B, Hq, S))
+    dk = np.empty((Hkv, P, d), dtype=np.float64)
+    dv = np.empty((Hkv, P, d), dtype=np.float64)
+    rc = _load().pskv_oracle_attn_bwd_prefix(_ptr(do), None if dl is None else _ptr(dl), _ptr(q), _ptr(pk), _ptr(pv),
+                                             _ptr(sk), _ptr(sv), float(scale), _ptr(dk), _ptr(dv), B, Hq, Hkv, S, P, d)
+    if rc != 0:
+        raise RuntimeError("pskv_oracle_attn_bwd_prefix failed with code %d" % rc)
+    return dk, dv
 
 
 def _mask_i32(mask, Bp, Pmax):

@@ -558,3 +558,73 @@ int pskv_oracle_target_ce_fwd(const double *hidden, const double *weight, const 
     }
     return failed ? 2 : 0;
 }
+
+/*
+ * Gradients of the shared prefix cache (full differentiability; the search itself keeps the
+ * prefix frozen, Sec. 4.2).  The same closed form as pskv_oracle_attn_bwd, keeping what that
+ * function discards: for every prefix key j < P of KV head g
+ *   dk_prefix[g, j, :] = scale * sum over candidates b, heads h of g, rows i of  ds_j q[b,h,i,:]
+ *   dv_prefix[g, j, :] =         sum over the same (b, h, i) of                  p_j dout[b,h,i,:]
+ * with ds_j = p_j (dp_j - D + dlse[b,h,i]) (dlse may be NULL).  Because the cache is shared, the sums
+ * run over ALL candidates: one KV head per thread, candidates in order, so the result does not
+ * depend on the thread count.  dk_prefix, dv_prefix are [Hkv][P][d].
+ */
+int pskv_oracle_attn_bwd_prefix(const double *dout, const double *dlse, const double *q,
+                                const double *prefix_k, const double *prefix_v,
+                                const double *suffix_k, const double *suffix_v, double scale,
+                                double *dk_prefix, double *dv_prefix,
+                                int B, int Hq, int Hkv, int S, int P, int d)
+{
+    if (B < 1 || Hq < 1 || Hkv < 1 || S < 1 || P < 0 || d < 1 || Hq % Hkv != 0) return 1;
+    const int n_rep = Hq / Hkv;
+    const int T = P + S;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int g = 0; g < Hkv; ++g) {
+        double *Kf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *Vf = (double *)malloc(sizeof(double) * (size_t)T * d);
+        double *p = (double *)malloc(sizeof(double) * (size_t)T);
+        double *o = (double *)malloc(sizeof(double) * (size_t)d);
+        double *dKp = dk_prefix + (size_t)g * P * d;
+        double *dVp = dv_prefix + (size_t)g * P * d;
+        for (size_t e = 0; e < (size_t)P * d; ++e) { dKp[e] = 0.0; dVp[e] = 0.0; }
+        if (!Kf || !Vf || !p || !o) {
+            failed = 1;
+        } else {
+            for (int b = 0; b < B; ++b) {
+                build_full_kv(prefix_k, suffix_k, Kf, b, g, Hkv, S, P, d);
+                build_full_kv(prefix_v, suffix_v, Vf, b, g, Hkv, S, P, d);
+                for (int r = 0; r < n_rep; ++r) {
+                    const int h = g * n_rep + r;
+                    for (int i = 0; i < S; ++i) {
+                        const size_t row = ((size_t)b * Hq + h) * S + i;
+                        const int n_vis = P + i + 1;
+                        const double *qr = q + row * d;
+                        const double *go = dout + row * d;
+                        softmax_row(qr, Kf, n_vis, d, scale, p);
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n_vis; ++j)
+                            for (int c = 0; c < d; ++c) o[c] += p[j] * Vf[(size_t)j * d + c];
+                        double D = 0.0;
+                        for (int c = 0; c < d; ++c) D += go[c] * o[c];
+                        const double gl = dlse ? dlse[row] : 0.0;
+                        for (int j = 0; j < P; ++j) {
+                            double dp = 0.0;
+                            for (int c = 0; c < d; ++c) dp += go[c] * Vf[(size_t)j * d + c];
+                            const double ds = p[j] * (dp - D + gl);
+                            for (int c = 0; c < d; ++c) {
+                                dKp[(size_t)j * d + c] += scale * ds * qr[c];
+                                dVp[(size_t)j * d + c] += p[j] * go[c];
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        free(Kf);
+        free(Vf);
+        free(p);
+        free(o);
+    }
+    return failed ? 2 : 0;
+}
