@@ -429,6 +429,25 @@ def detail_runs(pskv, device, peaks):
         res[name] = entry
         del layer
         torch.cuda.empty_cache()
+    # Gradients of the shared prefix cache at C2 (optional path: the search keeps the prefix frozen)
+    w = wl.WORKLOADS["C2"]
+    layer = Layer(pskv, w, device_inputs(w, w.seed, device))
+    layer.fwd()
+    dkp, dvp = torch.empty_like(layer.t["prefix_k"]), torch.empty_like(layer.t["prefix_v"])
+    ws_p = torch.empty(pskv.pskv_attn_bwd_prefix_workspace_bytes(w.B, w.Hq, w.Hkv, w.S, w.P, w.d), dtype=torch.uint8,
+                       device=device)
+
+    def pgrad():
+        t = layer.t
+        pskv.pskv_attn_bwd_prefix(t["dout"], None, t["q"], t["prefix_k"], t["prefix_v"], layer.out, layer.lse, w.scale,
+                                  dk_prefix=dkp, dv_prefix=dvp, workspace=ws_p)
+
+    ms = time_calls(pgrad, 10, 3)
+    fl = 8.0 * w.d * w.P * w.B * w.Hq * w.S  # four contractions over (rows x prefix keys x d)
+    res["C2_prefix_gradients"] = {"ms": ms, "tflops": fl / ms / 1e9,
+                                  "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"]}
+    del layer, dkp, dvp, ws_p
+    torch.cuda.empty_cache()
     # C2 over 32 layers back to back: 32 calls on distinct per-layer tensors, one stream, no host sync
     w = wl.WORKLOADS["C2"]
     layers = [Layer(pskv, w, device_inputs(w, w.seed + 100 + i, device)) for i in range(32)]

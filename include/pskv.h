@@ -113,6 +113,28 @@ pskv_status pskv_attn_bwd_lse(const void *dout,   /* bf16 [B,Hq,S,d] */
                               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Gradients of the shared prefix cache: what pskv_attn_bwd leaves out.  The search keeps the prefix
+ * frozen (Sec. 4.2) and never needs them; a caller that wants full differentiability (a trainable
+ * prefix, a check of the whole backward) gets them here.  With p_j, D and ds_j as in pskv_attn_bwd
+ * (dlse may be NULL), for every prefix key j < P of KV head g
+ *   dk_prefix[g,j,:] = scale * sum over ALL candidates b, heads h of g and rows i of  ds_j q[b,h,i,:]
+ *   dv_prefix[g,j,:] =         sum over the same (b, h, i) of                          p_j dout[b,h,i,:]
+ * (every row sees every prefix key).  The suffix K/V are not needed: they enter only through `out`
+ * and `lse`, the forward results.  Sums are accumulated in fp32 (atomic adds across candidate chunks on
+ * the tensor-core path, so the last bits may differ from run to run) and rounded to bf16 once.
+ * P must be at least 1.  dk_prefix, dv_prefix: bf16 [Hkv,P,d], fully overwritten.
+ */
+size_t pskv_attn_bwd_prefix_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d);
+pskv_status pskv_attn_bwd_prefix(const void *dout,     /* bf16 [B,Hq,S,d] */
+                                 const float *dlse,    /* fp32 [B,Hq,S] or NULL */
+                                 const void *q, const void *prefix_k, const void *prefix_v,
+                                 const void *out, const float *lse, float scale,
+                                 void *dk_prefix,      /* bf16 [Hkv,P,d] */
+                                 void *dv_prefix,      /* bf16 [Hkv,P,d] */
+                                 int B, int Hq, int Hkv, int S, int P, int d,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * pskv_attn_bwd without a workspace argument.  (The paper has no counterpart; this is a
  * convenience of this library.)  It is for callers that cannot allocate device memory: processes
  * in which a framework allocator owns the whole card, or loops with a fixed memory plan in which a

@@ -59,6 +59,10 @@ def lib() -> ctypes.CDLL:
         L.pskv_attn_bwd.restype = ci
         L.pskv_attn_bwd_lse.argtypes = [vp] * 9 + [cf] + [vp] * 3 + six + [vp, sz, vp]
         L.pskv_attn_bwd_lse.restype = ci
+        L.pskv_attn_bwd_prefix_workspace_bytes.argtypes = six
+        L.pskv_attn_bwd_prefix_workspace_bytes.restype = sz
+        L.pskv_attn_bwd_prefix.argtypes = [vp] * 7 + [cf] + [vp] * 2 + six + [vp, sz, vp]
+        L.pskv_attn_bwd_prefix.restype = ci
         seven = [ci] * 7
         L.pskv_attn_fwd_multi_workspace_bytes.argtypes = seven
         L.pskv_attn_fwd_multi_workspace_bytes.restype = sz
@@ -240,6 +244,29 @@ def pskv_attn_bwd_lse(dout, dlse, q, prefix_k, prefix_v, suffix_k, suffix_v, out
     if st != PSKV_OK:
         raise PskvError(st, "pskv_attn_bwd_lse")
     return dq, dk_suffix, dv_suffix
+
+
+def pskv_attn_bwd_prefix_workspace_bytes(B, Hq, Hkv, S, P, d) -> int:
+    return int(lib().pskv_attn_bwd_prefix_workspace_bytes(B, Hq, Hkv, S, P, d))
+
+
+def pskv_attn_bwd_prefix(dout, dlse, q, prefix_k, prefix_v, out, lse, scale, dk_prefix=None, dv_prefix=None,
+                         workspace=None):
+    """Gradients of the shared prefix cache, dk_prefix / dv_prefix [Hkv,P,d] (bf16), summed over all
+    candidates; dlse (fp32 [B,Hq,S]) may be None."""
+    B, Hq, S, d = (int(x) for x in q.shape)
+    Hkv, P = int(prefix_k.shape[0]), int(prefix_k.shape[1])
+    if dk_prefix is None:
+        dk_prefix = torch.empty_like(prefix_k)
+    if dv_prefix is None:
+        dv_prefix = torch.empty_like(prefix_v)
+    ws = _workspace(pskv_attn_bwd_prefix_workspace_bytes(B, Hq, Hkv, S, P, d), q.device, workspace)
+    st = lib().pskv_attn_bwd_prefix(_ptr(dout), _ptr(dlse), _ptr(q), _ptr(prefix_k), _ptr(prefix_v), _ptr(out),
+                                    _ptr(lse), float(scale), _ptr(dk_prefix), _ptr(dv_prefix), B, Hq, Hkv, S, P, d,
+                                    _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_attn_bwd_prefix")
+    return dk_prefix, dv_prefix
 
 
 def _multi_dims(q, prefix_k, suffix_k, prefix_len):

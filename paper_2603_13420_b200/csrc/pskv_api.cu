@@ -1,6 +1,7 @@
 // C ABI of libpskv: host-side validation, kernel-family choice and launch.  No device memory
 // is allocated here; everything the kernels touch is passed in by the caller.
 #include <stdio.h>
+#include <string.h>
 
 #include <atomic>
 #include <mutex>
@@ -103,7 +104,7 @@ std::vector<TimedLaunch> g_timed;
 const char *const kKernelNames[kKernelCount] = {
     "tc_fwd_kernel", "simt_row_dot_kernel", "tc_bwd_dq_kernel", "tc_bwd_dkv_kernel",
     "bwd_dkv_mma_kernel",
-    "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel", "ce_fwd_kernel", "ce_finalize_kernel"};
+    "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel", "ce_fwd_kernel", "ce_finalize_kernel", "tc_bwd_prefix_kernel", "simt_bwd_prefix_kernel"};
 
 }  // namespace
 
@@ -604,6 +605,60 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return PSKV_OK;
+}
+
+// ---- gradients of the shared prefix cache ---------------------------------------------------------------
+
+size_t pskv_attn_bwd_prefix_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d)
+{
+    Dims dm;
+    if (check_dims(B, Hq, Hkv, S, P, d, &dm) != PSKV_OK || P < 1) return 0;
+    // one fp32 per query row (D), then the fp32 accumulators of both gradients
+    return round256((size_t)B * Hq * S * sizeof(float)) + round256(2 * (size_t)Hkv * P * d * sizeof(float));
+}
+
+pskv_status pskv_attn_bwd_prefix(const void *dout, const float *dlse, const void *q, const void *prefix_k,
+                                 const void *prefix_v, const void *out, const float *lse, float scale,
+                                 void *dk_prefix, void *dv_prefix, int B, int Hq, int Hkv, int S, int P, int d,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Dims dm;
+    pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
+    if (st != PSKV_OK) return st;
+    if (P < 1) return PSKV_ERR_INVALID_ARG;
+    if (!dout || !q || !prefix_k || !prefix_v || !out || !lse || !dk_prefix || !dv_prefix) return PSKV_ERR_INVALID_ARG;
+    if (!aligned16(dout) || !aligned16(dlse) || !aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) ||
+        !aligned16(out) || !aligned16(lse) || !aligned16(dk_prefix) || !aligned16(dv_prefix))
+        return PSKV_ERR_INVALID_ARG;
+    if (!(scale == scale) || scale <= 0.f || scale > 1.0e6f) return PSKV_ERR_INVALID_ARG;
+    const size_t need = pskv_attn_bwd_prefix_workspace_bytes(B, Hq, Hkv, S, P, d);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return PSKV_ERR_WORKSPACE;
+    unsigned int *status_word = nullptr;
+    st = check_device(&status_word);
+    if (st != PSKV_OK) return st;
+
+    BwdArgs a;
+    memset(&a, 0, sizeof(a));
+    a.dout = static_cast<const __nv_bfloat16 *>(dout);
+    a.q = static_cast<const __nv_bfloat16 *>(q);
+    a.prefix_k = static_cast<const __nv_bfloat16 *>(prefix_k);
+    a.prefix_v = static_cast<const __nv_bfloat16 *>(prefix_v);
+    a.out = static_cast<const __nv_bfloat16 *>(out);
+    a.lse = lse;
+    a.row_dot = static_cast<float *>(workspace);
+    a.dlse = dlse;
+    a.scale = scale;
+    a.dims = dm;
+    float *acc32 = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)B * Hq * S * sizeof(float)));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = launch_simt_row_dot(a, stream);  // D = <dout, out> - dlse per row
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = tc_bwd_prefix_supported(dm)
+            ? launch_tc_bwd_prefix(a, static_cast<__nv_bfloat16 *>(dk_prefix), static_cast<__nv_bfloat16 *>(dv_prefix),
+                                   acc32, status_word, stream)
+            : launch_simt_bwd_prefix(a, static_cast<__nv_bfloat16 *>(dk_prefix), static_cast<__nv_bfloat16 *>(dv_prefix),
+                                     stream);
+    return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
 }
 
 // ---- masked target cross-entropy fused with the vocabulary projection ---------------------------------

@@ -58,6 +58,13 @@ cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
 bool mma_bwd_dkv_supported(const Dims &d);
 cudaError_t launch_mma_bwd_dkv(const BwdArgs &a, cudaStream_t stream);
 bool tc_bwd_dkv_supported(const Dims &d);
+// Gradients of the shared prefix cache (need row_dot): tensor-core kernel (d = 128; `acc32` holds
+// 2 * Hkv * P * d floats of scratch) or the general one.
+bool tc_bwd_prefix_supported(const Dims &d);
+cudaError_t launch_tc_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __nv_bfloat16 *dv_prefix, float *acc32,
+                                 unsigned int *status_word, cudaStream_t stream);
+cudaError_t launch_simt_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __nv_bfloat16 *dv_prefix,
+                                   cudaStream_t stream);
 cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream);
 
 // tcgen05/TMEM kernels.  `status_word` is the device status flag that bounded waits set.
@@ -93,7 +100,7 @@ void count_launches(int n);
 // its kernel with two CUDA events on the launch stream.
 enum KernelId {
     kKernelFwdTc = 0, kKernelRowDot, kKernelBwdDqTc, kKernelBwdDkvTc, kKernelBwdDkvMma,
-    kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCeFwd, kKernelCeFinalize, kKernelCount
+    kKernelFwdSimt, kKernelBwdDqSimt, kKernelBwdDkvSimt, kKernelCeFwd, kKernelCeFinalize, kKernelBwdPrefixTc, kKernelBwdPrefixSimt, kKernelCount
 };
 void *timing_begin(int kernel_id, cudaStream_t stream);  // returns nullptr when timing is off
 void timing_end(void *token, cudaStream_t stream);

@@ -203,6 +203,63 @@ simt_bwd_dkv_kernel(BwdArgs a)
     store_slice<D>(a.dv_suffix + (size_t)key * D, lane, dv);
 }
 
+// Gradients of the shared prefix cache, general version: one warp per prefix key (g, j); sums over
+// every candidate, the n_rep heads of the group and all their rows (every row sees every prefix key).
+// Needs row_dot.  Deterministic (no atomics), and slow: it serves the shapes the tensor-core kernel
+// does not take.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_bwd_prefix_kernel(BwdArgs a, __nv_bfloat16 *dk_prefix, __nv_bfloat16 *dv_prefix)
+{
+    __shared__ float k_s[kWarpsPerBlock][D];
+    __shared__ float v_s[kWarpsPerBlock][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Dims dm = a.dims;
+    const long long key = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    if (key >= (long long)dm.Hkv * dm.P) return;
+    const int j = (int)(key % dm.P);
+    const int g = (int)(key / dm.P);
+    stage_row<D>(k_s[warp], a.prefix_k + ((size_t)g * dm.Pstride + j) * D, lane);
+    stage_row<D>(v_s[warp], a.prefix_v + ((size_t)g * dm.Pstride + j) * D, lane);
+    __syncwarp();
+    const float scale2 = a.scale * kLog2e;
+    const int per_cand = dm.n_rep * dm.S;
+    const long long n_rows = (long long)dm.B * per_cand;
+    float dk[D / 32], dv[D / 32];
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) { dk[e] = 0.f; dv[e] = 0.f; }
+    for (long long r0 = 0; r0 < n_rows; r0 += 32) {
+        const long long r = r0 + lane;
+        float p = 0.f, ds = 0.f;
+        if (r < n_rows) {
+            const int b = (int)(r / per_cand), rem = (int)(r - (long long)b * per_cand);
+            const size_t row = ((size_t)b * dm.Hq + (size_t)g * dm.n_rep) * dm.S + rem;  // heads of a group are contiguous
+            p = exp2f(scale2 * dot_row<D>(k_s[warp], a.q + row * D) - a.lse[row] * kLog2e);
+            ds = p * (dot_row<D>(v_s[warp], a.dout + row * D) - a.row_dot[row]);
+        }
+        const int cnt = (int)(n_rows - r0 < 32 ? n_rows - r0 : 32);
+        for (int u = 0; u < cnt; ++u) {
+            const float pu = __shfl_sync(0xffffffffu, p, u);
+            const float dsu = __shfl_sync(0xffffffffu, ds, u);
+            const long long rr = r0 + u;
+            const int b = (int)(rr / per_cand), rem = (int)(rr - (long long)b * per_cand);
+            const size_t row = ((size_t)b * dm.Hq + (size_t)g * dm.n_rep) * dm.S + rem;
+            float qv[D / 32], gv[D / 32];
+            load_slice<D>(a.q + row * D, lane, qv);
+            load_slice<D>(a.dout + row * D, lane, gv);
+#pragma unroll
+            for (int e = 0; e < D / 32; ++e) {
+                dk[e] = fmaf(dsu, qv[e], dk[e]);
+                dv[e] = fmaf(pu, gv[e], dv[e]);
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < D / 32; ++e) dk[e] *= a.scale;
+    store_slice<D>(dk_prefix + (size_t)key * D, lane, dk);
+    store_slice<D>(dv_prefix + (size_t)key * D, lane, dv);
+}
+
 inline unsigned int blocks_for(long long items)
 {
     return (unsigned int)((items + kWarpsPerBlock - 1) / kWarpsPerBlock);
@@ -244,6 +301,18 @@ cudaError_t launch_simt_bwd_dkv(const BwdArgs &a, cudaStream_t stream)
         simt_bwd_dkv_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
     else
         simt_bwd_dkv_kernel<64><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simt_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __nv_bfloat16 *dv_prefix, cudaStream_t stream)
+{
+    const long long keys = (long long)a.dims.Hkv * a.dims.P;
+    KernelTiming timing(kKernelBwdPrefixSimt, stream);
+    if (a.dims.d == 128)
+        simt_bwd_prefix_kernel<128><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a, dk_prefix, dv_prefix);
+    else
+        simt_bwd_prefix_kernel<64><<<blocks_for(keys), kWarpsPerBlock * 32, 0, stream>>>(a, dk_prefix, dv_prefix);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -23,6 +23,15 @@
 //               query row) and, at the end of a group, the write-back of the two accumulators
 // The arithmetic is tiny next to the bytes moved (Q and dO are read once, nothing else is big):
 // the kernel is bound by HBM, and everything is arranged to keep two tiles of copies in flight.
+//
+// The same kernel, instantiated with PRE = true, produces the gradients of the shared PREFIX cache
+// (which the search keeps frozen, Sec. 4.2, but a caller may want: full differentiability).  A unit
+// of work is then (KV head, block of 64 prefix keys, chunk of candidates): the block's K/V rows are
+// the operands, every key of the block is visible to every row, the row tiles of all candidates of
+// the chunk accumulate into the same transposed accumulators, and the write-back adds them into an
+// fp32 array in global memory (the chunks of one block meet there), which a small kernel rounds to
+// bf16 afterwards.  The key blocks of one (head, chunk) are numbered consecutively, so the CTAs
+// that re-read the same Q / dO rows run together and find them in L2.
 #include <string.h>
 
 #include "pskv_common.cuh"
@@ -71,8 +80,11 @@ struct TcDkvParams {
     float sl2, scale;
     int B, Hq, Hkv, S, n_rep, Rg;
     int TP;                // S rounded up to 16: the N of every MMA
-    int ntile;             // 128-row tiles per group
-    int total_groups;      // B * Hkv
+    int ntile;             // 128-row tiles per (candidate, KV head)
+    int total_groups;      // B * Hkv; prefix mode: Hkv * nbc * nkb
+    // prefix mode
+    float *dkp32, *dvp32;  // [Hkv][P][128] fp32 accumulators in global memory (zeroed before the launch)
+    int P, nkb, nbc, cpc;  // prefix length, key blocks of 64, candidate chunks, candidates per chunk
     FastDiv fd_S, fd_Hkv;
     // shared-memory byte offsets from the 1024-byte aligned base
     int off_q, off_do, off_k, off_v, off_p, off_ds, off_bar, off_misc, kv_bytes;
@@ -80,24 +92,42 @@ struct TcDkvParams {
 
 // unit u of a CTA -> (index of the group within this CTA, tile within the group)
 struct Unit {
-    int gi, tt, bg, b, g;
+    int gi, tt, bg, b, g, kb;
     bool first, last;
 };
+template <bool PRE>
 __device__ __forceinline__ Unit unit_of(const TcDkvParams &p, int u)
 {
     Unit x;
-    x.gi = u / p.ntile;
-    x.tt = u - x.gi * p.ntile;
-    x.bg = blockIdx.x + x.gi * gridDim.x;
-    x.b = p.fd_Hkv.div(x.bg);
-    x.g = x.bg - x.b * p.Hkv;
-    x.first = x.tt == 0;
-    x.last = x.tt == p.ntile - 1;
+    if (PRE) {
+        // group = (KV head, candidate chunk, key block), key block fastest; cpc * ntile units each
+        const int upg = p.cpc * p.ntile;
+        x.gi = u / upg;
+        const int w = u - x.gi * upg;
+        const int cb = w / p.ntile;
+        x.tt = w - cb * p.ntile;
+        x.bg = blockIdx.x + x.gi * gridDim.x;
+        const int rest = x.bg / p.nkb;
+        x.kb = x.bg - rest * p.nkb;
+        x.g = rest / p.nbc;
+        x.b = (rest - x.g * p.nbc) * p.cpc + cb;  // may be >= B in the last chunk: such tiles read as zero
+        x.first = w == 0;
+        x.last = w == upg - 1;
+    } else {
+        x.gi = u / p.ntile;
+        x.tt = u - x.gi * p.ntile;
+        x.bg = blockIdx.x + x.gi * gridDim.x;
+        x.b = p.fd_Hkv.div(x.bg);
+        x.g = x.bg - x.b * p.Hkv;
+        x.kb = 0;
+        x.first = x.tt == 0;
+        x.last = x.tt == p.ntile - 1;
+    }
     return x;
 }
 
-// NP = TP / 16: 16-key pieces per row
-template <int NP>
+// NP = TP / 16: 16-key pieces per row.  PRE: prefix-gradient mode (NP = 4).
+template <int NP, bool PRE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                   const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -141,10 +171,10 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t tmem = *tmem_slot;
 
     const int my_groups = (int)blockIdx.x < p.total_groups ? (p.total_groups - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int total_units = my_groups * p.ntile;
+    const int total_units = my_groups * (PRE ? p.cpc * p.ntile : p.ntile);
     const int box_rows = p.Rg < kTileM ? p.Rg : kTileM;  // rows one Q / dO copy brings (rows past Rg read as zero)
     const uint32_t tile_tx = (uint32_t)(2 * 2 * box_rows * 128);
-    const uint32_t kv_tx = (uint32_t)(2 * 2 * p.S * 128);
+    const uint32_t kv_tx = PRE ? (uint32_t)(2 * 2 * 64 * 128) : (uint32_t)(2 * 2 * p.S * 128);  // (a full box, zero-filled past P)
     const int kv_slab = TP * 128;
 
     if (warp == 0) {
@@ -158,7 +188,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         bool ok = true;
 #pragma unroll 1
         for (int u = 0; u < total_units && ok; ++u) {
-            const Unit x = unit_of(p, u);
+            const Unit x = unit_of<PRE>(p, u);
             const int st = u & 1;
             if (x.first) {
                 const int ks = x.gi & 1;
@@ -168,10 +198,17 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     mbar_arrive_expect_tx(bar(kBarKvFull + ks), kv_tx);
 #pragma unroll
                     for (int sl = 0; sl < 2; ++sl) {
-                        tma_load_4d(sbase + p.off_k + ks * p.kv_bytes + sl * kv_slab, &tm_k, bar(kBarKvFull + ks), sl * 64,
-                                    0, x.g, x.b);
-                        tma_load_4d(sbase + p.off_v + ks * p.kv_bytes + sl * kv_slab, &tm_v, bar(kBarKvFull + ks), sl * 64,
-                                    0, x.g, x.b);
+                        if (PRE) {
+                            tma_load_3d(sbase + p.off_k + ks * p.kv_bytes + sl * kv_slab, &tm_k, bar(kBarKvFull + ks),
+                                        sl * 64, x.kb * 64, x.g);
+                            tma_load_3d(sbase + p.off_v + ks * p.kv_bytes + sl * kv_slab, &tm_v, bar(kBarKvFull + ks),
+                                        sl * 64, x.kb * 64, x.g);
+                        } else {
+                            tma_load_4d(sbase + p.off_k + ks * p.kv_bytes + sl * kv_slab, &tm_k, bar(kBarKvFull + ks),
+                                        sl * 64, 0, x.g, x.b);
+                            tma_load_4d(sbase + p.off_v + ks * p.kv_bytes + sl * kv_slab, &tm_v, bar(kBarKvFull + ks),
+                                        sl * 64, 0, x.g, x.b);
+                        }
                     }
                 }
                 __syncwarp();
@@ -179,13 +216,13 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             // the copies of unit u + 2 can only be issued when this stage is free again: ask for
             // its rows in L2 now, so that they are close by then
             if (u + 2 < total_units) {
-                const Unit y = unit_of(p, u + 2);
+                const Unit y = unit_of<PRE>(p, u + 2);
                 if (elect_one_sync()) {
 #pragma unroll
                     for (int sl = 0; sl < 2; ++sl) {
                         tma_prefetch_4d(&tm_q, sl * 64, y.tt * kTileM, y.g, y.b);
                         tma_prefetch_4d(&tm_do, sl * 64, y.tt * kTileM, y.g, y.b);
-                        if (y.first) {
+                        if (y.first && !PRE) {
                             tma_prefetch_4d(&tm_k, sl * 64, 0, y.g, y.b);
                             tma_prefetch_4d(&tm_v, sl * 64, 0, y.g, y.b);
                         }
@@ -215,7 +252,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         bool ok = true;
         // score side of unit u: S = Q K_s^T, dP = dO V_s^T
         auto score_pair = [&](int u) -> bool {
-            const Unit x = unit_of(p, u);
+            const Unit x = unit_of<PRE>(p, u);
             const int st = u & 1, ks = x.gi & 1;
             if (!mbar_wait_warp(bar(kBarQFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvMma)) return false;
             if (x.first && !mbar_wait_warp(bar(kBarKvFull + ks), (x.gi >> 1) & 1, abort_flag, p.status, kErrDkvMma))
@@ -243,7 +280,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         };
         // gradient side of unit v: dV^T += dO^T P, dK^T += Q^T dS
         auto grad_pair = [&](int v) -> bool {
-            const Unit x = unit_of(p, v);
+            const Unit x = unit_of<PRE>(p, v);
             const int st = v & 1, ks = x.gi & 1, as = x.gi & 1;
             if (!mbar_wait_warp(bar(kBarPReady), v & 1, abort_flag, p.status, kErrDkvMma)) return false;
             // the accumulator set must have been written back by the group that used it before
@@ -307,6 +344,10 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const int bg = blockIdx.x + gi * gridDim.x;
             __nv_bfloat16 *dvg = p.dv + (size_t)bg * p.S * kD + row;
             __nv_bfloat16 *dkg = p.dk + (size_t)bg * p.S * kD + row;
+            // prefix mode: key block and KV head of the group, keys of the block that exist
+            const int rest = PRE ? bg / p.nkb : 0;
+            const int kb = bg - rest * p.nkb, gh = PRE ? rest / p.nbc : 0;
+            const int nkeys = PRE ? min(64, p.P - kb * 64) : 0;
             if (wg < NP) {
                 uint32_t av[16], ak[16];
                 const uint32_t acc = tmem + lane_addr + kColAcc + as * kAccCols;
@@ -316,12 +357,26 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarAccFree + as));
+                if (PRE) {
+                    // the candidate chunks of a key block meet in global memory: lane <-> d, coalesced adds
+                    float *av32 = p.dvp32 + ((size_t)gh * p.P + (size_t)kb * 64) * kD + row;
+                    float *ak32 = p.dkp32 + ((size_t)gh * p.P + (size_t)kb * 64) * kD + row;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const int t = wg * 16 + c;
-                    if (t < p.S) {
-                        dvg[(size_t)t * kD] = __float2bfloat16_rn(__uint_as_float(av[c]));
-                        dkg[(size_t)t * kD] = __float2bfloat16_rn(__uint_as_float(ak[c]) * p.scale);
+                    for (int c = 0; c < 16; ++c) {
+                        const int t = wg * 16 + c;
+                        if (t < nkeys) {
+                            atomicAdd(av32 + (size_t)t * kD, __uint_as_float(av[c]));
+                            atomicAdd(ak32 + (size_t)t * kD, __uint_as_float(ak[c]) * p.scale);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const int t = wg * 16 + c;
+                        if (t < p.S) {
+                            dvg[(size_t)t * kD] = __float2bfloat16_rn(__uint_as_float(av[c]));
+                            dkg[(size_t)t * kD] = __float2bfloat16_rn(__uint_as_float(ak[c]) * p.scale);
+                        }
                     }
                 }
             } else {
@@ -334,12 +389,13 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         };
 #pragma unroll 1
         for (int u = 0; u < total_units && ok; ++u) {
-            const Unit x = unit_of(p, u);
+            const Unit x = unit_of<PRE>(p, u);
             const int st = u & 1;
             const int gr = x.tt * kTileM + row;  // row inside the group: head-major, then position
-            const bool valid = gr < p.Rg;
+            const bool valid = gr < p.Rg && (!PRE || x.b < p.B);
             const size_t row0 = ((size_t)x.b * p.Hq + (size_t)x.g * p.n_rep) * p.S;
-            const int i_pos = valid ? gr - p.fd_S.div(gr) * p.S : -1;  // causal: key t is visible when t <= i
+            // causal: suffix key t is visible when t <= i; prefix mode: every key of the block that exists
+            const int i_pos = !valid ? -1 : PRE ? min(64, p.P - x.kb * 64) - 1 : gr - p.fd_S.div(gr) * p.S;
             const float nl2 = valid ? -p.lse[row0 + gr] * kLog2e : 0.f;
             const float dr = valid ? p.row_dot[row0 + gr] : 0.f;
             ok = mbar_wait_warp(bar(kBarSFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
@@ -408,21 +464,31 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
 // ------------------------------------------------------------------------------ host side
 
-template <int NP>
+template <int NP, bool PRE>
 cudaError_t launch_np(const BwdArgs &a, const CUtensorMap &tm_q, const CUtensorMap &tm_do, const CUtensorMap &tm_k,
                       const CUtensorMap &tm_v, const TcDkvParams &p, int smem_bytes, cudaStream_t stream)
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_bwd_dkv_kernel<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        cudaError_t e = cudaFuncSetAttribute(tc_bwd_dkv_kernel<NP, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     const int grid = p.total_groups < sm_count() ? p.total_groups : sm_count();
-    KernelTiming timing(kKernelBwdDkvTc, stream);
-    tc_bwd_dkv_kernel<NP><<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_do, tm_k, tm_v, p);
+    KernelTiming timing(PRE ? kKernelBwdPrefixTc : kKernelBwdDkvTc, stream);
+    tc_bwd_dkv_kernel<NP, PRE><<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_do, tm_k, tm_v, p);
     count_launches(1);
     return cudaGetLastError();
+}
+
+// fp32 accumulators -> bf16 results
+__global__ void __launch_bounds__(256)
+prefix_grad_round_kernel(const float *acc_k, const float *acc_v, __nv_bfloat16 *dk, __nv_bfloat16 *dv, size_t n)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        dk[i] = __float2bfloat16_rn(acc_k[i]);
+        dv[i] = __float2bfloat16_rn(acc_v[i]);
+    }
 }
 
 }  // namespace
@@ -503,11 +569,86 @@ cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaS
         if (!encode_map(&tm_v, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
     switch (TP / 16) {
-    case 1: return launch_np<1>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
-    case 2: return launch_np<2>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
-    case 3: return launch_np<3>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
-    default: return launch_np<4>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    case 1: return launch_np<1, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    case 2: return launch_np<2, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    case 3: return launch_np<3, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    default: return launch_np<4, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
     }
+}
+
+bool tc_bwd_prefix_supported(const Dims &dm)
+{
+    if (dm.Skv != dm.S || dm.ragged) return false;
+    return dm.d == kD && dm.P >= 1 && (long long)dm.n_rep * dm.S < 2000000000ll &&
+           (long long)dm.Hkv * ((dm.P + 63) / 64) * 4096ll < 2000000000ll;
+}
+
+// dk_prefix / dv_prefix [Hkv][P][128] (bf16) from a.row_dot (already computed), through `acc32`
+// (2 * Hkv * P * 128 floats of scratch).
+cudaError_t launch_tc_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __nv_bfloat16 *dv_prefix, float *acc32,
+                                 unsigned int *status_word, cudaStream_t stream)
+{
+    const Dims &dm = a.dims;
+    const int Rg = dm.n_rep * dm.S;
+    const size_t n_acc = (size_t)dm.Hkv * dm.P * kD;
+    TcDkvParams p;
+    memset(&p, 0, sizeof(p));
+    p.lse = a.lse;
+    p.row_dot = a.row_dot;
+    p.status = status_word;
+    p.sl2 = a.scale * kLog2e;
+    p.scale = a.scale;
+    p.B = dm.B; p.Hq = dm.Hq; p.Hkv = dm.Hkv; p.S = dm.S; p.n_rep = dm.n_rep; p.Rg = Rg;
+    p.TP = 64;
+    p.ntile = (Rg + kTileM - 1) / kTileM;
+    p.P = dm.P;
+    p.nkb = (dm.P + 63) / 64;
+    // enough candidate chunks for about two groups per SM, so that the tail of the launch is short
+    int nbc = (2 * sm_count() + dm.Hkv * p.nkb - 1) / (dm.Hkv * p.nkb);
+    if (nbc > dm.B) nbc = dm.B;
+    if (nbc < 1) nbc = 1;
+    p.cpc = (dm.B + nbc - 1) / nbc;
+    p.nbc = (dm.B + p.cpc - 1) / p.cpc;
+    p.total_groups = dm.Hkv * p.nbc * p.nkb;
+    p.dkp32 = acc32;
+    p.dvp32 = acc32 + n_acc;
+    p.fd_S.init(dm.S);
+    p.fd_Hkv.init(dm.Hkv);
+    p.kv_bytes = round_up(2 * 64 * 128, 1024);
+    p.off_q = 0;
+    p.off_do = p.off_q + 2 * kTileBytes;
+    p.off_k = p.off_do + 2 * kTileBytes;
+    p.off_v = p.off_k + 2 * p.kv_bytes;
+    p.off_p = p.off_v + 2 * p.kv_bytes;
+    p.off_ds = p.off_p + kSlabBytes;
+    p.off_bar = p.off_ds + kSlabBytes;
+    p.off_misc = p.off_bar + 256;
+    const int smem_bytes = p.off_misc + 64;
+    if (smem_bytes > kMaxSmem) return cudaErrorInvalidConfiguration;
+
+    CUtensorMap tm_q, tm_do, tm_k, tm_v;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)Rg, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
+        cuuint64_t str[3] = {(cuuint64_t)kD * 2, (cuuint64_t)Rg * kD * 2, (cuuint64_t)dm.Hkv * Rg * kD * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)(Rg < kTileM ? Rg : kTileM), 1, 1};
+        if (!encode_map(&tm_q, a.q, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_do, a.dout, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
+        cuuint64_t str[2] = {(cuuint64_t)kD * 2, (cuuint64_t)dm.Pstride * kD * 2};
+        cuuint32_t box[3] = {64, 64, 1};
+        if (!encode_map(&tm_k, a.prefix_k, 3, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_v, a.prefix_v, 3, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    cudaError_t e = cudaMemsetAsync(acc32, 0, 2 * n_acc * sizeof(float), stream);
+    if (e != cudaSuccess) return e;
+    e = launch_np<4, true>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    if (e != cudaSuccess) return e;
+    const int blocks = (int)((n_acc + 255) / 256 < 1184 ? (n_acc + 255) / 256 : 1184);
+    prefix_grad_round_kernel<<<blocks, 256, 0, stream>>>(p.dkp32, p.dvp32, dk_prefix, dv_prefix, n_acc);
+    count_launches(1);
+    return cudaGetLastError();
 }
 
 }  // namespace pskv
