@@ -4,7 +4,11 @@ Candidates are independent given the prefix cache (each one reads the shared pre
 its own suffix K/V only), so the multi-GPU path splits the candidate dimension, replicates
 the small prefix cache on every rank and needs no collective on the data path -- the paper's
 data-parallel case, where every rank keeps the prefix caches of its local batch and no
-all-gather of caches takes place (Appendix G.6).  The helpers here are host-side only.
+all-gather of caches takes place (Appendix G.6).  The one exchange step belongs to the optional
+gradients of the shared prefix cache: they are sums over ALL candidates, so each rank's
+`pskv_attn_bwd_prefix` result covers only its own candidates and the ranks' results are summed
+(`allreduce_prefix_gradients`, one all-reduce of 2 * Hkv * P * d values).  The helpers here are
+host-side only.
 """
 from __future__ import annotations
 
@@ -36,3 +40,17 @@ def max_over_ranks(values, device=None):
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(x, op=dist.ReduceOp.MAX)
     return x.tolist()
+
+
+def allreduce_prefix_gradients(dk_prefix: torch.Tensor, dv_prefix: torch.Tensor):
+    """Sum the per-rank gradients of the shared prefix cache over all ranks, in place (NCCL on CUDA
+    tensors, gloo on CPU tensors).  The sum is taken in fp32: a bf16 all-reduce would round once per
+    rank.  No-op without an initialised process group."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1):
+        return dk_prefix, dv_prefix
+    both = torch.stack([dk_prefix.to(torch.float32), dv_prefix.to(torch.float32)])
+    dist.all_reduce(both, op=dist.ReduceOp.SUM)
+    dk_prefix.copy_(both[0])
+    dv_prefix.copy_(both[1])
+    return dk_prefix, dv_prefix

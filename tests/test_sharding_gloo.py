@@ -1,6 +1,8 @@
 """The N > 1 path on CPU: two gloo ranks shard the candidates, each evaluates its shard against
 a replicated prefix cache (here with the oracle standing in for the device), and the gathered
-result equals the unsharded one -- no collective is needed on the data path."""
+result equals the unsharded one -- no collective is needed on the data path.  The optional
+gradients of the shared prefix cache are the exception: sums over all candidates, so the ranks'
+partial results meet in one all-reduce."""
 import os
 import socket
 
@@ -52,6 +54,15 @@ def _worker(rank, world, port, ret):
         gathered = [None] * world
         dist.all_gather_object(gathered, (rank, out, lse))
         slow = shard.max_over_ranks([1.0 + rank, 5.0 - rank])
+        # prefix-cache gradients: each rank's covers its own candidates; one all-reduce sums them
+        gen = torch.Generator(device="cpu")
+        gen.manual_seed(11)
+        dout_full = torch.randn(t["q"].shape, generator=gen, dtype=torch.float64).numpy()
+        lo, hi = shard.candidate_range(t["q"].shape[0], world, rank)
+        pk_g, pv_g = oracle.attn_bwd_prefix(dout_full[lo:hi], f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"],
+                                            f["suffix_v"], w.scale)
+        dkp, dvp = torch.from_numpy(pk_g).to(torch.float32), torch.from_numpy(pv_g).to(torch.float32)
+        shard.allreduce_prefix_gradients(dkp, dvp)
         if rank == 0:
             full = {k: v.to(torch.float64).numpy() for k, v in t.items()}
             ro, rl = oracle.attn_fwd(full["q"], full["prefix_k"], full["prefix_v"], full["suffix_k"],
@@ -59,6 +70,9 @@ def _worker(rank, world, port, ret):
             go = np.concatenate([g[1] for g in sorted(gathered, key=lambda g: g[0])], axis=0)
             gl = np.concatenate([g[2] for g in sorted(gathered, key=lambda g: g[0])], axis=0)
             ret["ok"] = bool(np.array_equal(go, ro) and np.array_equal(gl, rl))
+            fk, fv = oracle.attn_bwd_prefix(dout_full, full["q"], full["prefix_k"], full["prefix_v"], full["suffix_k"],
+                                            full["suffix_v"], w.scale)
+            ret["prefix_grad_err"] = float(max(np.max(np.abs(dkp.numpy() - fk)), np.max(np.abs(dvp.numpy() - fv))))
             ret["max"] = slow
     finally:
         dist.destroy_process_group()
@@ -72,3 +86,4 @@ def test_two_rank_candidate_sharding_matches_unsharded():
     mp.spawn(_worker, args=(world, port, ret), nprocs=world, join=True)
     assert ret["ok"] is True
     assert ret["max"] == [2.0, 5.0]
+    assert ret["prefix_grad_err"] < 1e-5   # fp32 all-reduce of fp64-computed partial sums
