@@ -429,25 +429,7 @@ def detail_runs(pskv, device, peaks):
         res[name] = entry
         del layer
         torch.cuda.empty_cache()
-    # Gradients of the shared prefix cache at C2 (optional path: the search keeps the prefix frozen)
-    w = wl.WORKLOADS["C2"]
-    layer = Layer(pskv, w, device_inputs(w, w.seed, device))
-    layer.fwd()
-    dkp, dvp = torch.empty_like(layer.t["prefix_k"]), torch.empty_like(layer.t["prefix_v"])
-    ws_p = torch.empty(pskv.pskv_attn_bwd_prefix_workspace_bytes(w.B, w.Hq, w.Hkv, w.S, w.P, w.d), dtype=torch.uint8,
-                       device=device)
-
-    def pgrad():
-        t = layer.t
-        pskv.pskv_attn_bwd_prefix(t["dout"], None, t["q"], t["prefix_k"], t["prefix_v"], layer.out, layer.lse, w.scale,
-                                  dk_prefix=dkp, dv_prefix=dvp, workspace=ws_p)
-
-    ms = time_calls(pgrad, 10, 3)
-    fl = 8.0 * w.d * w.P * w.B * w.Hq * w.S  # four contractions over (rows x prefix keys x d)
-    res["C2_prefix_gradients"] = {"ms": ms, "tflops": fl / ms / 1e9,
-                                  "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"]}
-    del layer, dkp, dvp, ws_p
-    torch.cuda.empty_cache()
+    res["C2_prefix_gradients"] = prefix_grad_run(pskv, device, peaks, 10, 3)
     # C2 over 32 layers back to back: 32 calls on distinct per-layer tensors, one stream, no host sync
     w = wl.WORKLOADS["C2"]
     layers = [Layer(pskv, w, device_inputs(w, w.seed + 100 + i, device)) for i in range(32)]
@@ -614,6 +596,26 @@ def ce_run(pskv, device, peaks, iters, warmup, with_library=True):
     return out
 
 
+def prefix_grad_run(pskv, device, peaks, iters, warmup):
+    """Gradients of the shared prefix cache at C2 (optional path: the search keeps the prefix frozen)."""
+    w = wl.WORKLOADS["C2"]
+    layer = Layer(pskv, w, device_inputs(w, w.seed, device))
+    layer.fwd()
+    dkp, dvp = torch.empty_like(layer.t["prefix_k"]), torch.empty_like(layer.t["prefix_v"])
+    ws_p = torch.empty(pskv.pskv_attn_bwd_prefix_workspace_bytes(w.B, w.Hq, w.Hkv, w.S, w.P, w.d), dtype=torch.uint8,
+                       device=device)
+
+    def pgrad():
+        t = layer.t
+        pskv.pskv_attn_bwd_prefix(t["dout"], None, t["q"], t["prefix_k"], t["prefix_v"], layer.out, layer.lse, w.scale,
+                                  dk_prefix=dkp, dv_prefix=dvp, workspace=ws_p)
+
+    ms = time_calls(pgrad, iters, warmup)
+    fl = 8.0 * w.d * w.P * w.B * w.Hq * w.S  # four contractions over (rows x prefix keys x d)
+    return {"ms": ms, "tflops": fl / ms / 1e9, "pct_bf16_peak": 100 * fl / ms / 1e9 / peaks["bf16_tflops"],
+            "algorithmic_flops": fl}
+
+
 def run_variant(args):
     """One variant's timing loop alone (for profiling it without the rest of the benchmark)."""
     if not torch.cuda.is_available():
@@ -624,6 +626,8 @@ def run_variant(args):
     peaks = load_peaks()
     if args.variant == "prefill":
         res = prefill_run(pskv, device, peaks, args.steps, max(args.warmup, 3))
+    elif args.variant == "prefix_grad":
+        res = prefix_grad_run(pskv, device, peaks, args.steps, max(args.warmup, 3))
     elif args.variant == "target_ce":
         res = ce_run(pskv, device, peaks, args.steps, max(args.warmup, 3), with_library=False)
     else:
@@ -661,7 +665,7 @@ def main():
                     help="candidates of the one-off CPU oracle sample reported as cpu_baseline")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
-    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill", "target_ce"],
+    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill", "target_ce", "prefix_grad"],
                     help="time only this variant of the detail runs (1 GPU) and print its entry")
     args = ap.parse_args()
     if args.impl == "reference":
