@@ -122,6 +122,30 @@ def test_growing_the_suffix_token_by_token_reproduces_the_full_evaluation():
         assert (l1 - l_full[:, :, L - 1:L]).abs().max().item() <= 1e-3 * max(1.0, l_full.abs().max().item())
 
 
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", [(40, 8, 2, 1, 24, 200, 128), (3, 8, 2, 256, 256, 100, 128)])
+def test_rows_outside_the_safe_exponent_range_are_redone_in_every_tiling(shape):
+    """Scores of several hundred nats in a few rows: the tensor-core kernel marks those rows and recomputes
+    them with a running maximum, also when its tiles are whole candidates (decode) or lie inside one
+    candidate (long suffix)."""
+    B, Hq, Hkv, Sq, Skv, P, d = shape
+    t, _ = make(B, Hq, Hkv, Sq, Skv, P, d, False)
+    q = t["q"].float()
+    q[1, 2, 0] *= 60.0
+    q[B - 1, 0, Sq - 1] *= 45.0
+    q[0, Hq - 1, Sq // 2] *= -50.0
+    t["q"] = q.to(torch.bfloat16)
+    scale = 1.0 / np.sqrt(d)
+    out, lse = pskv.pskv_attn_fwd_decode(t["q"].cuda(), t["prefix_k"].cuda(), t["prefix_v"].cuda(), t["suffix_k"].cuda(),
+                                         t["suffix_v"].cuda(), None, scale)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    f = {k: parity.to_f64(v) for k, v in t.items()}
+    ro, rl = oracle.attn_fwd_decode(f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"], scale)
+    assert np.abs(rl).max() > 100.0
+    parity.check_tensor("out", parity.to_f64(out), ro)
+    parity.check_lse(parity.to_f64(lse), rl)
+
+
 def test_decode_arguments_are_checked_on_the_host():
     L = pskv.binding.lib()
     fake = ctypes.c_void_p(4096)
