@@ -136,7 +136,7 @@ using namespace pskv;
 
 extern "C" {
 
-int pskv_version(void) { return 100; }
+int pskv_version(void) { return 200; }
 
 long long pskv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
