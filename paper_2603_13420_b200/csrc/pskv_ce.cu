@@ -12,9 +12,9 @@
 // quarter of the CTA count; inside a group the units are numbered panel-major, row tile fastest, and
 // CTA c takes units c, c + G, c + 2G, ...: the CTAs running at any moment work on about four weight
 // panels (16 MB each) against one group of row tiles (1 MB each), a working set that stays in L2, so
-// the weight matrix comes from HBM once per row group and the hidden states once.  Each unit leaves one partial (max, sum) per row; a small second
-// kernel merges the partials of a row, forms nll = mask * (lse - target logit) and the masked
-// average per candidate.
+// the weight matrix comes from HBM once per row group and the hidden states once.  Each unit
+// leaves one partial (max, sum) per row; two small kernels merge the partials of a row into lse
+// and nll = mask * (lse - target logit) and form the masked average per candidate.
 //
 // Roles (256 threads): warp 0 TMA producer (hidden tile and weight block, 64 columns of the hidden
 // dimension per stage, 4 stages), warp 1 tcgen05.mma issuer, warp 2 owns the tensor-memory
@@ -250,31 +250,40 @@ ce_fwd_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ 
     if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
-// Merges the partials of every row and reduces per candidate: one warp per candidate.
+// Merges the partials of every row: one thread per row (consecutive threads read consecutive
+// addresses of every panel's partial arrays), lse and nll per row.
 __global__ void __launch_bounds__(256)
-ce_finalize_kernel(const float *part_m, const float *part_l, const float *tlogit, const int *target,
-                   const float *mask, float *nll, float *lse, float *loss, int N, int Lr, int Rpad, int npanel, int V)
+ce_rows_kernel(const float *part_m, const float *part_l, const float *tlogit, const int *target, const float *mask,
+               float *nll, float *lse, long long R, int Rpad, int npanel, int V)
+{
+    const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    float M = -INFINITY;
+    for (int pn = 0; pn < npanel; ++pn) M = fmaxf(M, part_m[(size_t)pn * Rpad + r]);
+    float L = 0.f;
+    for (int pn = 0; pn < npanel; ++pn) L += part_l[(size_t)pn * Rpad + r] * exp2f(part_m[(size_t)pn * Rpad + r] - M);
+    const float ls = (M + log2f(L)) * kLn2;
+    lse[r] = ls;
+    const float w = mask[r];
+    float v = 0.f;
+    if (w != 0.f) {
+        const int z = target[r];
+        v = (z >= 0 && z < V) ? w * (ls - tlogit[r]) : __int_as_float(0x7fc00000);  // a bad token id shows as NaN
+    }
+    nll[r] = v;
+}
+
+// Masked average per candidate: one warp per candidate.
+__global__ void __launch_bounds__(256)
+ce_finalize_kernel(const float *nll, const float *mask, float *loss, int N, int Lr)
 {
     const int warp = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
     if (warp >= N) return;
     float num = 0.f, den = 0.f;
     for (int i = lane; i < Lr; i += 32) {
         const size_t r = (size_t)warp * Lr + i;
-        float M = -INFINITY;
-        for (int pn = 0; pn < npanel; ++pn) M = fmaxf(M, part_m[(size_t)pn * Rpad + r]);
-        float L = 0.f;
-        for (int pn = 0; pn < npanel; ++pn) L += part_l[(size_t)pn * Rpad + r] * exp2f(part_m[(size_t)pn * Rpad + r] - M);
-        const float ls = (M + log2f(L)) * kLn2;
-        lse[r] = ls;
-        const float w = mask[r];
-        float v = 0.f;
-        if (w != 0.f) {
-            const int z = target[r];
-            v = (z >= 0 && z < V) ? w * (ls - tlogit[r]) : __int_as_float(0x7fc00000);  // a bad token id shows as NaN
-        }
-        nll[r] = v;
-        num += v;
-        den += w;
+        num += nll[r];
+        den += mask[r];
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -359,11 +368,13 @@ cudaError_t launch_ce_fwd(const CeArgs &a, void *workspace, unsigned int *status
     if (e != cudaSuccess) return e;
     {
         KernelTiming timing(kKernelCeFinalize, stream);
+        ce_rows_kernel<<<(unsigned)((R + 255) / 256), 256, 0, stream>>>(p.part_m, p.part_l, p.tlogit, a.target, a.mask, a.nll,
+                                                                       a.lse, R, pl.Rpad, pl.npanel, a.V);
         const int warps_per_block = 8;
         ce_finalize_kernel<<<(a.N + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, stream>>>(
-            p.part_m, p.part_l, p.tlogit, a.target, a.mask, a.nll, a.lse, a.loss, a.N, a.Lr, pl.Rpad, pl.npanel, a.V);
+            a.nll, a.mask, a.loss, a.N, a.Lr);
     }
-    count_launches(2);
+    count_launches(3);
     return cudaGetLastError();
 }
 
