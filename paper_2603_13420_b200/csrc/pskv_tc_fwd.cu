@@ -556,44 +556,54 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
         for (int i = 0; tl < n_tiles && ok; ++i) {
             const int slot = i % kSlots;
-            // the slot is free once the value MMAs of item i-3 (which read P from it) have completed
-            ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
-            if (!ok) break;
-            if (k == 0) {
-                ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaQk);
-                if (!ok) break;
-            }
-            uint32_t kaddr;
+            // everything that does not depend on a wait comes first, so that it is out of the way
+            // when the waits return
+            uint32_t kaddr, kbar, kpar;
             int n, slab;
+            bool kwait = true;
             if (k < p.nblk_p || SR) {
                 n = k < p.nblk_p ? prefix_block_rows(p, k)
                     : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
                 slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
                 if (RES) {
-                    if (t.first_of_g)
-                        ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaQk);
+                    kwait = t.first_of_g;
+                    kbar = bar(kBarKFull + k);
+                    kpar = (uint32_t)(t.g - g_first) & 1u;
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
                 } else {
                     const uint32_t ks = kuse % (uint32_t)p.stages;
-                    ok = mbar_wait_warp(bar(kBarKFull + ks), (kuse / (uint32_t)p.stages) & 1, abort_flag, p.status,
-                                        kErrMmaQk);
+                    kbar = bar(kBarKFull + ks);
+                    kpar = (kuse / (uint32_t)p.stages) & 1u;
                     kaddr = sbase + p.off_pk + ks * C::kTileBytes;
                 }
             } else {
                 n = t.n_sfx;
                 slab = sfx_slab;
-                ok = mbar_wait_warp(bar(kBarSKFull), tl & 1, abort_flag, p.status, kErrMmaQk);
+                kbar = bar(kBarSKFull);
+                kpar = (uint32_t)tl & 1u;
                 kaddr = sbase + p.off_sk;
             }
-            if (!ok) break;
-            PSKV_TRACE_EVENT(10, i);
-            tc_fence_after();
             const uint32_t idesc = make_idesc_bf16(kTileM, n, 0);
             const uint32_t d_tmem = tmem + slot * kBlockN;
             const uint64_t k_desc = make_smem_desc(kaddr, 0, 1024);
             const uint64_t k_slab = (uint64_t)(slab >> 4);
             const bool last_of_tile = k == nitems - 1;
             const bool free_stage = (k < p.nblk_p || SR) && !RES;
+            // the slot is free once the value MMAs of item i-3 (which read P from it) have completed
+            PSKV_TRACE_EVENT(16, i);
+            ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
+            if (!ok) break;
+            PSKV_TRACE_EVENT(18, i);
+            if (k == 0) {
+                ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaQk);
+                if (!ok) break;
+            }
+            if (kwait) {
+                ok = mbar_wait_warp(kbar, kpar, abort_flag, p.status, kErrMmaQk);
+                if (!ok) break;
+            }
+            PSKV_TRACE_EVENT(10, i);
+            tc_fence_after();
             if (elect_one_sync()) {
 #pragma unroll
                 for (int ks16 = 0; ks16 < D / 16; ++ks16) {
@@ -626,6 +636,39 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         bool ok = true;
         for (int i = 0; tl < n_tiles && ok; ++i) {
             const int slot = i % kSlots;
+            // everything that does not depend on a wait comes first
+            uint32_t vaddr, vbar, vpar;
+            int n, slab;
+            bool vwait = true;
+            if (k < p.nblk_p || SR) {
+                n = k < p.nblk_p ? prefix_block_rows(p, k)
+                    : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
+                slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
+                if (RES) {
+                    vwait = t.first_of_g;
+                    vbar = bar(kBarVFull + k);
+                    vpar = (uint32_t)(t.g - g_first) & 1u;
+                    vaddr = sbase + p.off_pv + k * C::kTileBytes;
+                } else {
+                    const uint32_t vs = vuse % (uint32_t)p.stages;
+                    vbar = bar(kBarVFull + vs);
+                    vpar = (vuse / (uint32_t)p.stages) & 1u;
+                    vaddr = sbase + p.off_pv + vs * C::kTileBytes;
+                }
+            } else {
+                n = t.n_sfx;
+                slab = sfx_slab;
+                vbar = bar(kBarSVFull);
+                vpar = (uint32_t)tl & 1u;
+                vaddr = sbase + p.off_sv;
+            }
+            const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
+            const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
+            const int nk = n >> 4;
+            const bool last_of_tile = k == nitems - 1;
+            const bool free_stage = (k < p.nblk_p || SR) && !RES;
+            const uint32_t acc0 = k > 0 ? 1u : 0u;
+            PSKV_TRACE_EVENT(17, i);
             ok = mbar_wait_warp(bar(kBarPReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaPv);
             if (!ok) break;
             if (k == 0 && tl > 0) {
@@ -634,38 +677,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 ok = mbar_wait_warp(bar(kBarOFree), (tl - 1) & 1, abort_flag, p.status, kErrMmaPv);
                 if (!ok) break;
             }
-            uint32_t vaddr;
-            int n, slab;
-            if (k < p.nblk_p || SR) {
-                n = k < p.nblk_p ? prefix_block_rows(p, k)
-                    : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
-                slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
-                if (RES) {
-                    if (t.first_of_g)
-                        ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaPv);
-                    vaddr = sbase + p.off_pv + k * C::kTileBytes;
-                } else {
-                    const uint32_t vs = vuse % (uint32_t)p.stages;
-                    ok = mbar_wait_warp(bar(kBarVFull + vs), (vuse / (uint32_t)p.stages) & 1, abort_flag, p.status,
-                                        kErrMmaPv);
-                    vaddr = sbase + p.off_pv + vs * C::kTileBytes;
-                }
-            } else {
-                n = t.n_sfx;
-                slab = sfx_slab;
+            if (vwait) {
                 PSKV_TRACE_EVENT(14, i);
-                ok = mbar_wait_warp(bar(kBarSVFull), tl & 1, abort_flag, p.status, kErrMmaPv);
-                vaddr = sbase + p.off_sv;
+                ok = mbar_wait_warp(vbar, vpar, abort_flag, p.status, kErrMmaPv);
+                if (!ok) break;
             }
-            if (!ok) break;
             PSKV_TRACE_EVENT(11, i);
             tc_fence_after();
-            const uint32_t p_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
-            const uint64_t v_desc = make_smem_desc(vaddr, (uint32_t)slab, 1024);
-            const int nk = n >> 4;
-            const bool last_of_tile = k == nitems - 1;
-            const bool free_stage = (k < p.nblk_p || SR) && !RES;
-            const uint32_t acc0 = k > 0 ? 1u : 0u;
             if (elect_one_sync()) {
 #pragma unroll
                 for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
@@ -861,6 +879,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // the TMA stores of the previous tile must have read the staging buffer
             ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
             if (!ok) break;
+            PSKV_TRACE_EVENT(33, te);
             // one 64-column slab per round; O is free for the next tile's first value MMA as soon
             // as the last round's loads have returned
 #pragma unroll 1
@@ -869,10 +888,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 tmem_ld32(tmem + lane_addr + kOCol + sl * 64, o0);
                 tmem_ld32(tmem + lane_addr + kOCol + sl * 64 + kPiece, o1);
                 tmem_wait_ld();
+                PSKV_TRACE_EVENT(34 + sl, te);
                 if (sl == C::kSlabs - 1) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarOFree));
+                    PSKV_TRACE_EVENT(32, te);
                 }
                 // 128-byte rows, 16-byte chunks swizzled by the row
                 uint8_t *srow = smem + p.off_stage + sl * kStagingBytes + row * 128;
