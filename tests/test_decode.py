@@ -158,3 +158,33 @@ def test_decode_arguments_are_checked_on_the_host():
     assert pskv.pskv_attn_fwd_decode_workspace_bytes(8, 4, 4, 1, 8, 16, 128) == 256
     assert pskv.pskv_attn_fwd_decode_workspace_bytes(8, 4, 4, 9, 8, 16, 128) == 0
     assert pskv.pskv_attn_bwd_decode_workspace_bytes(8, 4, 4, 2, 8, 16, 128) >= 8 * 4 * 2 * 4
+
+
+@pytest.mark.gpu
+def test_single_key_rows_are_exact_up_to_one_rounding_of_the_probability():
+    """One cached token and no prefix: the softmax has a single term, so out is that token's value row
+    and dQ is zero.  The tensor-core forward feeds bf16 probabilities to the value contraction and
+    divides by the fp32 sum of the unrounded ones, so `out` may differ from the value row by one bf16
+    rounding (2^-8 relative), and the backward, which takes that `out`, sees D = <dout, out> off by the
+    same amount: |dQ| stays below scale * 2^-7 * sum_c |dout_c v_c| * |k| instead of being exactly zero."""
+    B, Hq, Hkv, d = 18, 14, 2, 128
+    t, _ = make(B, Hq, Hkv, 1, 1, 0, d, False)
+    scale = 1.0 / np.sqrt(d)
+    dev = {k: v.cuda() for k, v in t.items()}
+    out, lse = pskv.pskv_attn_fwd_decode(dev["q"], None, None, dev["suffix_k"], dev["suffix_v"], None, scale)
+    n_rep = Hq // Hkv
+    v = t["suffix_v"][:, :, 0].float().repeat_interleave(n_rep, dim=1)          # [B, Hq, d]
+    k = t["suffix_k"][:, :, 0].float().repeat_interleave(n_rep, dim=1)
+    o = out.cpu().float()[:, :, 0]
+    assert torch.all((o - v).abs() <= 2.0 ** -7 * v.abs() + 1e-6)
+    s = (t["q"].float()[:, :, 0] * k).sum(-1) * scale
+    assert torch.all((lse.cpu()[:, :, 0] - s).abs() <= 1e-3 * torch.clamp(s.abs(), min=1.0))
+    dq, dk, dv = pskv.pskv_attn_bwd_decode(dev["dout"], dev["q"], None, None, dev["suffix_k"], dev["suffix_v"], None,
+                                           out, lse, scale)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    dp = (t["dout"].float()[:, :, 0] * v).abs().sum(-1)                           # sum |dout_c v_c|, [B, Hq]
+    bound = scale * 2.0 ** -7 * dp[..., None] * k.abs() + 1e-5
+    assert torch.all(dq.cpu().float()[:, :, 0].abs() <= bound)
+    # dV of the one key is the sum of dout over its query heads (p = 1)
+    ref_dv = t["dout"].float()[:, :, 0].reshape(B, Hkv, n_rep, d).sum(2)
+    assert torch.all((dv.cpu().float()[:, :, 0] - ref_dv).abs() <= 2.0 ** -7 * ref_dv.abs() + 2e-2)
