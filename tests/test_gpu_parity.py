@@ -79,6 +79,8 @@ EDGE = [
     (2, 8, 2, 256, 100, 128), # 1024 rows per group, two suffix blocks, causal limit inside each
     (1, 8, 2, 512, 0, 128),   # one sequence, no prefix: plain causal self-attention (a prefix prefill)
     (2, 4, 4, 131, 20, 128),  # a prime row count per group: no tiling, general kernels
+    (2, 8, 2, 48, 16384, 128),  # a long prefix: 128 key blocks streamed per tile
+    (3, 4, 4, 16, 4099, 64),    # long prefix with a ragged last block, head dim 64
 ]
 
 
