@@ -838,7 +838,7 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
         if (e != cudaSuccess) return e;
     }
     if (parts & kBwdPartDq) {
-        const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
+        const int grid = even_grid(p.total_tiles, sm_count());
         {
             KernelTiming timing(kKernelBwdDqTc, stream);
             kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,

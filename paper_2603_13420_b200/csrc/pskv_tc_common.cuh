@@ -86,6 +86,16 @@ __device__ __forceinline__ TileInfo tile_info(const Params &p, int tile, int t_b
 
 // ------------------------------------------------------------------------------ host side
 
+// Persistent grid for `units` equal work items on `sms` SMs: every CTA gets the same number of items (the
+// longest CTA sets the kernel's duration either way), so that a launch whose items do not fill the last
+// round leaves whole SMs free for a kernel running beside it instead of idling them one item early.
+inline int even_grid(int units, int sms)
+{
+    if (units <= sms) return units;
+    const int rounds = (units + sms - 1) / sms;
+    return (units + rounds - 1) / rounds;
+}
+
 inline int gcd_int(int a, int b) { return b == 0 ? a : gcd_int(b, a % b); }
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 

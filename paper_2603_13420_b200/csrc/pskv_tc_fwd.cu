@@ -1177,7 +1177,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
         if (e != cudaSuccess) return e;
         attr_set[plan.mode] = true;
     }
-    const int grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
+    const int grid = even_grid(p.total_tiles, sm_count());
     {
         KernelTiming timing(kKernelFwdTc, stream);
         kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail, tm_sk,
