@@ -398,9 +398,9 @@ def roofline(w, kernels, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (kernel, workload) -> bytes.
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("tc_fwd_kernel", "C2"): 473.9e6,        # profiles/tc_fwd_kernel_C2.md
-    ("tc_bwd_dq_kernel", "C2"): 693.2e6,     # profiles/tc_bwd_dq_kernel_C2.md
-    ("tc_bwd_dkv_kernel", "C2"): 594.5e6,    # profiles/tc_bwd_dkv_kernel_C2.md
+    ("tc_fwd_kernel", "C2"): 473.7e6,        # profiles/tc_fwd_kernel_C2.md
+    ("tc_bwd_dq_kernel", "C2"): 690.6e6,     # profiles/tc_bwd_dq_kernel_C2.md
+    ("tc_bwd_dkv_kernel", "C2"): 594.8e6,    # profiles/tc_bwd_dkv_kernel_C2.md
     ("simt_row_dot_kernel", "C2"): 410.1e6,  # profiles/simt_row_dot_kernel_C2.md
 }
 
