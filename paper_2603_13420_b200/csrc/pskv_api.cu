@@ -466,6 +466,26 @@ pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void 
         st = check_dims(Kq, Hq, Hkv, S, prefix_len[i], d, &dm);
         if (st != PSKV_OK) return st;
     }
+    {
+        // One launch over all instructions when every tile lies inside one instruction: the prefix caches
+        // are heads of one [Bp*Hkv][Pmax][d] tensor and the left padding is masked like a causal limit.
+        Dims dall;
+        if (Bp > 1 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK && tc_fwd_fused_supported(dall, Bp)) {
+            FwdArgs a;
+            a.q = static_cast<const __nv_bfloat16 *>(q);
+            a.prefix_k = static_cast<const __nv_bfloat16 *>(prefix_k);
+            a.prefix_v = static_cast<const __nv_bfloat16 *>(prefix_v);
+            a.suffix_k = static_cast<const __nv_bfloat16 *>(suffix_k);
+            a.suffix_v = static_cast<const __nv_bfloat16 *>(suffix_v);
+            a.out = static_cast<__nv_bfloat16 *>(out);
+            a.lse = lse;
+            a.suffix_len = nullptr;
+            a.scale = scale;
+            a.dims = dall;
+            cudaError_t e = launch_tc_fwd(a, workspace, status_word, stream, Bp, prefix_len);
+            return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
+        }
+    }
     std::lock_guard<std::mutex> lock(g_side_mutex);
     SideStream *side = Bp > 1 ? side_stream() : nullptr;
     if (side) {

@@ -70,8 +70,13 @@ cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaS
 // tcgen05/TMEM kernels.  `status_word` is the device status flag that bounded waits set.
 bool tc_fwd_supported(const Dims &d);
 size_t tc_fwd_workspace_bytes(const Dims &d);
+// Several instructions in one launch (Sec. 4.3): the B candidates fall into `n_instr` contiguous groups
+// of equal size, group i uses prefix cache i of prefix_k / prefix_v [n_instr][Hkv][P][d], whose last
+// prefix_len[i] rows (host array) are real tokens and whose first rows are left padding.
+constexpr int kMaxFusedInstructions = 64;
+bool tc_fwd_fused_supported(const Dims &d, int n_instr);
 cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word,
-                          cudaStream_t stream);
+                          cudaStream_t stream, int n_instr = 1, const int *prefix_len = nullptr);
 bool tc_bwd_supported(const Dims &d);
 size_t tc_bwd_workspace_bytes(const Dims &d);
 // `parts` selects which of the three steps run (all by default): the row statistic D and the suffix

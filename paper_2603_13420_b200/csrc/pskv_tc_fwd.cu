@@ -48,6 +48,7 @@ constexpr int kOCol = kSlots * kBlockN;  // first tensor-memory column of O
 constexpr float kMaxRowSum = 1.2676506002282294e30f;   // 2^100
 constexpr float kMinRowSum = 7.8886090522101181e-31f;  // 2^-100
 constexpr int kMaxStages = 4;
+constexpr int kMaxInstr = kMaxFusedInstructions;  // prefixes one launch can serve
 
 enum : unsigned int {
     kErrProducerK = 0x101, kErrProducerV = 0x102, kErrMmaQk = 0x103, kErrMmaPv = 0x104,
@@ -81,6 +82,12 @@ struct TcFwdParams {
     int deal_by_cost;     // long suffixes: hand tiles to CTAs by cost rank instead of in contiguous ranges
     int long_sfx;         // 1: a tile lies inside ONE candidate and that candidate's suffix keys come in
                           //    128-key blocks (suffix caches or row groups beyond 128); 0: whole-candidate tiles
+    // several instructions in one launch (Sec. 4.3): the candidates of instruction i are contiguous and use
+    // prefix cache i of [n_instr][Hkv][P][d], whose first pad[i] rows are left padding
+    int n_instr;          // 1: one shared prefix
+    int rpi;              // rows of one instruction inside a KV head's row list (a multiple of tile_rows)
+    FastDiv fd_rpi;
+    int pad[kMaxInstr];
     // shared-memory carve-up (byte offsets from the 1024-byte aligned base)
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml;
 };
@@ -157,7 +164,7 @@ __device__ __forceinline__ int sfx_long_rows(const TcFwdParams &p, int j)
 // in as many blocks as it takes -- the mode of the decode-shaped operator, where a 128-row tile
 // spans many candidates, and of full-suffix shapes the other two modes cannot tile.  A compile-time
 // switch so that each launch carries only the code of its own mode.
-template <int D, int MODE>
+template <int D, int MODE, bool MI>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_out,
               const __grid_constant__ CUtensorMap tm_pk, const __grid_constant__ CUtensorMap tm_pv,
@@ -236,7 +243,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     auto items_of = [&](const TileInfo &t) {
         return p.nblk_p + (!SR ? 1 : p.long_sfx ? sfx_blocks_long(p, t) : p.fd_cpb.div(t.nc + p.cpb - 1));
     };
-    const int g_first = p.fd_tpg.div(t_begin);
+    // A run of tiles that shares one prefix: a KV head, or (several instructions) one instruction's
+    // candidates inside a KV head.  Runs are numbered in tile order; the resident prefix is reloaded at the
+    // start of each run and the barrier parity of those loads follows the run number.
+    auto inst_of = [&](const TileInfo &t) { return MI ? p.fd_rpi.div(t.R0) : 0; };
+    auto run_of = [&](const TileInfo &t, int inst) { return MI ? t.g * p.n_instr + inst : t.g; };
+    auto first_of_run = [&](const TileInfo &t, int inst) {
+        return t.first_of_g || (MI && t.R0 == inst * p.rpi);
+    };
+    int run_first;
+    {
+        const TileInfo t0 = tile_info(p, t_begin < p.total_tiles ? t_begin : 0, t_begin);
+        run_first = run_of(t0, inst_of(t0));
+    }
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
 
@@ -307,8 +326,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
             }
             __syncwarp();
+            const int inst = inst_of(t);
+            const int ph = inst * p.Hkv + t.g;  // head index inside the prefix caches
             if (RES) {
-                if (t.first_of_g && elect_one_sync()) {
+                if (first_of_run(t, inst) && elect_one_sync()) {
 #pragma unroll 1
                     for (int k = 0; k < p.nblk_p; ++k) {
                         const bool tail = k == p.nblk_p - 1;
@@ -317,7 +338,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll 1
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pk + k * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
-                                        bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
+                                        bar(kBarKFull + k), sl * 64, k * kBlockN, ph);
                     }
                 }
                 __syncwarp();
@@ -335,7 +356,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll 1
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
-                                        bar(kBarKFull + ks), sl * 64, k * kBlockN, t.g);
+                                        bar(kBarKFull + ks), sl * 64, k * kBlockN, ph);
                     }
                     __syncwarp();
                     ++kload;
@@ -415,14 +436,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             bool pend_store = tl > 0, pend_sv = have_tile && !SR;
             TileInfo t;
             int nk = 0;  // V blocks still to fetch through the ring for this tile
+            int ph = 0;  // head index inside the prefix caches
             if (have_tile) {
                 t = tile_info(p, tile_at(tl), t_begin);
+                const int inst = inst_of(t);
+                ph = inst * p.Hkv + t.g;
                 if (RES) {
                     // the resident prefix V blocks are free once every value MMA of the previous tile
                     // has completed
                     ok = mbar_wait_warp(bar(kBarSVFree), (tl & 1) ^ 1, abort_flag, p.status, kErrProducerV);
                     if (!ok) break;
-                    if (t.first_of_g && elect_one_sync()) {
+                    if (first_of_run(t, inst) && elect_one_sync()) {
 #pragma unroll 1
                         for (int k = 0; k < p.nblk_p; ++k) {
                             const bool tail = k == p.nblk_p - 1;
@@ -431,7 +455,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll 1
                             for (int sl = 0; sl < C::kSlabs; ++sl)
                                 tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab,
-                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
+                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + k), sl * 64, k * kBlockN, ph);
                         }
                     }
                     __syncwarp();
@@ -481,7 +505,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 #pragma unroll 1
                             for (int sl = 0; sl < C::kSlabs; ++sl)
                                 tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab,
-                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                                            tail ? &tm_pv_tail : &tm_pv, bar(kBarVFull + vs), sl * 64, k * kBlockN, ph);
                         }
                     }
                     __syncwarp();
@@ -566,9 +590,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
                 slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
                 if (RES) {
-                    kwait = t.first_of_g;
+                    const int inst = inst_of(t);
+                    kwait = first_of_run(t, inst);
                     kbar = bar(kBarKFull + k);
-                    kpar = (uint32_t)(t.g - g_first) & 1u;
+                    kpar = (uint32_t)(run_of(t, inst) - run_first) & 1u;
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
                 } else {
                     const uint32_t ks = kuse % (uint32_t)p.stages;
@@ -645,9 +670,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     : p.long_sfx ? sfx_long_rows(p, k - p.nblk_p) : sfx_block_rows(p, t.nc, k - p.nblk_p);
                 slab = (SR && p.long_sfx && k >= p.nblk_p) ? C::kSlabBytes : n * 128;  // (full 128-row boxes)
                 if (RES) {
-                    vwait = t.first_of_g;
+                    const int inst = inst_of(t);
+                    vwait = first_of_run(t, inst);
                     vbar = bar(kBarVFull + k);
-                    vpar = (uint32_t)(t.g - g_first) & 1u;
+                    vpar = (uint32_t)(run_of(t, inst) - run_first) & 1u;
                     vaddr = sbase + p.off_pv + k * C::kTileBytes;
                 } else {
                     const uint32_t vs = vuse % (uint32_t)p.stages;
@@ -757,6 +783,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
             }
             lsum = 0.f;
+            // several instructions: the first `pad` prefix keys of this tile's instruction are left padding
+            const int pad = MI ? p.pad[inst_of(t)] : 0;
 #pragma unroll 1
             for (int k = 0; k < nitems && ok; ++k, ++item) {
                 {
@@ -768,7 +796,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     int n, lo, hi;
                     if (k < p.nblk_p) {
                         n = prefix_block_rows(p, k);
-                        lo = 0;
+                        lo = max(0, pad - k * kBlockN);
                         hi = min(kBlockN, p.P - k * kBlockN) - 1;
                     } else if (SR && p.long_sfx) {
                         n = sfx_long_rows(p, k - p.nblk_p);
@@ -953,7 +981,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int b = p.fd_Rg.div(R), rr = R - b * p.Rg;
                 const long long grow = ((long long)b * p.Hq + (long long)t.g * p.n_rep) * p.S + rr;
                 const float v = p.lse[grow];
-                if (v != v) fwd_row<D>(p.args, grow, q_s, lane);
+                if (v != v) {
+                    if (MI) {  // the row's own prefix cache, without its left padding
+                        const int inst = inst_of(t), pd = p.pad[inst];
+                        FwdArgs a2 = p.args;
+                        const size_t off = ((size_t)inst * p.Hkv * p.P + (size_t)pd) * D;
+                        a2.prefix_k += off;
+                        a2.prefix_v += off;
+                        a2.dims.P = p.P - pd;
+                        fwd_row<D>(a2, grow, q_s, lane);
+                    } else {
+                        fwd_row<D>(p.args, grow, q_s, lane);
+                    }
+                }
             }
         }
     }
@@ -1097,7 +1137,7 @@ TilePlan plan_tiles(const Dims &dm)
 
 template <int D>
 cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsigned int *status_word,
-                   cudaStream_t stream)
+                   cudaStream_t stream, int n_instr, const int *prefix_len)
 {
     const Dims &dm = a.dims;
     const int Rg = dm.n_rep * dm.S;
@@ -1126,7 +1166,7 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
         if (!encode_map(&tm_sv, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
     if (dm.P > 0) {
-        cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
+        cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv * (cuuint64_t)n_instr};
         cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.Pstride * D * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
         cuuint32_t box_tail[3] = {64, (cuuint32_t)plan.tail_rows, 1};
@@ -1162,6 +1202,10 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.cpb = plan.cpb > 0 ? plan.cpb : 1;
     p.fd_cpb.init(p.cpb);
     p.long_sfx = plan.long_sfx;
+    p.n_instr = n_instr;
+    p.rpi = dm.B / n_instr * Rg;
+    p.fd_rpi.init(p.rpi > 0 ? p.rpi : 1);
+    for (int i = 0; i < kMaxInstr; ++i) p.pad[i] = (n_instr > 1 && i < n_instr) ? dm.P - prefix_len[i] : 0;
     // Dealing by cost balances the causal skew but lets every CTA touch every candidate's suffix K/V
     // at several times; it pays when those tensors stay in L2 between the touches.
     p.deal_by_cost = plan.long_sfx && dm.S % plan.tile_rows == 0 && dm.S / plan.tile_rows > 1 &&
@@ -1170,12 +1214,15 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar; p.off_misc = plan.off_misc;
     p.off_ml = plan.off_ml;
 
-    auto kernel = plan.mode == 1 ? tc_fwd_kernel<D, 1> : plan.mode == 2 ? tc_fwd_kernel<D, 2> : tc_fwd_kernel<D, 0>;
-    static bool attr_set[3] = {false, false, false};
-    if (!attr_set[plan.mode]) {
+    const bool mi = n_instr > 1;  // (never with the suffix-ring tiling)
+    auto kernel = plan.mode == 2 ? tc_fwd_kernel<D, 2, false>
+                  : plan.mode == 1 ? (mi ? tc_fwd_kernel<D, 1, true> : tc_fwd_kernel<D, 1, false>)
+                                   : (mi ? tc_fwd_kernel<D, 0, true> : tc_fwd_kernel<D, 0, false>);
+    static bool attr_set[6] = {false, false, false, false, false, false};
+    if (!attr_set[plan.mode + (mi ? 3 : 0)]) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
-        attr_set[plan.mode] = true;
+        attr_set[plan.mode + (mi ? 3 : 0)] = true;
     }
     const int grid = even_grid(p.total_tiles, sm_count());
     {
@@ -1218,12 +1265,27 @@ bool tc_fwd_supported(const Dims &dm)
 
 size_t tc_fwd_workspace_bytes(const Dims &) { return 0; }
 
-cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word, cudaStream_t stream)
+// One launch can serve several instructions when every tile lies inside one instruction's candidates (an
+// instruction's rows in a KV head's row list are a whole number of tiles) and the tiles are the 128-row
+// tiles with one suffix block each (not the suffix-ring tiling).
+bool tc_fwd_fused_supported(const Dims &dm, int n_instr)
+{
+    if (n_instr < 2 || n_instr > kMaxFusedInstructions || dm.B % n_instr != 0 || dm.P < 1 || dm.Pstride != dm.P ||
+        dm.ragged || !tc_fwd_supported(dm))
+        return false;
+    const TilePlan pl = plan_tiles(dm);
+    return pl.ok && pl.mode != 2 && ((long long)(dm.B / n_instr) * dm.n_rep * dm.S) % pl.tile_rows == 0;
+}
+
+cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word, cudaStream_t stream,
+                          int n_instr, const int *prefix_len)
 {
     const TilePlan plan = plan_tiles(a.dims);
     if (!plan.ok) return cudaErrorInvalidValue;
-    return a.dims.d == 128 ? launch<128>(a, plan, workspace, status_word, stream)
-                           : launch<64>(a, plan, workspace, status_word, stream);
+    if (n_instr > 1 && (!prefix_len || !tc_fwd_fused_supported(a.dims, n_instr))) return cudaErrorInvalidValue;
+    if (n_instr < 1) n_instr = 1;
+    return a.dims.d == 128 ? launch<128>(a, plan, workspace, status_word, stream, n_instr, prefix_len)
+                           : launch<64>(a, plan, workspace, status_word, stream, n_instr, prefix_len);
 }
 
 }  // namespace pskv

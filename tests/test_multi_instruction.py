@@ -37,7 +37,15 @@ CASES = [
     (6, 3, 4, 2, 8, 64, 64, (0, 64, 17)),          # head dim 64, an empty prefix, odd length
     (4, 4, 2, 1, 5, 33, 128, (33, 1, 20, 7)),      # general kernels (S not a multiple of 8)
     (64, 2, 32, 8, 48, 256, 128, (256, 200)),      # the GQA layer shape, two instructions
+    (16, 4, 8, 2, 16, 600, 128, (600, 0, 130, 471)),  # one launch, prefix blocks streamed; an empty prefix and
+                                                   # one whose padding covers three whole key blocks
+    (8, 2, 4, 4, 32, 96, 64, (96, 50)),            # one launch, head dim 64
+    (40, 5, 8, 2, 32, 200, 128, (200, 199, 73, 128, 1)),  # one launch, five instructions, odd lengths
 ]
+
+# forward launches each case must take: 1 = all instructions in one launch (every tile inside one instruction),
+# else one launch per instruction
+FWD_LAUNCHES = {0: 1, 1: 2, 2: 3, 3: 4, 4: 1, 5: 1, 6: 1, 7: 1}
 
 
 @pytest.mark.gpu
@@ -49,8 +57,10 @@ def test_forward_and_backward_match_the_oracle(case):
     dev = {k: v.cuda() for k, v in t.items()}
     out = parity.Guarded((B, Hq, S, d), torch.bfloat16, "cuda")
     lse = parity.Guarded((B, Hq, S), torch.float32, "cuda")
+    n0 = pskv.pskv_kernel_launches()
     pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"], dev["suffix_v"],
                              scale, out=out.view, lse=lse.view)
+    assert pskv.pskv_kernel_launches() - n0 == FWD_LAUNCHES[CASES.index(case)]
     assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
     out.check("out"); lse.check("lse")
     f = {k: parity.to_f64(v) for k, v in t.items()}
@@ -72,6 +82,33 @@ def test_forward_and_backward_match_the_oracle(case):
     parity.check_tensor("dq", parity.to_f64(dq.view), rq)
     parity.check_tensor("dk_suffix", parity.to_f64(dk.view), rk)
     parity.check_tensor("dv_suffix", parity.to_f64(dv.view), rv)
+
+
+@pytest.mark.gpu
+def test_one_launch_redoes_rows_outside_the_safe_exponent_range_with_their_own_prefix():
+    """Scores of several hundred nats in rows of different instructions: the one-launch forward marks them
+    and recomputes each with a running maximum against its own instruction's unpadded prefix."""
+    case = (16, 4, 8, 2, 16, 300, 128, (300, 40, 170, 1))
+    B, Bp, Hq, Hkv, S, Pmax, d, lens = case
+    t = make(*case)
+    q = t["q"].float()
+    q[1, 2, 3] *= 60.0      # instruction 0
+    q[5, 0, 15] *= -50.0    # instruction 1
+    q[15, 7, 0] *= 45.0     # instruction 3
+    t["q"] = q.to(torch.bfloat16)
+    scale = 1.0 / np.sqrt(d)
+    dev = {k: v.cuda() for k, v in t.items()}
+    n0 = pskv.pskv_kernel_launches()
+    out, lse = pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
+                                        dev["suffix_v"], scale)
+    assert pskv.pskv_kernel_launches() - n0 == 1
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    f = {k: parity.to_f64(v) for k, v in t.items()}
+    mask = oracle.left_padding_mask(lens, Pmax)
+    ref_out, ref_lse = oracle.attn_fwd_multi(f["q"], f["prefix_k"], f["prefix_v"], mask, f["suffix_k"], f["suffix_v"], scale)
+    assert np.abs(ref_lse).max() > 100.0
+    parity.check_tensor("out", parity.to_f64(out), ref_out)
+    parity.check_lse(parity.to_f64(lse), ref_lse)
 
 
 @pytest.mark.gpu
