@@ -569,6 +569,17 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         a.scale = scale;
         a.dims = dm;
     };
+    {
+        // All instructions in one dQ launch when every tile lies inside one instruction (as in the forward);
+        // the row statistic before it and the suffix gradients after it never involved the prefix.
+        Dims dall;
+        if (Bp > 1 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK && tc_bwd_fused_supported(dall, Bp)) {
+            BwdArgs a;
+            fill(a, 0, dall, 0);
+            cudaError_t e = launch_tc_bwd(a, workspace, status_word, stream, kBwdPartAll, Bp, prefix_len);
+            return e == cudaSuccess ? PSKV_OK : cuda_fail(e);
+        }
+    }
     // The row statistic D = <dout, out> and the suffix gradients do not involve the prefix: when every
     // instruction's part runs on the tensor-core kernels they are done once over all B candidates, and
     // only the dQ step runs once per instruction.

@@ -83,8 +83,10 @@ size_t tc_bwd_workspace_bytes(const Dims &d);
 // gradients do not involve the prefix, so a caller with several prefixes runs them once over all
 // candidates and the dQ step once per prefix.
 enum { kBwdPartRowDot = 1, kBwdPartDq = 2, kBwdPartDkv = 4, kBwdPartAll = 7 };
+bool tc_bwd_fused_supported(const Dims &d, int n_instr);  // several instructions in one dQ launch (as for the forward)
 cudaError_t launch_tc_bwd(const BwdArgs &a, void *workspace, unsigned int *status_word,
-                          cudaStream_t stream, int parts = kBwdPartAll);
+                          cudaStream_t stream, int parts = kBwdPartAll, int n_instr = 1,
+                          const int *prefix_len = nullptr);
 
 // Masked target cross-entropy fused with the vocabulary projection (tcgen05 GEMM whose logits stay on chip).
 struct CeArgs {

@@ -36,6 +36,7 @@ constexpr int kThreads = 32 * (4 + 4 * kGroups + 4);
 constexpr int kDpCol = kSlots * kBlockN;
 constexpr int kDqCol = kDpCol + kBlockN;
 constexpr int kMaxStages = 4;
+constexpr int kMaxInstr = kMaxFusedInstructions;  // prefixes one launch can serve
 
 enum : unsigned int {
     kErrProdA = 0x201, kErrProdB = 0x202, kErrMmaS = 0x203, kErrMmaDq = 0x204, kErrElem = 0x205,
@@ -53,6 +54,12 @@ struct TcBwdParams {
     FastDiv fd_tpg, fd_Rg, fd_S, fd_seg;  // divisions by tiles_per_group, Rg, S, seg_rows
     int nblk_p, tail_rows, resident, stages_k, stages_v, sfx_rows;  // ring stages of prefix K / V (streaming mode)
     int off_pk, off_pv, off_q, off_do, off_sk, off_sv, off_stage, off_bar, off_misc;
+    // several instructions in one launch (Sec. 4.3): the candidates of instruction i are contiguous and use
+    // prefix cache i of [n_instr][Hkv][P][d], whose first pad[i] rows are left padding
+    int n_instr;  // 1: one shared prefix
+    int rpi;      // rows of one instruction inside a KV head's row list (a multiple of tile_rows)
+    FastDiv fd_rpi;
+    int pad[kMaxInstr];
 };
 
 template <int D>
@@ -96,7 +103,7 @@ __device__ __forceinline__ int prefix_block_rows(const TcBwdParams &p, int k)
 // (else they stream through rings).  A K block is needed through a whole item (the dQ MMA reads it
 // after the element-wise stage), a V block only for its dP MMA, so when not both fit it is K that
 // stays.  Compile-time, so that each launch carries only the code of its own mode.
-template <int D, int MODE>
+template <int D, int MODE, bool MI>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                  const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_pk,
@@ -146,7 +153,17 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
     const int n_tiles = t_end - t_begin;
     const int nitems = p.nblk_p + 1;
-    const int g_first = p.fd_tpg.div(t_begin);
+    // A run of tiles that shares one prefix: a KV head, or (several instructions) one instruction's
+    // candidates inside a KV head; resident prefix blocks are reloaded at the start of each run and the
+    // barrier parity of those loads follows the run number.
+    auto inst_of = [&](const TileInfo &t) { return MI ? p.fd_rpi.div(t.R0) : 0; };
+    auto run_of = [&](const TileInfo &t, int inst) { return MI ? t.g * p.n_instr + inst : t.g; };
+    auto first_of_run = [&](const TileInfo &t, int inst) { return t.first_of_g || (MI && t.R0 == inst * p.rpi); };
+    int run_first;
+    {
+        const TileInfo t0 = tile_info(p, t_begin < p.total_tiles ? t_begin : 0, t_begin);
+        run_first = run_of(t0, inst_of(t0));
+    }
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
     const uint32_t stages_k = (uint32_t)p.stages_k, stages_v = (uint32_t)p.stages_v;
@@ -217,7 +234,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         mbar_arrive_expect_tx(bar(kBarKFull + ks), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pk + ks * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
-                                        bar(kBarKFull + ks), sl * 64, k * kBlockN, t.g);
+                                        bar(kBarKFull + ks), sl * 64, k * kBlockN, inst_of(t) * p.Hkv + t.g);
                     }
                     __syncwarp();
                     ++kload;
@@ -230,14 +247,14 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 ok = mbar_wait_warp(bar(kBarDqFull), (tl - 1) & 1, abort_flag, p.status, kErrProdA);
                 if (!ok) break;
             }
-            if (RK && t.first_of_g && elect_one_sync()) {
+            if (RK && first_of_run(t, inst_of(t)) && elect_one_sync()) {
                 for (int k = 0; k < p.nblk_p; ++k) {
                     const bool tail = k == p.nblk_p - 1;
                     const int slab = tail ? tail_slab : C::kSlabBytes;
                     mbar_arrive_expect_tx(bar(kBarKFull + k), (uint32_t)(C::kSlabs * slab));
                     for (int sl = 0; sl < C::kSlabs; ++sl)
                         tma_load_3d(sbase + p.off_pk + k * C::kTileBytes + sl * slab, tail ? &tm_pk_tail : &tm_pk,
-                                    bar(kBarKFull + k), sl * 64, k * kBlockN, t.g);
+                                    bar(kBarKFull + k), sl * 64, k * kBlockN, inst_of(t) * p.Hkv + t.g);
                 }
             }
             __syncwarp();
@@ -299,14 +316,14 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         ++qb;
                     }
                 }
-                if (RV && t.first_of_g) {
+                if (RV && first_of_run(t, inst_of(t))) {
                     for (int k = 0; k < p.nblk_p; ++k) {
                         const bool tail = k == p.nblk_p - 1;
                         const int slab = tail ? tail_slab : C::kSlabBytes;
                         mbar_arrive_expect_tx(bar(kBarVFull + k), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pv + k * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
-                                        bar(kBarVFull + k), sl * 64, k * kBlockN, t.g);
+                                        bar(kBarVFull + k), sl * 64, k * kBlockN, inst_of(t) * p.Hkv + t.g);
                     }
                 }
                 mbar_arrive_expect_tx(bar(kBarSVFull), (uint32_t)(t.nc * C::kSlabs * p.S * 128));
@@ -328,7 +345,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         mbar_arrive_expect_tx(bar(kBarVFull + vs), (uint32_t)(C::kSlabs * slab));
                         for (int sl = 0; sl < C::kSlabs; ++sl)
                             tma_load_3d(sbase + p.off_pv + vs * C::kTileBytes + sl * slab, tail ? &tm_pv_tail : &tm_pv,
-                                        bar(kBarVFull + vs), sl * 64, k * kBlockN, t.g);
+                                        bar(kBarVFull + vs), sl * 64, k * kBlockN, inst_of(t) * p.Hkv + t.g);
                     }
                     __syncwarp();
                     ++vload;
@@ -361,8 +378,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             uint32_t kaddr;
             if (prefix) {
                 if (RK) {
-                    if (t.first_of_g)
-                        ok = mbar_wait_warp(bar(kBarKFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaS);
+                    if (first_of_run(t, inst_of(t)))
+                        ok = mbar_wait_warp(bar(kBarKFull + k), (run_of(t, inst_of(t)) - run_first) & 1, abort_flag,
+                                            p.status, kErrMmaS);
                     kaddr = sbase + p.off_pk + k * C::kTileBytes;
                 } else {
                     const uint32_t ks = kuse % stages_k;
@@ -432,8 +450,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 uint32_t vaddr;
                 if (prefix) {
                     if (RV) {
-                        if (t.first_of_g)
-                            ok = mbar_wait_warp(bar(kBarVFull + k), (t.g - g_first) & 1, abort_flag, p.status, kErrMmaDq);
+                        if (first_of_run(t, inst_of(t)))
+                            ok = mbar_wait_warp(bar(kBarVFull + k), (run_of(t, inst_of(t)) - run_first) & 1, abort_flag,
+                                                p.status, kErrMmaDq);
                         vaddr = sbase + p.off_pv + k * C::kTileBytes;
                     } else {
                         const uint32_t vs = vuse % stages_v;
@@ -541,13 +560,14 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             // padding rows: lse = +inf makes every probability (and so every dS) zero
             const float neg_lse2 = valid ? -p.lse[grow] * kLog2e : -INFINITY;
             const float drow = valid ? p.row_dot[grow] : 0.f;
+            const int pad = MI ? p.pad[inst_of(t)] : 0;
 #pragma unroll 1
             for (int k = 0; k < nitems && ok; ++k, ++item) {
                 const int slot = item % kSlots;
                 int n, lo, hi;
                 if (k < p.nblk_p) {
                     n = prefix_block_rows(p, k);
-                    lo = 0;
+                    lo = max(0, pad - k * kBlockN);  // left padding of this tile's instruction
                     hi = min(kBlockN, p.P - k * kBlockN) - 1;
                 } else {
                     n = t.n_sfx;
@@ -765,7 +785,7 @@ BwdPlan plan_bwd(const Dims &dm)
 }
 
 template <int D>
-cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_word, cudaStream_t stream, int parts)
+cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_word, cudaStream_t stream, int parts, int n_instr, const int *prefix_len)
 {
     const Dims &dm = a.dims;
     const int Rg = dm.n_rep * dm.S;
@@ -790,7 +810,7 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
         if (!encode_map(&tm_sv, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
     if (dm.P > 0) {
-        cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv};
+        cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)dm.P, (cuuint64_t)dm.Hkv * (cuuint64_t)n_instr};
         cuuint64_t str[2] = {(cuuint64_t)D * 2, (cuuint64_t)dm.Pstride * D * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
         cuuint32_t box_tail[3] = {64, (cuuint32_t)plan.tail_rows, 1};
@@ -823,13 +843,20 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     p.off_pk = plan.off_pk; p.off_pv = plan.off_pv; p.off_q = plan.off_q; p.off_do = plan.off_do;
     p.off_sk = plan.off_sk; p.off_sv = plan.off_sv; p.off_stage = plan.off_stage; p.off_bar = plan.off_bar;
     p.off_misc = plan.off_misc;
+    p.n_instr = n_instr;
+    p.rpi = dm.B / n_instr * Rg;
+    p.fd_rpi.init(p.rpi > 0 ? p.rpi : 1);
+    for (int i = 0; i < kMaxInstr; ++i) p.pad[i] = (n_instr > 1 && i < n_instr) ? dm.P - prefix_len[i] : 0;
 
-    auto kernel = plan.resident == 3 ? tc_bwd_dq_kernel<D, 3> : plan.resident == 1 ? tc_bwd_dq_kernel<D, 1> : tc_bwd_dq_kernel<D, 0>;
-    static bool attr_set[4] = {false, false, false, false};
-    if (!attr_set[plan.resident]) {
+    const bool mi = n_instr > 1;
+    auto kernel = plan.resident == 3 ? (mi ? tc_bwd_dq_kernel<D, 3, true> : tc_bwd_dq_kernel<D, 3, false>)
+                  : plan.resident == 1 ? (mi ? tc_bwd_dq_kernel<D, 1, true> : tc_bwd_dq_kernel<D, 1, false>)
+                                       : (mi ? tc_bwd_dq_kernel<D, 0, true> : tc_bwd_dq_kernel<D, 0, false>);
+    static bool attr_set[8] = {false, false, false, false, false, false, false, false};
+    if (!attr_set[plan.resident + (mi ? 4 : 0)]) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
-        attr_set[plan.resident] = true;
+        attr_set[plan.resident + (mi ? 4 : 0)] = true;
     }
     // D = <dout, out> per row, then dQ on the tensor cores, then dK_suffix / dV_suffix
     cudaError_t e = cudaSuccess;
@@ -885,12 +912,26 @@ bool tc_bwd_supported(const Dims &dm)
 
 size_t tc_bwd_workspace_bytes(const Dims &dm) { return (size_t)dm.B * dm.Hq * dm.S * sizeof(float); }
 
-cudaError_t launch_tc_bwd(const BwdArgs &a, void *, unsigned int *status_word, cudaStream_t stream, int parts)
+// One launch can serve several instructions when an instruction's rows in a KV head's row list are a whole
+// number of tiles (every tile then lies inside one instruction).
+bool tc_bwd_fused_supported(const Dims &dm, int n_instr)
+{
+    if (n_instr < 2 || n_instr > kMaxFusedInstructions || dm.B % n_instr != 0 || dm.P < 1 || dm.Pstride != dm.P ||
+        !tc_bwd_supported(dm))
+        return false;
+    const BwdPlan pl = plan_bwd(dm);
+    return pl.ok && ((long long)(dm.B / n_instr) * dm.n_rep * dm.S) % pl.tile_rows == 0;
+}
+
+cudaError_t launch_tc_bwd(const BwdArgs &a, void *, unsigned int *status_word, cudaStream_t stream, int parts,
+                          int n_instr, const int *prefix_len)
 {
     const BwdPlan plan = plan_bwd(a.dims);
     if (!plan.ok) return cudaErrorInvalidValue;
-    return a.dims.d == 128 ? launch<128>(a, plan, status_word, stream, parts)
-                           : launch<64>(a, plan, status_word, stream, parts);
+    if (n_instr > 1 && (!prefix_len || !tc_bwd_fused_supported(a.dims, n_instr))) return cudaErrorInvalidValue;
+    if (n_instr < 1) n_instr = 1;
+    return a.dims.d == 128 ? launch<128>(a, plan, status_word, stream, parts, n_instr, prefix_len)
+                           : launch<64>(a, plan, status_word, stream, parts, n_instr, prefix_len);
 }
 
 }  // namespace pskv

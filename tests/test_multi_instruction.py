@@ -72,9 +72,12 @@ def test_forward_and_backward_match_the_oracle(case):
     dq = parity.Guarded((B, Hq, S, d), torch.bfloat16, "cuda")
     dk = parity.Guarded((B, Hkv, S, d), torch.bfloat16, "cuda")
     dv = parity.Guarded((B, Hkv, S, d), torch.bfloat16, "cuda")
+    n0 = pskv.pskv_kernel_launches()
     pskv.pskv_attn_bwd_multi(dev["dout"], dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
                              dev["suffix_v"], out.view, lse.view, scale, dq=dq.view, dk_suffix=dk.view,
                              dv_suffix=dv.view)
+    if FWD_LAUNCHES[CASES.index(case)] == 1:   # row statistic, one dQ launch for all instructions, suffix gradients
+        assert pskv.pskv_kernel_launches() - n0 == 3
     assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
     dq.check("dq"); dk.check("dk_suffix"); dv.check("dv_suffix")
     rq, rk, rv = oracle.attn_bwd_multi(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], mask, f["suffix_k"],
