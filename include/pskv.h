@@ -163,15 +163,19 @@ long long pskv_attn_bwd_static_max_rows(void);
  * alignment) with the position rules of the appendix on position consistency under padding.
  * There are Bp prefix caches, one per instruction, stored left-padded to a common length Pmax:
  *   prefix_k, prefix_v   bf16 [Bp,Hkv,Pmax,d]; the real tokens of instruction i are its LAST
- *                        prefix_len[i] rows (0 <= prefix_len[i] <= Pmax); padding rows are never read
+ *                        prefix_len[i] rows (0 <= prefix_len[i] <= Pmax); padding rows may hold any FINITE
+ *                        values (they may be read; their scores are masked and their values meet zero
+ *                        probabilities)
  *   prefix_len           HOST array of Bp ints (read before the call returns)
  * The B candidates are grouped by instruction: candidate b belongs to instruction b / (B / Bp), so B
  * must be a multiple of Bp and each cache is reused by its B / Bp candidates.  Everything else (q,
  * suffix_k, suffix_v, out, lse, dout, dq, dk_suffix, dv_suffix; scale; causal rule; error codes) is as
  * in pskv_attn_fwd / pskv_attn_bwd, with P replaced per candidate by the true prefix length of its
- * instruction.  The work is one pass per instruction; the passes are independent, so every other one
- * is enqueued on a stream of the library's own that forks from `cuda_stream` at the start of the call
- * and joins it again before the call returns (to the caller everything is ordered as if it had run on
+ * instruction.  When (B / Bp) * (Hq / Hkv) * S is a multiple of the kernels' row tile (128 rows in the
+ * usual case), Bp <= 64 and the shape runs on the tensor-core kernels, all instructions are served by one
+ * launch per kernel.  Otherwise the work is one pass per instruction; the passes are independent, so every
+ * other one is enqueued on a stream of the library's own that forks from `cuda_stream` at the start of the
+ * call and joins it again before the call returns (to the caller everything is ordered as if it had run on
  * `cuda_stream`, also under stream capture).
  */
 size_t pskv_attn_fwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d);

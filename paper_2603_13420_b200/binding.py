@@ -294,7 +294,7 @@ def pskv_attn_fwd_multi(q, prefix_k, prefix_v, prefix_len, suffix_k, suffix_v, s
                         workspace=None):
     """Forward with one left-padded prefix cache per instruction: prefix_k / prefix_v are
     [Bp, Hkv, Pmax, d], prefix_len (host ints) the true lengths, candidate b uses instruction
-    b // (B // Bp)."""
+    b // (B // Bp).  Padding rows may hold any finite values."""
     dims = _multi_dims(q, prefix_k, suffix_k, prefix_len)
     if out is None:
         out = torch.empty_like(q)

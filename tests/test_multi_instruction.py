@@ -23,7 +23,7 @@ def make(B, Bp, Hq, Hkv, S, Pmax, d, lens, seed=SEED):
 
     t = dict(q=draw(B, Hq, S, d), prefix_k=draw(Bp, Hkv, Pmax, d), prefix_v=draw(Bp, Hkv, Pmax, d),
              suffix_k=draw(B, Hkv, S, d), suffix_v=draw(B, Hkv, S, d), dout=draw(B, Hq, S, d))
-    # padding rows hold large garbage: they must never be read
+    # padding rows hold large finite garbage: it must not reach any result
     for i, n in enumerate(lens):
         t["prefix_k"][i, :, : Pmax - n] = 3.0e4
         t["prefix_v"][i, :, : Pmax - n] = -3.0e4
