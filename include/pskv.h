@@ -172,10 +172,9 @@ long long pskv_attn_bwd_static_max_rows(void);
  * suffix_k, suffix_v, out, lse, dout, dq, dk_suffix, dv_suffix; scale; causal rule; error codes) is as
  * in pskv_attn_fwd / pskv_attn_bwd, with P replaced per candidate by the true prefix length of its
  * instruction.  When (B / Bp) * (Hq / Hkv) * S is a multiple of the kernels' row tile (128 rows in the
- * usual case), Bp <= 64, the shape runs on the tensor-core kernels and the padding is a small share of the
- * keys (all instructions padded to Pmax hold at most 1.5 times the keys of their true lengths; the
- * environment variable PSKV_MULTI_FORM = "one" or "passes", read at every call, overrides this last test),
- * all instructions are served by one launch per kernel, which also multiplies the padded keys.  Otherwise the work is one pass per instruction; the passes are independent, so every
+ * usual case), Bp <= 64 and the shape runs on the tensor-core kernels, all instructions are served by one
+ * launch per kernel (the environment variable PSKV_MULTI_FORM = "passes", read at every call, turns this
+ * off; "one" is the default).  Otherwise the work is one pass per instruction; the passes are independent, so every
  * other one is enqueued on a stream of the library's own that forks from `cuda_stream` at the start of the
  * call and joins it again before the call returns (to the caller everything is ordered as if it had run on
  * `cuda_stream`, also under stream capture).

@@ -426,19 +426,12 @@ SideStream *side_stream()
     return ss.state == 1 ? &ss : nullptr;
 }
 
-// The one-launch form multiplies every instruction's padded key blocks too.  It saves about 8 us of
-// start-up and drain per instruction, so it pays unless the padding is a large share of the keys: it is
-// taken while all instructions padded to Pmax hold at most 1.5 times the keys of their true lengths.
-// The environment variable PSKV_MULTI_FORM overrides the choice ("one" or "passes"), read at every call.
-bool fused_worthwhile(const int *prefix_len, int Bp, int Pmax, int S)
+// The environment variable PSKV_MULTI_FORM ("one" or "passes"), read at every call, overrides the
+// library's choice between one launch for all instructions and one pass per instruction.
+int multi_form_env()
 {
-    if (const char *form = getenv("PSKV_MULTI_FORM")) {
-        if (form[0] == 'o') return true;
-        if (form[0] == 'p') return false;
-    }
-    long long real = 0;
-    for (int i = 0; i < Bp; ++i) real += prefix_len[i] + S;
-    return 2ll * Bp * (Pmax + S) <= 3ll * real;
+    const char *form = getenv("PSKV_MULTI_FORM");
+    return !form ? 0 : form[0] == 'o' ? 1 : form[0] == 'p' ? 2 : 0;
 }
 
 // checks shared by the two multi-instruction calls; fills the per-instruction geometry
@@ -485,7 +478,7 @@ pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void 
         // One launch over all instructions when every tile lies inside one instruction: the prefix caches
         // are heads of one [Bp*Hkv][Pmax][d] tensor and the left padding is masked like a causal limit.
         Dims dall;
-        if (Bp > 1 && fused_worthwhile(prefix_len, Bp, Pmax, S) && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
+        if (Bp > 1 && multi_form_env() != 2 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
             tc_fwd_fused_supported(dall, Bp)) {
             FwdArgs a;
             a.q = static_cast<const __nv_bfloat16 *>(q);
@@ -589,7 +582,7 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         // All instructions in one dQ launch when every tile lies inside one instruction (as in the forward);
         // the row statistic before it and the suffix gradients after it never involved the prefix.
         Dims dall;
-        if (Bp > 1 && fused_worthwhile(prefix_len, Bp, Pmax, S) && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
+        if (Bp > 1 && multi_form_env() != 2 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
             tc_bwd_fused_supported(dall, Bp)) {
             BwdArgs a;
             fill(a, 0, dall, 0);

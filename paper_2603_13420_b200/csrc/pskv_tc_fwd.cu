@@ -251,6 +251,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     auto first_of_run = [&](const TileInfo &t, int inst) {
         return t.first_of_g || (MI && t.R0 == inst * p.rpi);
     };
+    // First prefix block a tile works on: the blocks that hold nothing but left padding are skipped by
+    // every role (the resident copy still holds them, so the block index stays absolute).
+    auto first_block = [&](int inst) { return MI ? p.pad[inst] / kBlockN : 0; };
     int run_first;
     {
         const TileInfo t0 = tile_info(p, t_begin < p.total_tiles ? t_begin : 0, t_begin);
@@ -344,7 +347,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 __syncwarp();
             } else {
 #pragma unroll 1
-                for (int k = 0; k < p.nblk_p; ++k) {
+                for (int k = first_block(inst); k < p.nblk_p; ++k) {
                     const uint32_t ks = kload % (uint32_t)p.stages;
                     ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / (uint32_t)p.stages) & 1) ^ 1, abort_flag,
                                         p.status, kErrProducerK);
@@ -437,10 +440,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             TileInfo t;
             int nk = 0;  // V blocks still to fetch through the ring for this tile
             int ph = 0;  // head index inside the prefix caches
+            int kfirst = 0;
             if (have_tile) {
                 t = tile_info(p, tile_at(tl), t_begin);
                 const int inst = inst_of(t);
                 ph = inst * p.Hkv + t.g;
+                kfirst = first_block(inst);
                 if (RES) {
                     // the resident prefix V blocks are free once every value MMA of the previous tile
                     // has completed
@@ -463,7 +468,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     nk = SR ? items_of(t) : p.nblk_p;
                 }
             }
-            int k = 0;
+            int k = nk > 0 ? kfirst : 0;  // (nk stays 0 when the prefix is resident)
 #pragma unroll 1
             while (ok && (k < nk || pend_store || pend_sv)) {
                 const bool block = k >= nk;  // nothing else left to do for this tile: wait for the jobs
@@ -572,10 +577,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         __syncwarp();
     } else if (role == 1) {
         // ------------------------------------------------------------------ score MMAs: S = Q K^T
-        int tl = 0, k = 0;
+        int tl = 0;
         uint32_t kuse = 0;  // streaming mode: K blocks consumed from the ring
         TileInfo t = tile_info(p, tile_at(0), t_begin);
         int nitems = items_of(t);
+        int kfirst = first_block(inst_of(t)), k = kfirst;
         const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
         bool ok = true;
         for (int i = 0; tl < n_tiles && ok; ++i) {
@@ -619,12 +625,22 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             ok = mbar_wait_warp(bar(kBarPvDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaQk);
             if (!ok) break;
             PSKV_TRACE_EVENT(18, i);
-            if (k == 0) {
+            if (k == kfirst) {
                 ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaQk);
                 if (!ok) break;
             }
             if (kwait) {
                 ok = mbar_wait_warp(kbar, kpar, abort_flag, p.status, kErrMmaQk);
+                if (!ok) break;
+            }
+            if (MI && RES && k == kfirst && first_of_run(t, inst_of(t))) {
+                // The resident copy of a run always loads every prefix block, also those this run skips as
+                // padding.  Nobody multiplies them, so their loads are waited for here: a load must have
+                // landed before its buffer and barrier are armed again for the next run, and before the
+                // CTA exits.
+                const uint32_t par = (uint32_t)(run_of(t, inst_of(t)) - run_first) & 1u;
+                for (int kk = 0; kk < kfirst && kk < p.nblk_p && ok; ++kk)
+                    ok = mbar_wait_warp(bar(kBarKFull + kk), par, abort_flag, p.status, kErrMmaQk);
                 if (!ok) break;
             }
             PSKV_TRACE_EVENT(10, i);
@@ -648,15 +664,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (++tl < n_tiles) {
                     t = tile_info(p, tile_at(tl), t_begin);
                     nitems = items_of(t);
+                    k = kfirst = first_block(inst_of(t));
                 }
             }
         }
     } else if (role == 2) {
         // ------------------------------------------------------------------ value MMAs: O += P V
-        int tl = 0, k = 0;
+        int tl = 0;
         uint32_t vuse = 0;
         TileInfo t = tile_info(p, tile_at(0), t_begin);
         int nitems = items_of(t);
+        int kfirst = first_block(inst_of(t)), k = kfirst;
         const uint32_t idesc_pv = make_idesc_bf16(kTileM, D, 1);
         bool ok = true;
         for (int i = 0; tl < n_tiles && ok; ++i) {
@@ -693,11 +711,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const int nk = n >> 4;
             const bool last_of_tile = k == nitems - 1;
             const bool free_stage = (k < p.nblk_p || SR) && !RES;
-            const uint32_t acc0 = k > 0 ? 1u : 0u;
+            const uint32_t acc0 = k > kfirst ? 1u : 0u;
             PSKV_TRACE_EVENT(17, i);
             ok = mbar_wait_warp(bar(kBarPReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaPv);
             if (!ok) break;
-            if (k == 0 && tl > 0) {
+            if (k == kfirst && tl > 0) {
                 // O of the previous tile must have been read out by the epilogue warps
                 PSKV_TRACE_EVENT(15, i);
                 ok = mbar_wait_warp(bar(kBarOFree), (tl - 1) & 1, abort_flag, p.status, kErrMmaPv);
@@ -706,6 +724,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (vwait) {
                 PSKV_TRACE_EVENT(14, i);
                 ok = mbar_wait_warp(vbar, vpar, abort_flag, p.status, kErrMmaPv);
+                if (!ok) break;
+            }
+            if (MI && RES && k == kfirst && first_of_run(t, inst_of(t))) {  // (as for the K blocks above)
+                const uint32_t par = (uint32_t)(run_of(t, inst_of(t)) - run_first) & 1u;
+                for (int kk = 0; kk < kfirst && kk < p.nblk_p && ok; ++kk)
+                    ok = mbar_wait_warp(bar(kBarVFull + kk), par, abort_flag, p.status, kErrMmaPv);
                 if (!ok) break;
             }
             PSKV_TRACE_EVENT(11, i);
@@ -732,6 +756,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (++tl < n_tiles) {
                     t = tile_info(p, tile_at(tl), t_begin);
                     nitems = items_of(t);
+                    k = kfirst = first_block(inst_of(t));
                 }
             }
         }
@@ -786,7 +811,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             // several instructions: the first `pad` prefix keys of this tile's instruction are left padding
             const int pad = MI ? p.pad[inst_of(t)] : 0;
 #pragma unroll 1
-            for (int k = 0; k < nitems && ok; ++k, ++item) {
+            for (int k = pad / kBlockN; k < nitems && ok; ++k, ++item) {
                 {
                     const int slot = item % kSlots;
                     const uint32_t s_tmem = tmem + lane_addr + slot * kBlockN + wg * kPiece;

@@ -148,12 +148,41 @@ def test_multi_arguments_are_checked_on_the_host():
 
 
 @pytest.mark.gpu
-def test_the_library_picks_one_launch_only_while_padding_is_a_small_share_of_the_keys(monkeypatch):
+def test_the_library_takes_one_launch_by_itself_whenever_the_shape_allows_it(monkeypatch):
     monkeypatch.delenv("PSKV_MULTI_FORM", raising=False)
-    for lens, launches in (((256, 200), 1), ((256, 16), 2)):
+    for lens in ((256, 200), (256, 16)):
         case = (64, 2, 32, 8, 48, 256, 128, lens)
         t = make(*case)
         dev = {k: v.cuda() for k, v in t.items()}
         n0 = pskv.pskv_kernel_launches()
-        pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"], dev["suffix_v"], 0.088)
-        assert pskv.pskv_kernel_launches() - n0 == launches
+        out, lse = pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
+                                            dev["suffix_v"], 0.088)
+        assert pskv.pskv_kernel_launches() - n0 == 1
+        n0 = pskv.pskv_kernel_launches()
+        pskv.pskv_attn_bwd_multi(dev["dout"], dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
+                                 dev["suffix_v"], out, lse, 0.088)
+        assert pskv.pskv_kernel_launches() - n0 == 3   # row statistic, dQ, suffix gradients
+
+
+@pytest.mark.gpu
+def test_back_to_back_one_launch_calls_with_prefixes_that_are_padding_only(monkeypatch):
+    """Instructions whose prefix is empty skip every prefix block, yet the resident copy of their run is
+    still loaded: those loads have to land before the CTA exits or arms the buffers again.  Many calls in a
+    row without a synchronisation in between, each checked against the first."""
+    monkeypatch.setenv("PSKV_MULTI_FORM", "one")
+    case = (64, 4, 32, 8, 48, 256, 128, (256, 0, 0, 130))
+    B, Bp, Hq, Hkv, S, Pmax, d, lens = case
+    t = make(*case)
+    dev = {k: v.cuda() for k, v in t.items()}
+    scale = 1.0 / np.sqrt(d)
+    ref_out, ref_lse = pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
+                                                dev["suffix_v"], scale)
+    torch.cuda.synchronize()
+    outs = []
+    for _ in range(40):
+        outs.append(pskv.pskv_attn_fwd_multi(dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
+                                             dev["suffix_v"], scale))
+    torch.cuda.synchronize()
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    for o, l in outs:
+        assert torch.equal(o, ref_out) and torch.equal(l, ref_lse)
