@@ -469,15 +469,18 @@ def detail_runs(pskv, device, peaks):
         pskv.pskv_attn_bwd_multi(do, q, pk, pv, lens, sk, sv, out, lse, w.scale, dq=dq, dk_suffix=dk, dv_suffix=dv,
                                  workspace=ws_b)
 
-    mfwd()
     kq = w.B // Bp
-    fl_f = sum(wl.fwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
-    fl_b = sum(wl.bwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
-    ms_f = time_calls(mfwd, 20, 3)
-    ms_b = time_calls(mbwd, 20, 3)
-    res["C2_multi_8x64"] = {"prefix_len": lens,
-                            "fwd": {"ms": ms_f, "tflops": fl_f / ms_f / 1e9, "candidates_per_s": w.B / ms_f * 1e3},
-                            "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
+    # ... and with very unequal instruction lengths (padding is more than half of the padded keys)
+    for key, ls in (("C2_multi_8x64", lens), ("C2_multi_8x64_unequal", [256, 32, 32, 32, 200, 100, 16, 64])):
+        lens = ls
+        mfwd()
+        fl_f = sum(wl.fwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
+        fl_b = sum(wl.bwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
+        ms_f = time_calls(mfwd, 20, 3)
+        ms_b = time_calls(mbwd, 20, 3)
+        res[key] = {"prefix_len": list(lens),
+                    "fwd": {"ms": ms_f, "tflops": fl_f / ms_f / 1e9, "candidates_per_s": w.B / ms_f * 1e3},
+                    "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
     del q, sk, sv, do, pk, pv, out, lse, dq, dk, dv
     torch.cuda.empty_cache()
     for Bd in (512, 2048):
