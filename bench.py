@@ -405,6 +405,48 @@ TRAFFIC_BYTES_PER_LAUNCH = {
 }
 
 
+MULTI_LENS = [256, 240, 224, 208, 192, 176, 160, 144]
+MULTI_LENS_UNEQUAL = [256, 32, 32, 32, 200, 100, 16, 64]
+
+
+def multi_run(pskv, device, lens, iters, warmup):
+    """pskv_attn_fwd_multi / pskv_attn_bwd_multi at the C2 shape: len(lens) instructions, B / len(lens)
+    candidates each, one left-padded prefix cache per instruction."""
+    w = wl.WORKLOADS["C2"]
+    Bp, Pmax = len(lens), w.P
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(w.seed + 500)
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16).to(device)
+
+    q, sk, sv, do = draw(w.B, w.Hq, w.S, w.d), draw(w.B, w.Hkv, w.S, w.d), draw(w.B, w.Hkv, w.S, w.d), draw(w.B, w.Hq, w.S, w.d)
+    pk, pv = draw(Bp, w.Hkv, Pmax, w.d), draw(Bp, w.Hkv, Pmax, w.d)
+    out = torch.empty_like(q)
+    lse = torch.empty((w.B, w.Hq, w.S), dtype=torch.float32, device=device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(sk), torch.empty_like(sv)
+    mdims = (w.B, Bp, w.Hq, w.Hkv, w.S, Pmax, w.d)
+    ws_f = torch.empty(max(pskv.pskv_attn_fwd_multi_workspace_bytes(*mdims), 256), dtype=torch.uint8, device=device)
+    ws_b = torch.empty(max(pskv.pskv_attn_bwd_multi_workspace_bytes(*mdims), 256), dtype=torch.uint8, device=device)
+
+    def mfwd():
+        pskv.pskv_attn_fwd_multi(q, pk, pv, lens, sk, sv, w.scale, out=out, lse=lse, workspace=ws_f)
+
+    def mbwd():
+        pskv.pskv_attn_bwd_multi(do, q, pk, pv, lens, sk, sv, out, lse, w.scale, dq=dq, dk_suffix=dk, dv_suffix=dv,
+                                 workspace=ws_b)
+
+    mfwd()
+    kq = w.B // Bp
+    fl_f = sum(wl.fwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
+    fl_b = sum(wl.bwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
+    ms_f = time_calls(mfwd, iters, warmup)
+    ms_b = time_calls(mbwd, iters, warmup)
+    return {"prefix_len": list(lens),
+            "fwd": {"ms": ms_f, "tflops": fl_f / ms_f / 1e9, "candidates_per_s": w.B / ms_f * 1e3},
+            "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
+
+
 def detail_runs(pskv, device, peaks):
     """Kernel-only timings of every workload (forward; backward where the workload asks for it)."""
     res = {}
@@ -444,45 +486,10 @@ def detail_runs(pskv, device, peaks):
     del layers
     torch.cuda.empty_cache()
     # Batched multi-instruction variant (Sec. 4.3) at the C2 shape: 8 instructions x 64 candidates, one
-    # left-padded prefix cache per instruction, true lengths 144..256
-    lens = [256, 240, 224, 208, 192, 176, 160, 144]
-    Bp, Pmax = len(lens), w.P
-    gen = torch.Generator(device="cpu")
-    gen.manual_seed(w.seed + 500)
-
-    def draw(*shape):
-        return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16).to(device)
-
-    q, sk, sv, do = draw(w.B, w.Hq, w.S, w.d), draw(w.B, w.Hkv, w.S, w.d), draw(w.B, w.Hkv, w.S, w.d), draw(w.B, w.Hq, w.S, w.d)
-    pk, pv = draw(Bp, w.Hkv, Pmax, w.d), draw(Bp, w.Hkv, Pmax, w.d)
-    out = torch.empty_like(q)
-    lse = torch.empty((w.B, w.Hq, w.S), dtype=torch.float32, device=device)
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(sk), torch.empty_like(sv)
-    mdims = (w.B, Bp, w.Hq, w.Hkv, w.S, Pmax, w.d)
-    ws_f = torch.empty(max(pskv.pskv_attn_fwd_multi_workspace_bytes(*mdims), 256), dtype=torch.uint8, device=device)
-    ws_b = torch.empty(max(pskv.pskv_attn_bwd_multi_workspace_bytes(*mdims), 256), dtype=torch.uint8, device=device)
-
-    def mfwd():
-        pskv.pskv_attn_fwd_multi(q, pk, pv, lens, sk, sv, w.scale, out=out, lse=lse, workspace=ws_f)
-
-    def mbwd():
-        pskv.pskv_attn_bwd_multi(do, q, pk, pv, lens, sk, sv, out, lse, w.scale, dq=dq, dk_suffix=dk, dv_suffix=dv,
-                                 workspace=ws_b)
-
-    kq = w.B // Bp
-    # ... and with very unequal instruction lengths (padding is more than half of the padded keys)
-    for key, ls in (("C2_multi_8x64", lens), ("C2_multi_8x64_unequal", [256, 32, 32, 32, 200, 100, 16, 64])):
-        lens = ls
-        mfwd()
-        fl_f = sum(wl.fwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
-        fl_b = sum(wl.bwd_flops(dataclasses.replace(w, B=kq, P=n)) for n in lens)
-        ms_f = time_calls(mfwd, 20, 3)
-        ms_b = time_calls(mbwd, 20, 3)
-        res[key] = {"prefix_len": list(lens),
-                    "fwd": {"ms": ms_f, "tflops": fl_f / ms_f / 1e9, "candidates_per_s": w.B / ms_f * 1e3},
-                    "bwd": {"ms": ms_b, "tflops": fl_b / ms_b / 1e9, "candidates_per_s": w.B / ms_b * 1e3}}
-    del q, sk, sv, do, pk, pv, out, lse, dq, dk, dv
-    torch.cuda.empty_cache()
+    # left-padded prefix cache per instruction, true lengths 144..256; then very unequal lengths (padding is
+    # more than half of the padded keys)
+    res["C2_multi_8x64"] = multi_run(pskv, device, MULTI_LENS, 20, 3)
+    res["C2_multi_8x64_unequal"] = multi_run(pskv, device, MULTI_LENS_UNEQUAL, 20, 3)
     for Bd in (512, 2048):
         res["C2_decode_1of48_B%d" % Bd] = decode_run(pskv, device, peaks, Bd, 40, 4)
     res["prefix_prefill_P%d" % wl.WORKLOADS["C3"].P] = prefill_run(pskv, device, peaks, 40, 4)
@@ -631,6 +638,8 @@ def run_variant(args):
         res = prefill_run(pskv, device, peaks, args.steps, max(args.warmup, 3))
     elif args.variant == "prefix_grad":
         res = prefix_grad_run(pskv, device, peaks, args.steps, max(args.warmup, 3))
+    elif args.variant == "multi":
+        res = multi_run(pskv, device, MULTI_LENS, args.steps, max(args.warmup, 3))
     elif args.variant == "target_ce":
         res = ce_run(pskv, device, peaks, args.steps, max(args.warmup, 3), with_library=False)
     else:
@@ -668,7 +677,7 @@ def main():
                     help="candidates of the one-off CPU oracle sample reported as cpu_baseline")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
-    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill", "target_ce", "prefix_grad"],
+    ap.add_argument("--variant", default=None, choices=["decode_B512", "decode_B2048", "prefill", "target_ce", "prefix_grad", "multi"],
                     help="time only this variant of the detail runs (1 GPU) and print its entry")
     args = ap.parse_args()
     if args.impl == "reference":
