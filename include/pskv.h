@@ -283,10 +283,21 @@ int pskv_version(void);
 
 /*
  * Which kernel family pskv_attn_fwd / pskv_attn_bwd pick for these sizes:
- * 1 = tcgen05 / TMEM tensor-core kernels, 0 = general CUDA-core kernels, negative = sizes rejected.
+ * 2 = tcgen05 kernels on CTA pairs (two SMs share every MMA, cta_group::2; only after
+ * pskv_enable_cta_pairs(1)), 1 = tcgen05 / TMEM
+ * tensor-core kernels, one CTA per tile, 0 = general CUDA-core kernels, negative = sizes rejected.
  * `backward` selects which call is asked about.  Pure host logic; touches no device.
  */
 int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d);
+
+/*
+ * The CTA-pair kernels compute the same operator (Eq. 2 over the shared prefix of Sec. 4.2) as the
+ * single-CTA tensor-core kernels, for the shapes they take (pskv_kernel_family tells, once they are
+ * switched on).  They are OFF by default: at the layer shapes measured so far they are 5-15 % slower
+ * than the single-CTA kernels.  on = 1 makes every later call of this process use them where they
+ * apply, e.g. to compare the two.  Process-wide, host-side switch; touches no device.
+ */
+void pskv_enable_cta_pairs(int on);
 
 /*
  * Number of kernels this library has launched in this process so far (all threads, all devices).

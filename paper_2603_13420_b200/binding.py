@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.pskv_kernel_launches.restype = ctypes.c_longlong
         L.pskv_kernel_family.argtypes = [ci] + six
         L.pskv_kernel_family.restype = ci
+        L.pskv_enable_cta_pairs.argtypes = [ci]
+        L.pskv_enable_cta_pairs.restype = None
         _lib = L
     return _lib
 
@@ -166,6 +168,10 @@ def pskv_last_cuda_error() -> int:
 
 def pskv_status_string(status: int) -> str:
     return lib().pskv_status_string(int(status)).decode()
+
+
+def pskv_enable_cta_pairs(on: bool) -> None:
+    lib().pskv_enable_cta_pairs(int(bool(on)))
 
 
 def pskv_kernel_family(backward, B, Hq, Hkv, S, P, d) -> int:

@@ -91,6 +91,7 @@ size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
 size_t simt_bwd_workspace(const Dims &dm) { return round256((size_t)dm.B * dm.Hq * dm.S * sizeof(float)); }
 
 std::atomic<long long> g_launches{0};
+std::atomic<int> g_cta_pairs{0};
 
 // ---- optional per-kernel timing: a bounded list of (kernel id, start event, stop event)
 constexpr int kMaxTimed = 8192;
@@ -107,6 +108,8 @@ const char *const kKernelNames[kKernelCount] = {
     "simt_fwd_kernel", "simt_bwd_dq_kernel", "simt_bwd_dkv_kernel", "ce_fwd_kernel", "ce_finalize_kernel", "tc_bwd_prefix_kernel", "simt_bwd_prefix_kernel"};
 
 }  // namespace
+
+bool cta_pairs_enabled() { return g_cta_pairs.load(std::memory_order_relaxed) != 0; }
 
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -198,8 +201,11 @@ int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d
     Dims dm;
     pskv_status st = check_dims(B, Hq, Hkv, S, P, d, &dm);
     if (st != PSKV_OK) return -(int)st;
+    if (!backward && tc_fwd_supported(dm) && cta_pairs_enabled() && tc_fwd_pair_supported(dm)) return 2;
     return (backward ? tc_bwd_supported(dm) : tc_fwd_supported(dm)) ? 1 : 0;
 }
+
+void pskv_enable_cta_pairs(int on) { g_cta_pairs.store(on != 0, std::memory_order_relaxed); }
 
 size_t pskv_attn_fwd_workspace_bytes(int B, int Hq, int Hkv, int S, int P, int d)
 {

@@ -77,6 +77,11 @@ constexpr int kMaxFusedInstructions = 64;
 bool tc_fwd_fused_supported(const Dims &d, int n_instr);
 cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *status_word,
                           cudaStream_t stream, int n_instr = 1, const int *prefix_len = nullptr);
+// The forward on CTA pairs (cta_group::2), for the shapes it takes; launch_tc_fwd goes there by itself
+// unless pairs are switched off (pskv_enable_cta_pairs).
+bool tc_fwd_pair_supported(const Dims &d);
+cudaError_t launch_tc_fwd_pair(const FwdArgs &a, unsigned int *status_word, cudaStream_t stream);
+bool cta_pairs_enabled();
 bool tc_bwd_supported(const Dims &d);
 size_t tc_bwd_workspace_bytes(const Dims &d);
 // `parts` selects which of the three steps run (all by default): the row statistic D and the suffix

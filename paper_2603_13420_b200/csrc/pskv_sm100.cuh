@@ -59,10 +59,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// try_wait that lets the hardware suspend the thread for up to `hint_ns` nanoseconds while the phase is
+// incomplete (it resumes at once when the phase completes).  Without the hint a failed try_wait returns
+// after a short, system-chosen time, and a warp that polls in a loop keeps taking issue slots from the
+// warps of its scheduler that have work: in these kernels more than half of all executed instructions
+// were such polls.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Every wait in the kernels goes through this: it gives up after `kWaitBudgetCycles`, or as soon
 // as another thread of the CTA has given up (the CTA-wide `abort_flag` in shared memory), records
 // `code` in the device status word and returns false; the caller then leaves its role loop.
 constexpr long long kWaitBudgetCycles = 2000000000ll;  // about one second at B200 clocks
+constexpr uint32_t kSuspendNs = 100000u;               // longest hardware suspension per poll
 
 // The polling loop is one shared out-of-line routine: the kernels' hot loops stay small enough for
 // the instruction cache, and a wait that is already satisfied costs one inlined try_wait.
@@ -70,15 +91,13 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
                                             unsigned int *status_word, unsigned int code)
 {
     const long long start = clock64();
-    for (unsigned int spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0u) {
-            if (*abort_flag != 0) return false;
-            if (clock64() - start > kWaitBudgetCycles) {
-                *abort_flag = 1;
-                atomicCAS(status_word, 0u, code);
-                return false;
-            }
+    for (;;) {
+        if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
+        if (*abort_flag != 0) return false;
+        if (clock64() - start > kWaitBudgetCycles) {
+            *abort_flag = 1;
+            atomicCAS(status_word, 0u, code);
+            return false;
         }
     }
 }
@@ -341,6 +360,130 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+
+// ---------------------------------------------------------------------------------------------
+// CTA pairs: a cluster of two CTAs on the two SMs of one TPC shares every MMA (cta_group::2).  One
+// thread of the CTA with cluster rank 0 issues an instruction of 256 rows; each CTA supplies its own
+// 128 rows of A and its own half of B's N rows from its own shared memory, and receives its 128 rows
+// of D in its own tensor memory.  Every copy stays a plain single-CTA TMA load; the CTAs talk
+// through mbarriers (remote arrives, commits that signal the same barrier in both CTAs).
+
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// Address (shared::cluster window) of this CTA's shared-memory address `addr` in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+
+// One arrival on an mbarrier of another CTA of the cluster (address from map_to_cta).  What the
+// arrival publishes here lives in tensor memory or was written by TMA, each ordered by its own
+// fences, so the arrival itself carries no cluster-wide release (which costs about a thousand cycles).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__device__ __forceinline__ void store_remote_u32(uint32_t cluster_addr, uint32_t v)
+{
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
+// try_wait of the pair kernels (the phase may have been completed by the other CTA)
+__device__ __forceinline__ bool mbar_try_wait_cl(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait of the pair kernels; all 32 lanes wait, true only if every lane saw the phase.
+__device__ __forceinline__ bool mbar_wait_warp_cl(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                  unsigned int *status_word, unsigned int code)
+{
+    bool ok = mbar_try_wait_cl(bar, parity);
+    if (!ok) ok = mbar_wait_slow(bar, parity, abort_flag, status_word, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// Tensor memory of a CTA pair: the same warp of BOTH CTAs executes each of these.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// One arrival on the mbarrier at this shared-memory offset in every CTA of `cta_mask` once all
+// tcgen05.mma issued so far by this thread have completed.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"(cta_mask)
+        : "memory");
+}
+
+// D[tmem, 2 x 128 rows] (+)= A[smem of each CTA] * B[smem, half of N per CTA]
+__device__ __forceinline__ void mma_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// D[tmem] (+)= A[tmem of each CTA] * B[smem, half of N per CTA]
+__device__ __forceinline__ void mma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+        "}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Registers move between the roles of a kernel: all four warps of a warpgroup (warps 4k .. 4k+3) give
+// up registers down to, or ask for registers up to, N per thread (a multiple of 8).  An increase waits
+// until other warpgroups have released enough.
+template <int N>
+__device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // 2^x on the special-function unit (flushes denormals; 2^-inf = 0)
 __device__ __forceinline__ float ex2_approx(float x)

@@ -18,13 +18,16 @@ constexpr int kMaxSmem = 232448;             // dynamic shared memory a CTA may 
 // Optional event trace of CTA 0 (lane 0 of each warp, a private buffer per warp so that an event
 // costs one clock read and two stores): compiled in only with -DPSKV_TRACE=<group mask>.
 #ifdef PSKV_TRACE
+#ifndef PSKV_TRACE_CTA
+#define PSKV_TRACE_CTA 0
+#endif
 constexpr int kTraceWarps = 28, kTraceCap = 4096;
 __device__ long long g_trace[kTraceWarps * kTraceCap * 2];
 __device__ unsigned int g_trace_n[kTraceWarps];
 #define PSKV_TRACE_DECL unsigned int trace_i_ = 0
 #define PSKV_TRACE_EVENT(tag, val)                                                                     \
     do {                                                                                               \
-        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == 0 && (threadIdx.x & 31) == 0 &&        \
+        if (((PSKV_TRACE >> ((tag) / 10)) & 1) && blockIdx.x == PSKV_TRACE_CTA && (threadIdx.x & 31) == 0 &&        \
             trace_i_ < (unsigned int)kTraceCap) {                                                      \
             long long *e_ = g_trace + ((size_t)(threadIdx.x >> 5) * kTraceCap + trace_i_) * 2;         \
             e_[0] = clock64();                                                                         \
@@ -34,7 +37,7 @@ __device__ unsigned int g_trace_n[kTraceWarps];
     } while (0)
 #define PSKV_TRACE_FLUSH                                                                               \
     do {                                                                                               \
-        if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
+        if (blockIdx.x == PSKV_TRACE_CTA && (threadIdx.x & 31) == 0) g_trace_n[threadIdx.x >> 5] = trace_i_;        \
     } while (0)
 #else
 #define PSKV_TRACE_DECL do { } while (0)

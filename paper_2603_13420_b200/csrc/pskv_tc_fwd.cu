@@ -1309,6 +1309,8 @@ cudaError_t launch_tc_fwd(const FwdArgs &a, void *workspace, unsigned int *statu
     if (!plan.ok) return cudaErrorInvalidValue;
     if (n_instr > 1 && (!prefix_len || !tc_fwd_fused_supported(a.dims, n_instr))) return cudaErrorInvalidValue;
     if (n_instr < 1) n_instr = 1;
+    if (n_instr == 1 && cta_pairs_enabled() && tc_fwd_pair_supported(a.dims))
+        return launch_tc_fwd_pair(a, status_word, stream);
     return a.dims.d == 128 ? launch<128>(a, plan, workspace, status_word, stream, n_instr, prefix_len)
                            : launch<64>(a, plan, workspace, status_word, stream, n_instr, prefix_len);
 }
