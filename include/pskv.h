@@ -173,13 +173,21 @@ long long pskv_attn_bwd_static_max_rows(void);
  * in pskv_attn_fwd / pskv_attn_bwd, with P replaced per candidate by the true prefix length of its
  * instruction.  When (B / Bp) * (Hq / Hkv) * S is a multiple of the kernels' row tile (128 rows in the
  * usual case), Bp <= 64 and the shape runs on the tensor-core kernels, all instructions are served by one
- * launch per kernel (the environment variable PSKV_MULTI_FORM = "passes", read at every call, turns this
- * off; "one" is the default).  Otherwise the work is one pass per instruction; the passes are independent, so every
+ * launch per kernel (pskv_set_multi_form(2) turns this off).  Otherwise the work is one pass per instruction; the passes are independent, so every
  * other one is enqueued on a stream of the library's own that forks from `cuda_stream` at the start of the
  * call and joins it again before the call returns (to the caller everything is ordered as if it had run on
  * `cuda_stream`, also under stream capture).
  */
 size_t pskv_attn_fwd_multi_workspace_bytes(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d);
+
+/*
+ * How the multi-instruction calls (Sec. 4.3) schedule their work: 0 = the library chooses (one launch for
+ * all instructions where the shapes allow it, else one pass per instruction), 1 = the same choice, stated
+ * explicitly, 2 = always one pass per instruction.  Both forms compute the same result; the switch exists
+ * to compare them.  Process-wide, host side; PSKV_ERR_INVALID_ARG for any other value.
+ */
+pskv_status pskv_set_multi_form(int form);
+
 pskv_status pskv_attn_fwd_multi(const void *q,        /* bf16 [B,Hq,S,d] */
                                 const void *prefix_k, /* bf16 [Bp,Hkv,Pmax,d] (may be NULL when Pmax == 0) */
                                 const void *prefix_v, /* bf16 [Bp,Hkv,Pmax,d] */
@@ -298,6 +306,23 @@ int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d
  * apply, e.g. to compare the two.  Process-wide, host-side switch; touches no device.
  */
 void pskv_enable_cta_pairs(int on);
+
+/*
+ * Self-test of the bounded device-side waits (the mechanism behind PSKV_ERR_DEVICE_TIMEOUT): enqueues one
+ * tiny kernel on `cuda_stream` in which a single warp waits, through the routine all tensor-core kernels
+ * wait with, for a barrier that nothing will ever complete, gives up after `budget_cycles` SM clock cycles
+ * (1 .. 1e9), records the time-out in the device status word and returns normally.  The next
+ * pskv_poll_device_status on that stream therefore returns PSKV_ERR_DEVICE_TIMEOUT once, and PSKV_OK after
+ * that; the device stays fully usable.  Returns PSKV_OK when the kernel was enqueued.  The paper has no
+ * counterpart: this checks the library's own failure detection.
+ */
+pskv_status pskv_selftest_wait_timeout(long long budget_cycles, void *cuda_stream);
+
+/*
+ * Self-test of the per-device bookkeeping of the launch sites (per-device opt-in to large dynamic shared
+ * memory), run on the host with made-up device ordinals; touches no device.  0 = passed.
+ */
+int pskv_selftest_per_device_once(void);
 
 /*
  * Number of kernels this library has launched in this process so far (all threads, all devices).

@@ -108,6 +108,12 @@ def lib() -> ctypes.CDLL:
         L.pskv_kernel_launches.restype = ctypes.c_longlong
         L.pskv_kernel_family.argtypes = [ci] + six
         L.pskv_kernel_family.restype = ci
+        L.pskv_selftest_wait_timeout.argtypes = [ctypes.c_longlong, vp]
+        L.pskv_selftest_wait_timeout.restype = ci
+        L.pskv_selftest_per_device_once.argtypes = []
+        L.pskv_selftest_per_device_once.restype = ci
+        L.pskv_set_multi_form.argtypes = [ci]
+        L.pskv_set_multi_form.restype = ci
         L.pskv_enable_cta_pairs.argtypes = [ci]
         L.pskv_enable_cta_pairs.restype = None
         _lib = L
@@ -168,6 +174,26 @@ def pskv_last_cuda_error() -> int:
 
 def pskv_status_string(status: int) -> str:
     return lib().pskv_status_string(int(status)).decode()
+
+
+def pskv_selftest_wait_timeout(budget_cycles: int = 100000) -> None:
+    """Enqueue the tiny kernel whose bounded wait runs out (see include/pskv.h)."""
+    st = lib().pskv_selftest_wait_timeout(int(budget_cycles), _stream())
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_selftest_wait_timeout")
+
+
+def pskv_selftest_per_device_once() -> int:
+    return int(lib().pskv_selftest_per_device_once())
+
+
+def pskv_set_multi_form(form) -> None:
+    """0 / "auto": the library chooses; 1 / "one": one launch for all instructions where the shapes allow
+    it; 2 / "passes": one pass per instruction."""
+    form = {"auto": 0, "one": 1, "passes": 2}.get(form, form)
+    st = lib().pskv_set_multi_form(int(form))
+    if st != PSKV_OK:
+        raise PskvError(st, "pskv_set_multi_form")
 
 
 def pskv_enable_cta_pairs(on: bool) -> None:

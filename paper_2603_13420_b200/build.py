@@ -14,7 +14,7 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libpskv.so")
 
-SOURCES = ["pskv_api.cu", "pskv_simt.cu", "pskv_tc_fwd.cu", "pskv_tc_fwd_pair.cu", "pskv_tc_bwd.cu", "pskv_tc_dkv.cu", "pskv_bwd_dkv.cu", "pskv_noalloc.cu", "pskv_ce.cu"]
+SOURCES = ["pskv_api.cu", "pskv_simt.cu", "pskv_tc_fwd.cu", "pskv_tc_fwd_pair.cu", "pskv_tc_bwd.cu", "pskv_tc_dkv.cu", "pskv_bwd_dkv.cu", "pskv_noalloc.cu", "pskv_selftest.cu", "pskv_ce.cu"]
 
 
 def _nvcc() -> str:

@@ -92,6 +92,7 @@ size_t simt_bwd_workspace(const Dims &dm) { return round256((size_t)dm.B * dm.Hq
 
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_cta_pairs{0};
+std::atomic<int> g_multi_form{0};  // see pskv_set_multi_form
 
 // ---- optional per-kernel timing: a bounded list of (kernel id, start event, stop event)
 constexpr int kMaxTimed = 8192;
@@ -110,6 +111,8 @@ const char *const kKernelNames[kKernelCount] = {
 }  // namespace
 
 bool cta_pairs_enabled() { return g_cta_pairs.load(std::memory_order_relaxed) != 0; }
+
+pskv_status device_status_word(unsigned int **status_word) { return check_device(status_word); }
 
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -203,6 +206,13 @@ int pskv_kernel_family(int backward, int B, int Hq, int Hkv, int S, int P, int d
     if (st != PSKV_OK) return -(int)st;
     if (!backward && tc_fwd_supported(dm) && cta_pairs_enabled() && tc_fwd_pair_supported(dm)) return 2;
     return (backward ? tc_bwd_supported(dm) : tc_fwd_supported(dm)) ? 1 : 0;
+}
+
+pskv_status pskv_set_multi_form(int form)
+{
+    if (form < 0 || form > 2) return PSKV_ERR_INVALID_ARG;
+    g_multi_form.store(form, std::memory_order_relaxed);
+    return PSKV_OK;
 }
 
 void pskv_enable_cta_pairs(int on) { g_cta_pairs.store(on != 0, std::memory_order_relaxed); }
@@ -432,13 +442,9 @@ SideStream *side_stream()
     return ss.state == 1 ? &ss : nullptr;
 }
 
-// The environment variable PSKV_MULTI_FORM ("one" or "passes"), read at every call, overrides the
-// library's choice between one launch for all instructions and one pass per instruction.
-int multi_form_env()
-{
-    const char *form = getenv("PSKV_MULTI_FORM");
-    return !form ? 0 : form[0] == 'o' ? 1 : form[0] == 'p' ? 2 : 0;
-}
+// pskv_set_multi_form: 0 = the library chooses between one launch for all instructions and one pass per
+// instruction, 1 = one launch wherever the shapes allow it (the same as 0 today), 2 = always passes.
+int multi_form() { return g_multi_form.load(std::memory_order_relaxed); }
 
 // checks shared by the two multi-instruction calls; fills the per-instruction geometry
 pskv_status check_multi(int B, int Bp, int Hq, int Hkv, int S, int Pmax, int d, const int *prefix_len)
@@ -484,7 +490,7 @@ pskv_status pskv_attn_fwd_multi(const void *q, const void *prefix_k, const void 
         // One launch over all instructions when every tile lies inside one instruction: the prefix caches
         // are heads of one [Bp*Hkv][Pmax][d] tensor and the left padding is masked like a causal limit.
         Dims dall;
-        if (Bp > 1 && multi_form_env() != 2 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
+        if (Bp > 1 && multi_form() != 2 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
             tc_fwd_fused_supported(dall, Bp)) {
             FwdArgs a;
             a.q = static_cast<const __nv_bfloat16 *>(q);
@@ -588,7 +594,7 @@ pskv_status pskv_attn_bwd_multi(const void *dout, const void *q, const void *pre
         // All instructions in one dQ launch when every tile lies inside one instruction (as in the forward);
         // the row statistic before it and the suffix gradients after it never involved the prefix.
         Dims dall;
-        if (Bp > 1 && multi_form_env() != 2 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
+        if (Bp > 1 && multi_form() != 2 && check_dims(B, Hq, Hkv, S, Pmax, d, &dall) == PSKV_OK &&
             tc_bwd_fused_supported(dall, Bp)) {
             BwdArgs a;
             fill(a, 0, dall, 0);

@@ -9,6 +9,7 @@
 // part is bound by its memory traffic, not by tensor throughput.  Sums over the heads of a group
 // happen in registers of one CTA, so the result is deterministic and needs no atomics.
 #include "pskv_common.cuh"
+#include "pskv_tc_common.cuh"
 
 namespace pskv {
 namespace {
@@ -274,31 +275,15 @@ bwd_dkv_mma_kernel(BwdArgs a)
     cp_async_wait_all();
 }
 
-inline int sm_count_dkv()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <int D, int TP>
 cudaError_t launch_one(const BwdArgs &a, cudaStream_t stream)
 {
     using L = DkvSmem<D, TP>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(bwd_dkv_mma_kernel<D, TP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             L::kBytes);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static PerDeviceOnce attr_set;
+    if (cudaError_t e = ensure_max_smem(bwd_dkv_mma_kernel<D, TP>, attr_set, L::kBytes); e != cudaSuccess) return e;
     KernelTiming timing(kKernelBwdDkvMma, stream);
     const int total_bg = a.dims.B * a.dims.Hkv;
-    const int max_ctas = 2 * sm_count_dkv();  // two resident CTAs per SM, each walking over its groups
+    const int max_ctas = 2 * sm_count();  // two resident CTAs per SM, each walking over its groups
     bwd_dkv_mma_kernel<D, TP><<<total_bg < max_ctas ? total_bg : max_ctas, kDkvThreads, L::kBytes, stream>>>(a);
     count_launches(1);
     return cudaGetLastError();

@@ -353,12 +353,8 @@ cudaError_t launch_ce_fwd(const CeArgs &a, void *workspace, unsigned int *status
     p.rg = sm_count() / 4 < 1 ? 1 : sm_count() / 4;
     if (p.rg > pl.nrt) p.rg = pl.nrt;
     const int smem_bytes = kCeStages * kCeStageBytes + 8 * kCeNumBars + 64;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(ce_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static PerDeviceOnce attr_set;
+    if (cudaError_t e = ensure_max_smem(ce_fwd_kernel, attr_set, smem_bytes); e != cudaSuccess) return e;
     const int grid = p.units < sm_count() ? p.units : sm_count();
     {
         KernelTiming timing(kKernelCeFwd, stream);

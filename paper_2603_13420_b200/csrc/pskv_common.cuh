@@ -105,6 +105,10 @@ bool ce_fwd_supported(int N, int Lr, int Dm, int V);
 size_t ce_fwd_workspace_bytes(int N, int Lr, int Dm, int V);
 cudaError_t launch_ce_fwd(const CeArgs &a, void *workspace, unsigned int *status_word, cudaStream_t stream);
 
+// PSKV_OK and the device address of the status word when the current device is an sm_100 part, else the
+// error the public calls return for it (PSKV_ERR_UNSUPPORTED_ARCH, PSKV_ERR_CUDA).
+pskv_status device_status_word(unsigned int **status_word);
+
 // Host-side count of kernel launches (read through pskv_kernel_launches()).
 void count_launches(int n);
 

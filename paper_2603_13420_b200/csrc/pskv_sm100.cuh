@@ -59,11 +59,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// try_wait that lets the hardware suspend the thread for up to `hint_ns` nanoseconds while the phase is
-// incomplete (it resumes at once when the phase completes).  Without the hint a failed try_wait returns
-// after a short, system-chosen time, and a warp that polls in a loop keeps taking issue slots from the
-// warps of its scheduler that have work: in these kernels more than half of all executed instructions
-// were such polls.
+// try_wait with a suspend-time hint: the thread may stay suspended for up to `hint_ns` nanoseconds while
+// the phase is incomplete (and resumes when it completes) instead of returning after a short,
+// system-chosen time.  About half of the instructions these kernels execute are polls of waiting warps;
+// the hint thins them out a little.  Measured: pollers do not slow the working warps of their scheduler
+// down (they only fill issue slots nobody else wants), so this is tidiness, not speed.
 __device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns)
 {
     uint32_t ok;
@@ -88,13 +88,14 @@ constexpr uint32_t kSuspendNs = 100000u;               // longest hardware suspe
 // The polling loop is one shared out-of-line routine: the kernels' hot loops stay small enough for
 // the instruction cache, and a wait that is already satisfied costs one inlined try_wait.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                            unsigned int *status_word, unsigned int code)
+                                            unsigned int *status_word, unsigned int code,
+                                            long long budget = kWaitBudgetCycles)
 {
     const long long start = clock64();
     for (;;) {
         if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
         if (*abort_flag != 0) return false;
-        if (clock64() - start > kWaitBudgetCycles) {
+        if (clock64() - start > budget) {
             *abort_flag = 1;
             atomicCAS(status_word, 0u, code);
             return false;
@@ -103,10 +104,11 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
 }
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          unsigned int *status_word, unsigned int code)
+                                          unsigned int *status_word, unsigned int code,
+                                          long long budget = kWaitBudgetCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status_word, code);
+    return mbar_wait_slow(bar, parity, abort_flag, status_word, code, budget);
 }
 
 // Bounded wait until a monotonically increasing shared-memory counter reaches `target`.
@@ -130,9 +132,10 @@ __device__ __forceinline__ bool spin_wait_ge(volatile int *counter, int target, 
 
 // All 32 lanes wait (the warp's control flow stays uniform); true only if every lane saw the phase.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                               unsigned int *status_word, unsigned int code)
+                                               unsigned int *status_word, unsigned int code,
+                                               long long budget = kWaitBudgetCycles)
 {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status_word, code));
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status_word, code, budget));
 }
 
 // One lane of a fully converged warp gets a non-zero result.

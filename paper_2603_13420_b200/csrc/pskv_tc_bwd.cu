@@ -852,12 +852,8 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
     auto kernel = plan.resident == 3 ? (mi ? tc_bwd_dq_kernel<D, 3, true> : tc_bwd_dq_kernel<D, 3, false>)
                   : plan.resident == 1 ? (mi ? tc_bwd_dq_kernel<D, 1, true> : tc_bwd_dq_kernel<D, 1, false>)
                                        : (mi ? tc_bwd_dq_kernel<D, 0, true> : tc_bwd_dq_kernel<D, 0, false>);
-    static bool attr_set[8] = {false, false, false, false, false, false, false, false};
-    if (!attr_set[plan.resident + (mi ? 4 : 0)]) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr_set[plan.resident + (mi ? 4 : 0)] = true;
-    }
+    static PerDeviceOnce attr_set[8];
+    if (cudaError_t e0 = ensure_max_smem(kernel, attr_set[plan.resident + (mi ? 4 : 0)]); e0 != cudaSuccess) return e0;
     // D = <dout, out> per row, then dQ on the tensor cores, then dK_suffix / dV_suffix
     cudaError_t e = cudaSuccess;
     if (parts & kBwdPartRowDot) {

@@ -4,6 +4,9 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
+
+#include <atomic>
 
 #include "pskv_common.cuh"
 
@@ -155,29 +158,102 @@ inline EncodeTiledFn get_encode_fn()
 }
 
 // bf16 tensor, innermost dimension contiguous, 128-byte swizzle, 64-column boxes.
+// A launch needs eight or nine of these and a search loop calls with the same buffers and shapes step
+// after step, so the encoded maps are kept in a small per-thread table keyed by everything that went
+// into them (base address, rank, extents, strides, box); a hit costs a compare and a 128-byte copy
+// instead of a driver call.  A tensor map holds no reference to the memory: a stale entry for a freed
+// and re-used address is still the right map for that address.
+struct MapKey {
+    const void *base;
+    int rank;
+    cuuint64_t dims[4], strides[3];
+    cuuint32_t box[4];
+};
+struct MapCacheEntry {
+    bool used;
+    MapKey key;
+    CUtensorMap map;
+};
+constexpr int kMapCacheSize = 64;  // direct-mapped
+
 inline bool encode_map(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims,
                 const cuuint64_t *strides_bytes, const cuuint32_t *box)
 {
+    static thread_local MapCacheEntry cache[kMapCacheSize];
+    MapKey key;
+    memset(&key, 0, sizeof(key));
+    key.base = base;
+    key.rank = rank;
+    for (int i = 0; i < rank && i < 4; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank && i < 3; ++i) key.strides[i] = strides_bytes[i];
+    unsigned long long h = (unsigned long long)(uintptr_t)base * 0x9E3779B97F4A7C15ull;
+    for (int i = 0; i < 4; ++i) h = (h ^ key.dims[i] ^ ((unsigned long long)key.box[i] << 40)) * 0x100000001B3ull;
+    MapCacheEntry &e = cache[(h >> 32) % kMapCacheSize];
+#ifndef PSKV_NO_MAP_CACHE  // (defined only to measure what the table saves)
+    if (e.used && memcmp(&e.key, &key, sizeof(key)) == 0) {
+        memcpy(map, &e.map, sizeof(CUtensorMap));
+        return true;
+    }
+#endif
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims,
                     strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    if (r != CUDA_SUCCESS) return false;
+    e.used = true;
+    e.key = key;
+    memcpy(&e.map, map, sizeof(CUtensorMap));
+    return true;
 }
 
+// Per-device state of the launch sites.  cudaFuncSetAttribute (the opt-in to more than 48 KB of
+// dynamic shared memory) and the SM count belong to a DEVICE, not to the process: a process that works
+// on several GPUs needs both once per device.
+constexpr int kMaxGuardDevices = 64;
+
+// One flag per device ordinal; first_time(dev) is true exactly once per device (ordinals beyond the
+// table are always "first", i.e. the caller simply repeats the cheap set-up).
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> done{0};
+    bool pending(int dev) const
+    {
+        return dev < 0 || dev >= kMaxGuardDevices || ((done.load(std::memory_order_acquire) >> dev) & 1ull) == 0;
+    }
+    void mark(int dev)
+    {
+        if (dev >= 0 && dev < kMaxGuardDevices) done.fetch_or(1ull << dev, std::memory_order_release);
+    }
+};
+
+// Raises a kernel's dynamic shared-memory limit on the current device if that has not been done there yet.
+template <class Kernel>
+inline cudaError_t ensure_max_smem(Kernel kernel, PerDeviceOnce &once, int bytes = kMaxSmem)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!once.pending(dev)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) once.mark(dev);
+    return e;
+}
+
+// SM count of the current device (looked up once per device).
 inline int sm_count()
 {
-    static int n = 0;
+    static std::atomic<int> count[kMaxGuardDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    const bool cached = dev >= 0 && dev < kMaxGuardDevices;
+    int n = cached ? count[dev].load(std::memory_order_relaxed) : 0;
     if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+        if (cached) count[dev].store(n, std::memory_order_relaxed);
     }
     return n;
 }
-
 
 }  // namespace
 }  // namespace pskv

@@ -468,12 +468,8 @@ template <int NP, bool PRE>
 cudaError_t launch_np(const BwdArgs &a, const CUtensorMap &tm_q, const CUtensorMap &tm_do, const CUtensorMap &tm_k,
                       const CUtensorMap &tm_v, const TcDkvParams &p, int smem_bytes, cudaStream_t stream)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_bwd_dkv_kernel<NP, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static PerDeviceOnce attr_set;
+    if (cudaError_t e = ensure_max_smem(tc_bwd_dkv_kernel<NP, PRE>, attr_set); e != cudaSuccess) return e;
     const int grid = p.total_groups < sm_count() ? p.total_groups : sm_count();
     KernelTiming timing(PRE ? kKernelBwdPrefixTc : kKernelBwdDkvTc, stream);
     tc_bwd_dkv_kernel<NP, PRE><<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_do, tm_k, tm_v, p);

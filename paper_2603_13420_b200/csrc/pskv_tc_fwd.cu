@@ -927,7 +927,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const float l = (mlt[0] + mlt[kTileM]) + (mlt[2 * kTileM] + mlt[3 * kTileM]);
             const bool row_ok = l >= kMinRowSum && l <= kMaxRowSum;  // false for overflow (inf, NaN), underflow
             // staged values must be finite (the buffer may double as suffix V, whose padding rows
-            // meet zero probabilities); rows that failed are redone anyway
+            // meet zero probabilities): rows that failed stage zeros, and are redone anyway
             const float inv = row_ok ? 1.f / l : 0.f;
             // the TMA stores of the previous tile must have read the staging buffer
             ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
@@ -957,6 +957,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * inv, __uint_as_float(o0[8 * c + 3]) * inv);
                     v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * inv, __uint_as_float(o0[8 * c + 5]) * inv);
                     v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * inv, __uint_as_float(o0[8 * c + 7]) * inv);
+                    if (!row_ok) v = make_uint4(0, 0, 0, 0);  // (inf or NaN accumulators times zero are not zero)
                     *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
                 }
 #pragma unroll
@@ -966,6 +967,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * inv, __uint_as_float(o1[8 * c + 3]) * inv);
                     v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * inv, __uint_as_float(o1[8 * c + 5]) * inv);
                     v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * inv, __uint_as_float(o1[8 * c + 7]) * inv);
+                    if (!row_ok) v = make_uint4(0, 0, 0, 0);
                     *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
                 }
             }
@@ -1243,12 +1245,8 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     auto kernel = plan.mode == 2 ? tc_fwd_kernel<D, 2, false>
                   : plan.mode == 1 ? (mi ? tc_fwd_kernel<D, 1, true> : tc_fwd_kernel<D, 1, false>)
                                    : (mi ? tc_fwd_kernel<D, 0, true> : tc_fwd_kernel<D, 0, false>);
-    static bool attr_set[6] = {false, false, false, false, false, false};
-    if (!attr_set[plan.mode + (mi ? 3 : 0)]) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr_set[plan.mode + (mi ? 3 : 0)] = true;
-    }
+    static PerDeviceOnce attr_set[6];
+    if (cudaError_t e = ensure_max_smem(kernel, attr_set[plan.mode + (mi ? 3 : 0)]); e != cudaSuccess) return e;
     const int grid = even_grid(p.total_tiles, sm_count());
     {
         KernelTiming timing(kKernelFwdTc, stream);

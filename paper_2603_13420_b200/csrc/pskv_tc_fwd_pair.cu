@@ -836,8 +836,8 @@ cudaError_t launch_tc_fwd_pair(const FwdArgs &a, unsigned int *status_word, cuda
     p.sk_bytes = plan.sk_bytes;
     p.sv_bytes = plan.sv_bytes;
 
-    cudaError_t e = cudaFuncSetAttribute(tc_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-    if (e != cudaSuccess) return e;
+    static PerDeviceOnce attr_set;
+    if (cudaError_t e = ensure_max_smem(tc_fwd_pair_kernel, attr_set); e != cudaSuccess) return e;
     const int pairs = even_grid(p.total_pt, sm_count() / 2);
     {
         KernelTiming timing(kKernelFwdTc, stream);

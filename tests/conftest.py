@@ -26,6 +26,18 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+@pytest.fixture(autouse=True)
+def _library_switches_back_to_default():
+    """Process-wide switches of the library a test may have flipped are put back after every test."""
+    yield
+    try:
+        import paper_2603_13420_b200 as pskv
+        pskv.pskv_set_multi_form("auto")
+        pskv.pskv_enable_cta_pairs(False)
+    except Exception:  # library not built: nothing to reset
+        pass
+
+
 @pytest.fixture(scope="session", autouse=True)
 def _built_libraries():
     """Compile the CUDA library and the C oracle once per session if their sources changed."""

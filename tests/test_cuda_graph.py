@@ -53,7 +53,7 @@ def test_forward_and_backward_replay_from_a_cuda_graph():
 @pytest.mark.gpu
 @pytest.mark.parametrize("form", ["passes", "one"])
 def test_multi_instruction_forward_replays_from_a_cuda_graph(form, monkeypatch):
-    monkeypatch.setenv("PSKV_MULTI_FORM", form)   # per-instruction passes on two streams / one launch
+    pskv.pskv_set_multi_form(form)   # per-instruction passes on two streams / one launch
     B, Bp, Hq, Hkv, S, Pmax, d = 32, 4, 8, 2, 16, 160, 128
     lens = (160, 120, 64, 33)
     gen = torch.Generator(device="cpu")

@@ -139,6 +139,28 @@ def test_rows_outside_the_safe_exponent_range_are_redone(kind):
     assert np.abs(ref_lse).max() > 100.0   # the case really is extreme
 
 
+def test_overflowing_rows_do_not_poison_the_next_tile_through_the_shared_staging_buffer():
+    """Head layout of the GQA layer with S = 40: the output staging buffer shares its memory with the
+    suffix V buffer, a CTA walks over five tiles, and every fifth tile holds ONE candidate (40 suffix keys
+    in a 48-row block, so rows 40..47 of the buffer keep what the previous tile staged there).  Rows
+    40..47 and 120..127 of the tile before it overflow (scores of several hundred nats): what they stage
+    must be finite, or the next tile's value contraction turns every one of its rows into NaN."""
+    w = Workload("alias", 4242, B=64, Hq=32, Hkv=8, d=128, P=256, S=40)
+    assert pskv.pskv_kernel_family(0, w.B, w.Hq, w.Hkv, w.S, w.P, w.d) == 1
+    t = make_inputs(w)
+    q = t["q"].float()
+    for g in (0, 5):                       # two KV heads; tile 3 of a head = rows 384..511 of its row list
+        q[2, 4 * g + 2, 24:32] *= 60.0     # tile rows 40..47  (candidate 2, third head of the group)
+        q[3, 4 * g + 0, 24:32] *= 60.0     # tile rows 120..127 (candidate 3, first head of the group)
+    t["q"] = q.to(torch.bfloat16)
+    out, lse, _ = parity.run_fwd_gpu(t, w.scale)   # (checks that nothing is NaN or unwritten)
+    cand = [1, 2, 3, 4]                    # the overflowing candidates and the one-candidate tile behind them
+    ref_out, ref_lse = parity.oracle_fwd(t, w.scale, cand)
+    parity.check_tensor("out", parity.to_f64(out[cand]), ref_out, max_abs=4e-2, mean_abs=4e-3)
+    parity.check_lse(parity.to_f64(lse[cand]), ref_lse)
+    assert np.abs(ref_lse).max() > 100.0
+
+
 # ---------------------------------------------------------------- properties that hold at any size
 
 def test_candidate_permutation_equivariance():

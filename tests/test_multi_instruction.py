@@ -50,7 +50,7 @@ ONE_LAUNCH_SHAPES = {0, 4, 5, 6, 7}
 
 @pytest.fixture(params=["one", "passes"])
 def form(request, monkeypatch):
-    monkeypatch.setenv("PSKV_MULTI_FORM", request.param)
+    pskv.pskv_set_multi_form(request.param)
     return request.param
 
 
@@ -98,7 +98,7 @@ def test_forward_and_backward_match_the_oracle(case, form):
 def test_one_launch_redoes_rows_outside_the_safe_exponent_range_with_their_own_prefix(monkeypatch):
     """Scores of several hundred nats in rows of different instructions: the one-launch forward marks them
     and recomputes each with a running maximum against its own instruction's unpadded prefix."""
-    monkeypatch.setenv("PSKV_MULTI_FORM", "one")
+    pskv.pskv_set_multi_form("one")
     case = (16, 4, 8, 2, 16, 300, 128, (300, 40, 170, 1))
     B, Bp, Hq, Hkv, S, Pmax, d, lens = case
     t = make(*case)
@@ -149,7 +149,7 @@ def test_multi_arguments_are_checked_on_the_host():
 
 @pytest.mark.gpu
 def test_the_library_takes_one_launch_by_itself_whenever_the_shape_allows_it(monkeypatch):
-    monkeypatch.delenv("PSKV_MULTI_FORM", raising=False)
+    pskv.pskv_set_multi_form("auto")
     for lens in ((256, 200), (256, 16)):
         case = (64, 2, 32, 8, 48, 256, 128, lens)
         t = make(*case)
@@ -169,7 +169,7 @@ def test_back_to_back_one_launch_calls_with_prefixes_that_are_padding_only(monke
     """Instructions whose prefix is empty skip every prefix block, yet the resident copy of their run is
     still loaded: those loads have to land before the CTA exits or arms the buffers again.  Many calls in a
     row without a synchronisation in between, each checked against the first."""
-    monkeypatch.setenv("PSKV_MULTI_FORM", "one")
+    pskv.pskv_set_multi_form("one")
     case = (64, 4, 32, 8, 48, 256, 128, (256, 0, 0, 130))
     B, Bp, Hq, Hkv, S, Pmax, d, lens = case
     t = make(*case)

@@ -91,7 +91,7 @@ def test_random_multi_instruction_shape_matches_the_oracle(case, monkeypatch):
     """Several instructions with random true prefix lengths (empty ones and whole padded key blocks included),
     in the one-launch form where the shape allows it and in per-instruction passes."""
     B, Bp, Hq, Hkv, S, Pmax, d, lens, form = case
-    monkeypatch.setenv("PSKV_MULTI_FORM", form)
+    pskv.pskv_set_multi_form(form)
     gen = torch.Generator(device="cpu")
     gen.manual_seed(B + 3 * Bp + 5 * S + 7 * Pmax + sum(lens))
     draw = lambda *s: torch.randn(s, generator=gen, dtype=torch.float32).to(torch.bfloat16)
