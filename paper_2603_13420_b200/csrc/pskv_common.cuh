@@ -65,7 +65,10 @@ cudaError_t launch_tc_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __n
                                  unsigned int *status_word, cudaStream_t stream);
 cudaError_t launch_simt_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __nv_bfloat16 *dv_prefix,
                                    cudaStream_t stream);
-cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream);
+// with_d: the kernel also forms D = <dout, out> - dlse per row and writes it to a.row_dot (it then needs
+// a.out and no pre-pass); tc_bwd_dkv_row_dot_supported tells whether the shape allows that.
+bool tc_bwd_dkv_row_dot_supported(const Dims &d);
+cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream, bool with_d = false);
 
 // tcgen05/TMEM kernels.  `status_word` is the device status flag that bounded waits set.
 bool tc_fwd_supported(const Dims &d);
@@ -86,7 +89,9 @@ bool tc_bwd_supported(const Dims &d);
 size_t tc_bwd_workspace_bytes(const Dims &d);
 // `parts` selects which of the three steps run (all by default): the row statistic D and the suffix
 // gradients do not involve the prefix, so a caller with several prefixes runs them once over all
-// candidates and the dQ step once per prefix.
+// candidates and the dQ step once per prefix.  Where one kernel produces both the row statistic and the
+// suffix gradients (tc_bwd_dkv_row_dot_supported) it runs for kBwdPartRowDot and kBwdPartDkv is empty;
+// a caller that splits the parts must ask for kBwdPartRowDot before kBwdPartDq either way.
 enum { kBwdPartRowDot = 1, kBwdPartDq = 2, kBwdPartDkv = 4, kBwdPartAll = 7 };
 bool tc_bwd_fused_supported(const Dims &d, int n_instr);  // several instructions in one dQ launch (as for the forward)
 cudaError_t launch_tc_bwd(const BwdArgs &a, void *workspace, unsigned int *status_word,

@@ -854,10 +854,14 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
                                        : (mi ? tc_bwd_dq_kernel<D, 0, true> : tc_bwd_dq_kernel<D, 0, false>);
     static PerDeviceOnce attr_set[8];
     if (cudaError_t e0 = ensure_max_smem(kernel, attr_set[plan.resident + (mi ? 4 : 0)]); e0 != cudaSuccess) return e0;
-    // D = <dout, out> per row, then dQ on the tensor cores, then dK_suffix / dV_suffix
+    // The suffix-gradient kernel streams every dO row anyway, so where the shape allows it forms the row
+    // statistic D = <dout, out> itself and runs FIRST (it then stands for both the "row statistic" and the
+    // "suffix gradients" part); the query-side kernel behind it reads D.  Otherwise: a streaming pre-pass
+    // for D, then dQ, then dK_suffix / dV_suffix.
+    const bool d_in_dkv = tc_bwd_dkv_row_dot_supported(dm);
     cudaError_t e = cudaSuccess;
     if (parts & kBwdPartRowDot) {
-        e = launch_simt_row_dot(a, stream);
+        e = d_in_dkv ? launch_tc_bwd_dkv(a, status_word, stream, true) : launch_simt_row_dot(a, stream);
         if (e != cudaSuccess) return e;
     }
     if (parts & kBwdPartDq) {
@@ -872,6 +876,7 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
         if (e != cudaSuccess) return e;
     }
     if (!(parts & kBwdPartDkv)) return cudaSuccess;
+    if (d_in_dkv) return cudaSuccess;  // done together with the row statistic (also for callers that ask part by part)
     if (tc_bwd_dkv_supported(dm)) return launch_tc_bwd_dkv(a, status_word, stream);
     return mma_bwd_dkv_supported(dm) ? launch_mma_bwd_dkv(a, stream) : launch_simt_bwd_dkv(a, stream);
 }

@@ -24,6 +24,13 @@
 // The arithmetic is tiny next to the bytes moved (Q and dO are read once, nothing else is big):
 // the kernel is bound by HBM, and everything is arranged to keep two tiles of copies in flight.
 //
+// Because it streams every dO row anyway and has issue slots to spare, the kernel (instantiated with
+// DROW = true) also forms the row statistic of the backward pass, D = <dO, O> (minus the gradient
+// arriving on lse, if any), instead of a pre-pass that would read dO a second time: the element-wise
+// warps read the O rows of the tile straight from global memory (32 of the 128 columns per warpgroup),
+// meet the dO tile in shared memory, exchange their four partial sums through shared memory and write
+// D for the query-side kernel, which runs behind this one.
+//
 // The same kernel, instantiated with PRE = true, produces the gradients of the shared PREFIX cache
 // (which the search keeps frozen, Sec. 4.2, but a caller may want: full differentiability).  A unit
 // of work is then (KV head, block of 64 prefix keys, chunk of candidates): the block's K/V rows are
@@ -68,12 +75,16 @@ enum {
     kBarPFree = 13,      // the MMAs that read them completed
     kBarAccFull = 14,    // [2] the accumulators of a group are final
     kBarAccFree = 16,    // [2] the write-back has read them out (one arrival per element-wise warp)
-    kNumBars = 18
+    kBarDFull = 18,      // [2] DROW: the four partial sums of D of a tile are in shared memory (16 arrivals)
+    kNumBars = 20
 };
 
 struct TcDkvParams {
     const float *lse;      // [B*Hq*S]
-    const float *row_dot;  // [B*Hq*S]
+    const float *row_dot;  // [B*Hq*S] D per row (read; DROW: written here by this kernel, never read)
+    float *row_dot_out;    // DROW: where D goes for the query-side kernel
+    const __nv_bfloat16 *out;  // DROW: [B,Hq,S,128] forward output
+    const float *dlse;     // DROW: gradient arriving on lse, or nullptr
     __nv_bfloat16 *dk;     // [B,Hkv,S,128]
     __nv_bfloat16 *dv;
     unsigned int *status;
@@ -87,7 +98,7 @@ struct TcDkvParams {
     int P, nkb, nbc, cpc;  // prefix length, key blocks of 64, candidate chunks, candidates per chunk
     FastDiv fd_S, fd_Hkv;
     // shared-memory byte offsets from the 1024-byte aligned base
-    int off_q, off_do, off_k, off_v, off_p, off_ds, off_bar, off_misc, kv_bytes;
+    int off_q, off_do, off_k, off_v, off_p, off_ds, off_bar, off_misc, off_dpart, kv_bytes;
 };
 
 // unit u of a CTA -> (index of the group within this CTA, tile within the group)
@@ -126,12 +137,13 @@ __device__ __forceinline__ Unit unit_of(const TcDkvParams &p, int u)
     return x;
 }
 
-// NP = TP / 16: 16-key pieces per row.  PRE: prefix-gradient mode (NP = 4).
-template <int NP, bool PRE>
+// NP = TP / 16: 16-key pieces per row.  PRE: prefix-gradient mode (NP = 4).  DROW: form D = <dO, O>
+// here and write it out (never together with PRE).
+template <int NP, bool PRE, bool DROW = false>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                   const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                  const TcDkvParams p)
+                  const __grid_constant__ CUtensorMap tm_o, const TcDkvParams p)
 {
     constexpr int TP = NP * 16;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -153,7 +165,8 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0) {
 #pragma unroll 1
         for (int i = 0; i < kNumBars; ++i) {
-            const bool elem = i == kBarSFree || i == kBarSFree + 1 || i == kBarPReady || i == kBarAccFree || i == kBarAccFree + 1;
+            const bool elem = i == kBarSFree || i == kBarSFree + 1 || i == kBarPReady || i == kBarAccFree ||
+                              i == kBarAccFree + 1 || i == kBarDFull || i == kBarDFull + 1;
             mbar_init(bar(i), elem ? (uint32_t)(4 * kElemGroups) : 1u);
         }
         *abort_flag = 0;
@@ -222,6 +235,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int sl = 0; sl < 2; ++sl) {
                         tma_prefetch_4d(&tm_q, sl * 64, y.tt * kTileM, y.g, y.b);
                         tma_prefetch_4d(&tm_do, sl * 64, y.tt * kTileM, y.g, y.b);
+                        if (DROW) tma_prefetch_4d(&tm_o, sl * 64, y.tt * kTileM, y.g, y.b);  // read by the element-wise warps
                         if (y.first && !PRE) {
                             tma_prefetch_4d(&tm_k, sl * 64, 0, y.g, y.b);
                             tma_prefetch_4d(&tm_v, sl * 64, 0, y.g, y.b);
@@ -335,6 +349,17 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         uint8_t *ds_row = smem + p.off_ds + row * 128;
         bool ok = true;
         int pending_gi = -1;  // group whose accumulators are still to be written back
+        float *dpart = reinterpret_cast<float *>(smem + p.off_dpart);  // DROW: [stage][warpgroup][row]
+        uint4 o_next[4] = {};                                            // DROW: this thread's O slice of the coming unit
+        if (DROW && total_units > 0) {
+            const Unit y = unit_of<PRE>(p, 0);
+            if (row < p.Rg) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(
+                    p.out + (((size_t)y.b * p.Hq + (size_t)y.g * p.n_rep) * p.S + row) * kD + 32 * wg);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) o_next[j] = __ldg(src + j);
+            }
+        }
         // write-back of group gi: lane <-> column d, tensor-memory column <-> key
         auto write_back = [&](int gi) -> bool {
             const int as = gi & 1;
@@ -397,9 +422,55 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             // causal: suffix key t is visible when t <= i; prefix mode: every key of the block that exists
             const int i_pos = !valid ? -1 : PRE ? min(64, p.P - x.kb * 64) - 1 : gr - p.fd_S.div(gr) * p.S;
             const float nl2 = valid ? -p.lse[row0 + gr] * kLog2e : 0.f;
-            const float dr = valid ? p.row_dot[row0 + gr] : 0.f;
+            float dr = (!DROW && valid) ? p.row_dot[row0 + gr] : 0.f;
+            if (DROW) {
+                // my 32 of the row's 128 columns: O from global memory (requested one unit ahead), dO from the
+                // tile in shared memory (64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row)
+                float part = 0.f;
+                ok = mbar_wait_warp(bar(kBarQFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
+                if (!ok) break;
+                if (valid) {
+                    const uint8_t *dorow = smem + p.off_do + st * kTileBytes + (wg >> 1) * kSlabBytes + row * 128;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 dv = *reinterpret_cast<const uint4 *>(dorow + ((((wg & 1) * 4 + j) ^ (row & 7)) << 4));
+                        const __nv_bfloat162 *a = reinterpret_cast<const __nv_bfloat162 *>(&dv);
+                        const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&o_next[j]);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 fa = __bfloat1622float2(a[e]), fb = __bfloat1622float2(b[e]);
+                            part = fmaf(fa.x, fb.x, part);
+                            part = fmaf(fa.y, fb.y, part);
+                        }
+                    }
+                }
+                dpart[(st * 4 + wg) * kTileM + row] = part;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarDFull + st));
+                // the O slice of the next unit's row, in flight while this unit is worked on
+                if (u + 1 < total_units) {
+                    const Unit y = unit_of<PRE>(p, u + 1);
+                    const int gy = y.tt * kTileM + row;
+                    if (gy < p.Rg) {
+                        const uint4 *src = reinterpret_cast<const uint4 *>(
+                            p.out + (((size_t)y.b * p.Hq + (size_t)y.g * p.n_rep) * p.S + gy) * kD + 32 * wg);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) o_next[j] = __ldg(src + j);
+                    }
+                }
+            }
             ok = mbar_wait_warp(bar(kBarSFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
             if (!ok) break;
+            if (DROW) {
+                ok = mbar_wait_warp(bar(kBarDFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
+                if (!ok) break;
+                const float *dp = dpart + st * 4 * kTileM + row;  // the four warpgroups' partial sums, in fixed order
+                dr = (dp[0] + dp[kTileM]) + (dp[2 * kTileM] + dp[3 * kTileM]);
+                if (valid) {
+                    if (p.dlse) dr -= p.dlse[row0 + gr];
+                    if (wg == 0) p.row_dot_out[row0 + gr] = dr;
+                }
+            }
             PSKV_TRACE_EVENT(20, u);
             tc_fence_after();
             // group wg takes the 16-key piece wg of the tile (groups past the last piece only join the barriers)
@@ -464,15 +535,16 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
 // ------------------------------------------------------------------------------ host side
 
-template <int NP, bool PRE>
+template <int NP, bool PRE, bool DROW = false>
 cudaError_t launch_np(const BwdArgs &a, const CUtensorMap &tm_q, const CUtensorMap &tm_do, const CUtensorMap &tm_k,
-                      const CUtensorMap &tm_v, const TcDkvParams &p, int smem_bytes, cudaStream_t stream)
+                      const CUtensorMap &tm_v, const CUtensorMap &tm_o, const TcDkvParams &p, int smem_bytes,
+                      cudaStream_t stream)
 {
     static PerDeviceOnce attr_set;
-    if (cudaError_t e = ensure_max_smem(tc_bwd_dkv_kernel<NP, PRE>, attr_set); e != cudaSuccess) return e;
+    if (cudaError_t e = ensure_max_smem(tc_bwd_dkv_kernel<NP, PRE, DROW>, attr_set); e != cudaSuccess) return e;
     const int grid = p.total_groups < sm_count() ? p.total_groups : sm_count();
     KernelTiming timing(PRE ? kKernelBwdPrefixTc : kKernelBwdDkvTc, stream);
-    tc_bwd_dkv_kernel<NP, PRE><<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_do, tm_k, tm_v, p);
+    tc_bwd_dkv_kernel<NP, PRE, DROW><<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_do, tm_k, tm_v, tm_o, p);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -515,11 +587,30 @@ bool tc_bwd_dkv_supported(const Dims &dm)
            (long long)dm.n_rep * dm.S < 2000000000ll && get_encode_fn() != nullptr;
 }
 
-cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream)
+// Shared-memory bytes of the suffix-gradient launch; with_d adds the partial sums of D.
+static int dkv_smem_bytes(int TP, bool with_d)
+{
+    const int kv_bytes = round_up(2 * TP * 128, 1024);
+    return 4 * kTileBytes + 4 * kv_bytes + 2 * kSlabBytes + 256 + 64 + (with_d ? 2 * 4 * kTileM * 4 : 0);
+}
+
+// The kernel can form D for any shape it takes whose shared memory has room for the partial sums; it is
+// asked to only where a (candidate, KV head) group fills whole 128-row tiles.  With small groups (one
+// query head per KV head and a short suffix: 40 rows of 128) the kernel runs at a little over half of
+// the HBM bandwidth, and reading O there costs more than the streaming pre-pass that reads dO twice
+// (measured at B = 128, 32 heads, S = 40: 151 against 137 us for the whole backward).
+bool tc_bwd_dkv_row_dot_supported(const Dims &dm)
+{
+    return tc_bwd_dkv_supported(dm) && dm.n_rep * dm.S >= kTileM &&
+           dkv_smem_bytes((dm.S + 15) / 16 * 16, true) <= kMaxSmem;
+}
+
+cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaStream_t stream, bool with_d)
 {
     const Dims &dm = a.dims;
     const int Rg = dm.n_rep * dm.S;
     const int TP = (dm.S + 15) / 16 * 16;
+    if (with_d && !tc_bwd_dkv_row_dot_supported(dm)) return cudaErrorInvalidValue;
 
     TcDkvParams p;
     memset(&p, 0, sizeof(p));
@@ -545,10 +636,14 @@ cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaS
     p.off_ds = p.off_p + kSlabBytes;
     p.off_bar = p.off_ds + kSlabBytes;
     p.off_misc = p.off_bar + 256;
-    const int smem_bytes = p.off_misc + 64;
+    p.off_dpart = p.off_misc + 64;
+    const int smem_bytes = dkv_smem_bytes(TP, with_d);
     if (smem_bytes > kMaxSmem) return cudaErrorInvalidConfiguration;
+    p.row_dot_out = a.row_dot;
+    p.out = a.out;
+    p.dlse = a.dlse;
 
-    CUtensorMap tm_q, tm_do, tm_k, tm_v;
+    CUtensorMap tm_q, tm_do, tm_k, tm_v, tm_o;
     {
         // q / dout viewed as [B][Hkv][Rg][D]: the n_rep heads of a KV head are contiguous rows
         cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)Rg, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
@@ -556,6 +651,7 @@ cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaS
         cuuint32_t box[4] = {64, (cuuint32_t)(Rg < kTileM ? Rg : kTileM), 1, 1};
         if (!encode_map(&tm_q, a.q, 4, dims, str, box)) return cudaErrorInvalidValue;
         if (!encode_map(&tm_do, a.dout, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!encode_map(&tm_o, with_d ? a.out : a.dout, 4, dims, str, box)) return cudaErrorInvalidValue;  // (L2 prefetch only)
     }
     {
         cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)dm.S, (cuuint64_t)dm.Hkv, (cuuint64_t)dm.B};
@@ -564,11 +660,19 @@ cudaError_t launch_tc_bwd_dkv(const BwdArgs &a, unsigned int *status_word, cudaS
         if (!encode_map(&tm_k, a.suffix_k, 4, dims, str, box)) return cudaErrorInvalidValue;
         if (!encode_map(&tm_v, a.suffix_v, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
+    if (with_d) {
+        switch (TP / 16) {
+        case 1: return launch_np<1, false, true>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+        case 2: return launch_np<2, false, true>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+        case 3: return launch_np<3, false, true>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+        default: return launch_np<4, false, true>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+        }
+    }
     switch (TP / 16) {
-    case 1: return launch_np<1, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
-    case 2: return launch_np<2, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
-    case 3: return launch_np<3, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
-    default: return launch_np<4, false>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    case 1: return launch_np<1, false>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+    case 2: return launch_np<2, false>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+    case 3: return launch_np<3, false>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
+    default: return launch_np<4, false>(a, tm_q, tm_do, tm_k, tm_v, tm_o, p, smem_bytes, stream);
     }
 }
 
@@ -639,7 +743,7 @@ cudaError_t launch_tc_bwd_prefix(const BwdArgs &a, __nv_bfloat16 *dk_prefix, __n
     }
     cudaError_t e = cudaMemsetAsync(acc32, 0, 2 * n_acc * sizeof(float), stream);
     if (e != cudaSuccess) return e;
-    e = launch_np<4, true>(a, tm_q, tm_do, tm_k, tm_v, p, smem_bytes, stream);
+    e = launch_np<4, true>(a, tm_q, tm_do, tm_k, tm_v, tm_do, p, smem_bytes, stream);
     if (e != cudaSuccess) return e;
     const int blocks = (int)((n_acc + 255) / 256 < 1184 ? (n_acc + 255) / 256 : 1184);
     prefix_grad_round_kernel<<<blocks, 256, 0, stream>>>(p.dkp32, p.dvp32, dk_prefix, dv_prefix, n_acc);

@@ -145,7 +145,8 @@ def kernel_work(w: Workload) -> dict:
     return {
         "tc_fwd_kernel": {"flops": fwd_flops(w), "bytes": fwd_bytes(w)},
         "tc_bwd_dq_kernel": {"flops": rows * 6.0 * w.d * (w.P + vis), "bytes": float(3 * q + 8 * rows + skv + pkv)},
-        "tc_bwd_dkv_kernel": {"flops": rows * 4.0 * w.d * vis, "bytes": float(2 * q + 8 * rows + 2 * skv)},
+        # (reads q, dout and out -- it also forms D = <dout, out> --, lse and the suffix K/V; writes D and the gradients)
+        "tc_bwd_dkv_kernel": {"flops": rows * (4.0 * w.d * vis + 2.0 * w.d), "bytes": float(3 * q + 8 * rows + 2 * skv)},
         "bwd_dkv_mma_kernel": {"flops": rows * 4.0 * w.d * vis, "bytes": float(2 * q + 8 * rows + 2 * skv)},
         "simt_row_dot_kernel": {"flops": rows * 2.0 * w.d, "bytes": float(2 * q + 4 * rows)},
     }

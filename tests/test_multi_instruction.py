@@ -83,8 +83,9 @@ def test_forward_and_backward_match_the_oracle(case, form):
     pskv.pskv_attn_bwd_multi(dev["dout"], dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
                              dev["suffix_v"], out.view, lse.view, scale, dq=dq.view, dk_suffix=dk.view,
                              dv_suffix=dv.view)
-    if one:   # row statistic, one dQ launch for all instructions, suffix gradients
-        assert pskv.pskv_kernel_launches() - n0 == 3
+    if one:   # suffix gradients together with the row statistic (a pre-pass of its own for suffixes beyond 48
+        # keys), then one dQ launch for all instructions
+        assert pskv.pskv_kernel_launches() - n0 == (2 if S <= 48 and (Hq // Hkv) * S >= 128 else 3)
     assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
     dq.check("dq"); dk.check("dk_suffix"); dv.check("dv_suffix")
     rq, rk, rv = oracle.attn_bwd_multi(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], mask, f["suffix_k"],
@@ -161,7 +162,7 @@ def test_the_library_takes_one_launch_by_itself_whenever_the_shape_allows_it(mon
         n0 = pskv.pskv_kernel_launches()
         pskv.pskv_attn_bwd_multi(dev["dout"], dev["q"], dev["prefix_k"], dev["prefix_v"], lens, dev["suffix_k"],
                                  dev["suffix_v"], out, lse, 0.088)
-        assert pskv.pskv_kernel_launches() - n0 == 3   # row statistic, dQ, suffix gradients
+        assert pskv.pskv_kernel_launches() - n0 == 2   # suffix gradients with the row statistic, then dQ
 
 
 @pytest.mark.gpu
