@@ -51,6 +51,28 @@ def test_backward_full_size_sampled():
     parity.bwd_parity(w, cand=cand)
 
 
+def test_benchmark_step_full_size_sampled():
+    """The exact launches the benchmark's headline times: forward and backward of the GQA layer at
+    B = 512, sampled candidates against the oracle."""
+    w = wl("C2", backward=True)
+    rng = np.random.default_rng(w.seed + 7)
+    cand = sorted(set([0, 1, w.B - 1] + rng.integers(0, w.B, size=4).tolist()))
+    t = make_inputs(w, with_dout=True)
+    parity.fwd_parity(w, t=t, cand=cand)
+    parity.bwd_parity(w, t=t, cand=cand)
+
+
+@pytest.mark.parametrize("name,B", [("C3", 64), ("C2", 64)])
+def test_backward_many_tiles_per_cta_sampled(name, B):
+    """Backward with several tiles per persistent CTA, so that the prefix K/V rings of the query-side kernel
+    wrap across tiles: the long-prefix shape (K and V streaming, 512 tiles for 148 CTAs) and the GQA layer
+    shape (K resident, V streaming, 768 tiles).  Sampled candidates against the oracle."""
+    w = wl(name, B=B, backward=True)
+    rng = np.random.default_rng(w.seed + 11)
+    cand = sorted(set([0, B // 2, B - 1] + rng.integers(0, B, size=2).tolist()))
+    parity.bwd_parity(w, cand=cand)
+
+
 # ---------------------------------------------------------------- edge cases and odd shapes
 
 EDGE = [
