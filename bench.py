@@ -281,6 +281,7 @@ def run_cuda(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     import paper_2603_13420_b200 as pskv
+    pskv.pskv_enable_cta_pairs(args.cta_pairs)
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if world > 1:
@@ -517,10 +518,9 @@ def roofline(w, kernels, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (kernel, workload) -> bytes.
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("tc_fwd_kernel", "C2"): 473.7e6,        # profiles/tc_fwd_kernel_C2.md
-    ("tc_bwd_dq_kernel", "C2"): 690.6e6,     # profiles/tc_bwd_dq_kernel_C2.md
-    ("tc_bwd_dkv_kernel", "C2"): 594.8e6,    # profiles/tc_bwd_dkv_kernel_C2.md
-    ("simt_row_dot_kernel", "C2"): 410.1e6,  # profiles/simt_row_dot_kernel_C2.md
+    ("tc_fwd_kernel", "C2"): 473.9e6,        # profiles/tc_fwd_kernel_C2.md
+    ("tc_bwd_dq_kernel", "C2"): 691.8e6,     # profiles/tc_bwd_dq_kernel_C2.md
+    ("tc_bwd_dkv_kernel", "C2"): 816.6e6,    # profiles/tc_bwd_dkv_kernel_C2.md (with the row statistic D)
 }
 
 
@@ -813,6 +813,8 @@ def main():
                     help="candidates of the one-off CPU oracle sample reported as cpu_baseline")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-workload kernel timings")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--cta-pairs", action="store_true",
+                    help="use the opt-in CTA-pair forward kernel (pskv_enable_cta_pairs) instead of the default one")
     ap.add_argument("--no-e2e", action="store_true",
                     help="skip the end-to-end leg (profiling captures that should hold full-size steps only)")
     ap.add_argument("--sustained-s", type=float, default=2.0,
