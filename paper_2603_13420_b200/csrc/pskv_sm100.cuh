@@ -415,12 +415,31 @@ __device__ __forceinline__ bool mbar_try_wait_cl(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait of the pair kernels; all 32 lanes wait, true only if every lane saw the phase.
+// Bounded wait of the pair kernels; all 32 lanes wait, true only if every lane saw the phase.  The polling
+// loop is in line here (no call to the shared out-of-line routine): measured on the pair forward kernel that
+// is 5 % faster (145 against 152 us on the GQA layer shape), while the same change made the single-CTA
+// forward kernel 3 % slower, so those keep the call.  A failed try_wait has already suspended the thread
+// for a short time, so the loop counts polls and reads the abort flag and the clock only every 256th.
 __device__ __forceinline__ bool mbar_wait_warp_cl(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                                   unsigned int *status_word, unsigned int code)
 {
     bool ok = mbar_try_wait_cl(bar, parity);
-    if (!ok) ok = mbar_wait_slow(bar, parity, abort_flag, status_word, code);
+    if (!ok) {
+        long long start = 0;
+#pragma unroll 1
+        for (unsigned int spin = 1; !(ok = mbar_try_wait_cl(bar, parity)); ++spin) {
+            if ((spin & 255u) == 0u) {
+                if (*abort_flag != 0) break;
+                const long long now = clock64();
+                if (start == 0) start = now;
+                if (now - start > kWaitBudgetCycles) {
+                    *abort_flag = 1;
+                    atomicCAS(status_word, 0u, code);
+                    break;
+                }
+            }
+        }
+    }
     return __all_sync(0xffffffffu, ok);
 }
 

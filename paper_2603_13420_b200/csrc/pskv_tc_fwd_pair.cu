@@ -17,7 +17,8 @@
 //   warp 2      rank 0: issues O += P V for the pair; rank 1: the same relay for the value side
 //               (owns the tensor-memory allocation in both CTAs)
 //   warp 3      TMA producer, value side: own 64 columns of the prefix V blocks and of the suffix values
-//   warps 4-19  softmax: four warpgroups, each one 32-column piece of every item (thread <-> query row)
+//   warps 4-19  softmax: two groups of eight warps take the items in turn (thread <-> query row, the
+//               group's warps split the tile by row quadrant and column half)
 //   warps 20-23 epilogue: O / row sum -> bf16 -> staging -> TMA store; lse
 // Every copy is a plain single-CTA TMA load into the CTA's own shared memory.  The CTAs meet only at
 // mbarriers: commits signal the same barrier in both CTAs, rank 1's warps arrive remotely on rank 0's
@@ -36,14 +37,19 @@ using namespace sm100;
 
 constexpr int kD = 128;
 constexpr int kSlots = 2;      // score slots (128 fp32 columns) and probability slots (64 columns of bf16 pairs)
-constexpr int kSoftmaxWarpgroups = 4;  // one 32-column piece of every item each
-constexpr int kParts = 4;      // partial row sums per row and tile: one per piece
-constexpr int kThreads = 32 * (4 + 4 * kSoftmaxWarpgroups + 4);
+constexpr int kPiece = 32;     // score columns a softmax thread handles at a time
+constexpr int kGroups = 2;     // softmax groups: they take the items in turn (group = the item's slot)
+constexpr int kColSplit = 2;   // warps per row quadrant in a group: each owns 128 / kColSplit score columns
+constexpr int kWarpCols = kBlockN / kColSplit;        // score columns of a softmax warp
+constexpr int kSub = 16;                              // columns per tensor-memory load of a softmax thread
+static_assert(kWarpCols % (2 * kSub) == 0, "pieces come in pairs");
+constexpr int kParts = kGroups * kColSplit;            // partial row sums per row and tile
+constexpr int kSoftmaxWarps = 4 * kGroups * kColSplit;
+constexpr int kThreads = 32 * (4 + kSoftmaxWarps + 4);
 constexpr int kPCol = kSlots * kBlockN;            // first tensor-memory column of the probability slots
 constexpr int kPSlotCols = kBlockN / 2;
 constexpr int kOCol = kPCol + kSlots * kPSlotCols;  // first tensor-memory column of O
 static_assert(kOCol + kD <= 512, "tensor memory");
-constexpr int kPiece = 32;
 constexpr float kMaxRowSum = 1.2676506002282294e30f;   // 2^100
 constexpr float kMinRowSum = 7.8886090522101181e-31f;  // 2^-100
 constexpr int kMaxBlocks = 4;            // resident prefix blocks
@@ -157,7 +163,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const bool both_land = (i >= kBarQFull && i < kBarQFull + 2) || (i >= kBarSKFull && i < kBarSKFull + 2) ||
                                    (i >= kBarSVFull && i < kBarSVFull + 2) || i >= kBarKFull;
             if (both_land) count = rank == 0 ? 2u : 1u;  // own copies + the other CTA's "landed" arrival
-            if (i >= kBarSFree && i < kBarPReady + kSlots) count = 32u;  // the sixteen softmax warps of both CTAs
+            if (i >= kBarSFree && i < kBarPReady + kSlots) count = 2u * 4u * kColSplit;  // the warps of the item's softmax group, both CTAs
             if (i == kBarOFree) count = 8u;                                             // epilogue warps of both CTAs
             if (i == kBarStageFull) count = 4u;
             mbar_init(bar(i), count);
@@ -457,113 +463,170 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             __syncwarp();
         }
     }
-    } else if (warp < 4 + 4 * kSoftmaxWarpgroups) {
-        // ------------------------------------------------------------------ softmax warps (4..19)
-        // Sixteen warps, four per tensor-memory quadrant (= per scheduler); every warp works on every
-        // item and takes one 32-column piece of its quadrant's rows (thread <-> query row).  Scores
-        // and probabilities have separate slots in tensor memory, two of each: a warp pulls its
-        // piece of the scores into registers and hands the score slot back AT ONCE, so the score
-        // MMAs run two items ahead of the softmax and this stage never waits for scores; the
-        // bf16 probabilities go to the item's probability slot, which only that item's value MMAs
-        // hold.  What is left in the stage's critical loop is the exponentials themselves (the
-        // special-function unit, 16 per clock and SM, is the resource this stage is bound by).
-        // p = 2^(s * sl2) with no running max (rows whose sum leaves [2^-100, 2^100] are redone at the
-        // end); partial row sums go to the epilogue through shared memory.  Both arrivals go to
-        // rank 0, whose threads issue the MMAs.
-        const int piece = (warp - 4) >> 2;
-        const int c0 = piece * kPiece;  // first column of my piece
+    } else if (warp < 4 + kSoftmaxWarps) {
+        // ------------------------------------------------------------------ softmax warps
+        // Two groups take the items in turn (group = item mod 2 = the item's score and probability
+        // slot), so that one group's loads, waits and stores fall under the other one's exponentials.
+        // In a group the warps split the tile by row quadrant (tensor memory gives a warp the 32
+        // lanes of its quadrant) and by column half; a thread owns one query row and walks its 64
+        // columns in 16-column pieces, the load of the next piece in flight while it works on
+        // the current one (a tensor-memory load takes 400 to 600 cycles while the MMAs run).  The
+        // piece loop is unrolled by two only: with a whole row unrolled the loop body no longer
+        // fits the instruction cache (2.4 warps per issue slot stalled for instructions,
+        // against 0.5 in this form) and every piece took twice as long.  The score slot goes back
+        // to the MMA issuer as soon as the last piece is in registers, the probabilities go to a
+        // slot of their own that only the item's value MMAs hold; the first load of the group's
+        // next item is issued before this item's bookkeeping.  p = 2^(s * sl2) with no running
+        // max (rows whose sum leaves [2^-100, 2^100] are redone at the end); partial row sums go to
+        // the epilogue through shared memory.  Both arrivals go to rank 0, whose threads issue
+        // the MMAs.
+        const int sw = warp - 4;
+        const int wg = sw / (4 * kColSplit);
+        const int half = (sw >> 2) % kColSplit;
+        const int part = wg * kColSplit + half;
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+        const uint32_t s_tmem = lane_base + wg * kBlockN + half * kWarpCols;
+        const uint32_t p_tmem = lane_base + kPCol + wg * kPSlotCols + half * (kWarpCols / 2);
+        const int col0 = half * kWarpCols;  // first score column of this warp
         bool ok = !misaligned;
-        int item = 0;
-#pragma unroll 1
-        for (int tl = 0; tl < n_tiles && ok; ++tl) {
-            const PairTile t = pair_tile(p, pt_begin + tl, pt_begin, rank);
-            const int R = t.R0 + row;
-            const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
-            const int lo_sfx = (b - t.b_first) * p.S;              // first suffix column of this row's candidate
-            const int hi_sfx = lo_sfx + (r - p.fd_S.div(r) * p.S); // causal: suffix keys 0..i
-            float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
-#pragma unroll 1
-            for (int k = 0; k < nitems && ok; ++k, ++item) {
-                const int slot = item & 1;
-                const uint32_t par = (uint32_t)(item >> 1) & 1u;
-                const bool prefix = k < p.nblk_p;
-                const int n = prefix ? block_keys(p, k) : p.n_sfx;
-                const int lo = prefix ? 0 : lo_sfx;
-                const int hi = prefix ? min(kBlockN, p.P - k * kBlockN) - 1 : hi_sfx;
-                // my piece: 0 = beyond the item's keys (never read by the value MMAs), 1 = no valid column
-                // for this warp (zeros), 2 = some masked, 3 = all valid (a prefix block is the same for
-                // every row, so it needs no vote)
-                int kind;
-                if (c0 >= n) {
-                    kind = 0;
-                } else if (prefix) {
-                    kind = hi >= c0 + kPiece - 1 ? 3 : hi < c0 ? 1 : 2;
-                } else {
-                    const bool all_valid = lo <= c0 && hi >= c0 + kPiece - 1;
-                    const bool none_valid = hi < lo || hi < c0 || lo > c0 + kPiece - 1;
-                    kind = __all_sync(0xffffffffu, all_valid) ? 3 : __all_sync(0xffffffffu, none_valid) ? 1 : 2;
+        int tl = 0, k = wg;  // item = tl * nitems + k
+        while (k >= nitems) { k -= nitems; ++tl; }
+        int tl_row = -1, lo_sfx = 0, hi_sfx = 0;
+        int n = 0, lo = 0, hi = -1;  // the current item: keys, and this row's valid columns [lo, hi]
+        float lsum = 0.f;
+        // 0 = beyond the item's keys (never read by the value MMAs), 1 = no valid column for this warp
+        // (zeros), 2 = some masked, 3 = all valid
+        auto piece_kind = [&](int c0) -> int {
+            if (c0 >= n) return 0;
+            const bool all_valid = lo <= c0 && hi >= c0 + kSub - 1;
+            const bool none_valid = hi < lo || hi < c0 || lo > c0 + kSub - 1;
+            return __all_sync(0xffffffffu, all_valid) ? 3 : __all_sync(0xffffffffu, none_valid) ? 1 : 2;
+        };
+        // this row's limits for item (tl, k); a new tile resets the row sum
+        auto begin_item = [&]() {
+            if (tl != tl_row) {
+                const PairTile t = pair_tile(p, pt_begin + tl, pt_begin, rank);
+                const int R = t.R0 + row;
+                const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
+                lo_sfx = (b - t.b_first) * p.S;              // first suffix column of this row's candidate
+                hi_sfx = lo_sfx + (r - p.fd_S.div(r) * p.S); // causal: suffix keys 0..i
+                lsum = 0.f;
+                tl_row = tl;
+            }
+            const bool prefix = k < p.nblk_p;
+            n = prefix ? block_keys(p, k) : p.n_sfx;
+            lo = prefix ? 0 : lo_sfx;
+            hi = prefix ? min(kBlockN, p.P - k * kBlockN) - 1 : hi_sfx;
+        };
+        float ls0 = 0.f, ls1 = 0.f;
+        // one 16-column piece: exponentials, row sum, bf16 pairs to the probability slot
+        auto piece = [&](const uint32_t (&rr)[kSub], int kind, int c0) {
+            uint32_t pk[kSub / 2];
+            if (kind == 3) {
+#pragma unroll
+                for (int j = 0; j < kSub; j += 2) {
+                    float x0 = __uint_as_float(rr[j]), x1 = __uint_as_float(rr[j + 1]);
+                    mul_f32x2(x0, x1, p.sl2);
+                    x0 = ex2_approx(x0);
+                    x1 = ex2_approx(x1);
+                    add_f32x2(ls0, ls1, x0, x1);
+                    pk[j >> 1] = pack_bf16x2(x0, x1);
                 }
-                PSKV_TRACE_EVENT(25, item);
-                ok = mbar_wait_warp_cl(bar(kBarSFull + slot), par, abort_flag, p.status, kErrSoftmax);
+            } else if (kind == 2) {
+                const unsigned span = (unsigned)(hi - lo);
+                const int base = c0 - lo;
+                const bool any_col = hi >= lo;
+#pragma unroll
+                for (int j = 0; j < kSub; j += 2) {
+                    float x0 = __uint_as_float(rr[j]), x1 = __uint_as_float(rr[j + 1]);
+                    mul_f32x2(x0, x1, p.sl2);
+                    x0 = ex2_approx(x0);
+                    x1 = ex2_approx(x1);
+                    x0 = (any_col && (unsigned)(base + j) <= span) ? x0 : 0.f;
+                    x1 = (any_col && (unsigned)(base + j + 1) <= span) ? x1 : 0.f;
+                    add_f32x2(ls0, ls1, x0, x1);
+                    pk[j >> 1] = pack_bf16x2(x0, x1);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kSub / 2; ++j) pk[j] = 0u;
+            }
+            if (kind != 0) tmem_st8(p_tmem + ((c0 - col0) >> 1), pk);
+        };
+        uint32_t ra[kSub], rb[kSub];
+        int kind_a = 0;
+        if (ok && tl < n_tiles) {  // the first item: its scores, and the load of its first piece
+            begin_item();
+            ok = mbar_wait_warp_cl(bar(kBarSFull + wg), 0, abort_flag, p.status, kErrSoftmax);
+            if (ok) {
+                tc_fence_after();
+                kind_a = piece_kind(col0);
+                if (kind_a >= 2) tmem_ld16(s_tmem, ra);
+            }
+        }
+#pragma unroll 1
+        for (int use = 0; tl < n_tiles && ok; ++use) {
+            PSKV_TRACE_EVENT(20, use * kGroups + wg);
+            ls0 = 0.f;
+            ls1 = 0.f;
+#pragma unroll 1
+            for (int it = 0; it < kWarpCols / (2 * kSub); ++it) {
+                const int ca = col0 + it * 2 * kSub, cb = ca + kSub;
+                const bool last = it == kWarpCols / (2 * kSub) - 1;
+                tmem_wait_ld();  // piece A is in registers
+                const int kind_b = piece_kind(cb);
+                if (kind_b >= 2) tmem_ld16(s_tmem + (cb - col0), rb);
+                if (it == 0) {
+                    // the probability slot is free once the value MMAs of this group's previous item have
+                    // completed (issued a whole item period ago, so this wait rarely spins)
+                    ok = mbar_wait_warp_cl(bar(kBarPvDone + wg), (use & 1) ^ 1, abort_flag, p.status, kErrSoftmax);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                piece(ra, kind_a, ca);
+                tmem_wait_ld();  // piece B is in registers
+                if (!last) {
+                    kind_a = piece_kind(cb + kSub);
+                    if (kind_a >= 2) tmem_ld16(s_tmem + (cb + kSub - col0), ra);
+                } else {
+                    // this warp holds all it needs of the scores: the score MMAs of the group's next item
+                    // may overwrite the slot once every warp of the group has said so
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(lead_bar(kBarSFree + wg));
+                    PSKV_TRACE_EVENT(21, use * kGroups + wg);
+                }
+                piece(rb, kind_b, cb);
+            }
+            if (!ok) break;
+            lsum += ls0 + ls1;
+            PSKV_TRACE_EVENT(23, use * kGroups + wg);
+            // on to the group's next item; a partial row sum is complete when that one lies in another
+            // tile, and goes to the epilogue warps through shared memory BEFORE the arrival below (the
+            // tile's last value MMAs, which the epilogue waits for, need it)
+            const int tl_done = tl;
+            k += kGroups;
+            while (k >= nitems) { k -= nitems; ++tl; }
+            if (tl != tl_done) {
+                ml[((tl_done & 3) * kParts + part) * kTileM + row] = lsum;
+                __threadfence_block();
+            }
+            // the probabilities of this item are complete
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(lead_bar(kBarPReady + wg));
+            PSKV_TRACE_EVENT(24, use * kGroups + wg);
+            // the scores of the next item, and the load of its first piece
+            if (tl < n_tiles) {
+                begin_item();
+                PSKV_TRACE_EVENT(25, (use + 1) * kGroups + wg);
+                ok = mbar_wait_warp_cl(bar(kBarSFull + wg), (use + 1) & 1, abort_flag, p.status, kErrSoftmax);
                 if (!ok) break;
                 tc_fence_after();
-                PSKV_TRACE_EVENT(20, item);
-                uint32_t rr[kPiece], pk[kPiece / 2];
-                if (kind >= 2) {
-                    tmem_ld32(lane_base + slot * kBlockN + c0, rr);
-                    tmem_wait_ld();
-                }
-                // the scores are in registers: the score MMAs of the item after next may overwrite the slot
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_remote(lead_bar(kBarSFree + slot));
-                PSKV_TRACE_EVENT(21, item);
-                if (kind >= 2) {
-                    float e[kPiece];
-#pragma unroll
-                    for (int j = 0; j < kPiece; j += 2) {
-                        float x0 = __uint_as_float(rr[j]), x1 = __uint_as_float(rr[j + 1]);
-                        mul_f32x2(x0, x1, p.sl2);
-                        e[j] = ex2_approx(x0);
-                        e[j + 1] = ex2_approx(x1);
-                    }
-                    if (kind == 2) {
-                        const unsigned span = (unsigned)(hi - lo);
-                        const int base = c0 - lo;
-                        const bool any_col = hi >= lo;
-#pragma unroll
-                        for (int j = 0; j < kPiece; ++j)
-                            e[j] = (any_col && (unsigned)(base + j) <= span) ? e[j] : 0.f;
-                    }
-#pragma unroll
-                    for (int j = 0; j < kPiece / 4; ++j) {
-                        add_f32x2(ls0, ls1, e[4 * j], e[4 * j + 1]);
-                        add_f32x2(ls2, ls3, e[4 * j + 2], e[4 * j + 3]);
-                        pk[2 * j] = pack_bf16x2(e[4 * j], e[4 * j + 1]);
-                        pk[2 * j + 1] = pack_bf16x2(e[4 * j + 2], e[4 * j + 3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < kPiece / 2; ++j) pk[j] = 0u;
-                }
-                // the probability slot is free once the value MMAs of the item two back have completed
-                ok = mbar_wait_warp_cl(bar(kBarPvDone + slot), par ^ 1u, abort_flag, p.status, kErrSoftmax);
-                if (!ok) break;
-                tc_fence_after();
-                if (kind != 0) tmem_st16(lane_base + kPCol + slot * kPSlotCols + piece * (kPiece / 2), pk);
-                if (k == nitems - 1) {
-                    // the tile's partial row sums go to the epilogue warps through shared memory
-                    ml[((tl & 3) * kParts + piece) * kTileM + row] = (ls0 + ls1) + (ls2 + ls3);
-                    __threadfence_block();
-                }
-                PSKV_TRACE_EVENT(23, item);
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_remote(lead_bar(kBarPReady + slot));
-                PSKV_TRACE_EVENT(24, item);
+                kind_a = piece_kind(col0);
+                if (kind_a >= 2) tmem_ld16(s_tmem, ra);
             }
         }
     } else {
@@ -573,7 +636,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int ew = warp & 3;
         const int row = 32 * ew + lane;
         const uint32_t lane_addr = (uint32_t)(32 * ew) << 16;
-        const bool issuer = warp == 4 + 4 * kSoftmaxWarpgroups;
+        const bool issuer = warp == 4 + kSoftmaxWarps;
         const uint32_t stage = sbase + p.off_stage;
         if (issuer && lane == 0) prefetch_tensormap(&tm_out);
         bool ok = !misaligned;
@@ -584,9 +647,21 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (!ok) break;
             PSKV_TRACE_EVENT(30, te);
             tc_fence_after();
-            // the row sum: the four softmax pieces' partial sums
+            // the row sum: partial sums of the softmax groups that had an item of this tile (items go to
+            // the groups in turn), added in a fixed order
             const float *mlt = ml + (te & 3) * kParts * kTileM + row;
-            const float l = (mlt[0] + mlt[kTileM]) + (mlt[2 * kTileM] + mlt[3 * kTileM]);
+            float l = 0.f;
+            {
+                const int first = (te * nitems) % kGroups;  // group of the tile's first item
+#pragma unroll
+                for (int g = 0; g < kGroups; ++g) {
+                    const int dist = g >= first ? g - first : g + kGroups - first;  // items until group g's turn
+                    if (dist < nitems) {
+#pragma unroll
+                        for (int h = 0; h < kColSplit; ++h) l += mlt[(g * kColSplit + h) * kTileM];
+                    }
+                }
+            }
             const bool row_ok = l >= kMinRowSum && l <= kMaxRowSum;  // false for overflow (inf, NaN), underflow
             const float inv = row_ok ? 1.f / l : 0.f;
             // the TMA stores of the previous tile must have read the staging buffer
