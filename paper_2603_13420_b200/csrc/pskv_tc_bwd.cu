@@ -164,6 +164,16 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const TileInfo t0 = tile_info(p, t_begin < p.total_tiles ? t_begin : 0, t_begin);
         run_first = run_of(t0, inst_of(t0));
     }
+    // Several instructions (Sec. 4.3): the prefix of instruction i starts with pad[i] rows of left padding;
+    // the key blocks that hold nothing else are left out of its tiles (their probabilities are all zero), so
+    // the items of a tile are the blocks from first_block on, then the suffix block.
+    auto first_block = [&](const TileInfo &t) { return MI ? p.pad[inst_of(t)] / kBlockN : 0; };
+    auto count_items = [&]() {
+        if (!MI) return n_tiles * nitems;
+        int n = 0;
+        for (int tl = 0; tl < n_tiles; ++tl) n += nitems - first_block(tile_info(p, t_begin + tl, t_begin));
+        return n;
+    };
     const int sfx_slab = p.sfx_rows * 128;
     const int tail_slab = p.tail_rows * 128;
     const uint32_t stages_k = (uint32_t)p.stages_k, stages_v = (uint32_t)p.stages_v;
@@ -224,7 +234,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             __syncwarp();
             if (!RK) {
 #pragma unroll 1
-                for (int k = 0; k < p.nblk_p; ++k) {
+                for (int k = first_block(t); k < p.nblk_p; ++k) {
                     const uint32_t ks = kload % stages_k;
                     ok = mbar_wait_warp(bar(kBarKFree + ks), ((kload / stages_k) & 1) ^ 1, abort_flag, p.status, kErrProdA);
                     if (!ok) break;
@@ -335,7 +345,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             __syncwarp();
             if (!RV) {
 #pragma unroll 1
-                for (int k = 0; k < p.nblk_p; ++k) {
+                for (int k = first_block(t); k < p.nblk_p; ++k) {
                     const uint32_t vs = vload % stages_v;
                     ok = mbar_wait_warp(bar(kBarVFree + vs), ((vload / stages_v) & 1) ^ 1, abort_flag, p.status, kErrProdB);
                     if (!ok) break;
@@ -354,10 +364,11 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ S = Q K^T
-        const int total_items = n_tiles * nitems;
-        int tl = 0, k = 0;
+        const int total_items = count_items();
+        int tl = 0;
         uint32_t kuse = 0;
         TileInfo t = tile_info(p, t_begin, t_begin);
+        int kf = first_block(t), k = kf;
         const uint64_t q_desc = make_smem_desc(sbase + p.off_q, 0, 1024);
         bool ok = true;
 #pragma unroll 1
@@ -373,8 +384,16 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             // ---- S: the slot is free once the dQ MMAs of item i-2 have completed
             ok = mbar_wait_warp(bar(kBarDqDone + slot), ((i / kSlots) & 1) ^ 1, abort_flag, p.status, kErrMmaS);
             if (!ok) break;
-            if (k == 0) ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaS);
+            if (k == kf) ok = mbar_wait_warp(bar(kBarQFull), tl & 1, abort_flag, p.status, kErrMmaS);
             if (!ok) break;
+            if (MI && RK && k == kf && first_of_run(t, inst_of(t))) {
+                // the resident blocks this run leaves out were fetched with the others: pass their barriers
+                // too, so that every block's barrier has completed once per run
+                for (int kk = 0; kk < kf && kk < p.nblk_p && ok; ++kk)
+                    ok = mbar_wait_warp(bar(kBarKFull + kk), (run_of(t, inst_of(t)) - run_first) & 1, abort_flag, p.status,
+                                        kErrMmaS);
+                if (!ok) break;
+            }
             uint32_t kaddr;
             if (prefix) {
                 if (RK) {
@@ -411,8 +430,11 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
             if (ring_k) ++kuse;
             if (++k == nitems) {
-                k = 0;
-                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+                if (++tl < n_tiles) {
+                    t = tile_info(p, t_begin + tl, t_begin);
+                    kf = first_block(t);
+                }
+                k = kf;
             }
         }
     } else if (warp == 2) {
@@ -420,15 +442,16 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // This warp alternates: dP of item i+1 (its buffer comes free early in the element-wise
         // stage of item i), then dQ of item i (whose dS comes at the end of that stage).  The score
         // MMAs of warp 1 run beside both, so two threads keep the tensor pipe fed.
-        const int total_items = n_tiles * nitems;
-        int tl = 0, k = 0;
+        const int total_items = count_items();
+        int tl = 0;
         uint32_t kuse = 0;
         TileInfo t = tile_info(p, t_begin, t_begin);
+        int kf = first_block(t), k = kf;
         const uint32_t idesc_dq = make_idesc_bf16(kTileM, D, 1);
         const uint64_t do_desc = make_smem_desc(sbase + p.off_do, 0, 1024);
         bool ok = true;
         // cursor of the dP stream
-        int ptl = 0, pk = 0;
+        int ptl = 0, pkf = kf, pk = kf;
         uint32_t vuse = 0;
         TileInfo pt = t;
         auto issue_dp = [&](int i) -> bool {
@@ -445,8 +468,14 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 // ---- dP: its single slot is free once the element-wise warps have read item i-1
                 ok = mbar_wait_warp(bar(kBarDpFree), (i & 1) ^ 1, abort_flag, p.status, kErrMmaDq);
                 if (!ok) return false;
-                if (k == 0) ok = mbar_wait_warp(bar(kBarDoFull), tl & 1, abort_flag, p.status, kErrMmaDq);
+                if (k == pkf) ok = mbar_wait_warp(bar(kBarDoFull), tl & 1, abort_flag, p.status, kErrMmaDq);
                 if (!ok) return false;
+                if (MI && RV && k == pkf && first_of_run(t, inst_of(t))) {  // (as for the K blocks in warp 1)
+                    for (int kk = 0; kk < pkf && kk < p.nblk_p && ok; ++kk)
+                        ok = mbar_wait_warp(bar(kBarVFull + kk), (run_of(t, inst_of(t)) - run_first) & 1, abort_flag,
+                                            p.status, kErrMmaDq);
+                    if (!ok) return false;
+                }
                 uint32_t vaddr;
                 if (prefix) {
                     if (RV) {
@@ -484,8 +513,11 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) return false;
             if (ring_v) ++vuse;
             if (++pk == nitems) {
-                pk = 0;
-                if (++ptl < n_tiles) pt = tile_info(p, t_begin + ptl, t_begin);
+                if (++ptl < n_tiles) {
+                    pt = tile_info(p, t_begin + ptl, t_begin);
+                    pkf = first_block(pt);
+                }
+                pk = pkf;
             }
             return true;
         };
@@ -504,7 +536,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const bool ring = prefix && !RK;
             ok = mbar_wait_warp(bar(kBarDsReady + slot), (i / kSlots) & 1, abort_flag, p.status, kErrMmaDq);
             if (!ok) break;
-            if (k == 0 && tl > 0) {
+            if (k == kf && tl > 0) {
                 ok = mbar_wait_warp(bar(kBarDqFree), (tl - 1) & 1, abort_flag, p.status, kErrMmaDq);
                 if (!ok) break;
             }
@@ -516,7 +548,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const uint32_t ds_tmem = tmem + slot * kBlockN;  // bf16 pairs: 8 columns per 16 keys
             const uint64_t k_desc = make_smem_desc(kaddr, (uint32_t)slab, 1024);  // K as [keys][d]: d contiguous
             const int nk = n >> 4;
-            const uint32_t acc0 = k > 0 ? 1u : 0u;
+            const uint32_t acc0 = k > kf ? 1u : 0u;
             if (elect_one_sync()) {
 #pragma unroll
                 for (int ks16 = 0; ks16 < kBlockN / 16; ++ks16) {
@@ -531,8 +563,11 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             __syncwarp();
             if (ring) ++kuse;
             if (++k == nitems) {
-                k = 0;
-                if (++tl < n_tiles) t = tile_info(p, t_begin + tl, t_begin);
+                if (++tl < n_tiles) {
+                    t = tile_info(p, t_begin + tl, t_begin);
+                    kf = first_block(t);
+                }
+                k = kf;
             }
         }
     } else if (warp < 4 + 4 * kGroups) {
@@ -562,7 +597,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const float drow = valid ? p.row_dot[grow] : 0.f;
             const int pad = MI ? p.pad[inst_of(t)] : 0;
 #pragma unroll 1
-            for (int k = 0; k < nitems && ok; ++k, ++item) {
+            for (int k = pad / kBlockN; k < nitems && ok; ++k, ++item) {
                 const int slot = item % kSlots;
                 int n, lo, hi;
                 if (k < p.nblk_p) {
