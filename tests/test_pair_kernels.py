@@ -71,9 +71,9 @@ def test_pair_forward_outliers_and_redo_rows():
 
 
 def test_pair_and_single_cta_kernels_agree():
-    """Same shape through both kernel families: same tiling of the reductions, so the results agree
-    to the last bits of bf16 (they are not required to be bit-identical: the row sums add the four
-    partial sums in the same order, but the MMAs accumulate 256-row instructions)."""
+    """Same shape through both kernel families: same tiling of the key blocks, so the results agree to
+    the last bits of bf16 (they are not required to be bit-identical: the row sums are added up in a
+    different order and the MMAs accumulate 256-row instructions)."""
     w = dataclasses.replace(WORKLOADS["C2"], B=16)
     t = make_inputs(w)
     try:
