@@ -73,6 +73,8 @@ struct TcFwdParams {
     int stages;           // streaming mode: stages of the prefix K and V rings
     int sfx_rows;         // rows of the suffix K / V buffers (multiple of 16, <= 128)
     int alias_stage;      // 1 when the output staging buffer shares its memory with the suffix V buffer
+    int slab_stage;       // 1 when the staging buffer holds one 64-column slab: staged and stored a slab at a time
+    int ml_mask;          // partial row sums are kept for ml_mask + 1 tiles (3, or 0 behind kBarMlFree)
     // suffix-ring mode (tiles of whole candidates, suffix keys in blocks through the K/V rings)
     const int *suffix_len;  // cached suffix tokens per candidate, or nullptr (= Skv)
     int Skv;              // rows of a candidate's suffix K/V buffer (S counts its query rows)
@@ -110,6 +112,7 @@ enum {
     kBarOFree,       // epilogue has read O out (one arrival per softmax warp)
     kBarStageFull,   // the output tile is staged (one arrival per softmax warp)
     kBarStageFree,   // the TMA stores of that slab have read it
+    kBarMlFree,      // the epilogue has read a tile's partial row sums (one arrival per epilogue warp)
     kBarSFull,                        // [kSlots] scores of an item are in tensor memory
     kBarPReady = kBarSFull + kSlots,  // [kSlots] probabilities written (one arrival per softmax warp)
     kBarPvDone = kBarPReady + kSlots, // [kSlots] value MMAs of an item completed
@@ -198,7 +201,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) {
             const bool all_sm = i >= kBarPReady && i < kBarPReady + kSlots;
-            const bool epi = i == kBarOFree || i == kBarStageFull;
+            const bool epi = i == kBarOFree || i == kBarStageFull || i == kBarMlFree;
             mbar_init(bar(i), all_sm ? (uint32_t)(4 * kGroups) : epi ? 4u : 1u);
         }
         *abort_flag = 0;
@@ -429,6 +432,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         // stores of tile t have read the staging buffer.
         const uint32_t stage = sbase + p.off_stage;
         uint32_t vload = 0;
+        int store_slab = 0;  // slab_stage: slabs of the previous tile's output stored so far
         bool ok = true;
 #pragma unroll 1
         for (int tl = 0; tl <= n_tiles && ok; ++tl) {
@@ -528,24 +532,28 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     if (!ok) break;
                 }
                 if (pend_store && !sv_ready) {
+                    // the staging buffer holds the whole tile, or (slab_stage) one 64-column slab per round
+                    const uint32_t round = p.slab_stage ? (uint32_t)((tl - 1) * C::kSlabs + store_slab) : (uint32_t)(tl - 1);
                     bool ready;
                     if (block)
-                        ready = ok = mbar_wait_warp(bar(kBarStageFull), (tl - 1) & 1, abort_flag, p.status, kErrEpilogue);
+                        ready = ok = mbar_wait_warp(bar(kBarStageFull), round & 1, abort_flag, p.status, kErrEpilogue);
                     else
-                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarStageFull), (tl - 1) & 1) ? 1 : 0, 0) != 0;
+                        ready = __shfl_sync(0xffffffffu, mbar_try_wait(bar(kBarStageFull), round & 1) ? 1 : 0, 0) != 0;
                     if (!ok) break;
                     if (ready) {
                         const TileInfo u = tile_info(p, tile_at(tl - 1), t_begin);
                         const int nseg = SR ? 1 : p.fd_seg.div(u.rows);  // (one box of whole candidates)
+                        const int sl_first = p.slab_stage ? store_slab : 0;
+                        const int sl_end = p.slab_stage ? store_slab + 1 : C::kSlabs;
                         if (elect_one_sync()) {
 #pragma unroll 1
-                            for (int sl = 0; sl < C::kSlabs; ++sl)
+                            for (int sl = sl_first; sl < sl_end; ++sl)
 #pragma unroll 1
                                 for (int s = 0; s < nseg; ++s) {
                                     const int R = u.R0 + s * p.seg_rows;
                                     const int b = p.fd_Rg.div(R), r = R - b * p.Rg;
-                                    tma_store_4d(&tm_out, stage + sl * kStagingBytes + s * p.seg_rows * 128, sl * 64, r,
-                                                 u.g, b);
+                                    tma_store_4d(&tm_out, stage + (p.slab_stage ? 0 : sl) * kStagingBytes + s * p.seg_rows * 128,
+                                                 sl * 64, r, u.g, b);
                                 }
                             tma_store_commit();
                             tma_store_wait_read();  // the staging buffer may be overwritten after this
@@ -553,7 +561,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         }
                         __syncwarp();
                         PSKV_TRACE_EVENT(4, tl - 1);
-                        pend_store = false;
+                        if (p.slab_stage && store_slab + 1 < C::kSlabs) {
+                            ++store_slab;
+                        } else {
+                            store_slab = 0;
+                            pend_store = false;
+                        }
                     }
                 }
                 if (pend_sv && p.alias_stage && !pend_store) sv_ready = true;
@@ -895,8 +908,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         tmem_st16(s_tmem, pk);
                     }
                     if (k == nitems - 1) {
-                        // the tile's partial row sums go to the epilogue warps through shared memory
-                        ml[((tl & 3) * kGroups + wg) * kTileM + row] = lsum;
+                        // the tile's partial row sums go to the epilogue warps through shared memory (kept
+                        // for four tiles, or for one: then the epilogue must have read the previous tile's)
+                        if (p.ml_mask == 0 && tl > 0) {
+                            ok = mbar_wait_warp(bar(kBarMlFree), (tl - 1) & 1, abort_flag, p.status, kErrSoftmax);
+                            if (!ok) break;
+                        }
+                        ml[((tl & p.ml_mask) * kGroups + wg) * kTileM + row] = lsum;
                         __threadfence_block();
                     }
                     PSKV_TRACE_EVENT(23, item);
@@ -923,57 +941,108 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (!ok) break;
             PSKV_TRACE_EVENT(30, te);
             tc_fence_after();
-            const float *mlt = ml + (te & 3) * kGroups * kTileM + row;
+            const float *mlt = ml + (te & p.ml_mask) * kGroups * kTileM + row;
             const float l = (mlt[0] + mlt[kTileM]) + (mlt[2 * kTileM] + mlt[3 * kTileM]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarMlFree));
             const bool row_ok = l >= kMinRowSum && l <= kMaxRowSum;  // false for overflow (inf, NaN), underflow
             // staged values must be finite (the buffer may double as suffix V, whose padding rows
             // meet zero probabilities): rows that failed stage zeros, and are redone anyway
             const float inv = row_ok ? 1.f / l : 0.f;
-            // the TMA stores of the previous tile must have read the staging buffer
-            ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
-            if (!ok) break;
-            PSKV_TRACE_EVENT(33, te);
-            // one 64-column slab per round; O is free for the next tile's first value MMA as soon
-            // as the last round's loads have returned
+            if (p.slab_stage) {
+                // One 64-column slab at a time through a staging buffer of one slab: load, hand O back after
+                // the last load, wait for the previous slab's stores to have read the buffer, stage, tell
+                // the storing warp.  The buffer is this kernel's own: suffix V of the next tile is fetched
+                // as soon as this tile's value MMAs have completed, not behind these stores.
 #pragma unroll 1
-            for (int sl = 0; sl < C::kSlabs; ++sl) {
-                uint32_t o0[kPiece], o1[kPiece];
-                tmem_ld32(tmem + lane_addr + kOCol + sl * 64, o0);
-                tmem_ld32(tmem + lane_addr + kOCol + sl * 64 + kPiece, o1);
-                tmem_wait_ld();
-                PSKV_TRACE_EVENT(34 + sl, te);
-                if (sl == C::kSlabs - 1) {
-                    tc_fence_before();
+                for (int sl = 0; sl < C::kSlabs; ++sl) {
+                    const uint32_t round = (uint32_t)(te * C::kSlabs + sl);
+                    uint32_t o0[kPiece], o1[kPiece];
+                    tmem_ld32(tmem + lane_addr + kOCol + sl * 64, o0);
+                    tmem_ld32(tmem + lane_addr + kOCol + sl * 64 + kPiece, o1);
+                    tmem_wait_ld();
+                    PSKV_TRACE_EVENT(34 + sl, te);
+                    if (sl == C::kSlabs - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kBarOFree));
+                        PSKV_TRACE_EVENT(32, te);
+                    }
+                    ok = mbar_wait_warp(bar(kBarStageFree), (round & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
+                    if (!ok) break;
+                    uint8_t *srow = smem + p.off_stage + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * inv, __uint_as_float(o0[8 * c + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * inv, __uint_as_float(o0[8 * c + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * inv, __uint_as_float(o0[8 * c + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * inv, __uint_as_float(o0[8 * c + 7]) * inv);
+                        if (!row_ok) v = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * inv, __uint_as_float(o1[8 * c + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * inv, __uint_as_float(o1[8 * c + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * inv, __uint_as_float(o1[8 * c + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * inv, __uint_as_float(o1[8 * c + 7]) * inv);
+                        if (!row_ok) v = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
+                    }
+                    fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(kBarOFree));
-                    PSKV_TRACE_EVENT(32, te);
+                    if (lane == 0) mbar_arrive(bar(kBarStageFull));
                 }
-                // 128-byte rows, 16-byte chunks swizzled by the row
-                uint8_t *srow = smem + p.off_stage + sl * kStagingBytes + row * 128;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * inv, __uint_as_float(o0[8 * c + 1]) * inv);
-                    v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * inv, __uint_as_float(o0[8 * c + 3]) * inv);
-                    v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * inv, __uint_as_float(o0[8 * c + 5]) * inv);
-                    v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * inv, __uint_as_float(o0[8 * c + 7]) * inv);
-                    if (!row_ok) v = make_uint4(0, 0, 0, 0);  // (inf or NaN accumulators times zero are not zero)
-                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                if (!ok) break;
+            } else {
+            // the TMA stores of the previous tile must have read the staging buffer
+                ok = mbar_wait_warp(bar(kBarStageFree), (te & 1) ^ 1, abort_flag, p.status, kErrEpilogue);
+                if (!ok) break;
+                PSKV_TRACE_EVENT(33, te);
+                // one 64-column slab per round; O is free for the next tile's first value MMA as soon
+                // as the last round's loads have returned
+    #pragma unroll 1
+                for (int sl = 0; sl < C::kSlabs; ++sl) {
+                    uint32_t o0[kPiece], o1[kPiece];
+                    tmem_ld32(tmem + lane_addr + kOCol + sl * 64, o0);
+                    tmem_ld32(tmem + lane_addr + kOCol + sl * 64 + kPiece, o1);
+                    tmem_wait_ld();
+                    PSKV_TRACE_EVENT(34 + sl, te);
+                    if (sl == C::kSlabs - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kBarOFree));
+                        PSKV_TRACE_EVENT(32, te);
+                    }
+                    // 128-byte rows, 16-byte chunks swizzled by the row
+                    uint8_t *srow = smem + p.off_stage + sl * kStagingBytes + row * 128;
+    #pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * inv, __uint_as_float(o0[8 * c + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * inv, __uint_as_float(o0[8 * c + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * inv, __uint_as_float(o0[8 * c + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * inv, __uint_as_float(o0[8 * c + 7]) * inv);
+                        if (!row_ok) v = make_uint4(0, 0, 0, 0);  // (inf or NaN accumulators times zero are not zero)
+                        *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                    }
+    #pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * inv, __uint_as_float(o1[8 * c + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * inv, __uint_as_float(o1[8 * c + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * inv, __uint_as_float(o1[8 * c + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * inv, __uint_as_float(o1[8 * c + 7]) * inv);
+                        if (!row_ok) v = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
+                    }
                 }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * inv, __uint_as_float(o1[8 * c + 1]) * inv);
-                    v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * inv, __uint_as_float(o1[8 * c + 3]) * inv);
-                    v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * inv, __uint_as_float(o1[8 * c + 5]) * inv);
-                    v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * inv, __uint_as_float(o1[8 * c + 7]) * inv);
-                    if (!row_ok) v = make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
-                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarStageFull));
             }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarStageFull));
             const bool stored = row < u.rows;
             if (stored) {
                 const int R = u.R0 + row;
@@ -1034,7 +1103,7 @@ struct TilePlan {
     int cbox, Spad, cpb;  // suffix-ring mode: candidates per tile, rows per candidate in a block, candidates per block
     int long_sfx;         // suffix-ring mode: tiles inside one candidate, its suffix keys in 128-key blocks
     int tile_rows, seg_rows, tiles_per_group, sfx_rows;
-    int nblk_p, tail_rows, resident, stages, alias_stage;
+    int nblk_p, tail_rows, resident, stages, alias_stage, slab_stage, ml_tiles;
     int off_pk, off_pv, off_q, off_sk, off_sv, off_stage, off_bar, off_misc, off_ml, smem_bytes;
 };
 
@@ -1128,6 +1197,16 @@ TilePlan plan_base(const Dims &dm)
         pl.stages = pl.nblk_p;
         kv_bytes = resident_bytes;
         pl.alias_stage = fixed_own + 2 * resident_bytes <= kMaxSmem ? 0 : 1;
+        // Sharing the staging buffer with suffix V chains the next tile's suffix V behind this tile's
+        // stores.  A staging buffer of one 64-column slab, with the partial row sums kept for one tile
+        // instead of four, may still fit beside everything else: then the output goes a slab at a time.
+        const int ml_one = kGroups * kTileM * 4;
+        const int fixed_slab = tile_bytes + 2 * sfx_bytes + kStagingBytes + ml_one + 64 + kBarBytes;
+        if (pl.alias_stage && slabs == 2 && fixed_slab + 2 * resident_bytes <= kMaxSmem) {
+            pl.alias_stage = 0;
+            pl.slab_stage = 1;
+            pl.ml_tiles = 1;
+        }
     } else {
         const int st = ring_stages(fixed_shared);
         if (st < 1) return pl;  // does not fit: the general kernels take the shape
@@ -1142,10 +1221,10 @@ TilePlan plan_base(const Dims &dm)
     pl.off_sk = pl.off_q + tile_bytes;
     pl.off_sv = pl.off_sk + sfx_bytes;
     pl.off_stage = pl.alias_stage ? pl.off_sv : pl.off_sv + sv_bytes;
-    pl.off_bar = pl.off_stage + (pl.alias_stage ? sv_bytes : stage_bytes);
+    pl.off_bar = pl.off_stage + (pl.alias_stage ? sv_bytes : pl.slab_stage ? kStagingBytes : stage_bytes);
     pl.off_misc = pl.off_bar + kBarBytes;
     pl.off_ml = pl.off_misc + 64;
-    pl.smem_bytes = pl.off_ml + ml_bytes;
+    pl.smem_bytes = pl.off_ml + (pl.ml_tiles == 1 ? ml_bytes / 4 : ml_bytes);
     pl.ok = pl.smem_bytes <= kMaxSmem;
     pl.mode = pl.resident ? 1 : 0;
     return pl;
@@ -1223,6 +1302,8 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     p.stages = plan.stages > 0 ? plan.stages : 1;
     p.sfx_rows = plan.sfx_rows;
     p.alias_stage = plan.alias_stage;
+    p.slab_stage = plan.slab_stage;
+    p.ml_mask = plan.ml_tiles == 1 ? 0 : 3;
     p.suffix_len = a.suffix_len;
     p.Skv = dm.Skv;
     p.Spad = plan.Spad > 0 ? plan.Spad : 8;
