@@ -693,38 +693,58 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) break;
             tc_fence_after();
             const int nseg = p.fd_seg.div(t.rows);
+            // dQ leaves tensor memory in two load round trips back to back (the first slab is scaled and packed
+            // to bf16 in registers while the second one is on its way) and goes back to the MMA issuer right
+            // after them: the first dQ MMAs of the next tile wait for exactly that, and with the first slab's
+            // staging and stores between the two loads they waited 2 500-4 100 cycles a tile.
+            uint32_t pk0[C::kSlabs > 1 ? 32 : 1];
+            uint32_t o0[32], o1[32];
+            tmem_ld32(tmem + lane_addr + kDqCol, o0);
+            tmem_ld32(tmem + lane_addr + kDqCol + 32, o1);
+            tmem_wait_ld();
+            if (C::kSlabs > 1) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    pk0[c] = pack_bf16x2(__uint_as_float(o0[2 * c]) * p.scale, __uint_as_float(o0[2 * c + 1]) * p.scale);
+                    pk0[16 + c] = pack_bf16x2(__uint_as_float(o1[2 * c]) * p.scale, __uint_as_float(o1[2 * c + 1]) * p.scale);
+                }
+                tmem_ld32(tmem + lane_addr + kDqCol + 64, o0);
+                tmem_ld32(tmem + lane_addr + kDqCol + 96, o1);
+                tmem_wait_ld();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarDqFree));
 #pragma unroll 1
             for (int sl = 0; sl < C::kSlabs; ++sl) {
                 const uint32_t round = (uint32_t)(tl * C::kSlabs + sl);
-                uint32_t o0[32], o1[32];
-                tmem_ld32(tmem + lane_addr + kDqCol + sl * 64, o0);
-                tmem_ld32(tmem + lane_addr + kDqCol + sl * 64 + 32, o1);
-                tmem_wait_ld();
-                if (sl == C::kSlabs - 1) {  // dQ is free for the next tile once the last slab is in registers
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(kBarDqFree));
-                }
                 ok = mbar_wait_warp(bar(kBarStageFree), (round & 1) ^ 1, abort_flag, p.status, kErrEpi);
                 if (!ok) break;
                 uint8_t *srow = smem + p.off_stage + row * 128;
+                if (C::kSlabs > 1 && sl == 0) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * p.scale, __uint_as_float(o0[8 * c + 1]) * p.scale);
-                    v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * p.scale, __uint_as_float(o0[8 * c + 3]) * p.scale);
-                    v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * p.scale, __uint_as_float(o0[8 * c + 5]) * p.scale);
-                    v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * p.scale, __uint_as_float(o0[8 * c + 7]) * p.scale);
-                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
-                }
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) =
+                            make_uint4(pk0[4 * c], pk0[4 * c + 1], pk0[4 * c + 2], pk0[4 * c + 3]);
+                } else {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * p.scale, __uint_as_float(o1[8 * c + 1]) * p.scale);
-                    v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * p.scale, __uint_as_float(o1[8 * c + 3]) * p.scale);
-                    v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * p.scale, __uint_as_float(o1[8 * c + 5]) * p.scale);
-                    v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * p.scale, __uint_as_float(o1[8 * c + 7]) * p.scale);
-                    *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o0[8 * c]) * p.scale, __uint_as_float(o0[8 * c + 1]) * p.scale);
+                        v.y = pack_bf16x2(__uint_as_float(o0[8 * c + 2]) * p.scale, __uint_as_float(o0[8 * c + 3]) * p.scale);
+                        v.z = pack_bf16x2(__uint_as_float(o0[8 * c + 4]) * p.scale, __uint_as_float(o0[8 * c + 5]) * p.scale);
+                        v.w = pack_bf16x2(__uint_as_float(o0[8 * c + 6]) * p.scale, __uint_as_float(o0[8 * c + 7]) * p.scale);
+                        *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o1[8 * c]) * p.scale, __uint_as_float(o1[8 * c + 1]) * p.scale);
+                        v.y = pack_bf16x2(__uint_as_float(o1[8 * c + 2]) * p.scale, __uint_as_float(o1[8 * c + 3]) * p.scale);
+                        v.z = pack_bf16x2(__uint_as_float(o1[8 * c + 4]) * p.scale, __uint_as_float(o1[8 * c + 5]) * p.scale);
+                        v.w = pack_bf16x2(__uint_as_float(o1[8 * c + 6]) * p.scale, __uint_as_float(o1[8 * c + 7]) * p.scale);
+                        *reinterpret_cast<uint4 *>(srow + (((4 + c) ^ (row & 7)) << 4)) = v;
+                    }
                 }
                 fence_proxy_async();
                 __syncwarp();
