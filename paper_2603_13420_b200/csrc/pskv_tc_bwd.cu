@@ -117,6 +117,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     PSKV_TRACE_DECL;
+    grid_dep_launch();  // the next kernel of the stream may take over SMs as this one's CTAs exit
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + p.off_bar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -148,6 +149,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // everything above touched shared and tensor memory only: it may run under the tail of the kernel before
+    grid_dep_wait();
 
     const int t_begin = (int)((long long)blockIdx.x * p.total_tiles / gridDim.x);
     const int t_end = (int)((long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x);
@@ -923,11 +926,11 @@ cudaError_t launch(const BwdArgs &a, const BwdPlan &plan, unsigned int *status_w
         const int grid = even_grid(p.total_tiles, sm_count());
         {
             KernelTiming timing(kKernelBwdDqTc, stream);
-            kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_do, tm_dq, tm_pk, tm_pv, tm_pk_tail,
-                                                                tm_pv_tail, tm_sk, tm_sv, p);
+            e = launch_dependent(kernel, grid, kThreads, plan.smem_bytes, stream, tm_q, tm_do, tm_dq, tm_pk, tm_pv,
+                                 tm_pk_tail, tm_pv_tail, tm_sk, tm_sv, p);
         }
         count_launches(1);
-        e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     if (!(parts & kBwdPartDkv)) return cudaSuccess;

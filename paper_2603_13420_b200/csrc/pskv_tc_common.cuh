@@ -240,6 +240,31 @@ inline cudaError_t ensure_max_smem(Kernel kernel, PerDeviceOnce &once, int bytes
     return e;
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while the kernel before it in the
+// stream is still running (that one calls grid_dep_launch() at its start), so that its CTAs take over SMs as
+// the other's CTAs exit and run their prologue -- shared-memory zeroing, barrier and tensor-memory set-up, about
+// 3 us -- under the other kernel's tail; grid_dep_wait() in the kernel then holds every access to global memory
+// back until the kernel before has completed and its writes are visible.  Behind anything that is not such
+// a kernel the launch orders as usual.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int threads, int smem_bytes, cudaStream_t stream,
+                                    Args &&...args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    memset(&attr, 0, sizeof(attr));
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // SM count of the current device (looked up once per device).
 inline int sm_count()
 {

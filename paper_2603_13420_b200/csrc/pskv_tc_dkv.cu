@@ -150,6 +150,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
     PSKV_TRACE_DECL;
+    grid_dep_launch();  // the next kernel of the stream may take over SMs as this one's CTAs exit
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + p.off_bar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -182,6 +183,8 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // everything above touched shared and tensor memory only: it may run under the tail of the kernel before
+    grid_dep_wait();
 
     const int my_groups = (int)blockIdx.x < p.total_groups ? (p.total_groups - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int total_units = my_groups * (PRE ? p.cpc * p.ntile : p.ntile);
@@ -544,9 +547,10 @@ cudaError_t launch_np(const BwdArgs &a, const CUtensorMap &tm_q, const CUtensorM
     if (cudaError_t e = ensure_max_smem(tc_bwd_dkv_kernel<NP, PRE, DROW>, attr_set); e != cudaSuccess) return e;
     const int grid = p.total_groups < sm_count() ? p.total_groups : sm_count();
     KernelTiming timing(PRE ? kKernelBwdPrefixTc : kKernelBwdDkvTc, stream);
-    tc_bwd_dkv_kernel<NP, PRE, DROW><<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_do, tm_k, tm_v, tm_o, p);
+    const cudaError_t e = launch_dependent(tc_bwd_dkv_kernel<NP, PRE, DROW>, grid, kThreads, smem_bytes, stream, tm_q, tm_do,
+                                           tm_k, tm_v, tm_o, p);
     count_launches(1);
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // fp32 accumulators -> bf16 results

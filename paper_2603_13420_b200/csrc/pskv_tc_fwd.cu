@@ -182,6 +182,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // warp-uniform by construction
     PSKV_TRACE_DECL;
+    grid_dep_launch();  // the next kernel of the stream may take over SMs as this one's CTAs exit
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + p.off_bar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -218,6 +219,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // everything above touched shared and tensor memory only: it may run under the tail of the kernel before
+    grid_dep_wait();
 
     // Tiles of this CTA.  Normally a contiguous range (tiles are ordered KV head major, so the
     // resident prefix of a head serves a whole run).  With long suffixes a tile's cost grows with the
@@ -1329,13 +1332,14 @@ cudaError_t launch(const FwdArgs &a, const TilePlan &plan, void *workspace, unsi
     static PerDeviceOnce attr_set[6];
     if (cudaError_t e = ensure_max_smem(kernel, attr_set[plan.mode + (mi ? 3 : 0)]); e != cudaSuccess) return e;
     const int grid = even_grid(p.total_tiles, sm_count());
+    cudaError_t launch_err;
     {
         KernelTiming timing(kKernelFwdTc, stream);
-        kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail, tm_pv_tail, tm_sk,
-                                                            tm_sv, p);
+        launch_err = launch_dependent(kernel, grid, kThreads, plan.smem_bytes, stream, tm_q, tm_out, tm_pk, tm_pv, tm_pk_tail,
+                                      tm_pv_tail, tm_sk, tm_sv, p);
     }
     count_launches(1);
-    return cudaGetLastError();
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 }  // namespace
