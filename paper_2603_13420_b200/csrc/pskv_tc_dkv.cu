@@ -354,15 +354,20 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         int pending_gi = -1;  // group whose accumulators are still to be written back
         float *dpart = reinterpret_cast<float *>(smem + p.off_dpart);  // DROW: [stage][warpgroup][row]
         uint4 o_next[4] = {};                                            // DROW: this thread's O slice of the coming unit
-        if (DROW && total_units > 0) {
-            const Unit y = unit_of<PRE>(p, 0);
-            if (row < p.Rg) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    p.out + (((size_t)y.b * p.Hq + (size_t)y.g * p.n_rep) * p.S + row) * kD + 32 * wg);
+        // DROW: the O rows of a unit are read four lanes to a row -- lane 4k+c takes the 16-byte chunk c of this
+        // warpgroup's 32 columns of rows 8j+k (j = 0..3) of the warp's 32 rows -- so that a load instruction
+        // covers eight 64-byte runs of full sectors instead of 32 half-used ones.
+        const int orow_k = lane >> 2, ochunk = lane & 3;
+        auto load_o = [&](const Unit &y) {
+            const int base = y.tt * kTileM + 32 * (warp & 3);
+            const __nv_bfloat16 *o0 = p.out + (((size_t)y.b * p.Hq + (size_t)y.g * p.n_rep) * p.S) * kD + 32 * wg + 8 * ochunk;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) o_next[j] = __ldg(src + j);
+            for (int j = 0; j < 4; ++j) {
+                const int gy = base + 8 * j + orow_k;
+                o_next[j] = gy < p.Rg ? __ldg(reinterpret_cast<const uint4 *>(o0 + (size_t)gy * kD)) : make_uint4(0, 0, 0, 0);
             }
-        }
+        };
+        if (DROW && total_units > 0) load_o(unit_of<PRE>(p, 0));
         // write-back of group gi: lane <-> column d, tensor-memory column <-> key
         auto write_back = [&](int gi) -> bool {
             const int as = gi & 1;
@@ -429,38 +434,31 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (DROW) {
                 // my 32 of the row's 128 columns: O from global memory (requested one unit ahead), dO from the
                 // tile in shared memory (64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row)
-                float part = 0.f;
                 ok = mbar_wait_warp(bar(kBarQFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
                 if (!ok) break;
-                if (valid) {
-                    const uint8_t *dorow = smem + p.off_do + st * kTileBytes + (wg >> 1) * kSlabBytes + row * 128;
+                const uint8_t *dotile = smem + p.off_do + st * kTileBytes + (wg >> 1) * kSlabBytes;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint4 dv = *reinterpret_cast<const uint4 *>(dorow + ((((wg & 1) * 4 + j) ^ (row & 7)) << 4));
-                        const __nv_bfloat162 *a = reinterpret_cast<const __nv_bfloat162 *>(&dv);
-                        const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&o_next[j]);
+                for (int j = 0; j < 4; ++j) {
+                    const int r = 32 * (warp & 3) + 8 * j + orow_k;  // row of the tile this lane works on in round j
+                    const uint4 dv = *reinterpret_cast<const uint4 *>(dotile + r * 128 + ((((wg & 1) * 4 + ochunk) ^ (r & 7)) << 4));
+                    const __nv_bfloat162 *a = reinterpret_cast<const __nv_bfloat162 *>(&dv);
+                    const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&o_next[j]);
+                    float part = 0.f;
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float2 fa = __bfloat1622float2(a[e]), fb = __bfloat1622float2(b[e]);
-                            part = fmaf(fa.x, fb.x, part);
-                            part = fmaf(fa.y, fb.y, part);
-                        }
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 fa = __bfloat1622float2(a[e]), fb = __bfloat1622float2(b[e]);
+                        part = fmaf(fa.x, fb.x, part);
+                        part = fmaf(fa.y, fb.y, part);
                     }
+                    // the four chunks of the row, added in a fixed order; rows past the group read zeros for O
+                    part += __shfl_xor_sync(0xffffffffu, part, 1);
+                    part += __shfl_xor_sync(0xffffffffu, part, 2);
+                    if (ochunk == 0) dpart[(st * 4 + wg) * kTileM + r] = part;
                 }
-                dpart[(st * 4 + wg) * kTileM + row] = part;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarDFull + st));
-                // the O slice of the next unit's row, in flight while this unit is worked on
-                if (u + 1 < total_units) {
-                    const Unit y = unit_of<PRE>(p, u + 1);
-                    const int gy = y.tt * kTileM + row;
-                    if (gy < p.Rg) {
-                        const uint4 *src = reinterpret_cast<const uint4 *>(
-                            p.out + (((size_t)y.b * p.Hq + (size_t)y.g * p.n_rep) * p.S + gy) * kD + 32 * wg);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) o_next[j] = __ldg(src + j);
-                    }
-                }
+                // the O slice of the next unit, in flight while this unit is worked on
+                if (u + 1 < total_units) load_o(unit_of<PRE>(p, u + 1));
             }
             ok = mbar_wait_warp(bar(kBarSFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
             if (!ok) break;
