@@ -101,6 +101,18 @@ struct TcDkvParams {
     int off_q, off_do, off_k, off_v, off_p, off_ds, off_bar, off_misc, off_dpart, kv_bytes;
 };
 
+// Warp-level MMA (16 x 8 x 16, bf16 in, fp32 accumulate): used only to form the row statistic D, whose dot
+// products over the columns of a row are a diagonal of dO O^T.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // unit u of a CTA -> (index of the group within this CTA, tile within the group)
 struct Unit {
     int gi, tt, bg, b, g, kb;
@@ -436,24 +448,33 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // tile in shared memory (64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row)
                 ok = mbar_wait_warp(bar(kBarQFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
                 if (!ok) break;
+                // <dO, O> over my 32 columns for the warp's 32 rows, on the warp-level tensor-core path: for a group
+                // of 16 rows, dO (16 x 16 columns) times the transpose of 8 rows of O gives a 16 x 8 block of
+                // dO O^T whose diagonal holds 8 of the wanted sums; two such products per 16 rows, two 16-column
+                // slices each.  (Conversions and FMAs on the CUDA cores took these warps 1 000 cycles a unit.)
+                // The k index is permuted the same way on both sides, which a dot product does not mind: lane
+                // 4g+c holds columns 8c..8c+7 of a row, and slice s takes 8c+4s..8c+4s+3 as its k = 2c, 2c+1, 2c+8,
+                // 2c+9 -- so a lane's 16-byte chunk of O is its B fragment of both slices as it stands.
                 const uint8_t *dotile = smem + p.off_do + st * kTileBytes + (wg >> 1) * kSlabBytes;
+                const int g = orow_k, c = ochunk;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int r = 32 * (warp & 3) + 8 * j + orow_k;  // row of the tile this lane works on in round j
-                    const uint4 dv = *reinterpret_cast<const uint4 *>(dotile + r * 128 + ((((wg & 1) * 4 + ochunk) ^ (r & 7)) << 4));
-                    const __nv_bfloat162 *a = reinterpret_cast<const __nv_bfloat162 *>(&dv);
-                    const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&o_next[j]);
-                    float part = 0.f;
+                for (int G = 0; G < 2; ++G) {
+                    const int r_lo = 32 * (warp & 3) + 16 * G + g, r_hi = r_lo + 8;
+                    const uint4 alo = *reinterpret_cast<const uint4 *>(dotile + r_lo * 128 + ((((wg & 1) * 4 + c) ^ (r_lo & 7)) << 4));
+                    const uint4 ahi = *reinterpret_cast<const uint4 *>(dotile + r_hi * 128 + ((((wg & 1) * 4 + c) ^ (r_hi & 7)) << 4));
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 fa = __bfloat1622float2(a[e]), fb = __bfloat1622float2(b[e]);
-                        part = fmaf(fa.x, fb.x, part);
-                        part = fmaf(fa.y, fb.y, part);
+                    for (int h = 0; h < 2; ++h) {
+                        const uint4 b = o_next[2 * G + h];  // O rows 16 G + 8 h + (0..7) of the warp's 32
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                        mma_bf16_16816(acc, alo.x, ahi.x, alo.y, ahi.y, b.x, b.y);
+                        mma_bf16_16816(acc, alo.z, ahi.z, alo.w, ahi.w, b.z, b.w);
+                        // the diagonal: row i of the 16 meets column i (h = 0) or i - 8 (h = 1); lane 4g+c holds
+                        // columns 2c, 2c+1 of rows g (acc[0], acc[1]) and g+8 (acc[2], acc[3])
+                        if (c == (g >> 1)) {
+                            const float v = h == 0 ? ((g & 1) ? acc[1] : acc[0]) : ((g & 1) ? acc[3] : acc[2]);
+                            dpart[(st * 4 + wg) * kTileM + 32 * (warp & 3) + 16 * G + 8 * h + g] = v;
+                        }
                     }
-                    // the four chunks of the row, added in a fixed order; rows past the group read zeros for O
-                    part += __shfl_xor_sync(0xffffffffu, part, 1);
-                    part += __shfl_xor_sync(0xffffffffu, part, 2);
-                    if (ochunk == 0) dpart[(st * 4 + wg) * kTileM + r] = part;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarDFull + st));
