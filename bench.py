@@ -518,9 +518,9 @@ def roofline(w, kernels, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (kernel, workload) -> bytes.
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("tc_fwd_kernel", "C2"): 474.2e6,        # profiles/tc_fwd_kernel_C2.md
-    ("tc_bwd_dq_kernel", "C2"): 691.4e6,     # profiles/tc_bwd_dq_kernel_C2.md
-    ("tc_bwd_dkv_kernel", "C2"): 814.0e6,    # profiles/tc_bwd_dkv_kernel_C2.md (with the row statistic D)
+    ("tc_fwd_kernel", "C2"): 475.3e6,        # profiles/tc_fwd_kernel_C2.md
+    ("tc_bwd_dq_kernel", "C2"): 691.0e6,     # profiles/tc_bwd_dq_kernel_C2.md
+    ("tc_bwd_dkv_kernel", "C2"): 823.0e6,    # profiles/tc_bwd_dkv_kernel_C2.md (with the row statistic D)
 }
 
 
