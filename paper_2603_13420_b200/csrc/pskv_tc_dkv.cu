@@ -432,9 +432,10 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             PSKV_TRACE_EVENT(31, gi);
             return true;
         };
+        Unit x_next = unit_of<PRE>(p, 0);  // (DROW: the next unit is worked out once, for the O loads and for its turn)
 #pragma unroll 1
         for (int u = 0; u < total_units && ok; ++u) {
-            const Unit x = unit_of<PRE>(p, u);
+            const Unit x = DROW ? x_next : unit_of<PRE>(p, u);
             const int st = u & 1;
             const int gr = x.tt * kTileM + row;  // row inside the group: head-major, then position
             const bool valid = gr < p.Rg && (!PRE || x.b < p.B);
@@ -479,7 +480,10 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarDFull + st));
                 // the O slice of the next unit, in flight while this unit is worked on
-                if (u + 1 < total_units) load_o(unit_of<PRE>(p, u + 1));
+                if (u + 1 < total_units) {
+                    x_next = unit_of<PRE>(p, u + 1);
+                    load_o(x_next);
+                }
             }
             ok = mbar_wait_warp(bar(kBarSFull + st), (u >> 1) & 1, abort_flag, p.status, kErrDkvElem);
             if (!ok) break;
