@@ -1140,7 +1140,23 @@ TilePlan plan_suffix_ring(const Dims &dm)
     } else {
         pl.Spad = round_up(dm.Skv, 8);
         pl.cpb = kBlockN / pl.Spad;
-        pl.cbox = kTileM / Rg < dm.B ? kTileM / Rg : dm.B;
+        const int cmax = kTileM / Rg < dm.B ? kTileM / Rg : dm.B;
+        // Candidates per tile: as many as fit, unless a few less give every SM a tile (or one round of tiles
+        // less): a CTA's time is its tiles times the key blocks of a tile.  With 512 candidates of one query row
+        // x 4 heads, 32 per tile are 128 tiles of 18 blocks on 148 SMs, 30 per tile are 144 tiles of 17.
+        const int sms = sm_count();
+        const int nblk = (dm.P + kBlockN - 1) / kBlockN;
+        long long best_cost = -1;
+        pl.cbox = cmax;
+        for (int c = cmax; c >= 1 && c >= cmax - 8; --c) {
+            const long long tiles = (long long)dm.Hkv * ((dm.B + c - 1) / c);
+            const long long rounds = (tiles + sms - 1) / sms;
+            const long long cost = rounds * (nblk + (c + pl.cpb - 1) / pl.cpb);
+            if (best_cost < 0 || cost < best_cost) {
+                best_cost = cost;
+                pl.cbox = c;
+            }
+        }
         pl.tile_rows = pl.seg_rows = Rg * pl.cbox;
         pl.tiles_per_group = (dm.B + pl.cbox - 1) / pl.cbox;
     }
