@@ -432,18 +432,30 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             PSKV_TRACE_EVENT(31, gi);
             return true;
         };
-        Unit x_next = unit_of<PRE>(p, 0);  // (DROW: the next unit is worked out once, for the O loads and for its turn)
+        // The next unit is worked out once, and the two per-row statistics of my row in it (lse, D) are asked for
+        // a unit ahead, before the write-back, so that their latency lies under it (about 1 % at 192-row groups).
+        Unit x_next = unit_of<PRE>(p, 0);
+        float lse_next = 0.f, dr_next = 0.f;
+        auto load_stats = [&](const Unit &y) {
+            const int gy = y.tt * kTileM + row;
+            const bool v = gy < p.Rg && (!PRE || y.b < p.B);
+            const size_t r0 = ((size_t)y.b * p.Hq + (size_t)y.g * p.n_rep) * p.S;
+            lse_next = v ? p.lse[r0 + gy] : 0.f;
+            dr_next = (!DROW && v) ? p.row_dot[r0 + gy] : 0.f;
+        };
+        if (total_units > 0) load_stats(x_next);
 #pragma unroll 1
         for (int u = 0; u < total_units && ok; ++u) {
-            const Unit x = DROW ? x_next : unit_of<PRE>(p, u);
+            const Unit x = x_next;
             const int st = u & 1;
             const int gr = x.tt * kTileM + row;  // row inside the group: head-major, then position
             const bool valid = gr < p.Rg && (!PRE || x.b < p.B);
             const size_t row0 = ((size_t)x.b * p.Hq + (size_t)x.g * p.n_rep) * p.S;
             // causal: suffix key t is visible when t <= i; prefix mode: every key of the block that exists
             const int i_pos = !valid ? -1 : PRE ? min(64, p.P - x.kb * 64) - 1 : gr - p.fd_S.div(gr) * p.S;
-            const float nl2 = valid ? -p.lse[row0 + gr] * kLog2e : 0.f;
-            float dr = (!DROW && valid) ? p.row_dot[row0 + gr] : 0.f;
+            const float nl2 = -lse_next * kLog2e;
+            float dr = dr_next;
+            if (!DROW && u + 1 < total_units) x_next = unit_of<PRE>(p, u + 1);
             if (DROW) {
                 // my 32 of the row's 128 columns: O from global memory (requested one unit ahead), dO from the
                 // tile in shared memory (64-column slabs of 128-byte rows, 16-byte chunks swizzled by the row)
@@ -541,6 +553,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarPReady));
             PSKV_TRACE_EVENT(24, u);
+            if (u + 1 < total_units) load_stats(x_next);
             // the write-back of a group runs one unit late, when its last MMAs have long completed
             if (pending_gi >= 0) {
                 ok = write_back(pending_gi);
