@@ -1,8 +1,9 @@
 """The secondary lines of the benchmark at the sizes and in the launch configuration it times them: the
 decode-shaped forward at B = 512 and B = 2048 (one new token on a ragged 48-token suffix cache, C2 layer
 shape) and the multi-instruction forward + backward with 8 instructions x 64 candidates (both prefix-length
-lists of the benchmark).  The GPU runs the whole batch; the fp64 oracle runs the sampled candidates one by
-one (candidates never meet in this operator, so a candidate evaluated alone is its row of the batch)."""
+lists of the benchmark), and the prefix-cache gradients over all 512 candidates.  The GPU runs the whole
+batch; the fp64 oracle runs the sampled candidates one by one (candidates never meet in this operator, so a
+candidate evaluated alone is its row of the batch), except for the prefix gradients, which sum over all."""
 import numpy as np
 import pytest
 import torch
@@ -99,3 +100,24 @@ def test_multi_instruction_step_at_benchmark_size_sampled(lens):
         parity.check_tensor("dq[%d]" % c, got["dq"][c:c + 1], rq)
         parity.check_tensor("dk_suffix[%d]" % c, got["dk"][c:c + 1], rk)
         parity.check_tensor("dv_suffix[%d]" % c, got["dv"][c:c + 1], rv)
+
+
+def test_prefix_gradients_at_benchmark_size():
+    """dK_p / dV_p at the C2 shape with all 512 candidates (every key's gradient is a sum over 98 304 query
+    rows of its KV head, so nothing can be sampled): the whole result against the oracle."""
+    from paper_2603_13420_b200.inputs import make_inputs
+    w = WORKLOADS["C2"]
+    t = make_inputs(w, with_dout=True)
+    dev = {k: v.cuda() for k, v in t.items()}
+    out, lse = pskv.pskv_attn_fwd(dev["q"], dev["prefix_k"], dev["prefix_v"], dev["suffix_k"], dev["suffix_v"], w.scale)
+    dk = parity.Guarded((w.Hkv, w.P, w.d), torch.bfloat16, "cuda")
+    dv = parity.Guarded((w.Hkv, w.P, w.d), torch.bfloat16, "cuda")
+    pskv.pskv_attn_bwd_prefix(dev["dout"], None, dev["q"], dev["prefix_k"], dev["prefix_v"], out, lse, w.scale,
+                              dk_prefix=dk.view, dv_prefix=dv.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    dk.check("dk_prefix"); dv.check("dv_prefix")
+    f = {k: parity.to_f64(v) for k, v in t.items()}
+    rk, rv = oracle.attn_bwd_prefix(f["dout"], f["q"], f["prefix_k"], f["prefix_v"], f["suffix_k"], f["suffix_v"],
+                                    w.scale, None)
+    parity.check_tensor("dk_prefix", parity.to_f64(dk.view), rk)
+    parity.check_tensor("dv_prefix", parity.to_f64(dv.view), rv)
