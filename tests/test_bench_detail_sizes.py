@@ -1,7 +1,7 @@
 """The secondary lines of the benchmark at the sizes and in the launch configuration it times them: the
 decode-shaped forward at B = 512 and B = 2048 (one new token on a ragged 48-token suffix cache, C2 layer
 shape) and the multi-instruction forward + backward with 8 instructions x 64 candidates (both prefix-length
-lists of the benchmark), and the prefix-cache gradients over all 512 candidates.  The GPU runs the whole
+lists of the benchmark), the prefix-cache gradients over all 512 candidates and the 2048-token prefill.  The GPU runs the whole
 batch; the fp64 oracle runs the sampled candidates one by one (candidates never meet in this operator, so a
 candidate evaluated alone is its row of the batch), except for the prefix gradients, which sum over all."""
 import numpy as np
@@ -121,3 +121,29 @@ def test_prefix_gradients_at_benchmark_size():
                                     w.scale, None)
     parity.check_tensor("dk_prefix", parity.to_f64(dk.view), rk)
     parity.check_tensor("dv_prefix", parity.to_f64(dv.view), rv)
+
+
+def test_prefill_of_a_2048_token_sequence_sampled_heads():
+    """The prefill line: causal self-attention of one 2048-token sequence in the C3 head layout (B = 1, P = 0,
+    the sequence's K/V passed as the suffix), launched whole; two KV heads with their query heads go through
+    the oracle (heads never meet either)."""
+    w = WORKLOADS["C3"]
+    S = w.P
+    n_rep = w.Hq // w.Hkv
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(SEED + S)
+    q, k, v = _draw(gen, 1, w.Hq, S, w.d), _draw(gen, 1, w.Hkv, S, w.d), _draw(gen, 1, w.Hkv, S, w.d)
+    out = parity.Guarded((1, w.Hq, S, w.d), torch.bfloat16, "cuda")
+    lse = parity.Guarded((1, w.Hq, S), torch.float32, "cuda")
+    pskv.pskv_attn_fwd(q.cuda(), None, None, k.cuda(), v.cuda(), w.scale, out=out.view, lse=lse.view)
+    assert pskv.pskv_poll_device_status() == pskv.PSKV_OK
+    out.check("out"); lse.check("lse")
+    got_out, got_lse = parity.to_f64(out.view), parity.to_f64(lse.view)
+    empty = np.zeros((1, 0, w.d))
+    for g in (0, w.Hkv - 1):
+        hs = slice(g * n_rep, (g + 1) * n_rep)
+        ref_out, ref_lse = oracle.attn_fwd(parity.to_f64(q[:, hs]), empty, empty, parity.to_f64(k[:, g:g + 1]),
+                                           parity.to_f64(v[:, g:g + 1]), w.scale)
+        # (the first rows see one or two keys: relative bounds, as everywhere a row has fewer than 128 keys)
+        parity.check_tensor("out[head group %d]" % g, got_out[:, hs], ref_out)
+        parity.check_lse(got_lse[:, hs], ref_lse)
